@@ -1,0 +1,196 @@
+/*
+ * apms.h - C ABI of the APMSqueeze compressed-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the data-parallel hot path of APMSqueeze on ONE GPU, with the n
+ * data-parallel workers simulated as n device-resident buffer sets and the two exchanges
+ * of the Gather-Scatter AllReduce (Figure 1) replaced by direct indexing of device memory:
+ *
+ *   warmup phase       full-precision Adam with bias correction on the worker-averaged
+ *                      gradient (Algorithm 1 line 2; Section 3.2);
+ *   phase switch       the variance v is frozen, all compression errors start at zero
+ *                      (Section 3.3, first paragraph; Algorithm 1 initialisation);
+ *   compression phase  per step, for every chunk: every worker forms its local momentum,
+ *                      adds its compression error, compresses to sign bits + one scale and
+ *                      keeps the new error; the chunk's server averages the n decompressed
+ *                      messages, adds its own error, recompresses and keeps its new error;
+ *                      every worker replaces its momentum by the decompressed server message
+ *                      and updates the model with the frozen variance
+ *                      (Section 3.3 steps 1-6 = Algorithm 1 lines 4-11; Supplement A).
+ *
+ * Compressor (Section 5.1): sign bits + scale = ||z||_2 / sqrt(L) per chunk of L elements,
+ * so that the decompressed chunk has the l2 norm of the compensated chunk z.
+ *
+ * Conventions
+ *   - All state is binary32; sums of squares are accumulated in binary64.  Every operation
+ *     is rounded once (no fused contraction except the momentum update's single fma).
+ *   - A chunk is `chunk` consecutive elements of the flat parameter vector (a positive
+ *     multiple of 32); the last chunk may be shorter and is scaled by its true length.
+ *     C = ceil(d / chunk) chunks, W = ceil(d / 32) sign words.
+ *   - Sign words: uint32 word w, bit j (LSB = bit 0) holds element 32*w + j; 1 means
+ *     value >= 0 (so +0.0 and -0.0 give 1, NaN gives 0); bits past d are 0.
+ *   - Scales: float[C] in chunk order.
+ *   - "dev" pointers are device pointers valid on the context's device; "host" pointers
+ *     are ordinary host memory.  Gradient arrays are HOST arrays of n pointers.
+ *   - Every call enqueues its work on the context's stream and returns without a host
+ *     synchronisation unless stated otherwise.  The library never traps or aborts; every
+ *     failure is a status code and a message available from apms_last_error().
+ *   - The library has no CPU fallback: without a CUDA device every device call fails with
+ *     APMS_ERR_CUDA.
+ *   - One context must not be used from two host threads at once.
+ */
+#ifndef APMS_H
+#define APMS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct apms_ctx apms_ctx;
+
+typedef enum {
+    APMS_OK = 0,
+    APMS_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, size out of range            */
+    APMS_ERR_BAD_STATE = 2,     /* call not allowed in the context's current phase         */
+    APMS_ERR_CUDA = 3,          /* a CUDA runtime call failed; see apms_last_error()       */
+    APMS_ERR_OOM = 4,           /* workspace too small, or allocation failed               */
+    APMS_ERR_TIMEOUT = 5,       /* reserved: a bounded device-side wait gave up            */
+    APMS_ERR_BOUNDS = 6         /* reserved: a checked build recorded an out-of-range index */
+} apms_status;
+
+/* Phases of Algorithm 1. */
+typedef enum {
+    APMS_PHASE_CREATED = 0,     /* no parameters yet                                       */
+    APMS_PHASE_WARMUP = 1,      /* Adam steps (Algorithm 1 line 2)                         */
+    APMS_PHASE_COMPRESSED = 2   /* v frozen, 1-bit steps (Algorithm 1 lines 3-12)          */
+} apms_phase;
+
+/* State arrays readable / writable through apms_get_state / apms_set_state. */
+typedef enum {
+    APMS_STATE_X = 0,              /* float[d]   model x                                   */
+    APMS_STATE_V = 1,              /* float[d]   variance v (frozen after the switch)      */
+    APMS_STATE_M = 2,              /* float[d]   momentum m shared by all workers          */
+    APMS_STATE_WORKER_ERR = 3,     /* float[d]   worker compression error delta^(i)        */
+    APMS_STATE_WORKER_BITS = 4,    /* uint32[W]  sign words worker i sent last step        */
+    APMS_STATE_WORKER_SCALES = 5,  /* float[C]   scales worker i sent last step            */
+    APMS_STATE_SERVER_ERR = 6,     /* float[d]   server compression error delta-bar        */
+    APMS_STATE_SERVER_BITS = 7,    /* uint32[W]  sign words the servers broadcast          */
+    APMS_STATE_SERVER_SCALES = 8   /* float[C]   scales the servers broadcast              */
+} apms_state_id;
+
+/* Kernels of the path, for apms_kernel_time(). */
+typedef enum {
+    APMS_KERNEL_WARMUP_ADAM = 0,   /* Section 3.2                                           */
+    APMS_KERNEL_WORKER = 1,        /* Section 3.3 steps 1-2 (momentum + EC compression)     */
+    APMS_KERNEL_SERVER = 2,        /* Section 3.3 step 4 (average + EC recompression)       */
+    APMS_KERNEL_APPLY = 3,         /* Section 3.3 steps 5-6 (momentum replace + model update) */
+    APMS_KERNEL_COUNT = 4
+} apms_kernel_id;
+
+#define APMS_MAX_WORKERS 64
+
+/* Bytes of device workspace a context of this shape needs (pure function; 0 if the shape
+ * is invalid).  Covers x, v, m, the n worker and one server compensated vectors, all sign
+ * words and scales, and two d-float staging buffers for the host-gradient entry point. */
+size_t apms_workspace_bytes(int64_t d, int n, int64_t chunk);
+
+/* Create a context on the current CUDA device for d parameters and n simulated workers
+ * (Problem Setting: n workers, one shared x).  beta1, beta2, eps (Adam's constant, also
+ * added to sqrt(v) in the compression phase) and lr (gamma_t, changeable with
+ * apms_set_lr) are the hyper-parameters of Algorithm 1.  Requires d >= 1,
+ * 1 <= n <= APMS_MAX_WORKERS, chunk a positive multiple of 32.  No device memory is
+ * touched until apms_bind() or the first call that needs the workspace.
+ * On failure *out is NULL and apms_last_error(NULL) describes why. */
+apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float beta2,
+                        float eps, float lr, int64_t chunk);
+
+/* Give the context caller-owned device memory (>= apms_workspace_bytes, 256-byte aligned)
+ * and a CUDA stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ * The caller keeps ownership and must keep both alive until apms_destroy().  If never
+ * called, the context allocates its own workspace with cudaMalloc on first use and works
+ * on the default stream.  Must be called before apms_set_params(). */
+apms_status apms_bind(apms_ctx* ctx, void* workspace_dev, size_t bytes, void* cuda_stream);
+
+/* x <- x0, m <- 0, v <- 0, t <- 0 (Algorithm 1 initialisation); phase becomes WARMUP.
+ * x0 holds d floats, on the device if src_is_device != 0, else on the host (the call then
+ * synchronises the stream before returning). */
+apms_status apms_set_params(apms_ctx* ctx, const float* x0, int src_is_device);
+
+/* gamma_t for the following steps (Algorithm 1 takes a per-step learning rate). */
+apms_status apms_set_lr(apms_ctx* ctx, float lr);
+
+/* One Adam step (Section 3.2) on gbar = (1/n) sum_i g_i, summed in worker order:
+ *   m <- b1 m + (1-b1) gbar ; v <- b2 v + (1-b2) gbar^2 ;
+ *   x <- x - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps),  t = 1 for the first call.
+ * grads_dev: host array of n device pointers, each d floats, 16-byte aligned, read-only,
+ * valid until the stream has passed this step.  Phase must be WARMUP. */
+apms_status apms_warmup_step(apms_ctx* ctx, const float* const* grads_dev);
+
+/* End of warmup (Section 3.3: v is no longer updated): phase becomes COMPRESSED, every
+ * worker error and the server error are zero, Adam's raw m carries over. */
+apms_status apms_freeze_v(apms_ctx* ctx);
+
+/* One compression-phase step (Section 3.3 steps 1-6), for every chunk c of length L:
+ *   worker i:  z_i = (b1 m + (1-b1) g_i) + delta_i ;  s_i = ||z_i||_2 / sqrt(L) ;
+ *              bits_i = (z_i >= 0) ;  delta_i <- z_i - (+-s_i)
+ *   server:    zbar = (1/n) sum_i (+-s_i) + dbar ;  S = ||zbar||_2 / sqrt(L) ;
+ *              bits = (zbar >= 0) ;  dbar <- zbar - (+-S)
+ *   workers:   m <- +-S ;  x <- x - (lr m) / (sqrt(v) + eps)
+ * Same gradient-array contract as apms_warmup_step.  Phase must be COMPRESSED. */
+apms_status apms_compressed_step(apms_ctx* ctx, const float* const* grads_dev);
+
+/* The same step with the n gradients in HOST memory (pinned memory gives asynchronous
+ * copies): worker i's gradient is copied to a device staging buffer while worker i-1 is
+ * being compressed.  If x_out_host is not NULL the updated x (d floats) is copied back.
+ * Synchronises the stream before returning. */
+apms_status apms_compressed_step_host(apms_ctx* ctx, const float* const* grads_host,
+                                      float* x_out_host);
+
+/* Copy x (d floats) to dst: device memory if dst_is_device != 0 (stream-ordered), else
+ * host memory (synchronises the stream). */
+apms_status apms_get_params(apms_ctx* ctx, float* dst, int dst_is_device);
+
+/* Copy one state array to host memory (synchronises).  `worker` is ignored for arrays
+ * that are not per worker.  Errors and momentum are produced from the stored form: the
+ * library keeps, per worker and for the server, the compensated vector z and the chunk
+ * scales, from which delta = z - (+-scale) and m = +-scale follow exactly. */
+apms_status apms_get_state(apms_ctx* ctx, apms_state_id which, int worker, void* dst_host);
+
+/* The same for elements [first, first + count) of the array (count floats or words). */
+apms_status apms_get_state_slice(apms_ctx* ctx, apms_state_id which, int worker, int64_t first,
+                                 int64_t count, void* dst_host);
+
+/* Overwrite X, V, M, WORKER_ERR or SERVER_ERR from host memory (teacher forcing, restoring
+ * a checkpoint).  Setting an error array resets that side's stored scales to zero (they
+ * read as 0 until the next step); sign words and scales themselves cannot be set.
+ * Synchronises. */
+apms_status apms_set_state(apms_ctx* ctx, apms_state_id which, int worker, const void* src_host);
+
+/* Restore the step counter and phase of a checkpoint (t = Adam steps taken so far). */
+apms_status apms_restore(apms_ctx* ctx, int t, apms_phase phase);
+
+apms_phase  apms_get_phase(const apms_ctx* ctx);
+int         apms_get_t(const apms_ctx* ctx);
+
+/* Kernel timing: when enabled, every kernel launch is bracketed by CUDA events on the
+ * context's stream.  apms_kernel_time() synchronises the stream, returns the total time
+ * and launch count of one kernel since the last call for that kernel, and resets them. */
+apms_status apms_set_timing(apms_ctx* ctx, int enabled);
+apms_status apms_kernel_time(apms_ctx* ctx, apms_kernel_id which, double* total_ms, int64_t* launches);
+
+/* Kernels launched by this context since creation. */
+int64_t     apms_launch_count(const apms_ctx* ctx);
+
+/* Message of the last failure on this context (ctx == NULL: of the last failed
+ * apms_create on this thread).  Never NULL. */
+const char* apms_last_error(const apms_ctx* ctx);
+
+/* Free the context (and its workspace if it allocated one).  NULL is ignored. */
+void        apms_destroy(apms_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* APMS_H */

@@ -1,0 +1,307 @@
+"""Thin Python binding of the C ABI declared in include/apms.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  The
+module-level functions carry the C names; `Context` bundles a handle with a
+torch-allocated workspace and stream (PyTorch is used for device memory and streams
+only).  There is no CPU fallback: if the shared library is missing or no CUDA device
+is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libapms.so")
+
+OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_CUDA, ERR_OOM, ERR_TIMEOUT, ERR_BOUNDS = range(7)
+PHASE_CREATED, PHASE_WARMUP, PHASE_COMPRESSED = range(3)
+(STATE_X, STATE_V, STATE_M, STATE_WORKER_ERR, STATE_WORKER_BITS, STATE_WORKER_SCALES,
+ STATE_SERVER_ERR, STATE_SERVER_BITS, STATE_SERVER_SCALES) = range(9)
+KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
+KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
+MAX_WORKERS = 64
+
+_FP = C.POINTER(C.c_float)
+_FPP = C.POINTER(_FP)
+
+# name -> (restype, argtypes); mirrors include/apms.h one to one
+SIGNATURES = {
+    "apms_workspace_bytes": (C.c_size_t, [C.c_int64, C.c_int, C.c_int64]),
+    "apms_create": (C.c_int, [C.POINTER(C.c_void_p), C.c_int64, C.c_int, C.c_float, C.c_float,
+                              C.c_float, C.c_float, C.c_int64]),
+    "apms_bind": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "apms_set_params": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
+    "apms_set_lr": (C.c_int, [C.c_void_p, C.c_float]),
+    "apms_warmup_step": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p)]),
+    "apms_freeze_v": (C.c_int, [C.c_void_p]),
+    "apms_compressed_step": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p)]),
+    "apms_compressed_step_host": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]),
+    "apms_get_params": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
+    "apms_get_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
+    "apms_get_state_slice": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
+    "apms_set_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
+    "apms_restore": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
+    "apms_get_phase": (C.c_int, [C.c_void_p]),
+    "apms_get_t": (C.c_int, [C.c_void_p]),
+    "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "apms_launch_count": (C.c_int64, [C.c_void_p]),
+    "apms_last_error": (C.c_char_p, [C.c_void_p]),
+    "apms_destroy": (None, [C.c_void_p]),
+}
+
+_lib: Optional[C.CDLL] = None
+
+
+class ApmsError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"apms status {status}: {message}")
+        self.status = status
+
+
+def load() -> C.CDLL:
+    """Load paper_2008_11343_b200/libapms.so (built by build.py); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is not built; run `python -m paper_2008_11343_b200.build` "
+                              "(there is no fallback path)")
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (C.c_void_p * len(ptrs))(*ptrs)
+
+
+# --- functions with the C names ------------------------------------------------------------
+
+def apms_workspace_bytes(d: int, n: int, chunk: int) -> int:
+    return int(load().apms_workspace_bytes(d, n, chunk))
+
+
+def apms_create(d, n, beta1, beta2, eps, lr, chunk) -> int:
+    h = C.c_void_p()
+    st = load().apms_create(C.byref(h), d, n, beta1, beta2, eps, lr, chunk)
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(None).decode())
+    return h.value
+
+
+def _check(h, st):
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(h).decode())
+
+
+def apms_bind(h, workspace_ptr: int, nbytes: int, stream: int):
+    _check(h, load().apms_bind(h, workspace_ptr, nbytes, stream))
+
+
+def apms_set_params(h, x0_ptr: int, src_is_device: bool):
+    _check(h, load().apms_set_params(h, x0_ptr, int(src_is_device)))
+
+
+def apms_set_lr(h, lr: float):
+    _check(h, load().apms_set_lr(h, lr))
+
+
+def apms_warmup_step(h, grad_ptrs: Sequence[int]):
+    _check(h, load().apms_warmup_step(h, _ptr_array(grad_ptrs)))
+
+
+def apms_freeze_v(h):
+    _check(h, load().apms_freeze_v(h))
+
+
+def apms_compressed_step(h, grad_ptrs: Sequence[int]):
+    _check(h, load().apms_compressed_step(h, _ptr_array(grad_ptrs)))
+
+
+def apms_compressed_step_host(h, grad_host_ptrs: Sequence[int], x_out_host_ptr: Optional[int]):
+    _check(h, load().apms_compressed_step_host(h, _ptr_array(grad_host_ptrs), x_out_host_ptr))
+
+
+def apms_get_params(h, dst_ptr: int, dst_is_device: bool):
+    _check(h, load().apms_get_params(h, dst_ptr, int(dst_is_device)))
+
+
+def apms_get_state(h, which: int, worker: int, dst_host_ptr: int):
+    _check(h, load().apms_get_state(h, which, worker, dst_host_ptr))
+
+
+def apms_get_state_slice(h, which: int, worker: int, first: int, count: int, dst_host_ptr: int):
+    _check(h, load().apms_get_state_slice(h, which, worker, first, count, dst_host_ptr))
+
+
+def apms_set_state(h, which: int, worker: int, src_host_ptr: int):
+    _check(h, load().apms_set_state(h, which, worker, src_host_ptr))
+
+
+def apms_restore(h, t: int, phase: int):
+    _check(h, load().apms_restore(h, t, phase))
+
+
+def apms_get_phase(h) -> int:
+    return int(load().apms_get_phase(h))
+
+
+def apms_get_t(h) -> int:
+    return int(load().apms_get_t(h))
+
+
+def apms_set_timing(h, enabled: bool):
+    _check(h, load().apms_set_timing(h, int(enabled)))
+
+
+def apms_kernel_time(h, which: int):
+    ms, cnt = C.c_double(0.0), C.c_int64(0)
+    _check(h, load().apms_kernel_time(h, which, C.byref(ms), C.byref(cnt)))
+    return ms.value, cnt.value
+
+
+def apms_launch_count(h) -> int:
+    return int(load().apms_launch_count(h))
+
+
+def apms_last_error(h) -> str:
+    return load().apms_last_error(h).decode()
+
+
+def apms_destroy(h):
+    load().apms_destroy(h)
+
+
+# --- convenience wrapper: handle + torch workspace + stream ---------------------------------
+
+class Context:
+    """An apms context whose workspace is a torch CUDA tensor and whose stream is torch's."""
+
+    def __init__(self, d: int, n: int, beta1: float, beta2: float, eps: float, lr: float, chunk: int,
+                 device: str = "cuda:0", stream=None):
+        import torch
+
+        if not torch.cuda.is_available():
+            raise RuntimeError("apms needs a CUDA device; there is no CPU path")
+        self.d, self.n, self.chunk = d, n, chunk
+        self.C = (d + chunk - 1) // chunk
+        self.W = (d + 31) // 32
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self._h = apms_create(d, n, beta1, beta2, eps, lr, chunk)
+        nbytes = apms_workspace_bytes(d, n, chunk)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        apms_bind(self._h, self.workspace.data_ptr(), nbytes, self.stream.cuda_stream)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            apms_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _dev_ptrs(grads) -> list:
+        import torch
+
+        ptrs = []
+        for g in grads:
+            assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
+            ptrs.append(g.data_ptr())
+        return ptrs
+
+    def set_params(self, x0):
+        """x0: torch CUDA float32 tensor or numpy float32 array of d elements."""
+        if isinstance(x0, np.ndarray):
+            x0 = np.ascontiguousarray(x0, dtype=np.float32)
+            assert x0.size == self.d
+            apms_set_params(self._h, x0.ctypes.data, False)
+        else:
+            assert x0.numel() == self.d and x0.is_contiguous()
+            apms_set_params(self._h, x0.data_ptr(), x0.is_cuda)
+
+    def set_lr(self, lr: float):
+        apms_set_lr(self._h, lr)
+
+    def warmup_step(self, grads):
+        assert len(grads) == self.n
+        apms_warmup_step(self._h, self._dev_ptrs(grads))
+
+    def freeze_v(self):
+        apms_freeze_v(self._h)
+
+    def compressed_step(self, grads):
+        assert len(grads) == self.n
+        apms_compressed_step(self._h, self._dev_ptrs(grads))
+
+    def compressed_step_host(self, grads_host, x_out_host=None):
+        """grads_host: n CPU float32 tensors/arrays (pinned for overlap); x_out_host: CPU buffer or None."""
+        assert len(grads_host) == self.n
+
+        def hp(a):
+            return a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
+
+        apms_compressed_step_host(self._h, [hp(g) for g in grads_host],
+                                  None if x_out_host is None else hp(x_out_host))
+
+    def get_params(self, out=None) -> np.ndarray:
+        if out is not None and not isinstance(out, np.ndarray):
+            apms_get_params(self._h, out.data_ptr(), out.is_cuda)
+            return out
+        out = np.empty(self.d, dtype=np.float32) if out is None else out
+        apms_get_params(self._h, out.ctypes.data, False)
+        return out
+
+    def get_state(self, which: int, worker: int = 0) -> np.ndarray:
+        if which in (STATE_WORKER_BITS, STATE_SERVER_BITS):
+            out = np.empty(self.W, dtype=np.uint32)
+        elif which in (STATE_WORKER_SCALES, STATE_SERVER_SCALES):
+            out = np.empty(self.C, dtype=np.float32)
+        else:
+            out = np.empty(self.d, dtype=np.float32)
+        apms_get_state(self._h, which, worker, out.ctypes.data)
+        return out
+
+    def get_state_slice(self, which: int, first: int, count: int, worker: int = 0) -> np.ndarray:
+        dtype = np.uint32 if which in (STATE_WORKER_BITS, STATE_SERVER_BITS) else np.float32
+        out = np.empty(count, dtype=dtype)
+        apms_get_state_slice(self._h, which, worker, first, count, out.ctypes.data)
+        return out
+
+    def set_state(self, which: int, value: np.ndarray, worker: int = 0):
+        value = np.ascontiguousarray(value, dtype=np.float32)
+        assert value.size == self.d
+        apms_set_state(self._h, which, worker, value.ctypes.data)
+
+    def restore(self, t: int, phase: int):
+        apms_restore(self._h, t, phase)
+
+    @property
+    def phase(self) -> int:
+        return apms_get_phase(self._h)
+
+    @property
+    def t(self) -> int:
+        return apms_get_t(self._h)
+
+    def set_timing(self, enabled: bool):
+        apms_set_timing(self._h, enabled)
+
+    def kernel_time(self, which: int):
+        return apms_kernel_time(self._h, which)
+
+    @property
+    def launch_count(self) -> int:
+        return apms_launch_count(self._h)

@@ -1,0 +1,927 @@
+// APMSqueeze compressed-step library for B200 (sm_100a): kernels and C ABI.
+//
+// Data layout in HBM (one context, the n workers simulated as n buffer sets):
+//   x, v            float[d]      model and (frozen) variance, one copy: every worker holds
+//                                 the same x after every step (Algorithm 1 lines 10-11)
+//   m32             float[d]      binary32 momentum; authoritative only during warmup, for the
+//                                 first compressed step and after apms_set_state(M)
+//   zbar            float[d]      the server's last compensated vector  zbar = avg + dbar_old
+//   Bbar, Sbar      uint32[W], float[C]   the server's last message.  Together with zbar they
+//                                 hold BOTH the shared momentum m = +-Sbar (Section 3.3 step 5)
+//                                 and the server error dbar = zbar - (+-Sbar) (step 4)
+//   z_i             n x float[d]  worker i's last compensated vector z_i = m_i + delta_i_old
+//   B_i, s_i        n x uint32[W], n x float[C]   worker i's last message; its error is
+//                                 delta_i = z_i - (+-s_i) (Section 3.3 step 2)
+//
+// Keeping z instead of delta removes the only intra-chunk dependency of the step (the error
+// needs the chunk's scale, the scale needs the whole chunk): the subtraction delta = z - C[z]
+// is performed, with the same single binary32 rounding, by the next step's read.  Every
+// element of g_i and z_i is then read once and z_i written once per step, in one streaming
+// pass, and nothing has to be held on chip across the chunk reduction.
+//
+// Arithmetic: explicit round-to-nearest intrinsics everywhere, so that the compiler can
+// neither contract nor reorder; sums of squares in binary64 (products of binary32 values are
+// exact in binary64, so only the order of the additions can differ from a sequential sum).
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+#include <math.h>
+#include <new>
+#include <vector>
+
+#include "apms.h"
+
+namespace {
+
+constexpr int kThreads = 256;            // threads per CTA in every kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kGroup = 128;              // elements one warp covers per 128-bit access (4 sign words)
+
+struct GradPtrs { const float* p[APMS_MAX_WORKERS]; };
+
+// ------------------------------------------------------------------------------------------
+// small device helpers
+
+__device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void st_stream4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+// Up to four consecutive floats starting at p[k]; elements at or past `len` read as 0.
+__device__ __forceinline__ float4 ld4_checked(const float* p, int k, int len, bool streaming) {
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k + 3 < len) {
+        r = streaming ? ld_stream4(p + k) : *reinterpret_cast<const float4*>(p + k);
+    } else {
+        if (k + 0 < len) r.x = p[k + 0];
+        if (k + 1 < len) r.y = p[k + 1];
+        if (k + 2 < len) r.z = p[k + 2];
+    }
+    return r;
+}
+__device__ __forceinline__ void st4_checked(float* p, int k, int len, float4 v) {
+    if (k + 3 < len) {
+        st_stream4(p + k, v);
+    } else {
+        if (k + 0 < len) p[k + 0] = v.x;
+        if (k + 1 < len) p[k + 1] = v.y;
+        if (k + 2 < len) p[k + 2] = v.z;
+    }
+}
+
+// +-s with the sign of the compressor: z >= 0 gives +s (so do +0 and -0), NaN gives -s.
+__device__ __forceinline__ float signed_scale(float z, float s) { return (z >= 0.0f) ? s : -s; }
+__device__ __forceinline__ float bit_scale(uint32_t bit, float s) { return bit ? s : -s; }
+
+// The compression error implied by a stored compensated value and its chunk's scale.
+__device__ __forceinline__ float implied_error(float z, float s) { return __fsub_rn(z, signed_scale(z, s)); }
+
+// Lane l of a warp holds the four sign bits (nibble) of elements 4l..4l+3 of a 128-element
+// group.  Returns, in lanes 0, 8, 16, 24, the LSB-first sign word of elements 32*(l/8)...
+__device__ __forceinline__ uint32_t pack_group_words(uint32_t nibble, int lane) {
+    uint32_t w = nibble << (4 * (lane & 7));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    w |= __shfl_xor_sync(0xffffffffu, w, 2);
+    w |= __shfl_xor_sync(0xffffffffu, w, 4);
+    return w;
+}
+
+__device__ __forceinline__ double warp_sum(double a) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_down_sync(0xffffffffu, a, o);
+    return a;
+}
+
+// Fixed-order block sum (lane tree, then warps in order); result valid in thread 0.
+__device__ __forceinline__ double block_sum(double a, double* smem) {
+    a = warp_sum(a);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) smem[warp] = a;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += smem[w];
+    }
+    return t;
+}
+
+// ------------------------------------------------------------------------------------------
+// Warmup: Adam with bias correction on the worker-averaged gradient (Section 3.2).
+
+struct AdamArgs {
+    float* x; float* m; float* v;
+    int64_t d; int n;
+    float beta1, beta2, omb1, omb2, bc1, bc2, lr, eps, nf;
+};
+
+__device__ __forceinline__ void adam_elem(const AdamArgs& a, float gs, float& m, float& v, float& x) {
+    const float gbar = __fdiv_rn(gs, a.nf);
+    m = __fmaf_rn(a.beta1, m, __fmul_rn(a.omb1, gbar));
+    v = __fmaf_rn(a.beta2, v, __fmul_rn(a.omb2, __fmul_rn(gbar, gbar)));
+    const float mhat = __fdiv_rn(m, a.bc1);
+    const float vhat = __fdiv_rn(v, a.bc2);
+    x = __fsub_rn(x, __fdiv_rn(__fmul_rn(a.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), a.eps)));
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
+{
+    const int64_t nvec = a.d / 4;
+    for (int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x; q < nvec;
+         q += (int64_t)gridDim.x * kThreads) {
+        const int64_t j = q * 4;
+        float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int i = 0; i < a.n; ++i) {
+            const float4 g = ld_stream4(G.p[i] + j);
+            gs.x = __fadd_rn(gs.x, g.x); gs.y = __fadd_rn(gs.y, g.y);
+            gs.z = __fadd_rn(gs.z, g.z); gs.w = __fadd_rn(gs.w, g.w);
+        }
+        float4 m = *reinterpret_cast<const float4*>(a.m + j);
+        float4 v = *reinterpret_cast<const float4*>(a.v + j);
+        float4 x = *reinterpret_cast<const float4*>(a.x + j);
+        adam_elem(a, gs.x, m.x, v.x, x.x); adam_elem(a, gs.y, m.y, v.y, x.y);
+        adam_elem(a, gs.z, m.z, v.z, x.z); adam_elem(a, gs.w, m.w, v.w, x.w);
+        *reinterpret_cast<float4*>(a.m + j) = m;
+        *reinterpret_cast<float4*>(a.v + j) = v;
+        *reinterpret_cast<float4*>(a.x + j) = x;
+    }
+    // ragged tail (d not a multiple of 4): one thread per element
+    const int64_t j = nvec * 4 + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (j < a.d) {
+        float gs = 0.f;
+        for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, G.p[i][j]);
+        float m = a.m[j], v = a.v[j], x = a.x[j];
+        adam_elem(a, gs, m, v, x);
+        a.m[j] = m; a.v[j] = v; a.x[j] = x;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Worker side: local momentum + error-compensated 1-bit compression (Section 3.3 steps 1-2).
+// One CTA per (chunk, worker); consecutive CTAs take the n workers of one chunk so that the
+// chunk's momentum bits are shared through L2.
+
+struct WorkerArgs {
+    float* z;  int64_t dz;        // n x d compensated vectors, stride dz
+    uint32_t* B; int64_t Wp;      // n x W sign words, stride Wp
+    float* s;  int64_t Cp;        // n x C scales, stride Cp
+    const float* m32;             // binary32 momentum (first step / forced)
+    const uint32_t* Bbar; const float* Sbar;   // momentum as the server's last message
+    int64_t d; int64_t chunk;
+    int i0, ni;                   // this launch covers workers i0 .. i0+ni-1
+    float beta1, omb1;
+};
+
+template <bool M32, bool CHECKED>
+__device__ __forceinline__ void worker_group(const WorkerArgs& a, const float* __restrict__ g,
+                                             float* __restrict__ z, const float* __restrict__ m32,
+                                             const uint32_t* __restrict__ mbits, uint32_t* __restrict__ obits,
+                                             int grp, int lane, int L, float s_old, float Sbar,
+                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc)
+{
+    const int k = grp * kGroup + lane * 4;
+    float mm[4];
+    if (M32) {
+        mm[0] = mv.x; mm[1] = mv.y; mm[2] = mv.z; mm[3] = mv.w;
+    } else {
+        const uint32_t nib = mw >> (4 * (lane & 7));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mm[e] = bit_scale((nib >> e) & 1u, Sbar);
+    }
+    const float gg[4] = {gv.x, gv.y, gv.z, gv.w};
+    const float zo[4] = {zv.x, zv.y, zv.z, zv.w};
+    float zn[4];
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));   // local momentum
+        const float err = implied_error(zo[e], s_old);                          // delta_i (old)
+        zn[e] = __fadd_rn(mi, err);                                             // compensated
+        const bool valid = !CHECKED || (k + e < L);
+        if (valid) {
+            const double zd = (double)zn[e];
+            acc = fma(zd, zd, acc);
+            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+        }
+    }
+    const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
+    if (CHECKED) st4_checked(z, k, L, out); else st_stream4(z + k, out);
+    const uint32_t word = pack_group_words(nibble, lane);
+    if ((lane & 7) == 0) {
+        const int wk = grp * 4 + (lane >> 3);
+        if (!CHECKED || wk * 32 < L) obits[wk] = word;
+    }
+}
+
+template <bool M32, int U>
+__global__ void __launch_bounds__(kThreads, 4)
+k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
+{
+    __shared__ double red[kWarps];
+    const int ii = blockIdx.x % a.ni;
+    const int64_t c = blockIdx.x / a.ni;
+    const int i = a.i0 + ii;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
+    const float* __restrict__ g = G.p[ii] + base;
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
+    const float* __restrict__ m32 = a.m32 + base;
+    const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
+    float* sptr = a.s + (int64_t)i * a.Cp + c;
+    const float s_old = *sptr;
+    const float Sbar = M32 ? 0.0f : a.Sbar[c];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int full = L / kGroup;                  // groups with all 128 elements present
+    const int ngroups = (L + kGroup - 1) / kGroup;
+    double acc = 0.0;
+
+    int g0 = warp;
+    // fast path: U groups per warp per iteration, all loads issued before any use
+    for (; g0 + kWarps * (U - 1) < full; g0 += kWarps * U) {
+        float4 gv[U], zv[U], mv[U];
+        uint32_t mw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int grp = g0 + kWarps * u;
+            const int k = grp * kGroup + lane * 4;
+            gv[u] = ld_stream4(g + k);
+            zv[u] = ld_stream4(z + k);
+            if (M32) mv[u] = *reinterpret_cast<const float4*>(m32 + k);
+            else     mw[u] = mbits[grp * 4 + (lane >> 3)];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            worker_group<M32, false>(a, g, z, m32, mbits, obits, g0 + kWarps * u, lane, L, s_old, Sbar,
+                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc);
+    }
+    // remainder: one group at a time, bounds-checked
+    for (; g0 < ngroups; g0 += kWarps) {
+        const int k = g0 * kGroup + lane * 4;
+        const float4 gv = ld4_checked(g, k, L, true);
+        const float4 zv = ld4_checked(z, k, L, true);
+        float4 mv = make_float4(0, 0, 0, 0);
+        uint32_t mw = 0;
+        if (M32) mv = ld4_checked(m32, k, L, false);
+        else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
+        worker_group<M32, true>(a, g, z, m32, mbits, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
+    }
+
+    const double total = block_sum(acc, red);
+    if (threadIdx.x == 0) *sptr = (float)sqrt(total / (double)L);   // ||z||_2 / sqrt(L)
+}
+
+// ------------------------------------------------------------------------------------------
+// Server side: average the n decompressed messages, add the server error, recompress
+// (Section 3.3 step 4).  One CTA per chunk.
+
+struct ServerArgs {
+    const uint32_t* B; int64_t Wp;
+    const float* s; int64_t Cp;
+    float* zbar; uint32_t* Bbar; float* Sbar;
+    int64_t d; int64_t chunk;
+    int n; float nf;
+};
+
+template <bool CHECKED>
+__device__ __forceinline__ void server_group(const ServerArgs& a, const float* s_sh, const uint32_t* __restrict__ wb,
+                                             float* __restrict__ zb, uint32_t* __restrict__ ob,
+                                             int grp, int lane, int L, float S_old, double& acc)
+{
+    const int k = grp * kGroup + lane * 4;
+    const int wk = grp * 4 + (lane >> 3);
+    const int sh = 4 * (lane & 7);
+    float sum[4] = {0.f, 0.f, 0.f, 0.f};
+    const bool any = !CHECKED || (k < L);
+    if (any) {
+#pragma unroll 8
+        for (int i = 0; i < a.n; ++i) {
+            const uint32_t nib = wb[(int64_t)i * a.Wp + wk] >> sh;
+            const float si = s_sh[i];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sum[e] = __fadd_rn(sum[e], bit_scale((nib >> e) & 1u, si));
+        }
+    }
+    const float4 zo4 = CHECKED ? ld4_checked(zb, k, L, true) : ld_stream4(zb + k);
+    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+    float zn[4];
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float avg = __fdiv_rn(sum[e], a.nf);
+        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+        const bool valid = !CHECKED || (k + e < L);
+        if (valid) {
+            const double zd = (double)zn[e];
+            acc = fma(zd, zd, acc);
+            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+        }
+    }
+    const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
+    if (CHECKED) st4_checked(zb, k, L, out); else st_stream4(zb + k, out);
+    const uint32_t word = pack_group_words(nibble, lane);
+    if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) ob[wk] = word;
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+k_server(const ServerArgs a)
+{
+    __shared__ double red[kWarps];
+    __shared__ float s_sh[APMS_MAX_WORKERS];
+    const int64_t c = blockIdx.x;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
+    if (threadIdx.x < a.n) s_sh[threadIdx.x] = a.s[(int64_t)threadIdx.x * a.Cp + c];
+    const float S_old = a.Sbar[c];
+    __syncthreads();
+    const uint32_t* __restrict__ wb = a.B + base / 32;
+    float* __restrict__ zb = a.zbar + base;
+    uint32_t* __restrict__ ob = a.Bbar + base / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int full = L / kGroup;
+    const int ngroups = (L + kGroup - 1) / kGroup;
+    double acc = 0.0;
+    int g0 = warp;
+    for (; g0 < full; g0 += kWarps) server_group<false>(a, s_sh, wb, zb, ob, g0, lane, L, S_old, acc);
+    for (; g0 < ngroups; g0 += kWarps) server_group<true>(a, s_sh, wb, zb, ob, g0, lane, L, S_old, acc);
+    const double total = block_sum(acc, red);
+    if (threadIdx.x == 0) a.Sbar[c] = (float)sqrt(total / (double)L);
+}
+
+// ------------------------------------------------------------------------------------------
+// Worker side again: the received chunk replaces the momentum (it stays in its compressed
+// form) and the model moves with the frozen variance (Section 3.3 steps 5-6).
+
+struct ApplyArgs {
+    const uint32_t* Bbar; const float* Sbar; const float* v; float* x;
+    int64_t d; int64_t chunk; float lr, eps;
+};
+
+__device__ __forceinline__ float apply_elem(float x, float v, float q, float lr, float eps) {
+    return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+k_apply(const ApplyArgs a)
+{
+    const int64_t c = blockIdx.x;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
+    const float S = a.Sbar[c];
+    const uint32_t* __restrict__ bits = a.Bbar + base / 32;
+    const float* __restrict__ v = a.v + base;
+    float* __restrict__ x = a.x + base;
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const uint32_t nib = bits[k >> 5] >> (k & 31);
+        if (k + 3 < L) {
+            const float4 vv = ld_stream4(v + k);
+            float4 xx = ld_stream4(x + k);
+            xx.x = apply_elem(xx.x, vv.x, bit_scale(nib & 1u, S), a.lr, a.eps);
+            xx.y = apply_elem(xx.y, vv.y, bit_scale(nib & 2u, S), a.lr, a.eps);
+            xx.z = apply_elem(xx.z, vv.z, bit_scale(nib & 4u, S), a.lr, a.eps);
+            xx.w = apply_elem(xx.w, vv.w, bit_scale(nib & 8u, S), a.lr, a.eps);
+            st_stream4(x + k, xx);
+        } else {
+            for (int e = 0; e < 4 && k + e < L; ++e)
+                x[k + e] = apply_elem(x[k + e], v[k + e], bit_scale((nib >> e) & 1u, S), a.lr, a.eps);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// State materialisation (parity, checkpoints): delta = z - (+-scale), m = +-Sbar.
+
+__global__ void k_materialise_error(const float* __restrict__ z, const float* __restrict__ s,
+                                    float* __restrict__ out, int64_t first, int64_t count, int64_t chunk)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += (int64_t)gridDim.x * blockDim.x)
+        out[j] = implied_error(z[first + j], s[(first + j) / chunk]);
+}
+
+__global__ void k_materialise_momentum(const uint32_t* __restrict__ bits, const float* __restrict__ S,
+                                       float* __restrict__ out, int64_t first, int64_t count, int64_t chunk)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = first + j;
+        out[j] = bit_scale((bits[e >> 5] >> (e & 31)) & 1u, S[e / chunk]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    int64_t d, chunk, C, W, dz, Wp, Cp;
+    int n;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_stage, total;
+};
+
+bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
+{
+    if (d < 1 || n < 1 || n > APMS_MAX_WORKERS || chunk < 32 || chunk % 32 != 0) return false;
+    if (chunk > (int64_t)1 << 30) return false;
+    L->d = d; L->n = n; L->chunk = chunk;
+    L->C = (d + chunk - 1) / chunk;
+    L->W = (d + 31) / 32;
+    L->dz = (int64_t)round_up((size_t)d, 64);
+    L->Wp = (int64_t)round_up((size_t)L->W, 64);
+    L->Cp = (int64_t)round_up((size_t)L->C, 64);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o += round_up(bytes, 256); return at; };
+    L->off_x = take((size_t)L->dz * 4);
+    L->off_v = take((size_t)L->dz * 4);
+    L->off_m = take((size_t)L->dz * 4);
+    L->off_zbar = take((size_t)L->dz * 4);
+    L->off_z = take((size_t)L->dz * 4 * (size_t)n);
+    L->off_B = take((size_t)L->Wp * 4 * (size_t)n);
+    L->off_Bbar = take((size_t)L->Wp * 4);
+    L->off_s = take((size_t)L->Cp * 4 * (size_t)n);
+    L->off_Sbar = take((size_t)L->Cp * 4);
+    L->off_stage = take((size_t)L->dz * 4 * 2);
+    L->total = o;
+    return true;
+}
+
+thread_local char g_create_error[256] = "";
+
+struct EventPair { cudaEvent_t a, b; };
+
+}  // namespace
+
+struct apms_ctx {
+    Layout L;
+    float beta1, beta2, eps, lr;
+    int t;
+    apms_phase phase;
+    bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar)
+    char* ws; size_t ws_bytes; bool owns_ws;
+    cudaStream_t stream;
+    cudaStream_t copy_stream; cudaEvent_t ev_copied[2], ev_used[2]; bool host_path_ready;
+    int device;
+    int sms;
+    bool timing;
+    std::vector<EventPair> events[APMS_KERNEL_COUNT];
+    std::vector<EventPair> pool;
+    int64_t launches;
+    char err[512];
+
+    float* x() { return (float*)(ws + L.off_x); }
+    float* v() { return (float*)(ws + L.off_v); }
+    float* m() { return (float*)(ws + L.off_m); }
+    float* zbar() { return (float*)(ws + L.off_zbar); }
+    float* z(int i) { return (float*)(ws + L.off_z) + (int64_t)i * L.dz; }
+    uint32_t* B(int i) { return (uint32_t*)(ws + L.off_B) + (int64_t)i * L.Wp; }
+    uint32_t* Bbar() { return (uint32_t*)(ws + L.off_Bbar); }
+    float* s(int i) { return (float*)(ws + L.off_s) + (int64_t)i * L.Cp; }
+    float* Sbar() { return (float*)(ws + L.off_Sbar); }
+    float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
+};
+
+namespace {
+
+apms_status fail(apms_ctx* c, apms_status st, const char* fmt, const char* detail = "")
+{
+    if (c) snprintf(c->err, sizeof c->err, fmt, detail);
+    return st;
+}
+
+#define APMS_CUDA(c, call)                                                                   \
+    do {                                                                                     \
+        cudaError_t e__ = (call);                                                            \
+        if (e__ != cudaSuccess) {                                                            \
+            snprintf((c)->err, sizeof (c)->err, "%s failed: %s", #call, cudaGetErrorString(e__)); \
+            return APMS_ERR_CUDA;                                                            \
+        }                                                                                    \
+    } while (0)
+
+apms_status ensure_workspace(apms_ctx* c)
+{
+    if (c->ws) return APMS_OK;
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, c->L.total);
+    if (e != cudaSuccess) {
+        snprintf(c->err, sizeof c->err, "cudaMalloc of %zu workspace bytes failed: %s", c->L.total,
+                 cudaGetErrorString(e));
+        return e == cudaErrorMemoryAllocation ? APMS_ERR_OOM : APMS_ERR_CUDA;
+    }
+    c->ws = (char*)p; c->ws_bytes = c->L.total; c->owns_ws = true;
+    return APMS_OK;
+}
+
+// Event bracket around one kernel launch when timing is on.
+struct Timed {
+    apms_ctx* c; int k; EventPair ev; bool on;
+    Timed(apms_ctx* ctx, int kernel) : c(ctx), k(kernel), on(ctx->timing) {
+        if (!on) return;
+        if (!c->pool.empty()) { ev = c->pool.back(); c->pool.pop_back(); }
+        else if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) { on = false; return; }
+        cudaEventRecord(ev.a, c->stream);
+    }
+    ~Timed() {
+        if (!on) return;
+        cudaEventRecord(ev.b, c->stream);
+        c->events[k].push_back(ev);
+    }
+};
+
+apms_status check_grads(apms_ctx* c, const float* const* g, GradPtrs* out, int count)
+{
+    if (!g) return fail(c, APMS_ERR_INVALID_ARG, "gradient pointer array is NULL");
+    for (int i = 0; i < count; ++i) {
+        if (!g[i]) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is NULL");
+        if (((uintptr_t)g[i] & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is not 16-byte aligned");
+        out->p[i] = g[i];
+    }
+    return APMS_OK;
+}
+
+apms_status launch_check(apms_ctx* c, const char* what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        snprintf(c->err, sizeof c->err, "launch of %s failed: %s", what, cudaGetErrorString(e));
+        return APMS_ERR_CUDA;
+    }
+    c->launches += 1;
+    return APMS_OK;
+}
+
+apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
+{
+    WorkerArgs a;
+    a.z = c->z(0); a.dz = c->L.dz;
+    a.B = c->B(0); a.Wp = c->L.Wp;
+    a.s = c->s(0); a.Cp = c->L.Cp;
+    a.m32 = c->m(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.i0 = i0; a.ni = ni;
+    a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
+    const int64_t blocks = c->L.C * ni;
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
+    Timed t(c, APMS_KERNEL_WORKER);
+    if (c->m_is_fp32) k_worker<true, 4><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
+    else              k_worker<false, 4><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
+    return launch_check(c, "k_worker");
+}
+
+apms_status launch_server_and_apply(apms_ctx* c)
+{
+    {
+        ServerArgs a;
+        a.B = c->B(0); a.Wp = c->L.Wp; a.s = c->s(0); a.Cp = c->L.Cp;
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
+        a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n;
+        Timed t(c, APMS_KERNEL_SERVER);
+        k_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
+        apms_status st = launch_check(c, "k_server");
+        if (st != APMS_OK) return st;
+    }
+    {
+        ApplyArgs a;
+        a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
+        a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
+        Timed t(c, APMS_KERNEL_APPLY);
+        k_apply<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
+        apms_status st = launch_check(c, "k_apply");
+        if (st != APMS_OK) return st;
+    }
+    c->m_is_fp32 = false;      // from now on the momentum is the server's message
+    return APMS_OK;
+}
+
+int grid_for(const apms_ctx* c, int64_t items, int per_sm)
+{
+    int64_t blocks = (items + kThreads - 1) / kThreads;
+    const int64_t cap = (int64_t)c->sms * per_sm;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// C ABI
+
+extern "C" {
+
+size_t apms_workspace_bytes(int64_t d, int n, int64_t chunk)
+{
+    Layout L;
+    return make_layout(d, n, chunk, &L) ? L.total : 0;
+}
+
+apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float beta2, float eps,
+                        float lr, int64_t chunk)
+{
+    if (!out) { snprintf(g_create_error, sizeof g_create_error, "out is NULL"); return APMS_ERR_INVALID_ARG; }
+    *out = nullptr;
+    Layout L;
+    if (!make_layout(d, n, chunk, &L)) {
+        snprintf(g_create_error, sizeof g_create_error,
+                 "invalid shape: need d >= 1, 1 <= n <= %d, chunk a positive multiple of 32 (got d=%lld n=%d chunk=%lld)",
+                 APMS_MAX_WORKERS, (long long)d, n, (long long)chunk);
+        return APMS_ERR_INVALID_ARG;
+    }
+    if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) || !isfinite(lr)) {
+        snprintf(g_create_error, sizeof g_create_error, "invalid hyper-parameters: need 0 <= beta < 1, eps >= 0, finite lr");
+        return APMS_ERR_INVALID_ARG;
+    }
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) {
+        snprintf(g_create_error, sizeof g_create_error, "no usable CUDA device: %s", cudaGetErrorString(e));
+        return APMS_ERR_CUDA;
+    }
+    apms_ctx* c = new (std::nothrow) apms_ctx();
+    if (!c) { snprintf(g_create_error, sizeof g_create_error, "host allocation failed"); return APMS_ERR_OOM; }
+    c->L = L; c->beta1 = beta1; c->beta2 = beta2; c->eps = eps; c->lr = lr;
+    c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true;
+    c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
+    c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
+    c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
+    *out = c;
+    return APMS_OK;
+}
+
+apms_status apms_bind(apms_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "apms_bind must precede apms_set_params");
+    if (c->ws) return fail(c, APMS_ERR_BAD_STATE, "a workspace is already attached");
+    if (!workspace_dev || ((uintptr_t)workspace_dev & 255u)) return fail(c, APMS_ERR_INVALID_ARG, "workspace must be non-NULL and 256-byte aligned");
+    if (bytes < c->L.total) return fail(c, APMS_ERR_OOM, "workspace smaller than apms_workspace_bytes()");
+    c->ws = (char*)workspace_dev; c->ws_bytes = bytes; c->owns_ws = false;
+    c->stream = (cudaStream_t)cuda_stream;
+    return APMS_OK;
+}
+
+apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!x0) return fail(c, APMS_ERR_INVALID_ARG, "x0 is NULL");
+    apms_status st = ensure_workspace(c);
+    if (st != APMS_OK) return st;
+    const size_t bytes = (size_t)c->L.d * 4;
+    APMS_CUDA(c, cudaMemcpyAsync(c->x(), x0, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->m(), 0, (size_t)c->L.dz * 4, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
+    if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    c->t = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
+    return APMS_OK;
+}
+
+apms_status apms_set_lr(apms_ctx* c, float lr)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!isfinite(lr)) return fail(c, APMS_ERR_INVALID_ARG, "lr must be finite");
+    c->lr = lr;
+    return APMS_OK;
+}
+
+apms_status apms_warmup_step(apms_ctx* c, const float* const* grads_dev)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_WARMUP) return fail(c, APMS_ERR_BAD_STATE, "apms_warmup_step needs the WARMUP phase (after apms_set_params, before apms_freeze_v)");
+    GradPtrs G;
+    apms_status st = check_grads(c, grads_dev, &G, c->L.n);
+    if (st != APMS_OK) return st;
+    c->t += 1;
+    AdamArgs a;
+    a.x = c->x(); a.m = c->m(); a.v = c->v(); a.d = c->L.d; a.n = c->L.n;
+    a.beta1 = c->beta1; a.beta2 = c->beta2; a.omb1 = 1.0f - c->beta1; a.omb2 = 1.0f - c->beta2;
+    a.bc1 = (float)(1.0 - pow((double)c->beta1, (double)c->t));
+    a.bc2 = (float)(1.0 - pow((double)c->beta2, (double)c->t));
+    a.lr = c->lr; a.eps = c->eps; a.nf = (float)c->L.n;
+    Timed t(c, APMS_KERNEL_WARMUP_ADAM);
+    k_warmup_adam<<<grid_for(c, (c->L.d + 3) / 4, 8), kThreads, 0, c->stream>>>(G, a);
+    return launch_check(c, "k_warmup_adam");
+}
+
+apms_status apms_freeze_v(apms_ctx* c)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_WARMUP) return fail(c, APMS_ERR_BAD_STATE, "apms_freeze_v needs the WARMUP phase");
+    // errors start at zero: z = 0 with scale 0 implies delta = 0 - (+0) = 0
+    APMS_CUDA(c, cudaMemsetAsync(c->ws + c->L.off_zbar, 0, c->L.off_stage - c->L.off_zbar, c->stream));
+    c->phase = APMS_PHASE_COMPRESSED;
+    c->m_is_fp32 = true;
+    return APMS_OK;
+}
+
+apms_status apms_compressed_step(apms_ctx* c, const float* const* grads_dev)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step needs the COMPRESSED phase (call apms_freeze_v first)");
+    GradPtrs G;
+    apms_status st = check_grads(c, grads_dev, &G, c->L.n);
+    if (st != APMS_OK) return st;
+    st = launch_worker(c, G, 0, c->L.n);
+    if (st != APMS_OK) return st;
+    return launch_server_and_apply(c);
+}
+
+apms_status apms_compressed_step_host(apms_ctx* c, const float* const* grads_host, float* x_out_host)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step_host needs the COMPRESSED phase (call apms_freeze_v first)");
+    if (!grads_host) return fail(c, APMS_ERR_INVALID_ARG, "gradient pointer array is NULL");
+    for (int i = 0; i < c->L.n; ++i)
+        if (!grads_host[i]) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is NULL");
+    if (!c->host_path_ready) {
+        APMS_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            APMS_CUDA(c, cudaEventCreateWithFlags(&c->ev_copied[b], cudaEventDisableTiming));
+            APMS_CUDA(c, cudaEventCreateWithFlags(&c->ev_used[b], cudaEventDisableTiming));
+        }
+        c->host_path_ready = true;
+    }
+    const size_t bytes = (size_t)c->L.d * 4;
+    // the staging buffers may still be read by work queued earlier on the compute stream
+    APMS_CUDA(c, cudaEventRecord(c->ev_used[0], c->stream));
+    APMS_CUDA(c, cudaEventRecord(c->ev_used[1], c->stream));
+    for (int i = 0; i < c->L.n; ++i) {
+        const int b = i & 1;
+        APMS_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_used[b], 0));
+        APMS_CUDA(c, cudaMemcpyAsync(c->stage(b), grads_host[i], bytes, cudaMemcpyHostToDevice, c->copy_stream));
+        APMS_CUDA(c, cudaEventRecord(c->ev_copied[b], c->copy_stream));
+        APMS_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
+        GradPtrs G;
+        G.p[0] = c->stage(b);
+        apms_status st = launch_worker(c, G, i, 1);
+        if (st != APMS_OK) return st;
+        APMS_CUDA(c, cudaEventRecord(c->ev_used[b], c->stream));
+    }
+    apms_status st = launch_server_and_apply(c);
+    if (st != APMS_OK) return st;
+    if (x_out_host) APMS_CUDA(c, cudaMemcpyAsync(x_out_host, c->x(), bytes, cudaMemcpyDeviceToHost, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    return APMS_OK;
+}
+
+apms_status apms_get_params(apms_ctx* c, float* dst, int dst_is_device)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!dst) return fail(c, APMS_ERR_INVALID_ARG, "dst is NULL");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "no parameters set yet");
+    APMS_CUDA(c, cudaMemcpyAsync(dst, c->x(), (size_t)c->L.d * 4, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream));
+    if (!dst_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    return APMS_OK;
+}
+
+apms_status apms_get_state_slice(apms_ctx* c, apms_state_id which, int worker, int64_t first,
+                                 int64_t count, void* dst)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!dst) return fail(c, APMS_ERR_INVALID_ARG, "dst is NULL");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "no state yet");
+    const bool per_worker = which == APMS_STATE_WORKER_ERR || which == APMS_STATE_WORKER_BITS || which == APMS_STATE_WORKER_SCALES;
+    if (per_worker && (worker < 0 || worker >= c->L.n)) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range");
+    int64_t extent = c->L.d;
+    if (which == APMS_STATE_WORKER_BITS || which == APMS_STATE_SERVER_BITS) extent = c->L.W;
+    if (which == APMS_STATE_WORKER_SCALES || which == APMS_STATE_SERVER_SCALES) extent = c->L.C;
+    if (first < 0 || count < 0 || first > extent || count > extent - first) return fail(c, APMS_ERR_INVALID_ARG, "slice out of range");
+    if (count == 0) return APMS_OK;
+    const char* src = nullptr;
+    const int grid = grid_for(c, count, 8);
+    bool staged = false;
+    switch (which) {
+    case APMS_STATE_X: src = (const char*)c->x(); break;
+    case APMS_STATE_V: src = (const char*)c->v(); break;
+    case APMS_STATE_M:
+        if (c->m_is_fp32) src = (const char*)c->m();
+        else {
+            k_materialise_momentum<<<grid, kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->stage(0), first, count, c->L.chunk);
+            staged = true;
+        }
+        break;
+    case APMS_STATE_WORKER_ERR:
+        k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->z(worker), c->s(worker), c->stage(0), first, count, c->L.chunk);
+        staged = true;
+        break;
+    case APMS_STATE_SERVER_ERR:
+        k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->zbar(), c->Sbar(), c->stage(0), first, count, c->L.chunk);
+        staged = true;
+        break;
+    case APMS_STATE_WORKER_BITS: src = (const char*)c->B(worker); break;
+    case APMS_STATE_SERVER_BITS: src = (const char*)c->Bbar(); break;
+    case APMS_STATE_WORKER_SCALES: src = (const char*)c->s(worker); break;
+    case APMS_STATE_SERVER_SCALES: src = (const char*)c->Sbar(); break;
+    default: return fail(c, APMS_ERR_INVALID_ARG, "unknown state id");
+    }
+    APMS_CUDA(c, cudaGetLastError());
+    const char* from = staged ? (const char*)c->stage(0) : src + (size_t)first * 4;
+    APMS_CUDA(c, cudaMemcpyAsync(dst, from, (size_t)count * 4, cudaMemcpyDeviceToHost, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    return APMS_OK;
+}
+
+apms_status apms_get_state(apms_ctx* c, apms_state_id which, int worker, void* dst)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    int64_t extent = c->L.d;
+    if (which == APMS_STATE_WORKER_BITS || which == APMS_STATE_SERVER_BITS) extent = c->L.W;
+    if (which == APMS_STATE_WORKER_SCALES || which == APMS_STATE_SERVER_SCALES) extent = c->L.C;
+    return apms_get_state_slice(c, which, worker, 0, extent, dst);
+}
+
+apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const void* src)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!src) return fail(c, APMS_ERR_INVALID_ARG, "src is NULL");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    const size_t bytes = (size_t)c->L.d * 4;
+    float* dst = nullptr;
+    switch (which) {
+    case APMS_STATE_X: dst = c->x(); break;
+    case APMS_STATE_V: dst = c->v(); break;
+    case APMS_STATE_M: dst = c->m(); c->m_is_fp32 = true; break;
+    case APMS_STATE_WORKER_ERR:
+        if (worker < 0 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range");
+        if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
+        // delta = z - (+-0) = z: store the error as z with all scales of this worker zero
+        APMS_CUDA(c, cudaMemsetAsync(c->s(worker), 0, (size_t)c->L.Cp * 4, c->stream));
+        dst = c->z(worker);
+        break;
+    case APMS_STATE_SERVER_ERR:
+        if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
+        if (!c->m_is_fp32) {   // Sbar is about to be zeroed: move the momentum it encodes to binary32 first
+            k_materialise_momentum<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->m(), 0, c->L.d, c->L.chunk);
+            APMS_CUDA(c, cudaGetLastError());
+            c->m_is_fp32 = true;
+        }
+        APMS_CUDA(c, cudaMemsetAsync(c->Sbar(), 0, (size_t)c->L.Cp * 4, c->stream));
+        dst = c->zbar();
+        break;
+    default: return fail(c, APMS_ERR_INVALID_ARG, "this state array cannot be set");
+    }
+    APMS_CUDA(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    return APMS_OK;
+}
+
+apms_status apms_restore(apms_ctx* c, int t, apms_phase phase)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    if (t < 0 || (phase != APMS_PHASE_WARMUP && phase != APMS_PHASE_COMPRESSED)) return fail(c, APMS_ERR_INVALID_ARG, "invalid t or phase");
+    if (phase == APMS_PHASE_COMPRESSED && c->phase == APMS_PHASE_WARMUP) {
+        apms_status st = apms_freeze_v(c);
+        if (st != APMS_OK) return st;
+    }
+    c->t = t; c->phase = phase;
+    return APMS_OK;
+}
+
+apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }
+int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
+
+apms_status apms_set_timing(apms_ctx* c, int enabled)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    c->timing = enabled != 0;
+    return APMS_OK;
+}
+
+apms_status apms_kernel_time(apms_ctx* c, apms_kernel_id which, double* total_ms, int64_t* launches)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if ((int)which < 0 || which >= APMS_KERNEL_COUNT) return fail(c, APMS_ERR_INVALID_ARG, "unknown kernel id");
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    double sum = 0.0;
+    for (EventPair& ev : c->events[which]) {
+        float ms = 0.f;
+        APMS_CUDA(c, cudaEventElapsedTime(&ms, ev.a, ev.b));
+        sum += ms;
+        c->pool.push_back(ev);
+    }
+    if (total_ms) *total_ms = sum;
+    if (launches) *launches = (int64_t)c->events[which].size();
+    c->events[which].clear();
+    return APMS_OK;
+}
+
+int64_t apms_launch_count(const apms_ctx* c) { return c ? c->launches : 0; }
+
+const char* apms_last_error(const apms_ctx* c) { return c ? c->err : g_create_error; }
+
+void apms_destroy(apms_ctx* c)
+{
+    if (!c) return;
+    if (c->stream || c->ws) cudaStreamSynchronize(c->stream);
+    for (int k = 0; k < APMS_KERNEL_COUNT; ++k)
+        for (EventPair& ev : c->events[k]) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }
+    for (EventPair& ev : c->pool) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }
+    if (c->host_path_ready) {
+        for (int b = 0; b < 2; ++b) { cudaEventDestroy(c->ev_copied[b]); cudaEventDestroy(c->ev_used[b]); }
+        cudaStreamDestroy(c->copy_stream);
+    }
+    if (c->owns_ws && c->ws) cudaFree(c->ws);
+    delete c;
+}
+
+}  // extern "C"

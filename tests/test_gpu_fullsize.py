@@ -1,0 +1,115 @@
+"""Parity at the benchmark's full size, in the launch configuration the benchmark times:
+BERT-Large-shaped parameter set, n = 16 workers, chunk = 32768, device-resident gradients.
+
+The oracle cannot run 335M x 16 elements in a test, but chunks are independent problems
+(Supplement A: the algorithm equals a parameter-server step per chunk), so a sample of chunks -
+the first, the ragged last one and random ones - is cut out of the device state before a step,
+replayed by the oracle as a small problem, and compared with the device state after the step."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+import gpu_harness as H
+from oracle import apms_oracle as ao
+from paper_2008_11343_b200 import binding as B
+from paper_2008_11343_b200 import workloads as wl
+
+
+def _slices(w, chunks):
+    return [(c * w.chunk, min(w.d, (c + 1) * w.chunk) - c * w.chunk) for c in chunks]
+
+
+def _gather(ctx, which, sl, worker=0):
+    return np.concatenate([ctx.get_state_slice(which, lo, cnt, worker=worker) for lo, cnt in sl])
+
+
+def _gather_words(ctx, which, sl, worker=0):
+    return np.concatenate([ctx.get_state_slice(which, lo // 32, (cnt + 31) // 32, worker=worker) for lo, cnt in sl])
+
+
+@pytest.mark.parametrize("cfg,samples", [(3, 10), (2, 6)])
+def test_sampled_chunks_at_full_size(cfg, samples):
+    import torch
+
+    w = wl.config(cfg)
+    free, _ = torch.cuda.mem_get_info()
+    need = B.apms_workspace_bytes(w.d, w.n, w.chunk) + 4 * w.d * w.n + (2 << 30)
+    if free < need:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory, {free / 2**30:.0f} GiB free")
+    chunks = list(wl.sample_chunks(w, samples))
+    assert chunks[-1] == w.n_chunks - 1                      # the ragged chunk is part of the sample
+    sl = _slices(w, chunks)
+    dsub = sum(cnt for _, cnt in sl)
+
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    x0 = torch.empty(w.d, dtype=torch.float32, device="cuda").normal_(0.0, w.x0_std)
+    ctx.set_params(x0)
+    grads = [torch.empty(w.d, dtype=torch.float32, device="cuda") for _ in range(w.n)]
+
+    def draw(step):
+        for i in range(w.n):
+            wl.device_gradient(w, step, i, grads[i])
+        return [np.concatenate([g[lo:lo + cnt].cpu().numpy() for lo, cnt in sl]) for g in grads]
+
+    orc = ao.Oracle(dsub, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    orc.set_threads(orc.max_threads())
+    orc.set_params(_gather(ctx, B.STATE_X, sl))
+    sub = wl.Workload("sample", 0, n=w.n, chunk=w.chunk, tensor_sizes=(dsub,), dist=w.dist,
+                      scale_lo=1, scale_hi=1, lr=w.lr, eps=w.eps)
+
+    # warmup steps: element-wise, so the sampled elements can simply be replayed
+    for step in range(2):
+        gsub = draw(step)
+        ctx.warmup_step(grads)
+        orc.warmup_step(gsub)
+    for which, ref in ((B.STATE_X, orc.x), (B.STATE_M, orc.m), (B.STATE_V, orc.v)):
+        got = _gather(ctx, which, sl)
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), f"warmup state {which}"
+    ctx.freeze_v()
+    orc.freeze_v()
+
+    mismatched_scales = 0
+    for step in range(2, 5):
+        # teacher-force the oracle from the device state of the sampled chunks
+        orc.x[:] = _gather(ctx, B.STATE_X, sl)
+        orc.m[:] = _gather(ctx, B.STATE_M, sl)
+        orc.server_err[:] = _gather(ctx, B.STATE_SERVER_ERR, sl)
+        for i in range(w.n):
+            orc.worker_err(i)[:] = _gather(ctx, B.STATE_WORKER_ERR, sl, worker=i)
+        gsub = draw(step)
+        ctx.compressed_step(grads)
+        orc.compressed_step(gsub)
+        # sign words: bit-exact
+        assert np.array_equal(_gather_words(ctx, B.STATE_SERVER_BITS, sl), orc.server_bits)
+        for i in range(w.n):
+            assert np.array_equal(_gather_words(ctx, B.STATE_WORKER_BITS, sl, worker=i), orc.worker_bits(i)), \
+                f"step {step}: worker {i} sign words differ"
+        # scales
+        idx = np.asarray(chunks)
+        Sg = np.array([ctx.get_state_slice(B.STATE_SERVER_SCALES, int(c), 1)[0] for c in idx])
+        np.testing.assert_allclose(Sg, orc.server_scales, rtol=H.REL)
+        mismatched_scales += int((Sg != orc.server_scales).sum())
+        cidx = H.chunk_of(w.chunk, dsub)
+        for i in range(w.n):
+            sg = np.array([ctx.get_state_slice(B.STATE_WORKER_SCALES, int(c), 1, worker=i)[0] for c in idx])
+            np.testing.assert_allclose(sg, orc.worker_scales(i), rtol=H.REL)
+            mismatched_scales += int((sg != orc.worker_scales(i)).sum())
+            e_ref = orc.worker_err(i)
+            tol = H.REL * np.maximum(np.abs(e_ref), orc.worker_scales(i)[cidx])
+            assert (np.abs(_gather(ctx, B.STATE_WORKER_ERR, sl, worker=i) - e_ref) <= tol).all()
+        e_ref = orc.server_err
+        tol = H.REL * np.maximum(np.abs(e_ref), orc.server_scales[cidx])
+        assert (np.abs(_gather(ctx, B.STATE_SERVER_ERR, sl) - e_ref) <= tol).all()
+        np.testing.assert_allclose(_gather(ctx, B.STATE_M, sl), orc.m, rtol=H.REL)
+        stepsize = w.lr * orc.server_scales[cidx] / (np.sqrt(orc.v.astype(np.float64)) + w.eps)
+        assert (np.abs(_gather(ctx, B.STATE_X, sl) - orc.x) <= H.REL * (np.abs(orc.x) + stepsize)).all()
+    # the binary64 sums make a differently rounded scale a rare event, not the rule
+    assert mismatched_scales <= 2
+
+    # properties that hold at any size, on the whole vector: payload and padding
+    W = (w.d + 31) // 32
+    last = ctx.get_state_slice(B.STATE_SERVER_BITS, W - 1, 1)[0]
+    if w.d % 32:
+        assert int(last) >> (w.d % 32) == 0
+    assert np.isfinite(ctx.get_state_slice(B.STATE_SERVER_SCALES, 0, w.n_chunks)).all()

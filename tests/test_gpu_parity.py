@@ -1,0 +1,269 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+import gpu_harness as H
+from oracle import apms_oracle as ao
+from paper_2008_11343_b200 import binding as B
+from paper_2008_11343_b200 import workloads as wl
+
+
+def tiny(d, n, chunk, cfg_id=100, **kw):
+    return wl.Workload(f"tiny-{d}-{n}-{chunk}", cfg_id, n=n, chunk=chunk, tensor_sizes=(d,), dist="gauss",
+                       scale_lo=1e-3, scale_hi=1e-1, **kw)
+
+
+# ------------------------------------------------------------------ edge sizes, bit-identical
+
+EDGE = [(1, 1, 32), (31, 2, 32), (32, 2, 32), (33, 3, 32), (127, 4, 128), (128, 4, 128), (129, 4, 128),
+        (4095, 2, 4096), (4096, 2, 4096), (4097, 2, 4096), (1000, 5, 96), (12345, 3, 1024),
+        (5 * 8192 + 77, 2, 8192), (3 * 65536 + 1, 2, 65536), (70000, 16, 160), (2050, 64, 2048)]
+
+
+@pytest.mark.parametrize("d,n,chunk", EDGE)
+def test_free_running_edge_sizes_bit_identical(d, n, chunk):
+    """Ragged tails, d below / at / above a word, a vector and a chunk; several tiles.  On these
+    sizes every scale is expected to round identically on both sides, so the whole state must be
+    bit-identical (the binary64 sums differ only in the order of additions)."""
+    w = tiny(d, n, chunk, warmup_steps=3, compressed_steps=4)
+    H.run_both(w, exact=True)
+
+
+def test_teacher_forced_steps_bits_exact():
+    """The oracle's state is uploaded before every step; after the step the packed sign words
+    must equal the oracle's exactly and every value must be bit-identical."""
+    w = tiny(6 * 1024 + 333, 4, 1024, cfg_id=101, lr=1e-3)
+    ctx, orc = H.make_pair(w)
+    for step in range(2):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs))
+        orc.warmup_step(gs)
+    ctx.freeze_v()
+    orc.freeze_v()
+    rng = np.random.default_rng(3)
+    for step in range(2, 7):
+        # disturb the oracle's state so that each step starts from a state the CUDA side never produced
+        orc.server_err[:] += (rng.standard_normal(w.d) * 1e-4).astype(np.float32)
+        for i in range(w.n):
+            orc.worker_err(i)[:] += (rng.standard_normal(w.d) * 1e-4).astype(np.float32)
+        orc.m[:] = (rng.standard_normal(w.d) * 1e-3).astype(np.float32)
+        H.teacher_force(ctx, orc, w)
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs))
+        orc.compressed_step(gs)
+        H.compare_state(ctx, orc, w, exact=True)
+
+
+# ------------------------------------------------------------------ the benchmark's small configurations
+
+def test_config0_free_running_10_steps():
+    """d = 2^20, n = 4, chunk = 4096: 5 warmup + 10 compressed steps, free-running.  Sign words
+    bit-exact (ties aside), scales / errors / parameters within 1e-5 after 10 steps."""
+    w = wl.config(0)
+    _, _, reports = H.run_both(w, check_every_step=False)
+    assert reports[-1]["server_tie_elems"] == 0
+
+
+def test_config1_mixed_tensors_zero_gradients():
+    """d = 2^24 in 64 tensors with per-tensor scales over three decades and 20 % zero gradient
+    entries, n = 8, chunk = 8192 (steps reduced to keep the oracle's share of the run short)."""
+    w = wl.config(1)
+    H.run_both(w, warmup=3, compressed=5, check_every_step=False)
+
+
+def test_structural_zero_gradients_stay_finite():
+    """Elements whose gradient is always zero have v = 0; the update divides by eps alone and must
+    stay finite and equal to the oracle's."""
+    w = tiny(4096 + 40, 2, 1024, cfg_id=102, eps=1e-8)
+    mask = np.ones(w.d, dtype=np.float32)
+    mask[::7] = 0.0
+
+    def grads(step):
+        return [g * mask for g in wl.host_gradients(w, step)]
+
+    ctx, orc, _ = H.run_both(w, warmup=2, compressed=3, exact=True, grads_fn=grads)
+    assert np.isfinite(ctx.get_params()).all()
+
+
+def test_all_zero_chunk_and_constant_magnitude():
+    """Degenerate chunks: an all-zero chunk gives scale 0, all bits 1 and zero error; a chunk whose
+    compensated entries all have one magnitude compresses without error."""
+    d, n, chunk = 256, 2, 64
+    w = tiny(d, n, chunk, cfg_id=103)
+    ctx, orc = H.make_pair(w, x0=np.zeros(d, np.float32))
+    ctx.freeze_v()
+    orc.freeze_v()
+    g = np.zeros(d, np.float32)
+    g[64:128] = 0.5 * np.where(np.arange(64) % 3 == 0, -1.0, 1.0)
+    g[128:192] = np.linspace(-1, 1, 64, dtype=np.float32)
+    ctx.compressed_step(H.upload([g, g]))
+    orc.compressed_step([g, g])
+    H.compare_state(ctx, orc, w, exact=True)
+    s0 = ctx.get_state(B.STATE_WORKER_SCALES, 0)
+    bits = ctx.get_state(B.STATE_WORKER_BITS, 0)
+    err = ctx.get_state(B.STATE_WORKER_ERR, 0)
+    assert s0[0] == 0.0 and bits[0] == 0xFFFFFFFF and bits[1] == 0xFFFFFFFF and not err[:64].any()
+    assert not err[64:128].any()                      # constant magnitude: C[z] = z
+
+
+def test_nonfinite_gradient_propagates_like_the_oracle():
+    w = tiny(300, 2, 64, cfg_id=104)
+    ctx, orc = H.make_pair(w)
+    ctx.freeze_v()
+    orc.freeze_v()
+    gs = wl.host_gradients(w, 0)
+    gs[1][17] = np.nan
+    ctx.compressed_step(H.upload(gs))
+    orc.compressed_step(gs)
+    for i in range(2):
+        assert np.array_equal(ctx.get_state(B.STATE_WORKER_BITS, i), orc.worker_bits(i))
+        a, b = ctx.get_state(B.STATE_WORKER_SCALES, i), orc.worker_scales(i)
+        assert np.array_equal(np.isnan(a), np.isnan(b)) and np.array_equal(a[~np.isnan(a)], b[~np.isnan(b)])
+
+
+# ------------------------------------------------------------------ properties of the CUDA path alone
+
+def test_run_twice_is_bitwise_deterministic():
+    w = tiny(9 * 4096 + 5, 4, 4096, cfg_id=105)
+
+    def run():
+        ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        ctx.set_params(wl.initial_params(w))
+        for s in range(2):
+            ctx.warmup_step(H.upload(wl.host_gradients(w, s)))
+        ctx.freeze_v()
+        for s in range(2, 6):
+            ctx.compressed_step(H.upload(wl.host_gradients(w, s)))
+        return [ctx.get_state(k, i) for k in range(9) for i in (range(w.n) if k in (3, 4, 5) else [0])]
+
+    for a, b in zip(run(), run()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_host_gradient_entry_point_matches_device_entry_point():
+    import torch
+
+    w = tiny(5 * 2048 + 100, 3, 2048, cfg_id=106)
+    outs = []
+    for host in (False, True):
+        ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        ctx.set_params(wl.initial_params(w))
+        ctx.warmup_step(H.upload(wl.host_gradients(w, 0)))
+        ctx.freeze_v()
+        x_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        for s in range(1, 4):
+            gs = wl.host_gradients(w, s)
+            if host:
+                pinned = [torch.from_numpy(g).pin_memory() for g in gs]
+                ctx.compressed_step_host(pinned, x_host)
+                assert np.array_equal(x_host.numpy(), ctx.get_params())
+            else:
+                ctx.compressed_step(H.upload(gs))
+        outs.append([ctx.get_state(k, i) for k in range(9) for i in (range(w.n) if k in (3, 4, 5) else [0])])
+    for a, b in zip(*outs):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_checkpoint_restore_continues_bit_identically():
+    w = tiny(3 * 1024 + 17, 2, 1024, cfg_id=107)
+    a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    a.set_params(wl.initial_params(w))
+    a.warmup_step(H.upload(wl.host_gradients(w, 0)))
+    a.freeze_v()
+    for s in range(1, 4):
+        a.compressed_step(H.upload(wl.host_gradients(w, s)))
+    saved = {k: a.get_state(k) for k in (B.STATE_X, B.STATE_V, B.STATE_M, B.STATE_SERVER_ERR)}
+    werr = [a.get_state(B.STATE_WORKER_ERR, i) for i in range(w.n)]
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b.set_params(np.zeros(w.d, np.float32))
+    b.restore(a.t, B.PHASE_COMPRESSED)
+    for k, val in saved.items():
+        b.set_state(k, val)
+    for i in range(w.n):
+        b.set_state(B.STATE_WORKER_ERR, werr[i], worker=i)
+    for s in range(4, 7):
+        gs = H.upload(wl.host_gradients(w, s))
+        a.compressed_step(gs)
+        b.compressed_step(gs)
+    for k in (B.STATE_X, B.STATE_M, B.STATE_SERVER_ERR, B.STATE_SERVER_BITS, B.STATE_SERVER_SCALES):
+        assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32))
+    for i in range(w.n):
+        assert np.array_equal(a.get_state(B.STATE_WORKER_ERR, i), b.get_state(B.STATE_WORKER_ERR, i))
+
+
+def test_state_slices_agree_with_full_arrays():
+    w = tiny(4 * 512 + 9, 2, 512, cfg_id=108)
+    ctx, _, _ = H.run_both(w, warmup=1, compressed=2, check_every_step=False)
+    for which in range(9):
+        full = ctx.get_state(which, 1)
+        lo, cnt = (3, 5) if full.size < 100 else (500, 777)
+        lo, cnt = min(lo, full.size - 1), min(cnt, full.size - min(lo, full.size - 1))
+        part = ctx.get_state_slice(which, lo, cnt, worker=1)
+        assert np.array_equal(part.view(np.uint32), full[lo:lo + cnt].view(np.uint32))
+
+
+# ------------------------------------------------------------------ boundary behaviour (error codes, no faults)
+
+def test_phase_and_argument_errors_are_status_codes():
+    import torch
+
+    w = tiny(100, 2, 32, cfg_id=109)
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    g = [torch.zeros(w.d, device="cuda") for _ in range(2)]
+    with pytest.raises(B.ApmsError) as e:
+        ctx.warmup_step(g)                      # no parameters yet
+    assert e.value.status == B.ERR_BAD_STATE
+    ctx.set_params(np.zeros(w.d, np.float32))
+    with pytest.raises(B.ApmsError) as e:
+        ctx.compressed_step(g)                  # before the phase switch
+    assert e.value.status == B.ERR_BAD_STATE
+    with pytest.raises(B.ApmsError) as e:
+        B.apms_warmup_step(ctx._h, [g[0].data_ptr(), 0])
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.ApmsError) as e:
+        B.apms_warmup_step(ctx._h, [g[0].data_ptr(), g[1].data_ptr() + 4])     # misaligned
+    assert e.value.status == B.ERR_INVALID_ARG
+    ctx.warmup_step(g)
+    ctx.freeze_v()
+    with pytest.raises(B.ApmsError) as e:
+        ctx.warmup_step(g)                      # after the phase switch
+    assert e.value.status == B.ERR_BAD_STATE
+    with pytest.raises(B.ApmsError) as e:
+        ctx.freeze_v()
+    assert e.value.status == B.ERR_BAD_STATE
+    with pytest.raises(B.ApmsError) as e:
+        ctx.get_state(B.STATE_WORKER_ERR, 5)
+    assert e.value.status == B.ERR_INVALID_ARG
+    for bad in [(0, 1, 32), (10, 0, 32), (10, 65, 32), (10, 1, 48), (10, 1, 0)]:
+        with pytest.raises(B.ApmsError):
+            B.apms_create(bad[0], bad[1], 0.9, 0.999, 1e-8, 1e-3, bad[2])
+        assert B.apms_workspace_bytes(*bad) == 0
+    ctx.compressed_step(g)                      # the context is still usable after all of the above
+    assert ctx.launch_count == 1 + 3
+
+
+def test_library_owned_workspace_and_default_stream():
+    """apms_create without apms_bind: the library allocates its own workspace."""
+    import torch
+
+    w = tiny(1000, 2, 128, cfg_id=110)
+    h = B.apms_create(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    x0 = wl.initial_params(w)
+    B.apms_set_params(h, x0.ctypes.data, False)
+    orc = ao.Oracle(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    orc.set_params(x0)
+    gs = wl.host_gradients(w, 0)
+    dev = H.upload(gs)
+    torch.cuda.synchronize()
+    B.apms_warmup_step(h, [t.data_ptr() for t in dev])
+    orc.warmup_step(gs)
+    B.apms_freeze_v(h)
+    orc.freeze_v()
+    B.apms_compressed_step(h, [t.data_ptr() for t in dev])
+    orc.compressed_step(gs)
+    out = np.empty(w.d, np.float32)
+    B.apms_get_params(h, out.ctypes.data, False)
+    assert np.array_equal(out, orc.x)
+    B.apms_destroy(h)

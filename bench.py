@@ -67,7 +67,7 @@ class ClockSampler:
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
 
-    def __init__(self, index: int, period_s: float = 0.05):
+    def __init__(self, index: int, period_s: float = 0.02):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -178,6 +178,110 @@ def time_oracle(w, steps: int, warmup: int, budget_s: float = 20.0) -> dict:
             "ms_per_step": per_step * 1e3, "steps": len(times)}
 
 
+# ------------------------------------------------------------------------------------------ GPU leg
+
+def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=True) -> dict:
+    """Set up one workload on this rank's GPU and time K compressed steps (device-resident
+    gradients, CUDA events on the context's stream), optionally the Adam step and the e2e path."""
+    import torch
+
+    from paper_2008_11343_b200 import binding as B
+    from paper_2008_11343_b200 import workloads as wl
+
+    dev = torch.device("cuda", local_rank)
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}")
+    x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)
+    ctx.set_params(x0)
+    del x0
+    ring = []
+    for r in range(2):
+        gs = [torch.empty(w.d, dtype=torch.float32, device=dev) for _ in range(w.n)]
+        for i in range(w.n):
+            wl.device_gradient(w, r + 1000 * rank, i, gs[i])
+        ring.append(gs)
+    torch.cuda.synchronize()
+    group = dist if world > 1 else None
+
+    # warmup phase (timed alone when asked), phase switch, first compressed step
+    adam = None
+    for k in range(3):
+        ctx.warmup_step(ring[k % 2])
+    if want_adam:
+        ctx.set_timing(True)
+        for k in range(10):
+            ctx.warmup_step(ring[k % 2])
+        ms, cnt = ctx.kernel_time(B.KERNEL_WARMUP_ADAM)
+        ctx.set_timing(False)
+        ab = algorithmic_bytes(w.d, w.n, w.chunk)["warmup_adam"]
+        adam = {"ms_per_step": ms / cnt, "achieved_gbs": ab / (ms / cnt * 1e-3) / 1e9,
+                "worker_elements_per_s": w.d * w.n / (ms / cnt * 1e-3)}
+    ctx.freeze_v()
+    ctx.compressed_step(ring[0])             # reads the binary32 momentum once; not representative
+    for k in range(args.warmup):
+        ctx.compressed_step(ring[(k + 1) % 2])
+    torch.cuda.synchronize()
+
+    # timed region: K steps between two events on the context's stream
+    ctx.set_timing(True)
+    for kid in range(len(B.KERNEL_NAMES)):
+        ctx.kernel_time(kid)
+    launches0 = ctx.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local_rank) as clocks:
+        e0.record(ctx.stream)
+        for k in range(args.steps):
+            ctx.compressed_step(ring[k % 2])
+        e1.record(ctx.stream)
+        torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    seconds = max_over_ranks(e0.elapsed_time(e1) * 1e-3, group)
+    launches = ctx.launch_count - launches0
+    kernel_ms = {}
+    for kid, name in enumerate(B.KERNEL_NAMES):
+        ms, cnt = ctx.kernel_time(kid)
+        if cnt:
+            kernel_ms[name] = ms / cnt
+    ctx.set_timing(False)
+    out = {"ms_per_step": seconds * 1e3 / args.steps, "value": world * w.d * w.n * args.steps / seconds,
+           "kernel_ms": kernel_ms, "launches": launches, "clocks": clocks.summary(), "adam": adam, "e2e": None}
+
+    # end to end through the host-gradient entry point: H2D of the n gradients and D2H of x
+    # inside the timed region, every step
+    if want_e2e:
+        try:
+            host = [torch.empty(w.d, dtype=torch.float32).pin_memory() for _ in range(w.n)]
+            for i in range(w.n):
+                host[i].copy_(ring[0][i])
+            x_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
+            torch.cuda.synchronize()
+            ctx.compressed_step_host(host, x_host)
+            if world > 1:
+                dist.barrier()
+            t0 = time.perf_counter()
+            e0.record(ctx.stream)
+            for _ in range(args.e2e_steps):
+                ctx.compressed_step_host(host, x_host)
+            e1.record(ctx.stream)
+            torch.cuda.synchronize()
+            wall = time.perf_counter() - t0
+            secs = max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, wall), group)
+            out["e2e"] = {"value": world * w.d * w.n * args.e2e_steps / secs, "unit": UNIT,
+                          "h2d_bytes_per_step": 4 * w.d * w.n, "d2h_bytes_per_step": 4 * w.d,
+                          "ms_per_step": secs * 1e3 / args.e2e_steps, "steps": args.e2e_steps,
+                          "api": "apms_compressed_step_host (pinned host gradients in, x out)"}
+            del host, x_host
+        except RuntimeError as exc:      # e.g. not enough host memory to pin n*d floats
+            out["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+    ctx.close()
+    del ring, ctx
+    torch.cuda.empty_cache()
+    return out
+
+
 # ------------------------------------------------------------------------------------------ main
 
 def main(argv=None) -> int:
@@ -194,6 +298,8 @@ def main(argv=None) -> int:
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--adam", action="store_true", help="also time the warmup-phase Adam step alone")
+    ap.add_argument("--sweep", action="store_true",
+                    help="n in {2,4,8,16,32} x chunk in {1K,4K,16K,64K} on the chosen parameter set")
     args = ap.parse_args(argv)
     if args.warmup < 3:
         args.warmup = 3
@@ -232,7 +338,6 @@ def main(argv=None) -> int:
     import torch
     import torch.distributed as dist
 
-    from paper_2008_11343_b200 import binding as B
     from paper_2008_11343_b200 import build as libbuild
 
     if not torch.cuda.is_available():
@@ -242,108 +347,42 @@ def main(argv=None) -> int:
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    dev = torch.device("cuda", local_rank)
-
-    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}")
-    x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)
-    ctx.set_params(x0)
-    del x0
-    ring = []
-    for r in range(2):
-        gs = [torch.empty(w.d, dtype=torch.float32, device=dev) for _ in range(w.n)]
-        for i in range(w.n):
-            wl.device_gradient(w, r + 1000 * rank, i, gs[i])
-        ring.append(gs)
-    torch.cuda.synchronize()
-
-    # warmup phase (also timed alone when asked), phase switch, first compressed step
-    adam = None
-    for k in range(3):
-        ctx.warmup_step(ring[k % 2])
-    if args.adam:
-        ctx.set_timing(True)
-        for k in range(10):
-            ctx.warmup_step(ring[k % 2])
-        ms, cnt = ctx.kernel_time(B.KERNEL_WARMUP_ADAM)
-        ctx.set_timing(False)
-        ab = algorithmic_bytes(w.d, w.n, w.chunk)["warmup_adam"]
-        adam = {"ms_per_step": ms / cnt, "achieved_gbs": ab / (ms / cnt * 1e-3) / 1e9,
-                "worker_elements_per_s": w.d * w.n / (ms / cnt * 1e-3)}
-    ctx.freeze_v()
-    ctx.compressed_step(ring[0])             # reads the binary32 momentum once; not representative
-    for k in range(args.warmup):
-        ctx.compressed_step(ring[(k + 1) % 2])
-    torch.cuda.synchronize()
-
-    # timed region: K steps between two events on the context's stream
-    ctx.set_timing(True)
-    for kid in range(4):
-        ctx.kernel_time(kid)
-    launches0 = ctx.launch_count
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    with ClockSampler(local_rank) as clocks:
-        e0.record(ctx.stream)
-        for k in range(args.steps):
-            ctx.compressed_step(ring[k % 2])
-        e1.record(ctx.stream)
-        torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    seconds = max_over_ranks(e0.elapsed_time(e1) * 1e-3, dist if world > 1 else None)
-    launches = ctx.launch_count - launches0
-    kernel_ms = {}
-    for kid, name in enumerate(B.KERNEL_NAMES):
-        ms, cnt = ctx.kernel_time(kid)
-        if cnt:
-            kernel_ms[name] = ms / cnt
-    ctx.set_timing(False)
-    ms_per_step = seconds * 1e3 / args.steps
-    value = world * w.d * w.n * args.steps / seconds
-
-    ab = algorithmic_bytes(w.d, w.n, w.chunk)
     peaks = measured_peaks()
+
+    if args.sweep:
+        rows = []
+        for n in (2, 4, 8, 16, 32):
+            for chunk in (1024, 4096, 16384, 65536):
+                ws = w.with_(n=n, chunk=chunk)
+                m = measure(ws, args, rank, world, local_rank, dist, want_adam=(chunk == 1024), want_e2e=False)
+                ab = algorithmic_bytes(ws.d, n, chunk)
+                gbs = ab["step"] / (m["ms_per_step"] * 1e-3) / 1e9
+                row = {"n": n, "chunk": chunk, "ms_per_step": m["ms_per_step"], "value": m["value"],
+                       "step_gbs": gbs, "step_frac": gbs / peaks["hbm_gbs"], "kernel_ms": m["kernel_ms"]}
+                if m["adam"]:
+                    row["warmup_adam"] = m["adam"]
+                rows.append(row)
+        if rank == 0:
+            print(json.dumps({"sweep": rows, "workload": w.name, "d": w.d, "unit": UNIT, "peak_gbs": peaks["hbm_gbs"],
+                              "peak_source": peaks["source"]}))
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    m = measure(w, args, rank, world, local_rank, dist, want_adam=args.adam, want_e2e=not args.no_e2e)
+    ms_per_step, kernel_ms = m["ms_per_step"], m["kernel_ms"]
+    ab = algorithmic_bytes(w.d, w.n, w.chunk)
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
+    step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * w.n
                if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT else None)
     roofline = {"bound": "hbm", "kernel": "k_worker", "achieved": wk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": wk_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": traffic,
                 "algorithmic_bytes_per_launch": ab["worker"],
-                "whole_step": {"algorithmic_bytes": ab["step"], "achieved": ab["step"] / (ms_per_step * 1e-3) / 1e9,
-                               "frac": ab["step"] / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                               "frac_of_8TBs_nominal": ab["step"] / (ms_per_step * 1e-3) / 8e12},
+                "whole_step": {"algorithmic_bytes": ab["step"], "achieved": step_gbs,
+                               "frac": step_gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": step_gbs / 8000.0},
                 "kernel_ms": kernel_ms,
                 "kernel_gbs": {k: ab[k] / (v * 1e-3) / 1e9 for k, v in kernel_ms.items() if k in ab}}
-
-    # end to end through the host-gradient entry point: H2D of n gradients + D2H of x inside the timed region
-    e2e = None
-    if not args.no_e2e:
-        try:
-            host = [torch.empty(w.d, dtype=torch.float32).pin_memory() for _ in range(w.n)]
-            for i in range(w.n):
-                host[i].copy_(ring[0][i])
-            x_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
-            torch.cuda.synchronize()
-            ctx.compressed_step_host(host, x_host)
-            if world > 1:
-                dist.barrier()
-            t0 = time.perf_counter()
-            e0.record(ctx.stream)
-            for _ in range(args.e2e_steps):
-                ctx.compressed_step_host(host, x_host)
-            e1.record(ctx.stream)
-            torch.cuda.synchronize()
-            wall = time.perf_counter() - t0
-            secs = max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, wall), dist if world > 1 else None)
-            e2e = {"value": world * w.d * w.n * args.e2e_steps / secs, "unit": UNIT,
-                   "h2d_bytes_per_step": 4 * w.d * w.n, "d2h_bytes_per_step": 4 * w.d,
-                   "ms_per_step": secs * 1e3 / args.e2e_steps, "steps": args.e2e_steps,
-                   "api": "apms_compressed_step_host (pinned host gradients in, x out)"}
-            del host, x_host
-        except RuntimeError as exc:      # e.g. not enough host memory to pin n*d floats
-            e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -351,13 +390,13 @@ def main(argv=None) -> int:
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-                "clocks": clocks.summary()}
-        if adam:
-            line["warmup_adam"] = adam
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": m["e2e"], "gpu_launches": m["launches"],
+                "clocks": m["clocks"]}
+        if m["adam"]:
+            line["warmup_adam"] = m["adam"]
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

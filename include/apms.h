@@ -89,6 +89,13 @@ typedef enum {
     APMS_KERNEL_COUNT = 4
 } apms_kernel_id;
 
+/* How threads are grouped on a tile of a chunk in the worker and server kernels. */
+typedef enum {
+    APMS_TEAM_AUTO = 0,   /* one warp per tile when that still fills the GPU, else one CTA per tile */
+    APMS_TEAM_CTA = 1,    /* always one CTA (8 warps) per tile                                      */
+    APMS_TEAM_WARP = 2    /* always one warp per tile, eight tiles per CTA                          */
+} apms_team_mode;
+
 #define APMS_MAX_WORKERS 64
 
 /* Bytes of device workspace a context of this shape needs (pure function; 0 if the shape
@@ -173,6 +180,10 @@ apms_status apms_restore(apms_ctx* ctx, int t, apms_phase phase);
 
 apms_phase  apms_get_phase(const apms_ctx* ctx);
 int         apms_get_t(const apms_ctx* ctx);
+
+/* Launch-shape override (tuning and tests); results do not depend on it except for the order
+ * of the binary64 additions inside a chunk's sum of squares. */
+apms_status apms_set_team_mode(apms_ctx* ctx, apms_team_mode mode);
 
 /* Kernel timing: when enabled, every kernel launch is bracketed by CUDA events on the
  * context's stream.  apms_kernel_time() synchronises the stream, returns the total time

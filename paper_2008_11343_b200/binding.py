@@ -23,6 +23,7 @@ PHASE_CREATED, PHASE_WARMUP, PHASE_COMPRESSED = range(3)
  STATE_SERVER_ERR, STATE_SERVER_BITS, STATE_SERVER_SCALES) = range(9)
 KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
 KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
+TEAM_AUTO, TEAM_CTA, TEAM_WARP = range(3)
 MAX_WORKERS = 64
 
 _FP = C.POINTER(C.c_float)
@@ -47,6 +48,7 @@ SIGNATURES = {
     "apms_restore": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "apms_get_phase": (C.c_int, [C.c_void_p]),
     "apms_get_t": (C.c_int, [C.c_void_p]),
+    "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "apms_launch_count": (C.c_int64, [C.c_void_p]),
@@ -155,6 +157,10 @@ def apms_get_phase(h) -> int:
 
 def apms_get_t(h) -> int:
     return int(load().apms_get_t(h))
+
+
+def apms_set_team_mode(h, mode: int):
+    _check(h, load().apms_set_team_mode(h, mode))
 
 
 def apms_set_timing(h, enabled: bool):
@@ -295,6 +301,9 @@ class Context:
     @property
     def t(self) -> int:
         return apms_get_t(self._h)
+
+    def set_team_mode(self, mode: int):
+        apms_set_team_mode(self._h, mode)
 
     def set_timing(self, enabled: bool):
         apms_set_timing(self._h, enabled)

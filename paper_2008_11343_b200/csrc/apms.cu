@@ -39,6 +39,20 @@ constexpr int kThreads = 256;            // threads per CTA in every kernel
 constexpr int kWarps = kThreads / 32;
 constexpr int kGroup = 128;              // elements one warp covers per 128-bit access (4 sign words)
 
+// Tunables (defaults chosen by measurement on B200; override with -D to re-tune).
+#ifndef APMS_WORKER_U
+#define APMS_WORKER_U 4                  // 128-element groups in flight per warp, worker kernel
+#endif
+#ifndef APMS_SERVER_U
+#define APMS_SERVER_U 2                  // the same for the server kernel
+#endif
+#ifndef APMS_WORKER_CTAS
+#define APMS_WORKER_CTAS 3               // resident CTAs per SM the worker kernel is compiled for
+#endif
+#ifndef APMS_SERVER_CTAS
+#define APMS_SERVER_CTAS 3
+#endif
+
 struct GradPtrs { const float* p[APMS_MAX_WORKERS]; };
 
 // ------------------------------------------------------------------------------------------
@@ -159,25 +173,68 @@ k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
 }
 
 // ------------------------------------------------------------------------------------------
+// Mapping of chunks to work items.  An item is one tile of one chunk (for one worker on the
+// worker side).  Chunks up to kTileMax elements are one tile; longer chunks (the paper's own
+// layout is chunk = d/n) are cut into tiles of kTileSplit elements whose binary64 partial sums
+// of squares go to a scratch array and are added up, in tile order, by k_finalize_scales.
+// A team of WPC warps works on an item: the whole CTA (WPC = 8) or, for short chunks, one warp
+// (WPC = 1, eight items per CTA and no CTA-wide barrier).
+
+constexpr int64_t kTileMax = 65536;
+constexpr int64_t kTileSplit = 32768;
+// A tile is given to a single warp (eight tiles per CTA, no CTA-wide barrier) whenever that
+// still leaves at least kWarpTeamMinCtasPerSm CTAs per SM; small problems use one CTA per tile.
+constexpr int kWarpTeamMinCtasPerSm = 6;
+
+struct Tiling {
+    int64_t d, chunk, tile;   // tile == chunk when P == 1
+    int P;                    // tiles per chunk
+    int64_t Pp;               // row stride of the partial-sum arrays (>= C * P)
+};
+
+struct Item { int64_t c; int p; int64_t base; int L; int Lc; };
+
+__device__ __forceinline__ Item decode_item(const Tiling& t, int64_t chunk_tile)
+{
+    Item it;
+    it.p = (t.P == 1) ? 0 : (int)(chunk_tile % t.P);
+    it.c = (t.P == 1) ? chunk_tile : chunk_tile / t.P;
+    const int64_t cbeg = it.c * t.chunk;
+    const int64_t cend = (t.d - cbeg < t.chunk) ? t.d : cbeg + t.chunk;
+    it.base = cbeg + (int64_t)it.p * t.tile;
+    const int64_t left = cend - it.base;
+    it.L = (int)(left < t.tile ? (left > 0 ? left : 0) : t.tile);
+    it.Lc = (int)(cend - cbeg);
+    return it;
+}
+
+template <int WPC>
+__device__ __forceinline__ double team_sum(double a, double* smem)
+{
+    if (WPC == 1) return warp_sum(a);      // valid in lane 0
+    return block_sum(a, smem);             // valid in thread 0
+}
+
+// ------------------------------------------------------------------------------------------
 // Worker side: local momentum + error-compensated 1-bit compression (Section 3.3 steps 1-2).
-// One CTA per (chunk, worker); consecutive CTAs take the n workers of one chunk so that the
-// chunk's momentum bits are shared through L2.
+// Items are ordered chunk-major, worker-minor, so that the n workers of one chunk run
+// together and share that chunk's momentum bits through L2.
 
 struct WorkerArgs {
     float* z;  int64_t dz;        // n x d compensated vectors, stride dz
     uint32_t* B; int64_t Wp;      // n x W sign words, stride Wp
     float* s;  int64_t Cp;        // n x C scales, stride Cp
+    double* partial;              // n x Pp partial sums (only when P > 1)
     const float* m32;             // binary32 momentum (first step / forced)
     const uint32_t* Bbar; const float* Sbar;   // momentum as the server's last message
-    int64_t d; int64_t chunk;
+    Tiling t;
+    int64_t items;                // C * P * ni
     int i0, ni;                   // this launch covers workers i0 .. i0+ni-1
     float beta1, omb1;
 };
 
 template <bool M32, bool CHECKED>
-__device__ __forceinline__ void worker_group(const WorkerArgs& a, const float* __restrict__ g,
-                                             float* __restrict__ z, const float* __restrict__ m32,
-                                             const uint32_t* __restrict__ mbits, uint32_t* __restrict__ obits,
+__device__ __forceinline__ void worker_group(const WorkerArgs& a, float* __restrict__ z, uint32_t* __restrict__ obits,
                                              int grp, int lane, int L, float s_old, float Sbar,
                                              float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc)
 {
@@ -215,37 +272,39 @@ __device__ __forceinline__ void worker_group(const WorkerArgs& a, const float* _
     }
 }
 
-template <bool M32, int U>
-__global__ void __launch_bounds__(kThreads, 4)
+template <bool M32, int U, int WPC>
+__global__ void __launch_bounds__(kThreads, APMS_WORKER_CTAS)
 k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 {
     __shared__ double red[kWarps];
-    const int ii = blockIdx.x % a.ni;
-    const int64_t c = blockIdx.x / a.ni;
-    const int i = a.i0 + ii;
-    const int64_t base = c * a.chunk;
-    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
-    const float* __restrict__ g = G.p[ii] + base;
-    float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
-    const float* __restrict__ m32 = a.m32 + base;
-    const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
-    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
-    float* sptr = a.s + (int64_t)i * a.Cp + c;
-    const float s_old = *sptr;
-    const float Sbar = M32 ? 0.0f : a.Sbar[c];
+    constexpr int TEAMS = kWarps / WPC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t item = (int64_t)blockIdx.x * TEAMS + (WPC == 1 ? warp : 0);
+    if (item >= a.items) return;                       // only in the last CTA of the WPC == 1 form
+    const int ii = (int)(item % a.ni);
+    const Item it = decode_item(a.t, item / a.ni);
+    const int i = a.i0 + ii;
+    const int L = it.L;
+    const float* __restrict__ g = G.p[ii] + it.base;
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + it.base;
+    const float* __restrict__ m32 = a.m32 + it.base;
+    const uint32_t* __restrict__ mbits = a.Bbar + it.base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + it.base / 32;
+    float* sptr = a.s + (int64_t)i * a.Cp + it.c;
+    const float s_old = *sptr;
+    const float Sbar = M32 ? 0.0f : a.Sbar[it.c];
     const int full = L / kGroup;                  // groups with all 128 elements present
     const int ngroups = (L + kGroup - 1) / kGroup;
     double acc = 0.0;
 
-    int g0 = warp;
+    int g0 = (WPC == 1) ? 0 : warp;
     // fast path: U groups per warp per iteration, all loads issued before any use
-    for (; g0 + kWarps * (U - 1) < full; g0 += kWarps * U) {
+    for (; g0 + WPC * (U - 1) < full; g0 += WPC * U) {
         float4 gv[U], zv[U], mv[U];
         uint32_t mw[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int grp = g0 + kWarps * u;
+            const int grp = g0 + WPC * u;
             const int k = grp * kGroup + lane * 4;
             gv[u] = ld_stream4(g + k);
             zv[u] = ld_stream4(z + k);
@@ -254,11 +313,11 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         }
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            worker_group<M32, false>(a, g, z, m32, mbits, obits, g0 + kWarps * u, lane, L, s_old, Sbar,
+            worker_group<M32, false>(a, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
                                      gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc);
     }
     // remainder: one group at a time, bounds-checked
-    for (; g0 < ngroups; g0 += kWarps) {
+    for (; g0 < ngroups; g0 += WPC) {
         const int k = g0 * kGroup + lane * 4;
         const float4 gv = ld4_checked(g, k, L, true);
         const float4 zv = ld4_checked(z, k, L, true);
@@ -266,93 +325,154 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         uint32_t mw = 0;
         if (M32) mv = ld4_checked(m32, k, L, false);
         else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
-        worker_group<M32, true>(a, g, z, m32, mbits, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
+        worker_group<M32, true>(a, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
     }
 
-    const double total = block_sum(acc, red);
-    if (threadIdx.x == 0) *sptr = (float)sqrt(total / (double)L);   // ||z||_2 / sqrt(L)
+    const double total = team_sum<WPC>(acc, red);
+    if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
+        if (a.t.P == 1) *sptr = (float)sqrt(total / (double)it.Lc);          // ||z||_2 / sqrt(L)
+        else a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p] = total;
+    }
+}
+
+// Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).
+__global__ void k_finalize_scales(const double* __restrict__ partial, float* __restrict__ scales,
+                                  int rows, int64_t C, int64_t Cp, Tiling t)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)rows * C) return;
+    const int r = (int)(idx / C);
+    const int64_t c = idx % C;
+    const int64_t cbeg = c * t.chunk;
+    const int64_t Lc = (t.d - cbeg < t.chunk) ? t.d - cbeg : t.chunk;
+    double total = 0.0;
+    for (int p = 0; p < t.P; ++p) total += partial[(int64_t)r * t.Pp + c * t.P + p];
+    scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
 // ------------------------------------------------------------------------------------------
 // Server side: average the n decompressed messages, add the server error, recompress
-// (Section 3.3 step 4).  One CTA per chunk.
+// (Section 3.3 step 4).
 
 struct ServerArgs {
     const uint32_t* B; int64_t Wp;
     const float* s; int64_t Cp;
     float* zbar; uint32_t* Bbar; float* Sbar;
-    int64_t d; int64_t chunk;
+    double* partial;
+    Tiling t;
+    int64_t items;                // C * P
     int n; float nf;
 };
 
-template <bool CHECKED>
-__device__ __forceinline__ void server_group(const ServerArgs& a, const float* s_sh, const uint32_t* __restrict__ wb,
-                                             float* __restrict__ zb, uint32_t* __restrict__ ob,
-                                             int grp, int lane, int L, float S_old, double& acc)
+// U groups of one warp: the n sign words of every group are fetched worker by worker while
+// the running sums (sequential in worker order, as the average is defined) are updated.
+// +-s_i is formed by moving the complemented sign bit onto s_i's sign: no selects, no branches.
+template <int U, bool CHECKED>
+__device__ __forceinline__ void server_groups(const ServerArgs& a, const float* s_sh, const uint32_t* __restrict__ wb,
+                                              float* __restrict__ zb, uint32_t* __restrict__ ob,
+                                              int g0, int gstride, int lane, int L, float S_old, double& acc)
 {
-    const int k = grp * kGroup + lane * 4;
-    const int wk = grp * 4 + (lane >> 3);
     const int sh = 4 * (lane & 7);
-    float sum[4] = {0.f, 0.f, 0.f, 0.f};
-    const bool any = !CHECKED || (k < L);
-    if (any) {
-#pragma unroll 8
-        for (int i = 0; i < a.n; ++i) {
-            const uint32_t nib = wb[(int64_t)i * a.Wp + wk] >> sh;
-            const float si = s_sh[i];
+    const int wl = lane >> 3;
+    float sum[U][4];
+    float4 zo4[U];
+    bool live[U];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) sum[e] = __fadd_rn(sum[e], bit_scale((nib >> e) & 1u, si));
+    for (int u = 0; u < U; ++u) {
+        const int k = (g0 + gstride * u) * kGroup + lane * 4;
+        live[u] = !CHECKED || (k < L);
+        zo4[u] = CHECKED ? ld4_checked(zb, k, L, true) : ld_stream4(zb + k);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sum[u][e] = 0.0f;
+    }
+#pragma unroll 4
+    for (int i = 0; i < a.n; ++i) {
+        const uint32_t sbits = __float_as_uint(s_sh[i]);
+        uint32_t w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            w[u] = live[u] ? wb[(int64_t)i * a.Wp + (g0 + gstride * u) * 4 + wl] : 0u;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t neg = ~w[u] >> sh;            // bit e set: element e of this lane is negative
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                sum[u][e] = __fadd_rn(sum[u][e], __uint_as_float(sbits ^ ((neg << (31 - e)) & 0x80000000u)));
         }
     }
-    const float4 zo4 = CHECKED ? ld4_checked(zb, k, L, true) : ld_stream4(zb + k);
-    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
-    float zn[4];
-    uint32_t nibble = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const float avg = __fdiv_rn(sum[e], a.nf);
-        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
-        const bool valid = !CHECKED || (k + e < L);
-        if (valid) {
-            const double zd = (double)zn[e];
-            acc = fma(zd, zd, acc);
-            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+    for (int u = 0; u < U; ++u) {
+        const int grp = g0 + gstride * u;
+        const int k = grp * kGroup + lane * 4;
+        const float zo[4] = {zo4[u].x, zo4[u].y, zo4[u].z, zo4[u].w};
+        float zn[4];
+        uint32_t nibble = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float avg = __fdiv_rn(sum[u][e], a.nf);
+            zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+            const bool valid = !CHECKED || (k + e < L);
+            if (valid) {
+                const double zd = (double)zn[e];
+                acc = fma(zd, zd, acc);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
         }
+        const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        if (CHECKED) st4_checked(zb, k, L, out); else st_stream4(zb + k, out);
+        const uint32_t word = pack_group_words(nibble, lane);
+        const int wk = grp * 4 + wl;
+        if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) ob[wk] = word;
     }
-    const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
-    if (CHECKED) st4_checked(zb, k, L, out); else st_stream4(zb + k, out);
-    const uint32_t word = pack_group_words(nibble, lane);
-    if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) ob[wk] = word;
 }
 
-__global__ void __launch_bounds__(kThreads, 4)
+template <int U, int WPC>
+__global__ void __launch_bounds__(kThreads, APMS_SERVER_CTAS)
 k_server(const ServerArgs a)
 {
     __shared__ double red[kWarps];
-    __shared__ float s_sh[APMS_MAX_WORKERS];
-    const int64_t c = blockIdx.x;
-    const int64_t base = c * a.chunk;
-    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
-    if (threadIdx.x < a.n) s_sh[threadIdx.x] = a.s[(int64_t)threadIdx.x * a.Cp + c];
-    const float S_old = a.Sbar[c];
-    __syncthreads();
-    const uint32_t* __restrict__ wb = a.B + base / 32;
-    float* __restrict__ zb = a.zbar + base;
-    uint32_t* __restrict__ ob = a.Bbar + base / 32;
+    __shared__ float s_all[kWarps / WPC][APMS_MAX_WORKERS];
+    constexpr int TEAMS = kWarps / WPC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int team = (WPC == 1) ? warp : 0;
+    const int64_t item = (int64_t)blockIdx.x * TEAMS + team;
+    if (item >= a.items) return;
+    const Item it = decode_item(a.t, item);
+    const int L = it.L;
+    float* s_sh = s_all[team];
+    const int tid_in_team = (WPC == 1) ? lane : (int)threadIdx.x;
+    for (int i = tid_in_team; i < a.n; i += WPC * 32) s_sh[i] = a.s[(int64_t)i * a.Cp + it.c];
+    const float S_old = a.Sbar[it.c];
+    if (WPC == 1) __syncwarp(); else __syncthreads();
+    const uint32_t* __restrict__ wb = a.B + it.base / 32;
+    float* __restrict__ zb = a.zbar + it.base;
+    uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
     const int full = L / kGroup;
     const int ngroups = (L + kGroup - 1) / kGroup;
     double acc = 0.0;
-    int g0 = warp;
-    for (; g0 < full; g0 += kWarps) server_group<false>(a, s_sh, wb, zb, ob, g0, lane, L, S_old, acc);
-    for (; g0 < ngroups; g0 += kWarps) server_group<true>(a, s_sh, wb, zb, ob, g0, lane, L, S_old, acc);
-    const double total = block_sum(acc, red);
-    if (threadIdx.x == 0) a.Sbar[c] = (float)sqrt(total / (double)L);
+    // Each warp takes a contiguous run of groups, so that the 128-byte line of sign words it
+    // fetches for a worker serves its next seven groups from L1.
+    const int per_warp = (WPC == 1) ? ngroups : (ngroups + WPC - 1) / WPC;
+    int g0 = (WPC == 1) ? 0 : warp * per_warp;
+    const int g_end = (g0 + per_warp < ngroups) ? g0 + per_warp : ngroups;
+    const int g_full = (full < g_end) ? full : g_end;
+    for (; g0 + (U - 1) < g_full; g0 += U)
+        server_groups<U, false>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+    for (; g0 < g_end; ++g0)
+        server_groups<1, true>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+    const double total = team_sum<WPC>(acc, red);
+    if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
+        if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+        else a.partial[it.c * a.t.P + it.p] = total;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
 // Worker side again: the received chunk replaces the momentum (it stays in its compressed
 // form) and the model moves with the frozen variance (Section 3.3 steps 5-6).
+// One CTA per 8192 consecutive elements, whatever the chunk length.
+
+constexpr int kApplyTile = 8192;
 
 struct ApplyArgs {
     const uint32_t* Bbar; const float* Sbar; const float* v; float* x;
@@ -366,14 +486,20 @@ __device__ __forceinline__ float apply_elem(float x, float v, float q, float lr,
 __global__ void __launch_bounds__(kThreads, 4)
 k_apply(const ApplyArgs a)
 {
-    const int64_t c = blockIdx.x;
-    const int64_t base = c * a.chunk;
-    const int L = (int)((a.d - base < a.chunk) ? (a.d - base) : a.chunk);
-    const float S = a.Sbar[c];
+    const int64_t base = (int64_t)blockIdx.x * kApplyTile;
+    const int64_t left = a.d - base;
+    const int L = (int)(left < kApplyTile ? left : kApplyTile);
+    const int64_t c0 = base / a.chunk;
+    const uint32_t off0 = (uint32_t)(base - c0 * a.chunk);
+    const uint32_t chunk32 = (uint32_t)a.chunk;
     const uint32_t* __restrict__ bits = a.Bbar + base / 32;
     const float* __restrict__ v = a.v + base;
     float* __restrict__ x = a.x + base;
+    const float* __restrict__ Sb = a.Sbar + c0;
+#pragma unroll 2
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const uint32_t rel = off0 + (uint32_t)k;
+        const float S = Sb[rel < chunk32 ? 0u : rel / chunk32];
         const uint32_t nib = bits[k >> 5] >> (k & 31);
         if (k + 3 < L) {
             const float4 vv = ld_stream4(v + k);
@@ -417,7 +543,8 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
     int n;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_stage, total;
+    Tiling t;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_stage, total;
 };
 
 bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
@@ -441,6 +568,11 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     L->off_Bbar = take((size_t)L->Wp * 4);
     L->off_s = take((size_t)L->Cp * 4 * (size_t)n);
     L->off_Sbar = take((size_t)L->Cp * 4);
+    L->t.d = d; L->t.chunk = chunk;
+    if (chunk <= kTileMax) { L->t.tile = chunk; L->t.P = 1; }
+    else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
+    L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
+    L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
     L->off_stage = take((size_t)L->dz * 4 * 2);
     L->total = o;
     return true;
@@ -464,6 +596,7 @@ struct apms_ctx {
     int device;
     int sms;
     bool timing;
+    apms_team_mode team_mode;
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
@@ -479,6 +612,7 @@ struct apms_ctx {
     float* s(int i) { return (float*)(ws + L.off_s) + (int64_t)i * L.Cp; }
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
+    double* partial(int row) { return (double*)(ws + L.off_part) + (int64_t)row * L.t.Pp; }   // row n = server
 };
 
 namespace {
@@ -550,21 +684,50 @@ apms_status launch_check(apms_ctx* c, const char* what)
     return APMS_OK;
 }
 
+bool use_warp_teams(const apms_ctx* c, int64_t items)
+{
+    if (c->team_mode == APMS_TEAM_CTA) return false;
+    if (c->team_mode == APMS_TEAM_WARP) return true;
+    return items / kWarps >= (int64_t)kWarpTeamMinCtasPerSm * c->sms;
+}
+
+apms_status launch_finalize(apms_ctx* c, int first_row, int rows, float* scales)
+{
+    const int64_t total = (int64_t)rows * c->L.C;
+    k_finalize_scales<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->partial(first_row), scales, rows,
+                                                                            c->L.C, c->L.Cp, c->L.t);
+    return launch_check(c, "k_finalize_scales");
+}
+
 apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
 {
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
     a.B = c->B(0); a.Wp = c->L.Wp;
     a.s = c->s(0); a.Cp = c->L.Cp;
+    a.partial = c->partial(0);
     a.m32 = c->m(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
-    a.d = c->L.d; a.chunk = c->L.chunk; a.i0 = i0; a.ni = ni;
+    a.t = c->L.t; a.i0 = i0; a.ni = ni;
+    a.items = c->L.C * c->L.t.P * ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
-    const int64_t blocks = c->L.C * ni;
+    const bool warp_teams = use_warp_teams(c, a.items);
+    const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
-    Timed t(c, APMS_KERNEL_WORKER);
-    if (c->m_is_fp32) k_worker<true, 4><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
-    else              k_worker<false, 4><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
-    return launch_check(c, "k_worker");
+    {
+        Timed t(c, APMS_KERNEL_WORKER);
+        const unsigned gridx = (unsigned)blocks;
+        if (c->m_is_fp32) {
+            if (warp_teams) k_worker<true, 2, 1><<<gridx, kThreads, 0, c->stream>>>(G, a);
+            else            k_worker<true, 4, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a);
+        } else {
+            if (warp_teams) k_worker<false, APMS_WORKER_U, 1><<<gridx, kThreads, 0, c->stream>>>(G, a);
+            else            k_worker<false, APMS_WORKER_U, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a);
+        }
+        apms_status st = launch_check(c, "k_worker");
+        if (st != APMS_OK) return st;
+    }
+    if (c->L.t.P > 1) return launch_finalize(c, i0, ni, c->s(i0));
+    return APMS_OK;
 }
 
 apms_status launch_server_and_apply(apms_ctx* c)
@@ -573,18 +736,28 @@ apms_status launch_server_and_apply(apms_ctx* c)
         ServerArgs a;
         a.B = c->B(0); a.Wp = c->L.Wp; a.s = c->s(0); a.Cp = c->L.Cp;
         a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
-        a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n;
-        Timed t(c, APMS_KERNEL_SERVER);
-        k_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
-        apms_status st = launch_check(c, "k_server");
-        if (st != APMS_OK) return st;
+        a.partial = c->partial(c->L.n);
+        a.t = c->L.t; a.items = c->L.C * c->L.t.P; a.n = c->L.n; a.nf = (float)c->L.n;
+        const bool warp_teams = use_warp_teams(c, a.items);
+        const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
+        {
+            Timed t(c, APMS_KERNEL_SERVER);
+            if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+            else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+            apms_status st = launch_check(c, "k_server");
+            if (st != APMS_OK) return st;
+        }
+        if (c->L.t.P > 1) {
+            apms_status st = launch_finalize(c, c->L.n, 1, c->Sbar());
+            if (st != APMS_OK) return st;
+        }
     }
     {
         ApplyArgs a;
         a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
         Timed t(c, APMS_KERNEL_APPLY);
-        k_apply<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
+        k_apply<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(a);
         apms_status st = launch_check(c, "k_apply");
         if (st != APMS_OK) return st;
     }
@@ -644,6 +817,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
+    c->team_mode = APMS_TEAM_AUTO;
     *out = c;
     return APMS_OK;
 }
@@ -707,7 +881,7 @@ apms_status apms_freeze_v(apms_ctx* c)
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_WARMUP) return fail(c, APMS_ERR_BAD_STATE, "apms_freeze_v needs the WARMUP phase");
     // errors start at zero: z = 0 with scale 0 implies delta = 0 - (+0) = 0
-    APMS_CUDA(c, cudaMemsetAsync(c->ws + c->L.off_zbar, 0, c->L.off_stage - c->L.off_zbar, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->ws + c->L.off_zbar, 0, c->L.off_part - c->L.off_zbar, c->stream));
     c->phase = APMS_PHASE_COMPRESSED;
     c->m_is_fp32 = true;
     return APMS_OK;
@@ -879,6 +1053,14 @@ apms_status apms_restore(apms_ctx* c, int t, apms_phase phase)
 
 apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }
 int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
+
+apms_status apms_set_team_mode(apms_ctx* c, apms_team_mode mode)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (mode != APMS_TEAM_AUTO && mode != APMS_TEAM_CTA && mode != APMS_TEAM_WARP) return fail(c, APMS_ERR_INVALID_ARG, "unknown team mode");
+    c->team_mode = mode;
+    return APMS_OK;
+}
 
 apms_status apms_set_timing(apms_ctx* c, int enabled)
 {

@@ -18,10 +18,12 @@ def upload(grads):
     return [torch.from_numpy(np.ascontiguousarray(g)).cuda() for g in grads]
 
 
-def make_pair(w: wl.Workload, x0=None):
+def make_pair(w: wl.Workload, x0=None, team_mode=None):
     """A CUDA context and an oracle with the same shape, hyper-parameters and x0."""
     x0 = wl.initial_params(w) if x0 is None else x0
     ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    if team_mode is not None:
+        ctx.set_team_mode(team_mode)
     ctx.set_params(x0)
     orc = ao.Oracle(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
     orc.set_threads(orc.max_threads())
@@ -117,12 +119,12 @@ def teacher_force(ctx, orc, w):
 
 
 def run_both(w: wl.Workload, warmup=None, compressed=None, check_every_step=True, exact=False,
-             grads_fn=None):
+             grads_fn=None, team_mode=None):
     """Free-running: both sides step from the same x0 on the same gradients."""
     warmup = w.warmup_steps if warmup is None else warmup
     compressed = w.compressed_steps if compressed is None else compressed
     grads_fn = grads_fn or (lambda step: wl.host_gradients(w, step))
-    ctx, orc = make_pair(w)
+    ctx, orc = make_pair(w, team_mode=team_mode)
     reports = []
     step = 0
     for _ in range(warmup):

@@ -19,16 +19,18 @@ def tiny(d, n, chunk, cfg_id=100, **kw):
 
 EDGE = [(1, 1, 32), (31, 2, 32), (32, 2, 32), (33, 3, 32), (127, 4, 128), (128, 4, 128), (129, 4, 128),
         (4095, 2, 4096), (4096, 2, 4096), (4097, 2, 4096), (1000, 5, 96), (12345, 3, 1024),
-        (5 * 8192 + 77, 2, 8192), (3 * 65536 + 1, 2, 65536), (70000, 16, 160), (2050, 64, 2048)]
+        (5 * 8192 + 77, 2, 8192), (3 * 65536 + 1, 2, 65536), (70000, 16, 160), (2050, 64, 2048),
+        (300000, 2, 131104), (4 * 70016, 4, 70016), (5000, 3, 1024), (40000, 2, 4096)]
 
 
+@pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP], ids=["cta-per-tile", "warp-per-tile"])
 @pytest.mark.parametrize("d,n,chunk", EDGE)
-def test_free_running_edge_sizes_bit_identical(d, n, chunk):
+def test_free_running_edge_sizes_bit_identical(d, n, chunk, team):
     """Ragged tails, d below / at / above a word, a vector and a chunk; several tiles.  On these
     sizes every scale is expected to round identically on both sides, so the whole state must be
     bit-identical (the binary64 sums differ only in the order of additions)."""
     w = tiny(d, n, chunk, warmup_steps=3, compressed_steps=4)
-    H.run_both(w, exact=True)
+    H.run_both(w, exact=True, team_mode=team)
 
 
 def test_teacher_forced_steps_bits_exact():

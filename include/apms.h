@@ -201,6 +201,48 @@ const char* apms_last_error(const apms_ctx* ctx);
 /* Free the context (and its workspace if it allocated one).  NULL is ignored. */
 void        apms_destroy(apms_ctx* ctx);
 
+/* Allocation-free compression of a flat vector.  (The paper has no counterpart: this entry
+ * point exists for callers, not for the algorithm.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated or freed - inside a
+ * region of a framework that forbids allocator calls (a step function that must not disturb a
+ * caching allocator or its memory accounting), a plugin that is handed a fixed set of buffers
+ * and a stream and nothing else, a latency-critical loop in which cudaMalloc's implicit
+ * device-wide synchronisation is unacceptable.  Such a caller cannot create a context with its
+ * own workspace and has no spare buffer to bind one to.
+ *
+ * What it does: the 1-bit compressor of Section 5.1 on every chunk of z, as the worker side of
+ * apms_compressed_step does for a vector z = m_i + delta_i that is already formed:
+ *   scales_dev[c] = ||z_c||_2 / sqrt(L_c),   bit j of bits_dev = (z[j] >= 0),
+ * with the sign-word and scale layout stated at the top of this file.  z is not modified.
+ *   z_dev       device, d floats, 16-byte aligned, read-only
+ *   bits_dev    device, ceil(d/32) uint32, written (padding bits 0)
+ *   scales_dev  device, ceil(d/chunk) floats, written
+ *   cuda_stream a cudaStream_t passed as void* (NULL = the legacy default stream) on the
+ *               current device; the call enqueues two kernels and returns without synchronising
+ * The caller owns all three buffers.  The only memory the kernels use beyond them is one
+ * binary64 partial sum of squares per 32768-element tile of a chunk; it lives in a fixed array
+ * of APMS_NOALLOC_MAX_TILES doubles (128 KiB) that is part of the library's device image, so
+ * every GPU that loads the library holds those 128 KiB until the process exits.  The call makes
+ * no cudaMalloc / cudaFree and calls no allocating routine of any library.
+ *
+ * Limits and rules
+ *   - ceil(d/chunk) * ceil(chunk/32768) must not exceed APMS_NOALLOC_MAX_TILES (for chunks up
+ *     to 32768 elements that is d <= 2^29); larger shapes, d < 1, or a chunk that is not a
+ *     positive multiple of 32 return APMS_ERR_INVALID_ARG before anything is launched.
+ *   - The first call on each device looks up the device address of the fixed array (once per
+ *     device, with that device current).  Make that first call before any stream capture.
+ *   - All calls on a device share the one array.  It needs no clearing - every tile's slot is
+ *     overwritten before it is read - but it keeps the last call's contents, and two calls
+ *     whose kernels may overlap on the GPU (different streams without an ordering between
+ *     them, or different host threads) race on it and give wrong scales.  Calls on one stream
+ *     are safe back to back.
+ *   - There is no context: the message of a failure is read with apms_last_error(NULL) on the
+ *     calling thread. */
+#define APMS_NOALLOC_MAX_TILES 16384
+apms_status apms_compress_noalloc(const float* z_dev, int64_t d, int64_t chunk,
+                                  uint32_t* bits_dev, float* scales_dev, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

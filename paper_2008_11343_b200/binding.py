@@ -25,6 +25,7 @@ KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
 KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
 TEAM_AUTO, TEAM_CTA, TEAM_WARP = range(3)
 MAX_WORKERS = 64
+NOALLOC_MAX_TILES = 16384
 
 _FP = C.POINTER(C.c_float)
 _FPP = C.POINTER(_FP)
@@ -54,6 +55,7 @@ SIGNATURES = {
     "apms_launch_count": (C.c_int64, [C.c_void_p]),
     "apms_last_error": (C.c_char_p, [C.c_void_p]),
     "apms_destroy": (None, [C.c_void_p]),
+    "apms_compress_noalloc": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]),
 }
 
 _lib: Optional[C.CDLL] = None
@@ -183,6 +185,17 @@ def apms_last_error(h) -> str:
 
 def apms_destroy(h):
     load().apms_destroy(h)
+
+
+def apms_compress_noalloc(z_ptr: int, d: int, chunk: int, bits_ptr: int, scales_ptr: int, stream: int = 0):
+    """Sign words and chunk scales of the d floats at device address z_ptr, written to the
+    caller's device buffers.  For callers that may not allocate device memory: the library
+    allocates nothing here (its only scratch is a fixed 128 KiB array inside the library), so
+    the shape is limited (see APMS_NOALLOC_MAX_TILES in apms.h) and calls that overlap on the
+    GPU must be ordered by the caller.  Raises ApmsError with the library's message otherwise."""
+    st = load().apms_compress_noalloc(z_ptr, d, chunk, bits_ptr, scales_ptr, stream or None)
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(None).decode())
 
 
 # --- convenience wrapper: handle + torch workspace + stream ---------------------------------

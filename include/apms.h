@@ -56,7 +56,8 @@ typedef enum {
     APMS_ERR_BAD_STATE = 2,     /* call not allowed in the context's current phase         */
     APMS_ERR_CUDA = 3,          /* a CUDA runtime call failed; see apms_last_error()       */
     APMS_ERR_OOM = 4,           /* workspace too small, or allocation failed               */
-    APMS_ERR_TIMEOUT = 5,       /* reserved: a bounded device-side wait gave up            */
+    APMS_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (reported by the next
+                                   synchronising call; the context's state is then undefined) */
     APMS_ERR_BOUNDS = 6         /* reserved: a checked build recorded an out-of-range index */
 } apms_status;
 
@@ -91,9 +92,11 @@ typedef enum {
 
 /* How threads are grouped on a tile of a chunk in the worker and server kernels. */
 typedef enum {
-    APMS_TEAM_AUTO = 0,   /* one warp per tile when that still fills the GPU, else one CTA per tile */
-    APMS_TEAM_CTA = 1,    /* always one CTA (8 warps) per tile                                      */
-    APMS_TEAM_WARP = 2    /* always one warp per tile, eight tiles per CTA                          */
+    APMS_TEAM_AUTO = 0,   /* the library's choice for the shape (the forms below, per kernel)      */
+    APMS_TEAM_CTA = 1,    /* always one CTA (8 warps) per tile, operands loaded by the threads      */
+    APMS_TEAM_WARP = 2,   /* always one warp per tile, eight tiles per CTA                          */
+    APMS_TEAM_STAGED = 3  /* one CTA per tile fed by bulk asynchronous copies through shared memory
+                             wherever the shape allows it (chunk a multiple of 2048), else as AUTO  */
 } apms_team_mode;
 
 #define APMS_MAX_WORKERS 64

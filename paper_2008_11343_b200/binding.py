@@ -23,7 +23,7 @@ PHASE_CREATED, PHASE_WARMUP, PHASE_COMPRESSED = range(3)
  STATE_SERVER_ERR, STATE_SERVER_BITS, STATE_SERVER_SCALES) = range(9)
 KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
 KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
-TEAM_AUTO, TEAM_CTA, TEAM_WARP = range(3)
+TEAM_AUTO, TEAM_CTA, TEAM_WARP, TEAM_STAGED = range(4)
 MAX_WORKERS = 64
 NOALLOC_MAX_TILES = 16384
 

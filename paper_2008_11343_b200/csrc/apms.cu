@@ -469,6 +469,190 @@ k_server(const ServerArgs a)
 }
 
 // ------------------------------------------------------------------------------------------
+// Server side, staged form: the chunk's zbar and the n workers' sign words stream through a
+// ring of shared-memory stages filled by bulk asynchronous copies (one elected thread issues
+// them, an mbarrier per stage counts the arriving bytes), so that the bytes in flight do not
+// depend on registers or occupancy.  Used when every slab of kSlab elements of a tile starts
+// on a 16-byte boundary in all streams (chunk a multiple of kSlab); other shapes use k_server.
+
+constexpr int kSlab = 2048;                      // elements per stage: 8 KiB of zbar + n x 256 B of sign words
+constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per warp
+constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker
+constexpr int kStages = 4;
+constexpr uint32_t kWaitLimit = 1u << 22;        // polls of one mbarrier before the kernel gives up
+
+enum { DEVICE_OK = 0, DEVICE_WAIT_TIMEOUT = 1 };
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait: false when the phase did not complete within kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 32) __nanosleep(32);
+    }
+    return false;
+}
+// Global -> this CTA's shared memory; 16-byte aligned addresses, size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+struct ServerStagedArgs {
+    ServerArgs a;
+    int* status;          // device status word: set when a bounded wait gave up
+    float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
+};
+
+__device__ __forceinline__ size_t staged_stage_bytes(int n) { return (size_t)kSlab * 4 + (size_t)n * kSlabWords * 4; }
+
+__global__ void __launch_bounds__(kThreads, 3)
+k_server_staged(const ServerStagedArgs sa)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const ServerArgs& a = sa.a;
+    __shared__ double red[kWarps];
+    __shared__ uint64_t full[kStages];
+    __shared__ uint32_t neg_s[APMS_MAX_WORKERS];      // bit patterns of -s_i of this chunk
+    __shared__ int failed;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const Item it = decode_item(a.t, (int64_t)blockIdx.x);
+    const int L = it.L;
+    const int n = a.n;
+    const size_t stage_bytes = staged_stage_bytes(n);
+    const int nslabs = (L + kSlab - 1) / kSlab;
+    const float* __restrict__ zb_g = a.zbar + it.base;
+    const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
+    uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+        failed = 0;
+        mbar_fence_init();
+    }
+    for (int i = threadIdx.x; i < n; i += kThreads)
+        neg_s[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
+    const float S_old = a.Sbar[it.c];
+    __syncthreads();
+
+    // producer: slab j into stage j % kStages (only whole 16-byte pieces that hold live elements)
+    auto issue = [&](int j) {
+        const int st = j % kStages;
+        unsigned char* base = smem + (size_t)st * stage_bytes;
+        const int left = L - j * kSlab;
+        const int live = left < kSlab ? left : kSlab;
+        const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
+        const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
+        mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
+        bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
+        uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
+        for (int i = 0; i < n; ++i)
+            bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
+    };
+    if (threadIdx.x == 0)
+        for (int j = 0; j < kStages && j < nslabs; ++j) issue(j);
+
+    const int sh = 4 * (lane & 7);
+    const int wl = lane >> 3;
+    double acc = 0.0;
+    int j = 0;
+    for (; j < nslabs; ++j) {
+        const int st = j % kStages;
+        if (!mbar_wait(&full[st], (uint32_t)(j / kStages) & 1u)) failed = 1;     // nothing of this slab is stored then
+        const unsigned char* base = smem + (size_t)st * stage_bytes;
+        const float* zs = reinterpret_cast<const float*>(base);
+        const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
+        const int g0 = warp, g1 = warp + kWarps;                     // this warp's two groups of the slab
+        const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
+        const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
+        float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
+        const uint32_t* r0 = rows + g0 * 4 + wl;
+        const uint32_t* r1 = rows + g1 * 4 + wl;
+#pragma unroll 4
+        for (int i = 0; i < n; ++i) {
+            const uint32_t ns = neg_s[i];
+            // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
+            const uint32_t y0 = r0[i * kSlabWords] << (28 - sh);
+            const uint32_t y1 = r1[i * kSlabWords] << (28 - sh);
+            float2 q;
+            q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns);
+            s01 = __fadd2_rn(s01, q);
+            q.x = __uint_as_float(((y0 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y0 & 0x80000000u) ^ ns);
+            s23 = __fadd2_rn(s23, q);
+            q.x = __uint_as_float(((y1 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y1 << 2) & 0x80000000u) ^ ns);
+            t01 = __fadd2_rn(t01, q);
+            q.x = __uint_as_float(((y1 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y1 & 0x80000000u) ^ ns);
+            t23 = __fadd2_rn(t23, q);
+        }
+        __syncthreads();                                              // the stage has been read by everyone
+        if (failed) break;
+        if (threadIdx.x == 0 && j + kStages < nslabs) issue(j + kStages);
+
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int grp = j * kSlabGroups + (u ? g1 : g0);
+            const int k = grp * kGroup + lane * 4;
+            const float4 zo4 = u ? zo1 : zo0;
+            const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+            const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
+            float zn[4];
+            uint32_t nibble = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
+                zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+                if (k + e < L) {
+                    const double zd = (double)zn[e];
+                    acc = fma(zd, zd, acc);
+                    nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                }
+            }
+            st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            const uint32_t word = pack_group_words(nibble, lane);
+            const int wk = grp * 4 + wl;
+            if ((lane & 7) == 0 && wk * 32 < L) ob[wk] = word;
+        }
+    }
+    if (failed) {
+        // give the copies still in flight a bounded chance to land before the CTA's shared memory is released
+        if (threadIdx.x == 0) {
+            const int last = (j + kStages < nslabs) ? j + kStages : nslabs;
+            for (int q = j; q < last; ++q) mbar_wait(&full[q % kStages], (uint32_t)(q / kStages) & 1u);
+            atomicExch(sa.status, DEVICE_WAIT_TIMEOUT);
+        }
+        return;
+    }
+    const double total = block_sum(acc, red);
+    if (threadIdx.x == 0) {
+        if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+        else a.partial[it.c * a.t.P + it.p] = total;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Worker side again: the received chunk replaces the momentum (it stays in its compressed
 // form) and the model moves with the frozen variance (Section 3.3 steps 5-6).
 // One CTA per 8192 consecutive elements, whatever the chunk length.
@@ -545,7 +729,7 @@ struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_stage, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_stage, off_status, total;
 };
 
 bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
@@ -575,6 +759,7 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
     L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
     L->off_stage = take((size_t)L->dz * 4 * 2);
+    L->off_status = take(256);
     L->total = o;
     return true;
 }
@@ -598,6 +783,7 @@ struct apms_ctx {
     int sms;
     bool timing;
     apms_team_mode team_mode;
+    bool staged_ready;       // the staged server kernel's shared-memory limit has been raised
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
@@ -613,6 +799,7 @@ struct apms_ctx {
     float* s(int i) { return (float*)(ws + L.off_s) + (int64_t)i * L.Cp; }
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
+    int* status() { return (int*)(ws + L.off_status); }
     double* partial(int row) { return (double*)(ws + L.off_part) + (int64_t)row * L.t.Pp; }   // row n = server
 };
 
@@ -685,6 +872,23 @@ apms_status launch_check(apms_ctx* c, const char* what)
     return APMS_OK;
 }
 
+// After a stream synchronisation: has a kernel recorded that one of its bounded waits gave up?
+apms_status device_status_check(apms_ctx* c)
+{
+    int st = 0;
+    APMS_CUDA(c, cudaMemcpy(&st, c->status(), sizeof st, cudaMemcpyDeviceToHost));
+    if (st != 0) return fail(c, APMS_ERR_TIMEOUT, "a kernel gave up waiting for its own asynchronous copies; the state of this context is undefined");
+    return APMS_OK;
+}
+
+// The staged server kernel needs every 2048-element slab of a tile to start on a 16-byte boundary
+// in zbar and in the sign words, i.e. chunks that are multiples of 2048 elements.
+bool use_staged_server(const apms_ctx* c)
+{
+    if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
+    return c->L.chunk % kSlab == 0;
+}
+
 bool use_warp_teams(const apms_ctx* c, int64_t items)
 {
     if (c->team_mode == APMS_TEAM_CTA) return false;
@@ -739,11 +943,24 @@ apms_status launch_server_and_apply(apms_ctx* c)
         a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
         a.partial = c->partial(c->L.n);
         a.t = c->L.t; a.items = c->L.C * c->L.t.P; a.n = c->L.n; a.nf = (float)c->L.n;
-        const bool warp_teams = use_warp_teams(c, a.items);
+        const bool staged = use_staged_server(c);
+        const bool warp_teams = !staged && use_warp_teams(c, a.items);
         const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
+        if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
+        const size_t staged_smem = (size_t)kStages * ((size_t)kSlab * 4 + (size_t)a.n * kSlabWords * 4);
+        if (staged && !c->staged_ready) {
+            APMS_CUDA(c, cudaFuncSetAttribute(k_server_staged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged_smem));
+            c->staged_ready = true;
+        }
         {
             Timed t(c, APMS_KERNEL_SERVER);
-            if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+            if (staged) {
+                ServerStagedArgs sa;
+                sa.a = a; sa.status = c->status();
+                sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
+                k_server_staged<<<(unsigned)blocks, kThreads, staged_smem, c->stream>>>(sa);
+            }
+            else if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
             else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
             apms_status st = launch_check(c, "k_server");
             if (st != APMS_OK) return st;
@@ -818,7 +1035,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
-    c->team_mode = APMS_TEAM_AUTO;
+    c->team_mode = APMS_TEAM_AUTO; c->staged_ready = false;
     *out = c;
     return APMS_OK;
 }
@@ -845,6 +1062,7 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemcpyAsync(c->x(), x0, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->m(), 0, (size_t)c->L.dz * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
     c->t = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
     return APMS_OK;
@@ -935,7 +1153,7 @@ apms_status apms_compressed_step_host(apms_ctx* c, const float* const* grads_hos
     if (st != APMS_OK) return st;
     if (x_out_host) APMS_CUDA(c, cudaMemcpyAsync(x_out_host, c->x(), bytes, cudaMemcpyDeviceToHost, c->stream));
     APMS_CUDA(c, cudaStreamSynchronize(c->stream));
-    return APMS_OK;
+    return device_status_check(c);
 }
 
 apms_status apms_get_params(apms_ctx* c, float* dst, int dst_is_device)
@@ -944,7 +1162,10 @@ apms_status apms_get_params(apms_ctx* c, float* dst, int dst_is_device)
     if (!dst) return fail(c, APMS_ERR_INVALID_ARG, "dst is NULL");
     if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "no parameters set yet");
     APMS_CUDA(c, cudaMemcpyAsync(dst, c->x(), (size_t)c->L.d * 4, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream));
-    if (!dst_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (!dst_is_device) {
+        APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+        return device_status_check(c);
+    }
     return APMS_OK;
 }
 
@@ -992,7 +1213,7 @@ apms_status apms_get_state_slice(apms_ctx* c, apms_state_id which, int worker, i
     const char* from = staged ? (const char*)c->stage(0) : src + (size_t)first * 4;
     APMS_CUDA(c, cudaMemcpyAsync(dst, from, (size_t)count * 4, cudaMemcpyDeviceToHost, c->stream));
     APMS_CUDA(c, cudaStreamSynchronize(c->stream));
-    return APMS_OK;
+    return device_status_check(c);
 }
 
 apms_status apms_get_state(apms_ctx* c, apms_state_id which, int worker, void* dst)
@@ -1058,7 +1279,7 @@ int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
 apms_status apms_set_team_mode(apms_ctx* c, apms_team_mode mode)
 {
     if (!c) return APMS_ERR_INVALID_ARG;
-    if (mode != APMS_TEAM_AUTO && mode != APMS_TEAM_CTA && mode != APMS_TEAM_WARP) return fail(c, APMS_ERR_INVALID_ARG, "unknown team mode");
+    if (mode != APMS_TEAM_AUTO && mode != APMS_TEAM_CTA && mode != APMS_TEAM_WARP && mode != APMS_TEAM_STAGED) return fail(c, APMS_ERR_INVALID_ARG, "unknown team mode");
     c->team_mode = mode;
     return APMS_OK;
 }

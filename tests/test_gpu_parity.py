@@ -23,8 +23,15 @@ EDGE = [(1, 1, 32), (31, 2, 32), (32, 2, 32), (33, 3, 32), (127, 4, 128), (128, 
         (300000, 2, 131104), (4 * 70016, 4, 70016), (5000, 3, 1024), (40000, 2, 4096)]
 
 
-@pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP], ids=["cta-per-tile", "warp-per-tile"])
-@pytest.mark.parametrize("d,n,chunk", EDGE)
+# shapes for the staged forms (chunk a multiple of 2048): one slab, many slabs, ragged last slab and chunk,
+# split chunks, n not a power of two (IEEE division instead of the exact multiplication by 1/n), n = 64
+STAGED = [(2048, 1, 2048), (10 * 2048 + 1, 5, 2048), (6144 * 3 + 33, 7, 6144), (3 * 131072 + 4099, 3, 131072),
+          (8 * 32768 + 23552, 16, 32768), (2 * 4096 + 2047, 64, 4096), (65536 + 2049, 2, 65536)]
+
+
+@pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP, B.TEAM_AUTO, B.TEAM_STAGED],
+                         ids=["cta-per-tile", "warp-per-tile", "auto", "staged"])
+@pytest.mark.parametrize("d,n,chunk", EDGE + STAGED)
 def test_free_running_edge_sizes_bit_identical(d, n, chunk, team):
     """Ragged tails, d below / at / above a word, a vector and a chunk; several tiles.  On these
     sizes every scale is expected to round identically on both sides, so the whole state must be

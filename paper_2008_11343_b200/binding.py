@@ -15,7 +15,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libapms.so")
+LIB_PATH = os.environ.get("APMS_LIBRARY") or os.path.join(HERE, "libapms.so")   # override: another build of the same ABI
 
 OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_CUDA, ERR_OOM, ERR_TIMEOUT, ERR_BOUNDS = range(7)
 PHASE_CREATED, PHASE_WARMUP, PHASE_COMPRESSED = range(3)

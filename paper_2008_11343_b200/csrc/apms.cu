@@ -235,7 +235,7 @@ struct WorkerArgs {
 };
 
 template <bool M32, bool CHECKED>
-__device__ __forceinline__ void worker_group(const WorkerArgs& a, float* __restrict__ z, uint32_t* __restrict__ obits,
+__device__ __forceinline__ void worker_group(float beta1, float omb1, float* __restrict__ z, uint32_t* __restrict__ obits,
                                              int grp, int lane, int L, float s_old, float Sbar,
                                              float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc)
 {
@@ -254,7 +254,7 @@ __device__ __forceinline__ void worker_group(const WorkerArgs& a, float* __restr
     uint32_t nibble = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));   // local momentum
+        const float mi = __fmaf_rn(beta1, mm[e], __fmul_rn(omb1, gg[e]));       // local momentum
         const float err = implied_error(zo[e], s_old);                          // delta_i (old)
         zn[e] = __fadd_rn(mi, err);                                             // compensated
         const bool valid = !CHECKED || (k + e < L);
@@ -314,7 +314,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         }
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            worker_group<M32, false>(a, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
+            worker_group<M32, false>(a.beta1, a.omb1, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
                                      gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc);
     }
     // remainder: one group at a time, bounds-checked
@@ -326,7 +326,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         uint32_t mw = 0;
         if (M32) mv = ld4_checked(m32, k, L, false);
         else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
-        worker_group<M32, true>(a, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
+        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
     }
 
     const double total = team_sum<WPC>(acc, red);
@@ -334,6 +334,101 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         if (a.t.P == 1) *sptr = (float)sqrt(total / (double)it.Lc);          // ||z||_2 / sqrt(L)
         else a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p] = total;
     }
+}
+
+// Worker side, fine-tiled form (steady state, chunk a multiple of kFineTile): one CTA per
+// (worker, 4096-element tile), every load of the tile issued before the first use, the tile's
+// binary64 sum of squares written to a partial-sum array that k_finalize_fine adds up per chunk
+// in tile order.  Short-lived CTAs that each touch 16 KiB of every stream once keep DRAM pages
+// and the memory pipeline busier than long-running warps that each follow their own stream.
+// Launch order: runs of kFineRun consecutive tiles of one worker, then the same tiles of the next
+// worker, so that every stream is read in long sequential pieces while the n workers of a stretch
+// still meet its momentum bits in L2.
+
+constexpr int kFineTile = 4096;           // 256 threads x 4 x (4 floats)
+constexpr int kFineU = kFineTile / (kThreads * 4);
+constexpr int kFineRun = 64;
+
+struct WorkerFineArgs {
+    float* z; int64_t dz;
+    uint32_t* B; int64_t Wp;
+    const float* s; int64_t Cp;       // the scales of the previous step (read only here)
+    double* partial; int64_t Pp;      // ni rows of `tiles` partial sums, row stride Pp
+    const uint32_t* Bbar; const float* Sbar;
+    int64_t d, chunk, tiles;
+    int i0, ni;
+    float beta1, omb1;
+};
+
+__global__ void __launch_bounds__(kThreads, 3)
+k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
+{
+    __shared__ double red[kWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t per_stretch = (int64_t)a.ni * kFineRun;
+    const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
+    const int rem = (int)((int64_t)blockIdx.x - stretch * per_stretch);
+    const int ii = rem / kFineRun;
+    const int64_t t = stretch * kFineRun + (rem % kFineRun);
+    if (t >= a.tiles) return;                                  // whole CTA: the last stretch may be short
+    const int i = a.i0 + ii;
+    const int64_t base = t * kFineTile;
+    const int64_t c = base / a.chunk;
+    const int64_t left = a.d - base;
+    const int L = (int)(left < kFineTile ? left : kFineTile);
+    const float* __restrict__ g = G.p[ii] + base;
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
+    const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
+    const float s_old = a.s[(int64_t)i * a.Cp + c];
+    const float Sbar = a.Sbar[c];
+    double acc = 0.0;
+    if (L == kFineTile) {
+        float4 gv[kFineU], zv[kFineU];
+        uint32_t mw[kFineU];
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            const int grp = u * kWarps + warp;
+            const int k = grp * kGroup + lane * 4;
+            gv[u] = ld_stream4(g + k);
+            zv[u] = ld_stream4(z + k);
+            mw[u] = mbits[grp * 4 + (lane >> 3)];
+        }
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u)
+            worker_group<false, false>(a.beta1, a.omb1, z, obits, u * kWarps + warp, lane, L, s_old, Sbar,
+                                       gv[u], zv[u], make_float4(0, 0, 0, 0), mw[u], acc);
+    } else {
+        const int ngroups = (L + kGroup - 1) / kGroup;
+        for (int grp = warp; grp < ngroups; grp += kWarps) {
+            const int k = grp * kGroup + lane * 4;
+            const float4 gv = ld4_checked(g, k, L, true);
+            const float4 zv = ld4_checked(z, k, L, true);
+            const uint32_t mw = (k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
+            worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
+                                      make_float4(0, 0, 0, 0), mw, acc);
+        }
+    }
+    const double total = block_sum(acc, red);
+    if (threadIdx.x == 0) a.partial[(int64_t)ii * a.Pp + t] = total;
+}
+
+// Scales from the fine tiles' partial sums: tiles of a chunk added in order, then sqrt(sum / L).
+__global__ void k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
+                                int rows, int64_t C, int64_t d, int64_t chunk, int64_t tiles)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)rows * C) return;
+    const int r = (int)(idx / C);
+    const int64_t c = idx % C;
+    const int64_t cbeg = c * chunk;
+    const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
+    const int64_t P = chunk / kFineTile;
+    int64_t t1 = (c + 1) * P;
+    if (t1 > tiles) t1 = tiles;
+    double total = 0.0;
+    for (int64_t t = c * P; t < t1; ++t) total += partial[(int64_t)r * Pp + t];
+    scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
 // Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).
@@ -727,9 +822,10 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
+    int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_stage, off_status, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_status, total;
 };
 
 bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
@@ -758,6 +854,9 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
     L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
+    L->fine_tiles = (chunk % kFineTile == 0) ? (d + kFineTile - 1) / kFineTile : 0;
+    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles, 64);
+    L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
     L->off_stage = take((size_t)L->dz * 4 * 2);
     L->off_status = take(256);
     L->total = o;
@@ -800,6 +899,7 @@ struct apms_ctx {
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
     int* status() { return (int*)(ws + L.off_status); }
+    double* fine_partial(int row) { return (double*)(ws + L.off_fine) + (int64_t)row * L.fine_Pp; }
     double* partial(int row) { return (double*)(ws + L.off_part) + (int64_t)row * L.t.Pp; }   // row n = server
 };
 
@@ -904,8 +1004,43 @@ apms_status launch_finalize(apms_ctx* c, int first_row, int rows, float* scales)
     return launch_check(c, "k_finalize_scales");
 }
 
+bool use_fine_worker(const apms_ctx* c)
+{
+    if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
+    return !c->m_is_fp32 && c->L.fine_tiles > 0;
+}
+
+apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
+{
+    WorkerFineArgs a;
+    a.z = c->z(0); a.dz = c->L.dz;
+    a.B = c->B(0); a.Wp = c->L.Wp;
+    a.s = c->s(0); a.Cp = c->L.Cp;
+    a.partial = c->fine_partial(i0); a.Pp = c->L.fine_Pp;
+    a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.tiles = c->L.fine_tiles;
+    a.i0 = i0; a.ni = ni;
+    a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
+    const int64_t stretches = (a.tiles + kFineRun - 1) / kFineRun;
+    const int64_t blocks = stretches * kFineRun * ni;
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
+    {
+        Timed t(c, APMS_KERNEL_WORKER);
+        k_worker_fine<<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
+        apms_status st = launch_check(c, "k_worker_fine");
+        if (st != APMS_OK) return st;
+        const int64_t total = (int64_t)ni * c->L.C;
+        k_finalize_fine<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0),
+                                                                             c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk, a.tiles);
+        st = launch_check(c, "k_finalize_fine");
+        if (st != APMS_OK) return st;
+    }
+    return APMS_OK;
+}
+
 apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
 {
+    if (use_fine_worker(c)) return launch_worker_fine(c, G, i0, ni);
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
     a.B = c->B(0); a.Wp = c->L.Wp;

@@ -372,6 +372,9 @@ def main(argv=None) -> int:
     m = measure(w, args, rank, world, local_rank, dist, want_adam=args.adam, want_e2e=not args.no_e2e)
     ms_per_step, kernel_ms = m["ms_per_step"], m["kernel_ms"]
     ab = algorithmic_bytes(w.d, w.n, w.chunk)
+    if "apply" not in kernel_ms:          # steps 4-6 ran as one kernel: it moves both kernels' bytes (Bbar is not re-read)
+        ab["server"] = ab["server"] + ab["apply"] - 4 * -(-w.d // 32)
+        ab["step"] = ab["worker"] + ab["server"]
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
     step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * w.n

@@ -88,6 +88,11 @@ __device__ __forceinline__ void st4_checked(float* p, int k, int len, float4 v) 
 __device__ __forceinline__ float signed_scale(float z, float s) { return (z >= 0.0f) ? s : -s; }
 __device__ __forceinline__ float bit_scale(uint32_t bit, float s) { return bit ? s : -s; }
 
+// Model update of one element with the frozen variance (Section 3.3 step 6).
+__device__ __forceinline__ float apply_elem(float x, float v, float q, float lr, float eps) {
+    return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));
+}
+
 // The compression error implied by a stored compensated value and its chunk's scale.
 __device__ __forceinline__ float implied_error(float z, float s) { return __fsub_rn(z, signed_scale(z, s)); }
 
@@ -139,13 +144,17 @@ __device__ __forceinline__ void adam_elem(const AdamArgs& a, float gs, float& m,
     x = __fsub_rn(x, __fdiv_rn(__fmul_rn(a.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), a.eps)));
 }
 
+// One short-lived CTA per 1024 elements (one float4 per thread and stream): the n gradient
+// loads of a thread are independent, and many small CTAs keep more of them in flight than a
+// resident grid-stride loop does.
 __global__ void __launch_bounds__(kThreads)
 k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
 {
-    const int64_t nvec = a.d / 4;
-    for (int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x; q < nvec;
-         q += (int64_t)gridDim.x * kThreads) {
-        const int64_t j = q * 4;
+    const int64_t j = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
+    if (j + 3 < a.d) {
+        float4 m = ld_stream4(a.m + j);
+        float4 v = ld_stream4(a.v + j);
+        float4 x = ld_stream4(a.x + j);
         float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
         for (int i = 0; i < a.n; ++i) {
@@ -153,23 +162,20 @@ k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
             gs.x = __fadd_rn(gs.x, g.x); gs.y = __fadd_rn(gs.y, g.y);
             gs.z = __fadd_rn(gs.z, g.z); gs.w = __fadd_rn(gs.w, g.w);
         }
-        float4 m = *reinterpret_cast<const float4*>(a.m + j);
-        float4 v = *reinterpret_cast<const float4*>(a.v + j);
-        float4 x = *reinterpret_cast<const float4*>(a.x + j);
         adam_elem(a, gs.x, m.x, v.x, x.x); adam_elem(a, gs.y, m.y, v.y, x.y);
         adam_elem(a, gs.z, m.z, v.z, x.z); adam_elem(a, gs.w, m.w, v.w, x.w);
-        *reinterpret_cast<float4*>(a.m + j) = m;
-        *reinterpret_cast<float4*>(a.v + j) = v;
-        *reinterpret_cast<float4*>(a.x + j) = x;
-    }
-    // ragged tail (d not a multiple of 4): one thread per element
-    const int64_t j = nvec * 4 + (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (j < a.d) {
-        float gs = 0.f;
-        for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, G.p[i][j]);
-        float m = a.m[j], v = a.v[j], x = a.x[j];
-        adam_elem(a, gs, m, v, x);
-        a.m[j] = m; a.v[j] = v; a.x[j] = x;
+        st_stream4(a.m + j, m);
+        st_stream4(a.v + j, v);
+        st_stream4(a.x + j, x);
+    } else {
+        // ragged tail (d not a multiple of 4): element by element
+        for (int64_t e = j; e < a.d; ++e) {
+            float gs = 0.f;
+            for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, G.p[i][e]);
+            float m = a.m[e], v = a.v[e], x = a.x[e];
+            adam_elem(a, gs, m, v, x);
+            a.m[e] = m; a.v[e] = v; a.x[e] = x;
+        }
     }
 }
 
@@ -564,17 +570,22 @@ k_server(const ServerArgs a)
 }
 
 // ------------------------------------------------------------------------------------------
-// Server side, staged form: the chunk's zbar and the n workers' sign words stream through a
-// ring of shared-memory stages filled by bulk asynchronous copies (one elected thread issues
-// them, an mbarrier per stage counts the arriving bytes), so that the bytes in flight do not
-// depend on registers or occupancy.  Used when every slab of kSlab elements of a tile starts
-// on a 16-byte boundary in all streams (chunk a multiple of kSlab); other shapes use k_server.
+// Server side, staged form.  One CTA per chunk tile: a producer warp streams the tile through a
+// ring of shared-memory stages with bulk asynchronous copies (an mbarrier per stage counts the
+// arriving bytes, a second one collects the eight consumer warps' releases), so the bytes in
+// flight depend neither on registers nor on occupancy, and no CTA-wide barrier sits in the loop.
+// When the tile is the whole chunk, the CTA goes on to steps 5-6 for the same chunk (its new
+// scale is known once the eight consumer warps have met): v and x travel through the same ring
+// while other CTAs of the SM are still in their arithmetic-bound averaging phase.
+// Needs every slab of kSlab elements to start on a 16-byte boundary in all streams, i.e.
+// chunks that are multiples of kSlab; other shapes use k_server and k_apply.
 
-constexpr int kSlab = 2048;                      // elements per stage: 8 KiB of zbar + n x 256 B of sign words
-constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per warp
-constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker
+constexpr int kSlab = 2048;                      // elements per ring stage
+constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per consumer warp
+constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker and slab
 constexpr int kStages = 4;
-constexpr uint32_t kWaitLimit = 1u << 22;        // polls of one mbarrier before the kernel gives up
+constexpr int kStagedThreads = kThreads + 32;    // eight consumer warps + one producer warp
+constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about a second of SM clocks
 
 enum { DEVICE_OK = 0, DEVICE_WAIT_TIMEOUT = 1 };
 
@@ -588,6 +599,10 @@ __device__ __forceinline__ void mbar_fence_init()
 {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
@@ -595,18 +610,21 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 {
     uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 1000;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return done != 0;
 }
-// Bounded wait: false when the phase did not complete within kWaitLimit polls.
+// Bounded wait: false when the phase did not complete within kWaitCycles.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
 {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 32) __nanosleep(32);
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int k = 0; k < 32; ++k)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > kWaitCycles) return false;
     }
-    return false;
 }
 // Global -> this CTA's shared memory; 16-byte aligned addresses, size a multiple of 16 bytes.
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
@@ -614,137 +632,210 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
+// Barrier among the 256 consumer threads only (the producer warp never joins it).
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 struct ServerStagedArgs {
     ServerArgs a;
     int* status;          // device status word: set when a bounded wait gave up
     float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
+    const float* v; float* x; float lr, eps;     // steps 5-6, used by the fused form only
 };
 
-__device__ __forceinline__ size_t staged_stage_bytes(int n) { return (size_t)kSlab * 4 + (size_t)n * kSlabWords * 4; }
+// Bytes of one ring stage: a slab of zbar plus n rows of sign words, or (fused form) a slab of v and of x.
+__host__ __device__ __forceinline__ size_t staged_stage_bytes(int n, bool fused)
+{
+    const size_t server = (size_t)kSlab * 4 + (size_t)n * kSlabWords * 4;
+    const size_t apply = (size_t)kSlab * 8;
+    return (fused && apply > server) ? apply : server;
+}
 
-__global__ void __launch_bounds__(kThreads, 3)
+// Sum over the workers, in worker order, of +-s_i for the lane's 2 x 4 elements of one slab.
+// NT > 0: the number of workers is the compile-time constant NT (fully unrolled).
+template <int NT>
+__device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r0, const uint32_t* __restrict__ r1,
+                                                  const uint32_t* __restrict__ neg_s, int n, int sh,
+                                                  float2& s01, float2& s23, float2& t01, float2& t23)
+{
+    const int nn = NT > 0 ? NT : n;
+#pragma unroll(NT > 0 ? NT : 4)
+    for (int i = 0; i < nn; ++i) {
+        const uint32_t ns = neg_s[i];
+        // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
+        const uint32_t y0 = r0[i * kSlabWords] << (28 - sh);
+        const uint32_t y1 = r1[i * kSlabWords] << (28 - sh);
+        float2 q;
+        q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns);
+        s01 = __fadd2_rn(s01, q);
+        q.x = __uint_as_float(((y0 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y0 & 0x80000000u) ^ ns);
+        s23 = __fadd2_rn(s23, q);
+        q.x = __uint_as_float(((y1 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y1 << 2) & 0x80000000u) ^ ns);
+        t01 = __fadd2_rn(t01, q);
+        q.x = __uint_as_float(((y1 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y1 & 0x80000000u) ^ ns);
+        t23 = __fadd2_rn(t23, q);
+    }
+}
+
+template <int NT, bool FUSED>
+__global__ void __launch_bounds__(kStagedThreads, 3)
 k_server_staged(const ServerStagedArgs sa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const ServerArgs& a = sa.a;
     __shared__ double red[kWarps];
-    __shared__ uint64_t full[kStages];
+    __shared__ uint64_t full[kStages], empty[kStages];
     __shared__ uint32_t neg_s[APMS_MAX_WORKERS];      // bit patterns of -s_i of this chunk
+    __shared__ uint32_t nb[kTileMax / 32];            // the tile's new sign words
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const Item it = decode_item(a.t, (int64_t)blockIdx.x);
     const int L = it.L;
-    const int n = a.n;
-    const size_t stage_bytes = staged_stage_bytes(n);
+    const int n = NT > 0 ? NT : a.n;
+    const size_t stage_bytes = staged_stage_bytes(n, FUSED);
     const int nslabs = (L + kSlab - 1) / kSlab;
-    const float* __restrict__ zb_g = a.zbar + it.base;
-    const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
-    uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+    const int njobs = FUSED ? 2 * nslabs : nslabs;    // jobs nslabs.. are the slabs of v and x
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
         failed = 0;
         mbar_fence_init();
     }
-    for (int i = threadIdx.x; i < n; i += kThreads)
+    for (int i = threadIdx.x; i < n; i += kStagedThreads)
         neg_s[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
     const float S_old = a.Sbar[it.c];
     __syncthreads();
 
-    // producer: slab j into stage j % kStages (only whole 16-byte pieces that hold live elements)
-    auto issue = [&](int j) {
-        const int st = j % kStages;
-        unsigned char* base = smem + (size_t)st * stage_bytes;
-        const int left = L - j * kSlab;
-        const int live = left < kSlab ? left : kSlab;
-        const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
-        const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
-        mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
-        bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
-        uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
-        for (int i = 0; i < n; ++i)
-            bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
-    };
-    if (threadIdx.x == 0)
-        for (int j = 0; j < kStages && j < nslabs; ++j) issue(j);
-
-    const int sh = 4 * (lane & 7);
-    const int wl = lane >> 3;
-    double acc = 0.0;
-    int j = 0;
-    for (; j < nslabs; ++j) {
-        const int st = j % kStages;
-        if (!mbar_wait(&full[st], (uint32_t)(j / kStages) & 1u)) failed = 1;     // nothing of this slab is stored then
-        const unsigned char* base = smem + (size_t)st * stage_bytes;
-        const float* zs = reinterpret_cast<const float*>(base);
-        const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
-        const int g0 = warp, g1 = warp + kWarps;                     // this warp's two groups of the slab
-        const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
-        const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
-        float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
-        const uint32_t* r0 = rows + g0 * 4 + wl;
-        const uint32_t* r1 = rows + g1 * 4 + wl;
-#pragma unroll 4
-        for (int i = 0; i < n; ++i) {
-            const uint32_t ns = neg_s[i];
-            // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
-            const uint32_t y0 = r0[i * kSlabWords] << (28 - sh);
-            const uint32_t y1 = r1[i * kSlabWords] << (28 - sh);
-            float2 q;
-            q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns);
-            s01 = __fadd2_rn(s01, q);
-            q.x = __uint_as_float(((y0 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y0 & 0x80000000u) ^ ns);
-            s23 = __fadd2_rn(s23, q);
-            q.x = __uint_as_float(((y1 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y1 << 2) & 0x80000000u) ^ ns);
-            t01 = __fadd2_rn(t01, q);
-            q.x = __uint_as_float(((y1 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y1 & 0x80000000u) ^ ns);
-            t23 = __fadd2_rn(t23, q);
+    if (warp == kWarps) {
+        // ---- producer warp: one lane feeds the ring (only whole 16-byte pieces that hold live elements)
+        if (lane == 0) {
+            const float* __restrict__ zb_g = a.zbar + it.base;
+            const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
+            int issued = 0;
+            for (int q = 0; q < njobs; ++q) {
+                const int st = q % kStages;
+                if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; break; }
+                unsigned char* base = smem + (size_t)st * stage_bytes;
+                const int j = q < nslabs ? q : q - nslabs;
+                const int left = L - j * kSlab;
+                const int live = left < kSlab ? left : kSlab;
+                const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
+                if (q < nslabs) {
+                    const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
+                    mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
+                    bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
+                    uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
+                    for (int i = 0; i < n; ++i)
+                        bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
+                } else {
+                    mbar_arrive_expect_tx(&full[st], 2 * zbytes);
+                    bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                    bulk_load(base + (size_t)kSlab * 4, sa.x + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                }
+                issued = q + 1;
+            }
+            if (failed) {
+                // give the copies still in flight a bounded chance to land before shared memory is released
+                const int first = issued > kStages ? issued - kStages : 0;
+                for (int q = first; q < issued; ++q) mbar_wait(&full[q % kStages], (uint32_t)(q / kStages) & 1u);
+            }
         }
-        __syncthreads();                                              // the stage has been read by everyone
-        if (failed) break;
-        if (threadIdx.x == 0 && j + kStages < nslabs) issue(j + kStages);
-
+    } else {
+        // ---- consumer warps: two 128-element groups of every slab each
+        const int sh = 4 * (lane & 7);
+        const int wl = lane >> 3;
+        const int g0 = warp, g1 = warp + kWarps;
+        double acc = 0.0;
+        bool ok = true;
+        for (int j = 0; j < nslabs; ++j) {
+            const int st = j % kStages;
+            if (!mbar_wait(&full[st], (uint32_t)(j / kStages) & 1u)) { failed = 1; ok = false; break; }
+            const unsigned char* base = smem + (size_t)st * stage_bytes;
+            const float* zs = reinterpret_cast<const float*>(base);
+            const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
+            const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
+            const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
+            float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
+            signed_scale_sums<NT>(rows + g0 * 4 + wl, rows + g1 * 4 + wl, neg_s, n, sh, s01, s23, t01, t23);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int grp = j * kSlabGroups + (u ? g1 : g0);
-            const int k = grp * kGroup + lane * 4;
-            const float4 zo4 = u ? zo1 : zo0;
-            const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
-            const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
-            float zn[4];
-            uint32_t nibble = 0;
+            for (int u = 0; u < 2; ++u) {
+                const int grp = j * kSlabGroups + (u ? g1 : g0);
+                const int k = grp * kGroup + lane * 4;
+                const float4 zo4 = u ? zo1 : zo0;
+                const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+                const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
+                float zn[4];
+                uint32_t nibble = 0;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
-                zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
-                if (k + e < L) {
-                    const double zd = (double)zn[e];
-                    acc = fma(zd, zd, acc);
-                    nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                for (int e = 0; e < 4; ++e) {
+                    const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
+                    zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+                    if (k + e < L) {
+                        const double zd = (double)zn[e];
+                        acc = fma(zd, zd, acc);
+                        nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                    }
+                }
+                st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                const uint32_t word = pack_group_words(nibble, lane);
+                if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) red[warp] = acc;
+        consumer_barrier();                            // partial sums and sign words of the tile are in shared memory
+        double total = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) total += red[w];
+        if (failed) ok = false;
+        if (FUSED) {
+            // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
+            const float S_new = (float)sqrt(total / (double)it.Lc);
+            if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
+            for (int j = 0; ok && j < nslabs; ++j) {
+                const int q = nslabs + j;
+                const int st = q % kStages;
+                if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
+                const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
+                const float* xs = vs + kSlab;
+                float4 vv[2], xx[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
+                    xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[st]);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int grp = j * kSlabGroups + (u ? g1 : g0);
+                    const int k = grp * kGroup + lane * 4;
+                    const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                    xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib & 1u, S_new), sa.lr, sa.eps);
+                    xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib & 2u, S_new), sa.lr, sa.eps);
+                    xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib & 4u, S_new), sa.lr, sa.eps);
+                    xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib & 8u, S_new), sa.lr, sa.eps);
+                    st4_checked(sa.x + it.base, k, L, xx[u]);
                 }
             }
-            st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
-            const uint32_t word = pack_group_words(nibble, lane);
-            const int wk = grp * 4 + wl;
-            if ((lane & 7) == 0 && wk * 32 < L) ob[wk] = word;
+        } else if (ok && threadIdx.x == 0) {
+            if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+            else a.partial[it.c * a.t.P + it.p] = total;
+        }
+        // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
+        if (ok) {
+            uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+            const int nwords = (L + 31) / 32;
+            for (int w4 = threadIdx.x * 4; w4 < nwords; w4 += kThreads * 4) {
+                if (w4 + 3 < nwords) *reinterpret_cast<uint4*>(ob + w4) = *reinterpret_cast<const uint4*>(nb + w4);
+                else for (int w = w4; w < nwords; ++w) ob[w] = nb[w];
+            }
         }
     }
-    if (failed) {
-        // give the copies still in flight a bounded chance to land before the CTA's shared memory is released
-        if (threadIdx.x == 0) {
-            const int last = (j + kStages < nslabs) ? j + kStages : nslabs;
-            for (int q = j; q < last; ++q) mbar_wait(&full[q % kStages], (uint32_t)(q / kStages) & 1u);
-            atomicExch(sa.status, DEVICE_WAIT_TIMEOUT);
-        }
-        return;
-    }
-    const double total = block_sum(acc, red);
-    if (threadIdx.x == 0) {
-        if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
-        else a.partial[it.c * a.t.P + it.p] = total;
-    }
+    __syncthreads();                                   // every warp has left its loops; shared memory may go
+    if (threadIdx.x == 0 && failed) atomicExch(sa.status, DEVICE_WAIT_TIMEOUT);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -752,18 +843,15 @@ k_server_staged(const ServerStagedArgs sa)
 // form) and the model moves with the frozen variance (Section 3.3 steps 5-6).
 // One CTA per 8192 consecutive elements, whatever the chunk length.
 
-constexpr int kApplyTile = 8192;
+constexpr int kApplyTile = 4096;
+constexpr int kApplyU = kApplyTile / (kThreads * 4);
 
 struct ApplyArgs {
     const uint32_t* Bbar; const float* Sbar; const float* v; float* x;
     int64_t d; int64_t chunk; float lr, eps;
 };
 
-__device__ __forceinline__ float apply_elem(float x, float v, float q, float lr, float eps) {
-    return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));
-}
-
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads)
 k_apply(const ApplyArgs a)
 {
     const int64_t base = (int64_t)blockIdx.x * kApplyTile;
@@ -776,7 +864,30 @@ k_apply(const ApplyArgs a)
     const float* __restrict__ v = a.v + base;
     float* __restrict__ x = a.x + base;
     const float* __restrict__ Sb = a.Sbar + c0;
-#pragma unroll 2
+    if (L == kApplyTile) {
+        float4 vv[kApplyU], xx[kApplyU];
+        uint32_t nib[kApplyU];
+        float S[kApplyU];
+#pragma unroll
+        for (int u = 0; u < kApplyU; ++u) {
+            const int k = (u * kThreads + threadIdx.x) * 4;
+            vv[u] = ld_stream4(v + k);
+            xx[u] = ld_stream4(x + k);
+            nib[u] = bits[k >> 5] >> (k & 31);
+            const uint32_t rel = off0 + (uint32_t)k;
+            S[u] = Sb[rel < chunk32 ? 0u : rel / chunk32];
+        }
+#pragma unroll
+        for (int u = 0; u < kApplyU; ++u) {
+            const int k = (u * kThreads + threadIdx.x) * 4;
+            xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib[u] & 1u, S[u]), a.lr, a.eps);
+            xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib[u] & 2u, S[u]), a.lr, a.eps);
+            xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib[u] & 4u, S[u]), a.lr, a.eps);
+            xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib[u] & 8u, S[u]), a.lr, a.eps);
+            st_stream4(x + k, xx[u]);
+        }
+        return;
+    }
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
         const uint32_t rel = off0 + (uint32_t)k;
         const float S = Sb[rel < chunk32 ? 0u : rel / chunk32];
@@ -882,7 +993,6 @@ struct apms_ctx {
     int sms;
     bool timing;
     apms_team_mode team_mode;
-    bool staged_ready;       // the staged server kernel's shared-memory limit has been raised
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
@@ -1070,8 +1180,32 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
     return APMS_OK;
 }
 
+// Launch of one instantiation of the staged server kernel (its shared-memory limit is raised first).
+template <int NT, bool FUSED>
+cudaError_t launch_staged(const ServerStagedArgs& sa, unsigned blocks, size_t smem, cudaStream_t stream)
+{
+    cudaError_t e = cudaFuncSetAttribute(k_server_staged<NT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_server_staged<NT, FUSED><<<blocks, kStagedThreads, smem, stream>>>(sa);
+    return cudaSuccess;
+}
+
+template <bool FUSED>
+cudaError_t launch_staged_n(const ServerStagedArgs& sa, unsigned blocks, size_t smem, cudaStream_t stream)
+{
+    switch (sa.a.n) {        // the usual worker counts get a fully unrolled sum; any other count the generic loop
+    case 2:  return launch_staged<2, FUSED>(sa, blocks, smem, stream);
+    case 4:  return launch_staged<4, FUSED>(sa, blocks, smem, stream);
+    case 8:  return launch_staged<8, FUSED>(sa, blocks, smem, stream);
+    case 16: return launch_staged<16, FUSED>(sa, blocks, smem, stream);
+    case 32: return launch_staged<32, FUSED>(sa, blocks, smem, stream);
+    default: return launch_staged<0, FUSED>(sa, blocks, smem, stream);
+    }
+}
+
 apms_status launch_server_and_apply(apms_ctx* c)
 {
+    bool applied = false;      // steps 5-6 already done by the fused server kernel
     {
         ServerArgs a;
         a.B = c->B(0); a.Wp = c->L.Wp; a.s = c->s(0); a.Cp = c->L.Cp;
@@ -1082,18 +1216,22 @@ apms_status launch_server_and_apply(apms_ctx* c)
         const bool warp_teams = !staged && use_warp_teams(c, a.items);
         const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
         if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
-        const size_t staged_smem = (size_t)kStages * ((size_t)kSlab * 4 + (size_t)a.n * kSlabWords * 4);
-        if (staged && !c->staged_ready) {
-            APMS_CUDA(c, cudaFuncSetAttribute(k_server_staged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged_smem));
-            c->staged_ready = true;
-        }
         {
             Timed t(c, APMS_KERNEL_SERVER);
             if (staged) {
+                const bool fused = c->L.t.P == 1;        // the CTA sees the whole chunk, so it knows the new scale
                 ServerStagedArgs sa;
                 sa.a = a; sa.status = c->status();
                 sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
-                k_server_staged<<<(unsigned)blocks, kThreads, staged_smem, c->stream>>>(sa);
+                sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
+                const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
+                cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)blocks, smem, c->stream)
+                                      : launch_staged_n<false>(sa, (unsigned)blocks, smem, c->stream);
+                if (e != cudaSuccess) {
+                    snprintf(c->err, sizeof c->err, "setting up k_server_staged failed: %s", cudaGetErrorString(e));
+                    return APMS_ERR_CUDA;
+                }
+                applied = fused;
             }
             else if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
             else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
@@ -1105,7 +1243,7 @@ apms_status launch_server_and_apply(apms_ctx* c)
             if (st != APMS_OK) return st;
         }
     }
-    {
+    if (!applied) {
         ApplyArgs a;
         a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
@@ -1170,7 +1308,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
-    c->team_mode = APMS_TEAM_AUTO; c->staged_ready = false;
+    c->team_mode = APMS_TEAM_AUTO;
     *out = c;
     return APMS_OK;
 }
@@ -1226,7 +1364,9 @@ apms_status apms_warmup_step(apms_ctx* c, const float* const* grads_dev)
     a.bc2 = (float)(1.0 - pow((double)c->beta2, (double)c->t));
     a.lr = c->lr; a.eps = c->eps; a.nf = (float)c->L.n;
     Timed t(c, APMS_KERNEL_WARMUP_ADAM);
-    k_warmup_adam<<<grid_for(c, (c->L.d + 3) / 4, 8), kThreads, 0, c->stream>>>(G, a);
+    const int64_t adam_blocks = (c->L.d + (int64_t)kThreads * 4 - 1) / ((int64_t)kThreads * 4);
+    if (adam_blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "d too large for one launch");
+    k_warmup_adam<<<(unsigned)adam_blocks, kThreads, 0, c->stream>>>(G, a);
     return launch_check(c, "k_warmup_adam");
 }
 

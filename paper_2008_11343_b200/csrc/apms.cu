@@ -26,6 +26,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 #include <math.h>
 #include <mutex>
@@ -275,7 +276,7 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
     const uint32_t word = pack_group_words(nibble, lane);
     if ((lane & 7) == 0) {
         const int wk = grp * 4 + (lane >> 3);
-        if (!CHECKED || wk * 32 < L) obits[wk] = word;
+        if (!CHECKED || wk * 32 < L) __stcs(obits + wk, word);     // streaming: a plain store here costs ~4 % of the kernel
     }
 }
 
@@ -347,13 +348,15 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 // binary64 sum of squares written to a partial-sum array that k_finalize_fine adds up per chunk
 // in tile order.  Short-lived CTAs that each touch 16 KiB of every stream once keep DRAM pages
 // and the memory pipeline busier than long-running warps that each follow their own stream.
-// Launch order: runs of kFineRun consecutive tiles of one worker, then the same tiles of the next
-// worker, so that every stream is read in long sequential pieces while the n workers of a stretch
-// still meet its momentum bits in L2.
+// Warp w owns the tile's groups 4w..4w+3 (512 consecutive elements), so its 16 momentum words
+// are one 64-byte load handed round by shuffles and its 16 new sign words one 64-byte store.
+// Launch order: runs of `run` consecutive tiles of one worker, then the same tiles of the next
+// worker: every stream is read in long sequential pieces (measured: the longer the better for
+// DRAM), while the momentum bits of a run (run * 512 bytes) stay in L2 for the other workers.
 
 constexpr int kFineTile = 4096;           // 256 threads x 4 x (4 floats)
 constexpr int kFineU = kFineTile / (kThreads * 4);
-constexpr int kFineRun = 64;
+constexpr int kFineRunDefault = 4096;
 
 struct WorkerFineArgs {
     float* z; int64_t dz;
@@ -362,20 +365,20 @@ struct WorkerFineArgs {
     double* partial; int64_t Pp;      // ni rows of `tiles` partial sums, row stride Pp
     const uint32_t* Bbar; const float* Sbar;
     int64_t d, chunk, tiles;
-    int i0, ni;
+    int i0, ni, run;
     float beta1, omb1;
 };
 
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
     __shared__ double red[kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t per_stretch = (int64_t)a.ni * kFineRun;
+    const int64_t per_stretch = (int64_t)a.ni * a.run;
     const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
     const int rem = (int)((int64_t)blockIdx.x - stretch * per_stretch);
-    const int ii = rem / kFineRun;
-    const int64_t t = stretch * kFineRun + (rem % kFineRun);
+    const int ii = rem / a.run;
+    const int64_t t = stretch * a.run + (rem - ii * a.run);
     if (t >= a.tiles) return;                                  // whole CTA: the last stretch may be short
     const int i = a.i0 + ii;
     const int64_t base = t * kFineTile;
@@ -391,19 +394,37 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     double acc = 0.0;
     if (L == kFineTile) {
         float4 gv[kFineU], zv[kFineU];
-        uint32_t mw[kFineU];
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
-            const int grp = u * kWarps + warp;
-            const int k = grp * kGroup + lane * 4;
+            const int k = (warp * kFineU + u) * kGroup + lane * 4;
             gv[u] = ld_stream4(g + k);
             zv[u] = ld_stream4(z + k);
-            mw[u] = mbits[grp * 4 + (lane >> 3)];
         }
+        const uint32_t mine = (lane < 4 * kFineU) ? mbits[warp * 4 * kFineU + lane] : 0u;
+        uint32_t outw = 0;
 #pragma unroll
-        for (int u = 0; u < kFineU; ++u)
-            worker_group<false, false>(a.beta1, a.omb1, z, obits, u * kWarps + warp, lane, L, s_old, Sbar,
-                                       gv[u], zv[u], make_float4(0, 0, 0, 0), mw[u], acc);
+        for (int u = 0; u < kFineU; ++u) {
+            const int k = (warp * kFineU + u) * kGroup + lane * 4;
+            const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
+            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+            const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
+            float zn[4];
+            uint32_t nibble = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
+                const float mi = __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
+                zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
+                const double zd = (double)zn[e];
+                acc = fma(zd, zd, acc);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
+            st_stream4(z + k, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+            const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
+            if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
+        }
+        if (lane < 4 * kFineU) __stcs(obits + warp * 4 * kFineU + lane, outw);
     } else {
         const int ngroups = (L + kGroup - 1) / kGroup;
         for (int grp = warp; grp < ngroups; grp += kWarps) {
@@ -993,6 +1014,7 @@ struct apms_ctx {
     int sms;
     bool timing;
     apms_team_mode team_mode;
+    int fine_run;            // tiles of one worker launched back to back in the fine worker form
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
@@ -1131,8 +1153,9 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
     a.d = c->L.d; a.chunk = c->L.chunk; a.tiles = c->L.fine_tiles;
     a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
-    const int64_t stretches = (a.tiles + kFineRun - 1) / kFineRun;
-    const int64_t blocks = stretches * kFineRun * ni;
+    a.run = c->fine_run;
+    const int64_t stretches = (a.tiles + a.run - 1) / a.run;
+    const int64_t blocks = stretches * a.run * ni;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
     {
         Timed t(c, APMS_KERNEL_WORKER);
@@ -1309,6 +1332,9 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
+    c->fine_run = kFineRunDefault;
+    if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
+    if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
     *out = c;
     return APMS_OK;
 }

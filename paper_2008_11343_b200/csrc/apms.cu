@@ -343,26 +343,28 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
     }
 }
 
-// Worker side, fine-tiled form (steady state, chunk a multiple of kFineTile): one CTA per
-// (worker, 4096-element tile), every load of the tile issued before the first use, the tile's
-// binary64 sum of squares written to a partial-sum array that k_finalize_fine adds up per chunk
-// in tile order.  Short-lived CTAs that each touch 16 KiB of every stream once keep DRAM pages
-// and the memory pipeline busier than long-running warps that each follow their own stream.
-// Warp w owns the tile's groups 4w..4w+3 (512 consecutive elements), so its 16 momentum words
-// are one 64-byte load handed round by shuffles and its 16 new sign words one 64-byte store.
+// Worker side, fine-tiled form (steady state, chunk a multiple of kFineSub): one CTA per
+// (worker, 4096-element tile), every load of the tile issued before the first use.  Short-lived
+// CTAs that each touch 16 KiB of every stream once keep DRAM pages and the memory pipeline busier
+// than long-running warps that each follow their own stream.
+// Warp w owns the tile's groups 4w..4w+3 (kFineSub = 512 consecutive elements, all of one chunk),
+// so its 16 momentum words are one 64-byte load handed round by shuffles, its 16 new sign words
+// one 64-byte store, and its binary64 sum of squares one slot of a partial-sum array that
+// k_finalize_fine adds up per chunk in element order: the kernel has no barrier at all.
 // Launch order: runs of `run` consecutive tiles of one worker, then the same tiles of the next
 // worker: every stream is read in long sequential pieces (measured: the longer the better for
 // DRAM), while the momentum bits of a run (run * 512 bytes) stay in L2 for the other workers.
 
 constexpr int kFineTile = 4096;           // 256 threads x 4 x (4 floats)
 constexpr int kFineU = kFineTile / (kThreads * 4);
+constexpr int kFineSub = kFineTile / kWarps;      // elements per warp = per partial sum
 constexpr int kFineRunDefault = 4096;
 
 struct WorkerFineArgs {
     float* z; int64_t dz;
     uint32_t* B; int64_t Wp;
     const float* s; int64_t Cp;       // the scales of the previous step (read only here)
-    double* partial; int64_t Pp;      // ni rows of `tiles` partial sums, row stride Pp
+    double* partial; int64_t Pp;      // ni rows of tiles * kWarps partial sums, row stride Pp
     const uint32_t* Bbar; const float* Sbar;
     int64_t d, chunk, tiles;
     int i0, ni, run;
@@ -372,7 +374,6 @@ struct WorkerFineArgs {
 __global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
-    __shared__ double red[kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t per_stretch = (int64_t)a.ni * a.run;
     const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
@@ -381,10 +382,15 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     const int64_t t = stretch * a.run + (rem - ii * a.run);
     if (t >= a.tiles) return;                                  // whole CTA: the last stretch may be short
     const int i = a.i0 + ii;
-    const int64_t base = t * kFineTile;
-    const int64_t c = base / a.chunk;
+    const int64_t base = t * kFineTile + (int64_t)warp * kFineSub;     // this warp's 512 elements
+    double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + t * kWarps + warp;
     const int64_t left = a.d - base;
-    const int L = (int)(left < kFineTile ? left : kFineTile);
+    if (left <= 0) {                                           // past the end of the vector
+        if (lane == 0) *slot = 0.0;
+        return;
+    }
+    const int L = (int)(left < kFineSub ? left : kFineSub);
+    const int64_t c = base / a.chunk;
     const float* __restrict__ g = G.p[ii] + base;
     float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
     const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
@@ -392,19 +398,17 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     const float s_old = a.s[(int64_t)i * a.Cp + c];
     const float Sbar = a.Sbar[c];
     double acc = 0.0;
-    if (L == kFineTile) {
+    if (L == kFineSub) {
         float4 gv[kFineU], zv[kFineU];
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
-            const int k = (warp * kFineU + u) * kGroup + lane * 4;
-            gv[u] = ld_stream4(g + k);
-            zv[u] = ld_stream4(z + k);
+            gv[u] = ld_stream4(g + u * kGroup + lane * 4);
+            zv[u] = ld_stream4(z + u * kGroup + lane * 4);
         }
-        const uint32_t mine = (lane < 4 * kFineU) ? mbits[warp * 4 * kFineU + lane] : 0u;
+        const uint32_t mine = (lane < 4 * kFineU) ? mbits[lane] : 0u;
         uint32_t outw = 0;
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
-            const int k = (warp * kFineU + u) * kGroup + lane * 4;
             const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
             const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
             const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
@@ -419,15 +423,15 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
                 acc = fma(zd, zd, acc);
                 nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
             }
-            st_stream4(z + k, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
             const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
             const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
             if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
         }
-        if (lane < 4 * kFineU) __stcs(obits + warp * 4 * kFineU + lane, outw);
+        if (lane < 4 * kFineU) __stcs(obits + lane, outw);
     } else {
         const int ngroups = (L + kGroup - 1) / kGroup;
-        for (int grp = warp; grp < ngroups; grp += kWarps) {
+        for (int grp = 0; grp < ngroups; ++grp) {
             const int k = grp * kGroup + lane * 4;
             const float4 gv = ld4_checked(g, k, L, true);
             const float4 zv = ld4_checked(z, k, L, true);
@@ -436,13 +440,14 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
                                       make_float4(0, 0, 0, 0), mw, acc);
         }
     }
-    const double total = block_sum(acc, red);
-    if (threadIdx.x == 0) a.partial[(int64_t)ii * a.Pp + t] = total;
+    acc = warp_sum(acc);
+    if (lane == 0) *slot = acc;
 }
 
-// Scales from the fine tiles' partial sums: tiles of a chunk added in order, then sqrt(sum / L).
+// Scales from the fine form's partial sums (one per 512 elements): a chunk's slots added in
+// element order, then sqrt(sum / L).
 __global__ void k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
-                                int rows, int64_t C, int64_t d, int64_t chunk, int64_t tiles)
+                                int rows, int64_t C, int64_t d, int64_t chunk)
 {
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (int64_t)rows * C) return;
@@ -450,11 +455,9 @@ __global__ void k_finalize_fine(const double* __restrict__ partial, int64_t Pp, 
     const int64_t c = idx % C;
     const int64_t cbeg = c * chunk;
     const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
-    const int64_t P = chunk / kFineTile;
-    int64_t t1 = (c + 1) * P;
-    if (t1 > tiles) t1 = tiles;
+    const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
     double total = 0.0;
-    for (int64_t t = c * P; t < t1; ++t) total += partial[(int64_t)r * Pp + t];
+    for (int64_t q = q0; q < q1; ++q) total += partial[(int64_t)r * Pp + q];
     scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
@@ -986,8 +989,8 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
     L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
-    L->fine_tiles = (chunk % kFineTile == 0) ? (d + kFineTile - 1) / kFineTile : 0;
-    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles, 64);
+    L->fine_tiles = (chunk % kFineSub == 0) ? (d + kFineTile - 1) / kFineTile : 0;
+    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles * kWarps, 64);
     L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
     L->off_stage = take((size_t)L->dz * 4 * 2);
     L->off_status = take(256);
@@ -1164,7 +1167,7 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
         if (st != APMS_OK) return st;
         const int64_t total = (int64_t)ni * c->L.C;
         k_finalize_fine<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0),
-                                                                             c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk, a.tiles);
+                                                                             c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk);
         st = launch_check(c, "k_finalize_fine");
         if (st != APMS_OK) return st;
     }

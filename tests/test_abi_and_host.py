@@ -40,6 +40,7 @@ def test_workspace_bytes_is_pure_and_covers_the_state(lib):
     nbytes = B.apms_workspace_bytes(d, n, chunk)
     C, W = -(-d // chunk), -(-d // 32)
     need = 4 * d * (n + 4 + 2) + 4 * W * (n + 1) + 4 * C * (n + 1)
+    need += 8 * n * -(-d // 512)                     # one binary64 partial sum per worker and 512 elements
     assert need <= nbytes <= need * 1.001 + (1 << 20)
     assert B.apms_workspace_bytes(d, n, chunk) == nbytes
     for bad in [(0, 1, 32), (1, 0, 32), (1, 65, 32), (1, 1, 31), (1, 1, 0), (1, 1, -32)]:

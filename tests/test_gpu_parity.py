@@ -26,7 +26,8 @@ EDGE = [(1, 1, 32), (31, 2, 32), (32, 2, 32), (33, 3, 32), (127, 4, 128), (128, 
 # shapes for the staged forms (chunk a multiple of 2048): one slab, many slabs, ragged last slab and chunk,
 # split chunks, n not a power of two (IEEE division instead of the exact multiplication by 1/n), n = 64
 STAGED = [(2048, 1, 2048), (10 * 2048 + 1, 5, 2048), (6144 * 3 + 33, 7, 6144), (3 * 131072 + 4099, 3, 131072),
-          (8 * 32768 + 23552, 16, 32768), (2 * 4096 + 2047, 64, 4096), (65536 + 2049, 2, 65536)]
+          (8 * 32768 + 23552, 16, 32768), (2 * 4096 + 2047, 64, 4096), (65536 + 2049, 2, 65536),
+          (3 * 512 + 100, 3, 512), (7 * 1536 + 511, 2, 1536), (9 * 4096 + 513, 4, 1024)]
 
 
 @pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP, B.TEAM_AUTO, B.TEAM_STAGED],

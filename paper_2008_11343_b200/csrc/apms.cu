@@ -608,6 +608,7 @@ constexpr int kSlab = 2048;                      // elements per ring stage
 constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per consumer warp
 constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker and slab
 constexpr int kStages = 4;
+constexpr int64_t kStagedSpanElems = 32768;   // a CTA of the fused form walks enough chunks to stream about this many elements
 constexpr int kStagedThreads = kThreads + 32;    // eight consumer warps + one producer warp
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about a second of SM clocks
 
@@ -664,6 +665,7 @@ struct ServerStagedArgs {
     int* status;          // device status word: set when a bounded wait gave up
     float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
     const float* v; float* x; float lr, eps;     // steps 5-6, used by the fused form only
+    int span;             // chunks per CTA of the fused form
 };
 
 // Bytes of one ring stage: a slab of zbar plus n rows of sign words, or (fused form) a slab of v and of x.
@@ -700,7 +702,11 @@ __device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r
     }
 }
 
-template <int NT, bool FUSED>
+// A CTA of the fused form walks `span` consecutive chunks (short chunks are grouped so that a CTA
+// still streams about 32768 elements and the ring never drains between chunks); the unfused form
+// (chunks cut into tiles) handles one tile.  Jobs are numbered across the CTA's whole walk: per
+// chunk first its server slabs, then (fused) its slabs of v and x; job q uses stage q % kStages.
+template <int NT, bool FUSED, bool MULTI>
 __global__ void __launch_bounds__(kStagedThreads, 3)
 k_server_staged(const ServerStagedArgs sa)
 {
@@ -708,60 +714,62 @@ k_server_staged(const ServerStagedArgs sa)
     const ServerArgs& a = sa.a;
     __shared__ double red[kWarps];
     __shared__ uint64_t full[kStages], empty[kStages];
-    __shared__ uint32_t neg_s[APMS_MAX_WORKERS];      // bit patterns of -s_i of this chunk
-    __shared__ uint32_t nb[kTileMax / 32];            // the tile's new sign words
+    __shared__ uint32_t neg_s[2][APMS_MAX_WORKERS];   // bit patterns of -s_i, double-buffered over the walk
+    __shared__ uint32_t nb[kTileMax / 32];            // the current tile's new sign words
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const Item it = decode_item(a.t, (int64_t)blockIdx.x);
-    const int L = it.L;
     const int n = NT > 0 ? NT : a.n;
     const size_t stage_bytes = staged_stage_bytes(n, FUSED);
-    const int nslabs = (L + kSlab - 1) / kSlab;
-    const int njobs = FUSED ? 2 * nslabs : nslabs;    // jobs nslabs.. are the slabs of v and x
+    const int span = MULTI ? sa.span : 1;                  // MULTI = false: one item, the walk's loops fold away
+    const int64_t item0 = (int64_t)blockIdx.x * span;
+    const int nitems = MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
         failed = 0;
         mbar_fence_init();
     }
-    for (int i = threadIdx.x; i < n; i += kStagedThreads)
-        neg_s[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
-    const float S_old = a.Sbar[it.c];
     __syncthreads();
 
     if (warp == kWarps) {
         // ---- producer warp: one lane feeds the ring (only whole 16-byte pieces that hold live elements)
         if (lane == 0) {
-            const float* __restrict__ zb_g = a.zbar + it.base;
-            const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
-            int issued = 0;
-            for (int q = 0; q < njobs; ++q) {
-                const int st = q % kStages;
-                if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; break; }
-                unsigned char* base = smem + (size_t)st * stage_bytes;
-                const int j = q < nslabs ? q : q - nslabs;
-                const int left = L - j * kSlab;
-                const int live = left < kSlab ? left : kSlab;
-                const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
-                if (q < nslabs) {
-                    const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
-                    mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
-                    bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
-                    uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
-                    for (int i = 0; i < n; ++i)
-                        bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
-                } else {
-                    mbar_arrive_expect_tx(&full[st], 2 * zbytes);
-                    bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
-                    bulk_load(base + (size_t)kSlab * 4, sa.x + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+            int q = 0;
+            bool stop = false;
+            for (int w = 0; w < nitems && !stop; ++w) {
+                const Item it = decode_item(a.t, item0 + w);
+                const int L = it.L;
+                const int nslabs = (L + kSlab - 1) / kSlab;
+                const int njobs = FUSED ? 2 * nslabs : nslabs;
+                const float* __restrict__ zb_g = a.zbar + it.base;
+                const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
+                for (int r = 0; r < njobs; ++r, ++q) {
+                    const int st = q % kStages;
+                    if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; stop = true; break; }
+                    unsigned char* base = smem + (size_t)st * stage_bytes;
+                    const int j = r < nslabs ? r : r - nslabs;
+                    const int left = L - j * kSlab;
+                    const int live = left < kSlab ? left : kSlab;
+                    const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
+                    if (r < nslabs) {
+                        const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
+                        mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
+                        bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
+                        uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
+                        for (int i = 0; i < n; ++i)
+                            bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
+                    } else {
+                        mbar_arrive_expect_tx(&full[st], 2 * zbytes);
+                        bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                        bulk_load(base + (size_t)kSlab * 4, sa.x + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                    }
                 }
-                issued = q + 1;
             }
             if (failed) {
                 // give the copies still in flight a bounded chance to land before shared memory is released
-                const int first = issued > kStages ? issued - kStages : 0;
-                for (int q = first; q < issued; ++q) mbar_wait(&full[q % kStages], (uint32_t)(q / kStages) & 1u);
+                const int first = q > kStages ? q - kStages : 0;
+                for (int p = first; p < q; ++p) mbar_wait(&full[p % kStages], (uint32_t)(p / kStages) & 1u);
             }
         }
     } else {
@@ -769,92 +777,105 @@ k_server_staged(const ServerStagedArgs sa)
         const int sh = 4 * (lane & 7);
         const int wl = lane >> 3;
         const int g0 = warp, g1 = warp + kWarps;
-        double acc = 0.0;
-        bool ok = true;
-        for (int j = 0; j < nslabs; ++j) {
-            const int st = j % kStages;
-            if (!mbar_wait(&full[st], (uint32_t)(j / kStages) & 1u)) { failed = 1; ok = false; break; }
-            const unsigned char* base = smem + (size_t)st * stage_bytes;
-            const float* zs = reinterpret_cast<const float*>(base);
-            const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
-            const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
-            const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
-            float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
-            signed_scale_sums<NT>(rows + g0 * 4 + wl, rows + g1 * 4 + wl, neg_s, n, sh, s01, s23, t01, t23);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int grp = j * kSlabGroups + (u ? g1 : g0);
-                const int k = grp * kGroup + lane * 4;
-                const float4 zo4 = u ? zo1 : zo0;
-                const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
-                const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
-                float zn[4];
-                uint32_t nibble = 0;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
-                    zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
-                    if (k + e < L) {
-                        const double zd = (double)zn[e];
-                        acc = fma(zd, zd, acc);
-                        nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
-                    }
-                }
-                st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
-                const uint32_t word = pack_group_words(nibble, lane);
-                if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
-            }
-        }
-        acc = warp_sum(acc);
-        if (lane == 0) red[warp] = acc;
-        consumer_barrier();                            // partial sums and sign words of the tile are in shared memory
-        double total = 0.0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) total += red[w];
-        if (failed) ok = false;
-        if (FUSED) {
-            // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
-            const float S_new = (float)sqrt(total / (double)it.Lc);
-            if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
-            for (int j = 0; ok && j < nslabs; ++j) {
-                const int q = nslabs + j;
+        // A warp whose wait gives up sets `failed`, skips the rest of its phase and still arrives at the next
+        // consumer barrier; after every barrier all consumers read `failed` and leave together.
+        int q = 0;
+        for (int w = 0; w < nitems; ++w) {
+            const Item it = decode_item(a.t, item0 + w);
+            const int L = it.L;
+            const int nslabs = (L + kSlab - 1) / kSlab;
+            uint32_t* negs = neg_s[w & 1];
+            for (int i = threadIdx.x; i < n; i += kThreads)
+                negs[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
+            const float S_old = a.Sbar[it.c];
+            consumer_barrier();                        // -s_i in place; everybody is done with the previous chunk
+            if (failed) break;
+            bool ok = true;
+            double acc = 0.0;
+            for (int j = 0; j < nslabs; ++j, ++q) {
                 const int st = q % kStages;
                 if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
-                const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
-                const float* xs = vs + kSlab;
-                float4 vv[2], xx[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
-                    xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
-                }
+                const unsigned char* base = smem + (size_t)st * stage_bytes;
+                const float* zs = reinterpret_cast<const float*>(base);
+                const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
+                const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
+                const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
+                float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
+                signed_scale_sums<NT>(rows + g0 * 4 + wl, rows + g1 * 4 + wl, negs, n, sh, s01, s23, t01, t23);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);
+                if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int grp = j * kSlabGroups + (u ? g1 : g0);
                     const int k = grp * kGroup + lane * 4;
-                    const uint32_t nib = nb[grp * 4 + wl] >> sh;
-                    xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib & 1u, S_new), sa.lr, sa.eps);
-                    xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib & 2u, S_new), sa.lr, sa.eps);
-                    xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib & 4u, S_new), sa.lr, sa.eps);
-                    xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib & 8u, S_new), sa.lr, sa.eps);
-                    st4_checked(sa.x + it.base, k, L, xx[u]);
+                    const float4 zo4 = u ? zo1 : zo0;
+                    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+                    const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
+                    float zn[4];
+                    uint32_t nibble = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
+                        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+                        if (k + e < L) {
+                            const double zd = (double)zn[e];
+                            acc = fma(zd, zd, acc);
+                            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                        }
+                    }
+                    st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                    const uint32_t word = pack_group_words(nibble, lane);
+                    if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
                 }
             }
-        } else if (ok && threadIdx.x == 0) {
-            if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
-            else a.partial[it.c * a.t.P + it.p] = total;
-        }
-        // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
-        if (ok) {
-            uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
-            const int nwords = (L + 31) / 32;
-            for (int w4 = threadIdx.x * 4; w4 < nwords; w4 += kThreads * 4) {
-                if (w4 + 3 < nwords) *reinterpret_cast<uint4*>(ob + w4) = *reinterpret_cast<const uint4*>(nb + w4);
-                else for (int w = w4; w < nwords; ++w) ob[w] = nb[w];
+            acc = warp_sum(acc);
+            if (lane == 0) red[warp] = acc;
+            consumer_barrier();                        // partial sums and sign words of the tile are in shared memory
+            double total = 0.0;
+#pragma unroll
+            for (int r = 0; r < kWarps; ++r) total += red[r];
+            if (failed) break;
+            if (FUSED) {
+                // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
+                const float S_new = (float)sqrt(total / (double)it.Lc);
+                if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
+                for (int j = 0; ok && j < nslabs; ++j, ++q) {
+                    const int st = q % kStages;
+                    if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
+                    const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
+                    const float* xs = vs + kSlab;
+                    float4 vv[2], xx[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
+                        xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[st]);
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int grp = j * kSlabGroups + (u ? g1 : g0);
+                        const int k = grp * kGroup + lane * 4;
+                        const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                        xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib & 1u, S_new), sa.lr, sa.eps);
+                        xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib & 2u, S_new), sa.lr, sa.eps);
+                        xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib & 4u, S_new), sa.lr, sa.eps);
+                        xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib & 8u, S_new), sa.lr, sa.eps);
+                        st4_checked(sa.x + it.base, k, L, xx[u]);
+                    }
+                }
+            } else if (ok && threadIdx.x == 0) {
+                if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+                else a.partial[it.c * a.t.P + it.p] = total;
+            }
+            // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
+            if (ok) {
+                uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+                const int nwords = (L + 31) / 32;
+                for (int w4 = threadIdx.x * 4; w4 < nwords; w4 += kThreads * 4) {
+                    if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
+                    else for (int r = w4; r < nwords; ++r) ob[r] = nb[r];
+                }
             }
         }
     }
@@ -1210,9 +1231,15 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
 template <int NT, bool FUSED>
 cudaError_t launch_staged(const ServerStagedArgs& sa, unsigned blocks, size_t smem, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(k_server_staged<NT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k_server_staged<NT, FUSED><<<blocks, kStagedThreads, smem, stream>>>(sa);
+    if (FUSED && sa.span > 1) {
+        cudaError_t e = cudaFuncSetAttribute(k_server_staged<NT, FUSED, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_server_staged<NT, FUSED, FUSED><<<blocks, kStagedThreads, smem, stream>>>(sa);
+    } else {
+        cudaError_t e = cudaFuncSetAttribute(k_server_staged<NT, FUSED, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_server_staged<NT, FUSED, false><<<blocks, kStagedThreads, smem, stream>>>(sa);
+    }
     return cudaSuccess;
 }
 
@@ -1251,8 +1278,10 @@ apms_status launch_server_and_apply(apms_ctx* c)
                 sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
                 sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
                 const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
-                cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)blocks, smem, c->stream)
-                                      : launch_staged_n<false>(sa, (unsigned)blocks, smem, c->stream);
+                sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
+                const int64_t ctas = (a.items + sa.span - 1) / sa.span;
+                cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)ctas, smem, c->stream)
+                                      : launch_staged_n<false>(sa, (unsigned)ctas, smem, c->stream);
                 if (e != cudaSuccess) {
                     snprintf(c->err, sizeof c->err, "setting up k_server_staged failed: %s", cudaGetErrorString(e));
                     return APMS_ERR_CUDA;

@@ -41,15 +41,15 @@ UNIT = "worker-elements/s"
 NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT = 11.95    # k_worker_fine, profiles/k_worker_fine_small_case.md
 
 
-def algorithmic_bytes(d: int, n: int, chunk: int) -> dict:
+def algorithmic_bytes(d: int, n: int, chunk: int, grad_bytes: int = 4) -> dict:
     """Bytes each kernel must move per step (state kept as compensated vectors + messages)."""
     C = -(-d // chunk)
     W4 = 4 * -(-d // 32)
-    worker = n * (12 * d + W4) + W4 + n * 8 * C + 4 * C      # g, z read, z write, bits out; Bbar once; scales
+    worker = n * ((8 + grad_bytes) * d + W4) + W4 + n * 8 * C + 4 * C      # g, z read, z write, bits out; Bbar once; scales
     server = n * (W4 + 4 * C) + 8 * d + W4 + 8 * C           # n bit streams + scales in; zbar r/w; Bbar, Sbar
     apply_ = W4 + 4 * C + 12 * d                             # Bbar, Sbar, v, x in; x out
     return {"worker": worker, "server": server, "apply": apply_, "step": worker + server + apply_,
-            "warmup_adam": (4 * n + 24) * d}
+            "warmup_adam": (grad_bytes * n + 24) * d}
 
 
 def measured_peaks() -> dict:
@@ -193,12 +193,20 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
     x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)
     ctx.set_params(x0)
     del x0
+    gdt = getattr(torch, args.grad_dtype)
+    gbytes = 4 if gdt == torch.float32 else 2
     ring = []
+    scratch = torch.empty(w.d, dtype=torch.float32, device=dev) if gbytes == 2 else None
     for r in range(2):
-        gs = [torch.empty(w.d, dtype=torch.float32, device=dev) for _ in range(w.n)]
+        gs = [torch.empty(w.d, dtype=gdt, device=dev) for _ in range(w.n)]
         for i in range(w.n):
-            wl.device_gradient(w, r + 1000 * rank, i, gs[i])
+            if scratch is None:
+                wl.device_gradient(w, r + 1000 * rank, i, gs[i])
+            else:                                    # drawn in binary32, rounded once to the 16-bit type
+                wl.device_gradient(w, r + 1000 * rank, i, scratch)
+                gs[i].copy_(scratch)
         ring.append(gs)
+    del scratch
     torch.cuda.synchronize()
     group = dist if world > 1 else None
 
@@ -212,7 +220,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
             ctx.warmup_step(ring[k % 2])
         ms, cnt = ctx.kernel_time(B.KERNEL_WARMUP_ADAM)
         ctx.set_timing(False)
-        ab = algorithmic_bytes(w.d, w.n, w.chunk)["warmup_adam"]
+        ab = algorithmic_bytes(w.d, w.n, w.chunk, gbytes)["warmup_adam"]
         adam = {"ms_per_step": ms / cnt, "achieved_gbs": ab / (ms / cnt * 1e-3) / 1e9,
                 "worker_elements_per_s": w.d * w.n / (ms / cnt * 1e-3)}
     ctx.freeze_v()
@@ -253,7 +261,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
     # inside the timed region, every step
     if want_e2e:
         try:
-            host = [torch.empty(w.d, dtype=torch.float32).pin_memory() for _ in range(w.n)]
+            host = [torch.empty(w.d, dtype=gdt).pin_memory() for _ in range(w.n)]
             for i in range(w.n):
                 host[i].copy_(ring[0][i])
             x_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
@@ -270,7 +278,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
             wall = time.perf_counter() - t0
             secs = max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, wall), group)
             out["e2e"] = {"value": world * w.d * w.n * args.e2e_steps / secs, "unit": UNIT,
-                          "h2d_bytes_per_step": 4 * w.d * w.n, "d2h_bytes_per_step": 4 * w.d,
+                          "h2d_bytes_per_step": gbytes * w.d * w.n, "d2h_bytes_per_step": 4 * w.d,
                           "ms_per_step": secs * 1e3 / args.e2e_steps, "steps": args.e2e_steps,
                           "api": "apms_compressed_step_host (pinned host gradients in, x out)"}
             del host, x_host
@@ -294,6 +302,8 @@ def main(argv=None) -> int:
     ap.add_argument("--chunk", type=int, default=None, help="override the chunk length")
     ap.add_argument("--d", type=int, default=None, help="use only the first d elements of the parameter set")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16", "float16"],
+                    help="element type of the gradient arrays (the configurations of record use float32)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -317,7 +327,8 @@ def main(argv=None) -> int:
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": f"{w.name}: d={w.d}, n={w.n} simulated workers, chunk={w.chunk}, {w.dist} gradients",
-              "d": w.d, "n_workers": w.n, "chunk": w.chunk, "parallelism": f"replicas x{world}",
+              "d": w.d, "n_workers": w.n, "chunk": w.chunk, "gradient_dtype": args.grad_dtype,
+              "parallelism": f"replicas x{world}",
               "l2_policy": "inputs_exceed_l2" if 12 * w.d * w.n > (256 << 20) else "l2_resident",
               "gradient_ring": 2}
 
@@ -355,7 +366,7 @@ def main(argv=None) -> int:
             for chunk in (1024, 4096, 16384, 65536):
                 ws = w.with_(n=n, chunk=chunk)
                 m = measure(ws, args, rank, world, local_rank, dist, want_adam=(chunk == 1024), want_e2e=False)
-                ab = algorithmic_bytes(ws.d, n, chunk)
+                ab = algorithmic_bytes(ws.d, n, chunk, 4 if args.grad_dtype == "float32" else 2)
                 gbs = ab["step"] / (m["ms_per_step"] * 1e-3) / 1e9
                 row = {"n": n, "chunk": chunk, "ms_per_step": m["ms_per_step"], "value": m["value"],
                        "step_gbs": gbs, "step_frac": gbs / peaks["hbm_gbs"], "kernel_ms": m["kernel_ms"]}
@@ -371,14 +382,14 @@ def main(argv=None) -> int:
 
     m = measure(w, args, rank, world, local_rank, dist, want_adam=args.adam, want_e2e=not args.no_e2e)
     ms_per_step, kernel_ms = m["ms_per_step"], m["kernel_ms"]
-    ab = algorithmic_bytes(w.d, w.n, w.chunk)
+    ab = algorithmic_bytes(w.d, w.n, w.chunk, 4 if args.grad_dtype == "float32" else 2)
     if "apply" not in kernel_ms:          # steps 4-6 ran as one kernel: it moves both kernels' bytes (Bbar is not re-read)
         ab["server"] = ab["server"] + ab["apply"] - 4 * -(-w.d // 32)
         ab["step"] = ab["worker"] + ab["server"]
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
     step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * w.n
-               if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT else None)
+               if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32" else None)
     roofline = {"bound": "hbm", "kernel": "k_worker", "achieved": wk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": wk_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": traffic,
                 "algorithmic_bytes_per_launch": ab["worker"],

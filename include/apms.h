@@ -90,6 +90,16 @@ typedef enum {
     APMS_KERNEL_COUNT = 4
 } apms_kernel_id;
 
+/* Element type of the gradient arrays given to the *_typed step functions.  Section 5.1 counts
+ * the compressor's saving for float32 and for float16 training; with 16-bit gradients a step reads
+ * 2 instead of 4 bytes per worker and element.  A 16-bit gradient is widened to binary32 exactly
+ * before its first use; all state and all arithmetic stay binary32 as stated above. */
+typedef enum {
+    APMS_GRAD_F32 = 0,    /* IEEE binary32 */
+    APMS_GRAD_BF16 = 1,   /* bfloat16: the upper 16 bits of a binary32 */
+    APMS_GRAD_F16 = 2     /* IEEE binary16 */
+} apms_grad_type;
+
 /* How threads are grouped on a tile of a chunk in the worker and server kernels. */
 typedef enum {
     APMS_TEAM_AUTO = 0,   /* the library's choice for the shape (the forms below, per kernel)      */
@@ -157,6 +167,15 @@ apms_status apms_compressed_step(apms_ctx* ctx, const float* const* grads_dev);
  * Synchronises the stream before returning. */
 apms_status apms_compressed_step_host(apms_ctx* ctx, const float* const* grads_host,
                                       float* x_out_host);
+
+/* The three step functions for gradients of another element type: the same operations on
+ * g_i widened to binary32.  grads_*: host array of n pointers to d elements of `type` each,
+ * aligned to 16 bytes (binary32) or 8 bytes (16-bit types).  apms_warmup_step(ctx, g) is
+ * apms_warmup_step_typed(ctx, g, APMS_GRAD_F32), and so on. */
+apms_status apms_warmup_step_typed(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
+apms_status apms_compressed_step_typed(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
+apms_status apms_compressed_step_host_typed(apms_ctx* ctx, const void* const* grads_host, apms_grad_type type,
+                                            float* x_out_host);
 
 /* Copy x (d floats) to dst: device memory if dst_is_device != 0 (stream-ordered), else
  * host memory (synchronises the stream). */

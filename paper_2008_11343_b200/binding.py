@@ -24,6 +24,7 @@ PHASE_CREATED, PHASE_WARMUP, PHASE_COMPRESSED = range(3)
 KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
 KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
 TEAM_AUTO, TEAM_CTA, TEAM_WARP, TEAM_STAGED = range(4)
+GRAD_F32, GRAD_BF16, GRAD_F16 = range(3)
 MAX_WORKERS = 64
 NOALLOC_MAX_TILES = 16384
 
@@ -42,6 +43,9 @@ SIGNATURES = {
     "apms_freeze_v": (C.c_int, [C.c_void_p]),
     "apms_compressed_step": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p)]),
     "apms_compressed_step_host": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p]),
+    "apms_warmup_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
+    "apms_compressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
+    "apms_compressed_step_host_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int, C.c_void_p]),
     "apms_get_params": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
     "apms_get_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "apms_get_state_slice": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
@@ -131,6 +135,18 @@ def apms_compressed_step(h, grad_ptrs: Sequence[int]):
 
 def apms_compressed_step_host(h, grad_host_ptrs: Sequence[int], x_out_host_ptr: Optional[int]):
     _check(h, load().apms_compressed_step_host(h, _ptr_array(grad_host_ptrs), x_out_host_ptr))
+
+
+def apms_warmup_step_typed(h, grad_ptrs: Sequence[int], grad_type: int):
+    _check(h, load().apms_warmup_step_typed(h, _ptr_array(grad_ptrs), grad_type))
+
+
+def apms_compressed_step_typed(h, grad_ptrs: Sequence[int], grad_type: int):
+    _check(h, load().apms_compressed_step_typed(h, _ptr_array(grad_ptrs), grad_type))
+
+
+def apms_compressed_step_host_typed(h, grad_host_ptrs: Sequence[int], grad_type: int, x_out_host_ptr: Optional[int]):
+    _check(h, load().apms_compressed_step_host_typed(h, _ptr_array(grad_host_ptrs), grad_type, x_out_host_ptr))
 
 
 def apms_get_params(h, dst_ptr: int, dst_is_device: bool):
@@ -232,12 +248,19 @@ class Context:
             pass
 
     @staticmethod
-    def _dev_ptrs(grads) -> list:
+    def _grad_type(grads) -> int:
+        """GRAD_* constant of a list of torch tensors or numpy arrays that share one dtype."""
         import torch
 
+        names = {str(g.dtype).replace("torch.", "") for g in grads}
+        assert len(names) == 1, f"gradients of mixed types: {names}"
+        return {"float32": GRAD_F32, "bfloat16": GRAD_BF16, "float16": GRAD_F16}[names.pop()]
+
+    @staticmethod
+    def _dev_ptrs(grads) -> list:
         ptrs = []
         for g in grads:
-            assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
+            assert g.is_cuda and g.is_contiguous()
             ptrs.append(g.data_ptr())
         return ptrs
 
@@ -256,14 +279,14 @@ class Context:
 
     def warmup_step(self, grads):
         assert len(grads) == self.n
-        apms_warmup_step(self._h, self._dev_ptrs(grads))
+        apms_warmup_step_typed(self._h, self._dev_ptrs(grads), self._grad_type(grads))
 
     def freeze_v(self):
         apms_freeze_v(self._h)
 
     def compressed_step(self, grads):
         assert len(grads) == self.n
-        apms_compressed_step(self._h, self._dev_ptrs(grads))
+        apms_compressed_step_typed(self._h, self._dev_ptrs(grads), self._grad_type(grads))
 
     def compressed_step_host(self, grads_host, x_out_host=None):
         """grads_host: n CPU float32 tensors/arrays (pinned for overlap); x_out_host: CPU buffer or None."""
@@ -272,8 +295,8 @@ class Context:
         def hp(a):
             return a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
 
-        apms_compressed_step_host(self._h, [hp(g) for g in grads_host],
-                                  None if x_out_host is None else hp(x_out_host))
+        apms_compressed_step_host_typed(self._h, [hp(g) for g in grads_host], self._grad_type(grads_host),
+                                        None if x_out_host is None else hp(x_out_host))
 
     def get_params(self, out=None) -> np.ndarray:
         if out is not None and not isinstance(out, np.ndarray):

@@ -24,6 +24,7 @@
 // exact in binary64, so only the order of the additions can differ from a sequential sum).
 
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -55,7 +56,7 @@ constexpr int kGroup = 128;              // elements one warp covers per 128-bit
 #define APMS_SERVER_CTAS 3
 #endif
 
-struct GradPtrs { const float* p[APMS_MAX_WORKERS]; };
+struct GradPtrs { const void* p[APMS_MAX_WORKERS]; };     // element type given by the kernel's GT template argument
 
 // ------------------------------------------------------------------------------------------
 // small device helpers
@@ -83,6 +84,45 @@ __device__ __forceinline__ void st4_checked(float* p, int k, int len, float4 v) 
         if (k + 1 < len) p[k + 1] = v.y;
         if (k + 2 < len) p[k + 2] = v.z;
     }
+}
+
+// Gradient element types (apms_grad_type): binary32, bfloat16, binary16.  A 16-bit gradient is
+// widened to binary32 exactly before its first use, so the arithmetic of a step does not change.
+template <int GT> struct Grad;
+template <> struct Grad<APMS_GRAD_F32> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const float*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return ((const float*)p)[e]; }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) { return ld_stream4((const float*)p + k); }
+};
+template <> struct Grad<APMS_GRAD_BF16> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const uint16_t*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __uint_as_float((uint32_t)((const uint16_t*)p)[e] << 16); }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const uint16_t*)p + k));
+        return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                           __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+    }
+};
+template <> struct Grad<APMS_GRAD_F16> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const __half*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __half2float(((const __half*)p)[e]); }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const __half*)p + k));
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&r.y));
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+};
+// Up to four consecutive gradient elements starting at element k; elements at or past `len` read as 0.
+template <int GT>
+__device__ __forceinline__ float4 ld_grad4_checked(const void* p, int k, int len)
+{
+    if (k + 3 < len) return Grad<GT>::ld4(p, k);
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k + 0 < len) r.x = Grad<GT>::ld1(p, k + 0);
+    if (k + 1 < len) r.y = Grad<GT>::ld1(p, k + 1);
+    if (k + 2 < len) r.z = Grad<GT>::ld1(p, k + 2);
+    return r;
 }
 
 // +-s with the sign of the compressor: z >= 0 gives +s (so do +0 and -0), NaN gives -s.
@@ -148,6 +188,7 @@ __device__ __forceinline__ void adam_elem(const AdamArgs& a, float gs, float& m,
 // One short-lived CTA per 1024 elements (one float4 per thread and stream): the n gradient
 // loads of a thread are independent, and many small CTAs keep more of them in flight than a
 // resident grid-stride loop does.
+template <int GT>
 __global__ void __launch_bounds__(kThreads)
 k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
 {
@@ -159,7 +200,7 @@ k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
         float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
         for (int i = 0; i < a.n; ++i) {
-            const float4 g = ld_stream4(G.p[i] + j);
+            const float4 g = Grad<GT>::ld4(Grad<GT>::at(G.p[i], j), 0);
             gs.x = __fadd_rn(gs.x, g.x); gs.y = __fadd_rn(gs.y, g.y);
             gs.z = __fadd_rn(gs.z, g.z); gs.w = __fadd_rn(gs.w, g.w);
         }
@@ -172,7 +213,7 @@ k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
         // ragged tail (d not a multiple of 4): element by element
         for (int64_t e = j; e < a.d; ++e) {
             float gs = 0.f;
-            for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, G.p[i][e]);
+            for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, Grad<GT>::ld1(G.p[i], e));
             float m = a.m[e], v = a.v[e], x = a.x[e];
             adam_elem(a, gs, m, v, x);
             a.m[e] = m; a.v[e] = v; a.x[e] = x;
@@ -280,7 +321,7 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
     }
 }
 
-template <bool M32, int U, int WPC>
+template <int GT, bool M32, int U, int WPC>
 __global__ void __launch_bounds__(kThreads, APMS_WORKER_CTAS)
 k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 {
@@ -293,7 +334,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
     const Item it = decode_item(a.t, item / a.ni);
     const int i = a.i0 + ii;
     const int L = it.L;
-    const float* __restrict__ g = G.p[ii] + it.base;
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], it.base);
     float* __restrict__ z = a.z + (int64_t)i * a.dz + it.base;
     const float* __restrict__ m32 = a.m32 + it.base;
     const uint32_t* __restrict__ mbits = a.Bbar + it.base / 32;
@@ -314,7 +355,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         for (int u = 0; u < U; ++u) {
             const int grp = g0 + WPC * u;
             const int k = grp * kGroup + lane * 4;
-            gv[u] = ld_stream4(g + k);
+            gv[u] = Grad<GT>::ld4(g, k);
             zv[u] = ld_stream4(z + k);
             if (M32) mv[u] = *reinterpret_cast<const float4*>(m32 + k);
             else     mw[u] = mbits[grp * 4 + (lane >> 3)];
@@ -327,7 +368,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
     // remainder: one group at a time, bounds-checked
     for (; g0 < ngroups; g0 += WPC) {
         const int k = g0 * kGroup + lane * 4;
-        const float4 gv = ld4_checked(g, k, L, true);
+        const float4 gv = ld_grad4_checked<GT>(g, k, L);
         const float4 zv = ld4_checked(z, k, L, true);
         float4 mv = make_float4(0, 0, 0, 0);
         uint32_t mw = 0;
@@ -371,6 +412,7 @@ struct WorkerFineArgs {
     float beta1, omb1;
 };
 
+template <int GT>
 __global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
@@ -391,7 +433,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     }
     const int L = (int)(left < kFineSub ? left : kFineSub);
     const int64_t c = base / a.chunk;
-    const float* __restrict__ g = G.p[ii] + base;
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
     float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
     const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
     uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
@@ -402,7 +444,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
         float4 gv[kFineU], zv[kFineU];
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
-            gv[u] = ld_stream4(g + u * kGroup + lane * 4);
+            gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
             zv[u] = ld_stream4(z + u * kGroup + lane * 4);
         }
         const uint32_t mine = (lane < 4 * kFineU) ? mbits[lane] : 0u;
@@ -433,7 +475,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
         const int ngroups = (L + kGroup - 1) / kGroup;
         for (int grp = 0; grp < ngroups; ++grp) {
             const int k = grp * kGroup + lane * 4;
-            const float4 gv = ld4_checked(g, k, L, true);
+            const float4 gv = ld_grad4_checked<GT>(g, k, L);
             const float4 zv = ld4_checked(z, k, L, true);
             const uint32_t mw = (k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
             worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
@@ -1106,12 +1148,26 @@ struct Timed {
     }
 };
 
-apms_status check_grads(apms_ctx* c, const float* const* g, GradPtrs* out, int count)
+bool valid_grad_type(int t) { return t == APMS_GRAD_F32 || t == APMS_GRAD_BF16 || t == APMS_GRAD_F16; }
+size_t grad_elem_bytes(int t) { return t == APMS_GRAD_F32 ? 4 : 2; }
+
+// Runs `call` with GT bound to the compile-time constant that equals the run-time gradient type.
+#define APMS_DISPATCH_GRAD(type, ...)                                              \
+    do {                                                                           \
+        if ((type) == APMS_GRAD_BF16)     { constexpr int GT = APMS_GRAD_BF16; __VA_ARGS__; } \
+        else if ((type) == APMS_GRAD_F16) { constexpr int GT = APMS_GRAD_F16;  __VA_ARGS__; } \
+        else                              { constexpr int GT = APMS_GRAD_F32;  __VA_ARGS__; } \
+    } while (0)
+
+apms_status check_grads(apms_ctx* c, const void* const* g, int type, GradPtrs* out, int count)
 {
+    if (!valid_grad_type(type)) return fail(c, APMS_ERR_INVALID_ARG, "unknown gradient type");
     if (!g) return fail(c, APMS_ERR_INVALID_ARG, "gradient pointer array is NULL");
+    const uintptr_t mask = type == APMS_GRAD_F32 ? 15u : 7u;          // one lane's four elements per access
     for (int i = 0; i < count; ++i) {
         if (!g[i]) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is NULL");
-        if (((uintptr_t)g[i] & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is not 16-byte aligned");
+        if (((uintptr_t)g[i] & mask) != 0)
+            return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is not aligned (16 bytes for binary32, 8 bytes for 16-bit gradients)");
         out->p[i] = g[i];
     }
     return APMS_OK;
@@ -1166,7 +1222,7 @@ bool use_fine_worker(const apms_ctx* c)
     return !c->m_is_fp32 && c->L.fine_tiles > 0;
 }
 
-apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
+apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
 {
     WorkerFineArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
@@ -1183,7 +1239,7 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
     {
         Timed t(c, APMS_KERNEL_WORKER);
-        k_worker_fine<<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a);
+        APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
         apms_status st = launch_check(c, "k_worker_fine");
         if (st != APMS_OK) return st;
         const int64_t total = (int64_t)ni * c->L.C;
@@ -1195,9 +1251,9 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int i0, int ni)
     return APMS_OK;
 }
 
-apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
+apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
 {
-    if (use_fine_worker(c)) return launch_worker_fine(c, G, i0, ni);
+    if (use_fine_worker(c)) return launch_worker_fine(c, G, gtype, i0, ni);
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
     a.B = c->B(0); a.Wp = c->L.Wp;
@@ -1214,11 +1270,11 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int i0, int ni)
         Timed t(c, APMS_KERNEL_WORKER);
         const unsigned gridx = (unsigned)blocks;
         if (c->m_is_fp32) {
-            if (warp_teams) k_worker<true, 2, 1><<<gridx, kThreads, 0, c->stream>>>(G, a);
-            else            k_worker<true, 4, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a);
+            if (warp_teams) APMS_DISPATCH_GRAD(gtype, k_worker<GT, true, 2, 1><<<gridx, kThreads, 0, c->stream>>>(G, a));
+            else            APMS_DISPATCH_GRAD(gtype, k_worker<GT, true, 4, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a));
         } else {
-            if (warp_teams) k_worker<false, APMS_WORKER_U, 1><<<gridx, kThreads, 0, c->stream>>>(G, a);
-            else            k_worker<false, APMS_WORKER_U, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a);
+            if (warp_teams) APMS_DISPATCH_GRAD(gtype, k_worker<GT, false, APMS_WORKER_U, 1><<<gridx, kThreads, 0, c->stream>>>(G, a));
+            else            APMS_DISPATCH_GRAD(gtype, k_worker<GT, false, APMS_WORKER_U, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a));
         }
         apms_status st = launch_check(c, "k_worker");
         if (st != APMS_OK) return st;
@@ -1409,10 +1465,15 @@ apms_status apms_set_lr(apms_ctx* c, float lr)
 
 apms_status apms_warmup_step(apms_ctx* c, const float* const* grads_dev)
 {
+    return apms_warmup_step_typed(c, (const void* const*)grads_dev, APMS_GRAD_F32);
+}
+
+apms_status apms_warmup_step_typed(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
+{
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_WARMUP) return fail(c, APMS_ERR_BAD_STATE, "apms_warmup_step needs the WARMUP phase (after apms_set_params, before apms_freeze_v)");
     GradPtrs G;
-    apms_status st = check_grads(c, grads_dev, &G, c->L.n);
+    apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
     c->t += 1;
     AdamArgs a;
@@ -1424,7 +1485,7 @@ apms_status apms_warmup_step(apms_ctx* c, const float* const* grads_dev)
     Timed t(c, APMS_KERNEL_WARMUP_ADAM);
     const int64_t adam_blocks = (c->L.d + (int64_t)kThreads * 4 - 1) / ((int64_t)kThreads * 4);
     if (adam_blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "d too large for one launch");
-    k_warmup_adam<<<(unsigned)adam_blocks, kThreads, 0, c->stream>>>(G, a);
+    APMS_DISPATCH_GRAD((int)type, k_warmup_adam<GT><<<(unsigned)adam_blocks, kThreads, 0, c->stream>>>(G, a));
     return launch_check(c, "k_warmup_adam");
 }
 
@@ -1441,20 +1502,31 @@ apms_status apms_freeze_v(apms_ctx* c)
 
 apms_status apms_compressed_step(apms_ctx* c, const float* const* grads_dev)
 {
+    return apms_compressed_step_typed(c, (const void* const*)grads_dev, APMS_GRAD_F32);
+}
+
+apms_status apms_compressed_step_typed(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
+{
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step needs the COMPRESSED phase (call apms_freeze_v first)");
     GradPtrs G;
-    apms_status st = check_grads(c, grads_dev, &G, c->L.n);
+    apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
-    st = launch_worker(c, G, 0, c->L.n);
+    st = launch_worker(c, G, (int)type, 0, c->L.n);
     if (st != APMS_OK) return st;
     return launch_server_and_apply(c);
 }
 
 apms_status apms_compressed_step_host(apms_ctx* c, const float* const* grads_host, float* x_out_host)
 {
+    return apms_compressed_step_host_typed(c, (const void* const*)grads_host, APMS_GRAD_F32, x_out_host);
+}
+
+apms_status apms_compressed_step_host_typed(apms_ctx* c, const void* const* grads_host, apms_grad_type type, float* x_out_host)
+{
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step_host needs the COMPRESSED phase (call apms_freeze_v first)");
+    if (!valid_grad_type((int)type)) return fail(c, APMS_ERR_INVALID_ARG, "unknown gradient type");
     if (!grads_host) return fail(c, APMS_ERR_INVALID_ARG, "gradient pointer array is NULL");
     for (int i = 0; i < c->L.n; ++i)
         if (!grads_host[i]) return fail(c, APMS_ERR_INVALID_ARG, "a gradient pointer is NULL");
@@ -1467,18 +1539,19 @@ apms_status apms_compressed_step_host(apms_ctx* c, const float* const* grads_hos
         c->host_path_ready = true;
     }
     const size_t bytes = (size_t)c->L.d * 4;
+    const size_t gbytes = (size_t)c->L.d * grad_elem_bytes((int)type);
     // the staging buffers may still be read by work queued earlier on the compute stream
     APMS_CUDA(c, cudaEventRecord(c->ev_used[0], c->stream));
     APMS_CUDA(c, cudaEventRecord(c->ev_used[1], c->stream));
     for (int i = 0; i < c->L.n; ++i) {
         const int b = i & 1;
         APMS_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_used[b], 0));
-        APMS_CUDA(c, cudaMemcpyAsync(c->stage(b), grads_host[i], bytes, cudaMemcpyHostToDevice, c->copy_stream));
+        APMS_CUDA(c, cudaMemcpyAsync(c->stage(b), grads_host[i], gbytes, cudaMemcpyHostToDevice, c->copy_stream));
         APMS_CUDA(c, cudaEventRecord(c->ev_copied[b], c->copy_stream));
         APMS_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
         GradPtrs G;
         G.p[0] = c->stage(b);
-        apms_status st = launch_worker(c, G, i, 1);
+        apms_status st = launch_worker(c, G, (int)type, i, 1);
         if (st != APMS_OK) return st;
         APMS_CUDA(c, cudaEventRecord(c->ev_used[b], c->stream));
     }

@@ -119,11 +119,12 @@ def teacher_force(ctx, orc, w):
 
 
 def run_both(w: wl.Workload, warmup=None, compressed=None, check_every_step=True, exact=False,
-             grads_fn=None, team_mode=None):
+             grads_fn=None, team_mode=None, upload_fn=None):
     """Free-running: both sides step from the same x0 on the same gradients."""
     warmup = w.warmup_steps if warmup is None else warmup
     compressed = w.compressed_steps if compressed is None else compressed
     grads_fn = grads_fn or (lambda step: wl.host_gradients(w, step))
+    upload = upload_fn or globals()["upload"]
     ctx, orc = make_pair(w, team_mode=team_mode)
     reports = []
     step = 0

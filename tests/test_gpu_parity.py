@@ -66,6 +66,53 @@ def test_teacher_forced_steps_bits_exact():
         H.compare_state(ctx, orc, w, exact=True)
 
 
+# ------------------------------------------------------------------ 16-bit gradients
+
+@pytest.mark.parametrize("team", [B.TEAM_AUTO, B.TEAM_WARP], ids=["auto", "warp-per-tile"])
+@pytest.mark.parametrize("kind", ["bfloat16", "float16"])
+@pytest.mark.parametrize("d,n,chunk", [(5 * 4096 + 1234, 3, 4096), (3 * 1024 + 5, 2, 96), (70000, 16, 160),
+                                       (2 * 32768 + 23552, 4, 32768), (1 * 512 + 3, 2, 512)])
+def test_sixteen_bit_gradients_bit_identical(d, n, chunk, kind, team):
+    """Gradients given as bfloat16 / binary16 arrays: the library widens them exactly, so the state must be
+    bit-identical to the oracle's run on the same values held in binary32 (warmup and compressed steps)."""
+    import torch
+
+    dt = getattr(torch, kind)
+    w = tiny(d, n, chunk, cfg_id=120, warmup_steps=2, compressed_steps=3)
+
+    def grads(step):          # the values the 16-bit arrays hold, as binary32, for the oracle
+        return [torch.from_numpy(g).to(dt).to(torch.float32).numpy() for g in wl.host_gradients(w, step)]
+
+    def upload16(gs):
+        return [torch.from_numpy(g).to(dt).cuda() for g in gs]
+
+    H.run_both(w, exact=True, grads_fn=grads, upload_fn=upload16, team_mode=team)
+
+
+def test_sixteen_bit_host_gradients_and_alignment():
+    import torch
+
+    w = tiny(3 * 2048 + 77, 2, 2048, cfg_id=121)
+    ref = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    for c in (ref, ctx):
+        c.set_params(wl.initial_params(w))
+        c.freeze_v()
+    for step in range(3):
+        g16 = [torch.from_numpy(g).to(torch.bfloat16) for g in wl.host_gradients(w, step)]
+        ref.compressed_step([g.cuda() for g in g16])
+        ctx.compressed_step_host([g.pin_memory() for g in g16])
+    for k in (B.STATE_X, B.STATE_SERVER_BITS, B.STATE_SERVER_SCALES, B.STATE_SERVER_ERR):
+        assert np.array_equal(ref.get_state(k).view(np.uint32), ctx.get_state(k).view(np.uint32))
+    g = torch.zeros(w.d + 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.ApmsError) as e:                       # 2-byte offset: not 8-byte aligned
+        B.apms_compressed_step_typed(ctx._h, [g.data_ptr() + 2, g.data_ptr()], B.GRAD_BF16)
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.ApmsError) as e:
+        B.apms_compressed_step_typed(ctx._h, [g.data_ptr(), g.data_ptr()], 7)
+    assert e.value.status == B.ERR_INVALID_ARG
+
+
 # ------------------------------------------------------------------ the benchmark's small configurations
 
 def test_config0_free_running_10_steps():

@@ -200,6 +200,40 @@ apms_status apms_set_state(apms_ctx* ctx, apms_state_id which, int worker, const
 /* Restore the step counter and phase of a checkpoint (t = Adam steps taken so far). */
 apms_status apms_restore(apms_ctx* ctx, int t, apms_phase phase);
 
+/* Algorithm 1 end to end: T_w Adam steps, then compression-phase steps, with the learning rate
+ * gamma_t of the paper's BERT runs (Section 5.2: linear increase to the peak over the first
+ * steps, then multiplied by a constant factor after every so many steps).  Step k = 0, 1, ...:
+ *   k <  lr_ramp_steps :  lr = peak_lr * (k + 1) / lr_ramp_steps
+ *   k >= lr_ramp_steps :  lr = peak_lr * lr_decay ^ floor((k - lr_ramp_steps) / lr_decay_every)
+ * (lr_ramp_steps = 0: no ramp; lr_decay_every = 0: no decay), evaluated in binary64 and rounded
+ * once.  The paper's BERT-Large values would be {23000, 4e-4f, 12500, 0.99f, 520}. */
+typedef struct {
+    int64_t warmup_steps;     /* T_w: Adam steps before v is frozen                  */
+    float   peak_lr;
+    int64_t lr_ramp_steps;
+    float   lr_decay;
+    int64_t lr_decay_every;
+} apms_schedule;
+
+/* gamma_k of a schedule (pure function; 0 for a NULL schedule or k < 0). */
+float apms_schedule_lr(const apms_schedule* schedule, int64_t step);
+
+/* Attach a schedule (copied) for apms_step; NULL detaches it. */
+apms_status apms_set_schedule(apms_ctx* ctx, const apms_schedule* schedule);
+
+/* One step of Algorithm 1 under the attached schedule: sets gamma_k, runs a warmup step while
+ * fewer than T_w steps have been taken, calls apms_freeze_v when T_w is reached, and a
+ * compression-phase step from then on.  Same gradient contract as the *_typed functions.
+ * The step counter starts at 0 at apms_set_params and counts only successful apms_step calls. */
+apms_status apms_step(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
+int64_t     apms_get_step(const apms_ctx* ctx);
+
+/* Monitor for Assumption 1 (the compression errors stay bounded): squared l2 norms of the n
+ * worker errors delta^(i) (worker_sq_host, n doubles, may be NULL) and of the server error
+ * delta-bar (server_sq_host, may be NULL), summed in binary64 in a fixed order.  Reads every
+ * compensated vector once ((n+1) d floats) and synchronises.  Phase must be COMPRESSED.  Not part of a step; call it as often as wanted. */
+apms_status apms_error_norms(apms_ctx* ctx, double* worker_sq_host, double* server_sq_host);
+
 apms_phase  apms_get_phase(const apms_ctx* ctx);
 int         apms_get_t(const apms_ctx* ctx);
 

@@ -51,6 +51,11 @@ SIGNATURES = {
     "apms_get_state_slice": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
     "apms_set_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "apms_restore": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
+    "apms_schedule_lr": (C.c_float, [C.c_void_p, C.c_int64]),
+    "apms_set_schedule": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "apms_step": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
+    "apms_get_step": (C.c_int64, [C.c_void_p]),
+    "apms_error_norms": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "apms_get_phase": (C.c_int, [C.c_void_p]),
     "apms_get_t": (C.c_int, [C.c_void_p]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
@@ -167,6 +172,36 @@ def apms_set_state(h, which: int, worker: int, src_host_ptr: int):
 
 def apms_restore(h, t: int, phase: int):
     _check(h, load().apms_restore(h, t, phase))
+
+
+class Schedule(C.Structure):
+    """Mirror of the C struct apms_schedule."""
+    _fields_ = [("warmup_steps", C.c_int64), ("peak_lr", C.c_float), ("lr_ramp_steps", C.c_int64),
+                ("lr_decay", C.c_float), ("lr_decay_every", C.c_int64)]
+
+
+def apms_schedule_lr(schedule: Schedule, step: int) -> float:
+    return float(load().apms_schedule_lr(C.byref(schedule), step))
+
+
+def apms_set_schedule(h, schedule: Optional[Schedule]):
+    _check(h, load().apms_set_schedule(h, None if schedule is None else C.byref(schedule)))
+
+
+def apms_step(h, grad_ptrs: Sequence[int], grad_type: int):
+    _check(h, load().apms_step(h, _ptr_array(grad_ptrs), grad_type))
+
+
+def apms_get_step(h) -> int:
+    return int(load().apms_get_step(h))
+
+
+def apms_error_norms(h, n: int):
+    """(worker squared norms [n], server squared norm) as Python floats."""
+    w = (C.c_double * n)()
+    s = C.c_double(0.0)
+    _check(h, load().apms_error_norms(h, w, C.byref(s)))
+    return [float(v) for v in w], float(s.value)
 
 
 def apms_get_phase(h) -> int:
@@ -326,6 +361,21 @@ class Context:
         value = np.ascontiguousarray(value, dtype=np.float32)
         assert value.size == self.d
         apms_set_state(self._h, which, worker, value.ctypes.data)
+
+    def set_schedule(self, schedule: Optional[Schedule]):
+        apms_set_schedule(self._h, schedule)
+
+    def step(self, grads):
+        """One step of Algorithm 1 under the attached schedule (warmup, phase switch or compressed step)."""
+        assert len(grads) == self.n
+        apms_step(self._h, self._dev_ptrs(grads), self._grad_type(grads))
+
+    @property
+    def steps_taken(self) -> int:
+        return apms_get_step(self._h)
+
+    def error_norms(self):
+        return apms_error_norms(self._h, self.n)
 
     def restore(self, t: int, phase: int):
         apms_restore(self._h, t, phase)

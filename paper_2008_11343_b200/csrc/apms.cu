@@ -1014,6 +1014,47 @@ __global__ void k_materialise_momentum(const uint32_t* __restrict__ bits, const 
 }
 
 // ------------------------------------------------------------------------------------------
+// Error monitor: squared l2 norms of the compression errors (the quantities Assumption 1 bounds).
+// Row r < n is worker r (delta = z_r - (+-s_r)), row n the server.  One CTA per (row, 4096-element
+// tile) writes a binary64 partial sum; k_error_norm_rows adds a row's tiles in order.
+
+struct ErrNormArgs {
+    const float* z; int64_t dz; const float* s; int64_t Cp;      // worker rows
+    const float* zbar; const float* Sbar;                         // server row
+    double* partial; int64_t tiles; int n; int64_t d, chunk;
+};
+
+__global__ void __launch_bounds__(kThreads)
+k_error_norm_tiles(const ErrNormArgs a)
+{
+    __shared__ double red[kWarps];
+    const int row = (int)(blockIdx.x / a.tiles);
+    const int64_t t = blockIdx.x % a.tiles;
+    const float* __restrict__ z = row < a.n ? a.z + (int64_t)row * a.dz : a.zbar;
+    const float* __restrict__ s = row < a.n ? a.s + (int64_t)row * a.Cp : a.Sbar;
+    const int64_t base = t * 4096;
+    double acc = 0.0;
+    for (int k = threadIdx.x; k < 4096; k += kThreads) {
+        const int64_t j = base + k;
+        if (j < a.d) {
+            const double e = (double)implied_error(z[j], s[j / a.chunk]);
+            acc = fma(e, e, acc);
+        }
+    }
+    const double total = block_sum(acc, red);
+    if (threadIdx.x == 0) a.partial[(int64_t)row * a.tiles + t] = total;
+}
+
+__global__ void k_error_norm_rows(const double* __restrict__ partial, int64_t tiles, int rows, double* __restrict__ out)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    double total = 0.0;
+    for (int64_t t = 0; t < tiles; ++t) total += partial[(int64_t)r * tiles + t];
+    out[r] = total;
+}
+
+// ------------------------------------------------------------------------------------------
 // host side
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -1023,7 +1064,7 @@ struct Layout {
     int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_status, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_status, total;
 };
 
 bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
@@ -1056,6 +1097,7 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles * kWarps, 64);
     L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
     L->off_stage = take((size_t)L->dz * 4 * 2);
+    L->off_mon = take(((size_t)(n + 1) * (size_t)((d + 4095) / 4096) + (size_t)(n + 1)) * 8);   // error monitor: tile sums + row sums
     L->off_status = take(256);
     L->total = o;
     return true;
@@ -1071,6 +1113,8 @@ struct apms_ctx {
     Layout L;
     float beta1, beta2, eps, lr;
     int t;
+    int64_t steps;           // steps taken through apms_step (warmup and compressed)
+    apms_schedule sched; bool has_sched;
     apms_phase phase;
     bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar)
     char* ws; size_t ws_bytes; bool owns_ws;
@@ -1420,6 +1464,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
+    c->steps = 0; c->has_sched = false;
     c->fine_run = kFineRunDefault;
     if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
@@ -1451,7 +1496,7 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
-    c->t = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
+    c->t = 0; c->steps = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
     return APMS_OK;
 }
 
@@ -1677,6 +1722,74 @@ apms_status apms_restore(apms_ctx* c, int t, apms_phase phase)
     }
     c->t = t; c->phase = phase;
     return APMS_OK;
+}
+
+float apms_schedule_lr(const apms_schedule* sc, int64_t step)
+{
+    if (!sc || step < 0) return 0.0f;
+    if (sc->lr_ramp_steps > 0 && step < sc->lr_ramp_steps)
+        return (float)((double)sc->peak_lr * (double)(step + 1) / (double)sc->lr_ramp_steps);
+    if (sc->lr_decay_every <= 0) return sc->peak_lr;
+    const int64_t past = step - (sc->lr_ramp_steps > 0 ? sc->lr_ramp_steps : 0);
+    return (float)((double)sc->peak_lr * pow((double)sc->lr_decay, (double)(past / sc->lr_decay_every)));
+}
+
+apms_status apms_set_schedule(apms_ctx* c, const apms_schedule* sc)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!sc) { c->has_sched = false; return APMS_OK; }
+    if (sc->warmup_steps < 0 || !isfinite(sc->peak_lr) || sc->lr_ramp_steps < 0 || sc->lr_decay_every < 0 ||
+        !(sc->lr_decay > 0.0f) || !isfinite(sc->lr_decay))
+        return fail(c, APMS_ERR_INVALID_ARG, "invalid schedule: need warmup_steps >= 0, finite peak_lr, lr_ramp_steps >= 0, lr_decay > 0, lr_decay_every >= 0");
+    c->sched = *sc; c->has_sched = true;
+    return APMS_OK;
+}
+
+apms_status apms_step(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!c->has_sched) return fail(c, APMS_ERR_BAD_STATE, "apms_step needs a schedule (apms_set_schedule)");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    const float lr = apms_schedule_lr(&c->sched, c->steps);
+    apms_status st = apms_set_lr(c, lr);
+    if (st != APMS_OK) return st;
+    if (c->phase == APMS_PHASE_WARMUP && c->steps >= c->sched.warmup_steps) {       // T_w Adam steps are done
+        st = apms_freeze_v(c);
+        if (st != APMS_OK) return st;
+    }
+    st = (c->phase == APMS_PHASE_WARMUP) ? apms_warmup_step_typed(c, grads_dev, type)
+                                         : apms_compressed_step_typed(c, grads_dev, type);
+    if (st == APMS_OK) c->steps += 1;
+    return st;
+}
+
+int64_t apms_get_step(const apms_ctx* c) { return c ? c->steps : -1; }
+
+apms_status apms_error_norms(apms_ctx* c, double* worker_sq_host, double* server_sq_host)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
+    if (!worker_sq_host && !server_sq_host) return fail(c, APMS_ERR_INVALID_ARG, "both outputs are NULL");
+    const int rows = c->L.n + 1;
+    ErrNormArgs a;
+    a.z = c->z(0); a.dz = c->L.dz; a.s = c->s(0); a.Cp = c->L.Cp; a.zbar = c->zbar(); a.Sbar = c->Sbar();
+    a.tiles = (c->L.d + 4095) / 4096; a.n = c->L.n; a.d = c->L.d; a.chunk = c->L.chunk;
+    a.partial = reinterpret_cast<double*>(c->ws + c->L.off_mon);
+    double* out = a.partial + (size_t)rows * (size_t)a.tiles;
+    const int64_t blocks = (int64_t)rows * a.tiles;
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many tiles for one launch");
+    k_error_norm_tiles<<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+    apms_status st = launch_check(c, "k_error_norm_tiles");
+    if (st != APMS_OK) return st;
+    k_error_norm_rows<<<(rows + 63) / 64, 64, 0, c->stream>>>(a.partial, a.tiles, rows, out);
+    st = launch_check(c, "k_error_norm_rows");
+    if (st != APMS_OK) return st;
+    double host[APMS_MAX_WORKERS + 1];
+    APMS_CUDA(c, cudaMemcpyAsync(host, out, (size_t)rows * sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (worker_sq_host) for (int i = 0; i < c->L.n; ++i) worker_sq_host[i] = host[i];
+    if (server_sq_host) *server_sq_host = host[c->L.n];
+    return device_status_check(c);
 }
 
 apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }

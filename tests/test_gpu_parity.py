@@ -113,6 +113,51 @@ def test_sixteen_bit_host_gradients_and_alignment():
     assert e.value.status == B.ERR_INVALID_ARG
 
 
+# ------------------------------------------------------------------ phase driver and error monitor
+
+def test_scheduled_steps_follow_algorithm_1():
+    """apms_step under a schedule = T_w Adam steps, the phase switch, then compression-phase steps, each with
+    the schedule's learning rate; compared with the oracle driven by hand, bit for bit."""
+    w = tiny(4 * 2048 + 300, 3, 2048, cfg_id=130)
+    sc = B.Schedule(3, 2e-3, 4, 0.5, 2)                      # T_w = 3; ramp over 4 steps; halve every 2 steps
+    ctx, orc = H.make_pair(w)
+    ctx.set_schedule(sc)
+    for k in range(9):
+        gs = wl.host_gradients(w, k)
+        lr = B.apms_schedule_lr(sc, k)
+        orc.set_lr(lr)
+        if k == 3:
+            orc.freeze_v()
+        (orc.warmup_step if k < 3 else orc.compressed_step)(gs)
+        ctx.step(H.upload(gs))
+        assert ctx.steps_taken == k + 1 and ctx.phase == (B.PHASE_WARMUP if k < 3 else B.PHASE_COMPRESSED)
+        H.compare_state(ctx, orc, w, phase_compressed=k >= 3, exact=True)
+    assert ctx.t == 3
+    ctx.set_schedule(None)
+    with pytest.raises(B.ApmsError) as e:
+        ctx.step(H.upload(wl.host_gradients(w, 9)))
+    assert e.value.status == B.ERR_BAD_STATE
+
+
+def test_error_norms_match_the_oracle_state():
+    """The monitor's squared norms of the worker and server errors against binary64 sums over the oracle's errors."""
+    w = tiny(9 * 4096 + 777, 5, 4096, cfg_id=131)
+    ctx, orc, _ = H.run_both(w, warmup=2, compressed=4, check_every_step=False)
+    workers, server = ctx.error_norms()
+    for i in range(w.n):
+        ref = float(np.sum(orc.worker_err(i).astype(np.float64) ** 2))
+        assert abs(workers[i] - ref) <= 1e-12 * ref
+    ref = float(np.sum(orc.server_err.astype(np.float64) ** 2))
+    assert abs(server - ref) <= 1e-12 * ref
+    fresh = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    fresh.set_params(wl.initial_params(w))
+    with pytest.raises(B.ApmsError) as e:
+        fresh.error_norms()                                  # no errors exist before the phase switch
+    assert e.value.status == B.ERR_BAD_STATE
+    fresh.freeze_v()
+    assert fresh.error_norms() == ([0.0] * w.n, 0.0)
+
+
 # ------------------------------------------------------------------ the benchmark's small configurations
 
 def test_config0_free_running_10_steps():

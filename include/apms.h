@@ -177,6 +177,38 @@ apms_status apms_compressed_step_typed(apms_ctx* ctx, const void* const* grads_d
 apms_status apms_compressed_step_host_typed(apms_ctx* ctx, const void* const* grads_host, apms_grad_type type,
                                             float* x_out_host);
 
+/* A compression-phase step in its phases, for callers that carry out the two exchanges of the
+ * Gather-Scatter AllReduce themselves (Figure 1; Section 3.3 steps 3 and 5) - one process per
+ * GPU, each context holding its GPU's workers and serving a range of chunks:
+ *
+ *   apms_worker_phase   steps 1-2 for the context's n workers: leaves worker i's message (sign
+ *                       words of the whole vector, one scale per chunk) where apms_get_message
+ *                       points;
+ *   [exchange 1: every process sends, of each of its workers' messages, the part that belongs
+ *    to the chunks a peer serves, to that peer]
+ *   apms_server_phase   step 4 for chunks [chunk_begin, chunk_end) from `rows` received
+ *                       messages, averaged in row order: row j occupies row_words sign words
+ *                       starting at bits_rows_dev + j * row_words - its word 0 is the first word
+ *                       of chunk chunk_begin - and row_scales scales starting at
+ *                       scale_rows_dev + j * row_scales.  row_words must be a multiple of 4 that
+ *                       covers the range's words rounded up to 4; bits_rows_dev 16-byte aligned.
+ *                       Writes that range of the server's message (apms_get_message(ctx, -1)).
+ *                       May be called for several ranges in one step.
+ *   [exchange 2: every process sends its range of the server's message to all peers, so that
+ *    each holds the whole of it]
+ *   apms_apply_phase    steps 5-6 over the whole vector from the server's message; ends the step.
+ *
+ * With rows = the total number of workers in global worker order and the ranges covering every
+ * chunk once, the result equals apms_compressed_step of one context that holds all workers.
+ * apms_get_message: device addresses of worker i's message (worker = -1: the server's), valid
+ * while the workspace lives; the buffers hold W words / C scales, rows padded to 256 bytes. */
+apms_status apms_worker_phase(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
+apms_status apms_get_message(apms_ctx* ctx, int worker, uint32_t** bits_dev, float** scales_dev);
+apms_status apms_server_phase(apms_ctx* ctx, const uint32_t* bits_rows_dev, int64_t row_words,
+                              const float* scale_rows_dev, int64_t row_scales, int rows,
+                              int64_t chunk_begin, int64_t chunk_end);
+apms_status apms_apply_phase(apms_ctx* ctx);
+
 /* Copy x (d floats) to dst: device memory if dst_is_device != 0 (stream-ordered), else
  * host memory (synchronises the stream). */
 apms_status apms_get_params(apms_ctx* ctx, float* dst, int dst_is_device);

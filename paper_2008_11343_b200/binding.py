@@ -46,6 +46,10 @@ SIGNATURES = {
     "apms_warmup_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_compressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_compressed_step_host_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int, C.c_void_p]),
+    "apms_worker_phase": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
+    "apms_get_message": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
+    "apms_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64]),
+    "apms_apply_phase": (C.c_int, [C.c_void_p]),
     "apms_get_params": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
     "apms_get_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "apms_get_state_slice": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
@@ -152,6 +156,27 @@ def apms_compressed_step_typed(h, grad_ptrs: Sequence[int], grad_type: int):
 
 def apms_compressed_step_host_typed(h, grad_host_ptrs: Sequence[int], grad_type: int, x_out_host_ptr: Optional[int]):
     _check(h, load().apms_compressed_step_host_typed(h, _ptr_array(grad_host_ptrs), grad_type, x_out_host_ptr))
+
+
+def apms_worker_phase(h, grad_ptrs: Sequence[int], grad_type: int):
+    _check(h, load().apms_worker_phase(h, _ptr_array(grad_ptrs), grad_type))
+
+
+def apms_get_message(h, worker: int):
+    """(device address of the sign words, device address of the scales) of worker `worker` (-1: the server)."""
+    bits, scales = C.c_void_p(), C.c_void_p()
+    _check(h, load().apms_get_message(h, worker, C.byref(bits), C.byref(scales)))
+    return bits.value, scales.value
+
+
+def apms_server_phase(h, bits_rows_ptr: int, row_words: int, scale_rows_ptr: int, row_scales: int, rows: int,
+                      chunk_begin: int, chunk_end: int):
+    _check(h, load().apms_server_phase(h, bits_rows_ptr, row_words, scale_rows_ptr, row_scales, rows,
+                                       chunk_begin, chunk_end))
+
+
+def apms_apply_phase(h):
+    _check(h, load().apms_apply_phase(h))
 
 
 def apms_get_params(h, dst_ptr: int, dst_is_device: bool):
@@ -361,6 +386,32 @@ class Context:
         value = np.ascontiguousarray(value, dtype=np.float32)
         assert value.size == self.d
         apms_set_state(self._h, which, worker, value.ctypes.data)
+
+    # phase-wise step (the caller carries out the exchanges; see paper_2008_11343_b200/sharded.py)
+    def worker_phase(self, grads):
+        assert len(grads) == self.n
+        apms_worker_phase(self._h, self._dev_ptrs(grads), self._grad_type(grads))
+
+    def message(self, worker: int):
+        """Torch views (int32 sign words [W], float32 scales [C]) onto worker `worker`'s message inside the
+        workspace (-1: the server's message).  No copy: the library writes these buffers."""
+        import torch
+
+        bits_ptr, scales_ptr = apms_get_message(self._h, worker)
+        base = self.workspace.data_ptr()
+        b0, s0 = bits_ptr - base, scales_ptr - base
+        bits = self.workspace[b0:b0 + 4 * self.W].view(torch.int32)
+        scales = self.workspace[s0:s0 + 4 * self.C].view(torch.float32)
+        return bits, scales
+
+    def server_phase(self, bits_rows, scale_rows, chunk_begin: int, chunk_end: int):
+        """bits_rows: int32 CUDA tensor [rows, row_words]; scale_rows: float32 CUDA tensor [rows, row_scales]."""
+        assert bits_rows.is_contiguous() and scale_rows.is_contiguous() and bits_rows.shape[0] == scale_rows.shape[0]
+        apms_server_phase(self._h, bits_rows.data_ptr(), bits_rows.shape[1], scale_rows.data_ptr(), scale_rows.shape[1],
+                          bits_rows.shape[0], chunk_begin, chunk_end)
+
+    def apply_phase(self):
+        apms_apply_phase(self._h)
 
     def set_schedule(self, schedule: Optional[Schedule]):
         apms_set_schedule(self._h, schedule)

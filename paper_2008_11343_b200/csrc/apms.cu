@@ -528,7 +528,7 @@ struct ServerArgs {
     float* zbar; uint32_t* Bbar; float* Sbar;
     double* partial;
     Tiling t;
-    int64_t items;                // C * P
+    int64_t item0, items;         // items [item0, items) of the C * P chunk tiles
     int n; float nf;
 };
 
@@ -603,7 +603,7 @@ k_server(const ServerArgs a)
     constexpr int TEAMS = kWarps / WPC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int team = (WPC == 1) ? warp : 0;
-    const int64_t item = (int64_t)blockIdx.x * TEAMS + team;
+    const int64_t item = a.item0 + (int64_t)blockIdx.x * TEAMS + team;
     if (item >= a.items) return;
     const Item it = decode_item(a.t, item);
     const int L = it.L;
@@ -764,7 +764,7 @@ k_server_staged(const ServerStagedArgs sa)
     const int n = NT > 0 ? NT : a.n;
     const size_t stage_bytes = staged_stage_bytes(n, FUSED);
     const int span = MULTI ? sa.span : 1;                  // MULTI = false: one item, the walk's loops fold away
-    const int64_t item0 = (int64_t)blockIdx.x * span;
+    const int64_t item0 = a.item0 + (int64_t)blockIdx.x * span;
     const int nitems = MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1;
 
     if (threadIdx.x == 0) {
@@ -1114,6 +1114,7 @@ struct apms_ctx {
     float beta1, beta2, eps, lr;
     int t;
     int64_t steps;           // steps taken through apms_step (warmup and compressed)
+    int substep;             // phase-wise step: 0 = between steps, 1 = worker phase done, 2 = a server phase done
     apms_schedule sched; bool has_sched;
     apms_phase phase;
     bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar)
@@ -1356,55 +1357,81 @@ cudaError_t launch_staged_n(const ServerStagedArgs& sa, unsigned blocks, size_t 
     }
 }
 
+// Where the server finds the workers' messages: `rows` senders, row j holding sign words and scales
+// addressed by ABSOLUTE word / chunk index (a pointer into a shard is shifted back by the caller).
+struct ServerSource { const uint32_t* B; int64_t Wp; const float* s; int64_t Cp; int rows; };
+
+// Section 3.3 step 4 for chunks [cb, ce).  With may_fuse and a shape that allows it, steps 5-6 for
+// the same chunks run in the same kernel (*applied = true).
+apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int64_t ce, bool may_fuse, bool* applied)
+{
+    *applied = false;
+    ServerArgs a;
+    a.B = src.B; a.Wp = src.Wp; a.s = src.s; a.Cp = src.Cp;
+    a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
+    a.partial = c->partial(c->L.n);
+    a.t = c->L.t; a.item0 = cb * c->L.t.P; a.items = ce * c->L.t.P; a.n = src.rows; a.nf = (float)src.rows;
+    const int64_t count = a.items - a.item0;
+    if (count <= 0) return APMS_OK;
+    const bool staged = use_staged_server(c);
+    const bool warp_teams = !staged && use_warp_teams(c, count);
+    const int64_t blocks = warp_teams ? (count + kWarps - 1) / kWarps : count;
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
+    {
+        Timed t(c, APMS_KERNEL_SERVER);
+        if (staged) {
+            const bool fused = may_fuse && c->L.t.P == 1;   // the CTA sees the whole chunk, so it knows the new scale
+            ServerStagedArgs sa;
+            sa.a = a; sa.status = c->status();
+            sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
+            sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
+            const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
+            sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
+            const int64_t ctas = (count + sa.span - 1) / sa.span;
+            cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)ctas, smem, c->stream)
+                                  : launch_staged_n<false>(sa, (unsigned)ctas, smem, c->stream);
+            if (e != cudaSuccess) {
+                snprintf(c->err, sizeof c->err, "setting up k_server_staged failed: %s", cudaGetErrorString(e));
+                return APMS_ERR_CUDA;
+            }
+            *applied = fused;
+        }
+        else if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+        else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
+        apms_status st = launch_check(c, "k_server");
+        if (st != APMS_OK) return st;
+    }
+    if (c->L.t.P > 1) {
+        // scales of the range's split chunks: the same kernel on the range as a vector of its own
+        Tiling t = c->L.t;
+        t.d = c->L.d - cb * c->L.chunk;
+        const int64_t nchunks = ce - cb;
+        k_finalize_scales<<<(unsigned)((nchunks + 255) / 256), 256, 0, c->stream>>>(c->partial(c->L.n) + cb * c->L.t.P, c->Sbar() + cb,
+                                                                                 1, nchunks, c->L.Cp, t);
+        return launch_check(c, "k_finalize_scales");
+    }
+    return APMS_OK;
+}
+
+// Section 3.3 steps 5-6 over the whole vector, from the server message held in Bbar / Sbar.
+apms_status launch_apply(apms_ctx* c)
+{
+    ApplyArgs a;
+    a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
+    Timed t(c, APMS_KERNEL_APPLY);
+    k_apply<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(a);
+    return launch_check(c, "k_apply");
+}
+
 apms_status launch_server_and_apply(apms_ctx* c)
 {
+    const ServerSource own = {c->B(0), c->L.Wp, c->s(0), c->L.Cp, c->L.n};
     bool applied = false;      // steps 5-6 already done by the fused server kernel
-    {
-        ServerArgs a;
-        a.B = c->B(0); a.Wp = c->L.Wp; a.s = c->s(0); a.Cp = c->L.Cp;
-        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
-        a.partial = c->partial(c->L.n);
-        a.t = c->L.t; a.items = c->L.C * c->L.t.P; a.n = c->L.n; a.nf = (float)c->L.n;
-        const bool staged = use_staged_server(c);
-        const bool warp_teams = !staged && use_warp_teams(c, a.items);
-        const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
-        if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
-        {
-            Timed t(c, APMS_KERNEL_SERVER);
-            if (staged) {
-                const bool fused = c->L.t.P == 1;        // the CTA sees the whole chunk, so it knows the new scale
-                ServerStagedArgs sa;
-                sa.a = a; sa.status = c->status();
-                sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
-                sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
-                const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
-                sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
-                const int64_t ctas = (a.items + sa.span - 1) / sa.span;
-                cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)ctas, smem, c->stream)
-                                      : launch_staged_n<false>(sa, (unsigned)ctas, smem, c->stream);
-                if (e != cudaSuccess) {
-                    snprintf(c->err, sizeof c->err, "setting up k_server_staged failed: %s", cudaGetErrorString(e));
-                    return APMS_ERR_CUDA;
-                }
-                applied = fused;
-            }
-            else if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
-            else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
-            apms_status st = launch_check(c, "k_server");
-            if (st != APMS_OK) return st;
-        }
-        if (c->L.t.P > 1) {
-            apms_status st = launch_finalize(c, c->L.n, 1, c->Sbar());
-            if (st != APMS_OK) return st;
-        }
-    }
+    apms_status st = launch_server(c, own, 0, c->L.C, true, &applied);
+    if (st != APMS_OK) return st;
     if (!applied) {
-        ApplyArgs a;
-        a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
-        a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
-        Timed t(c, APMS_KERNEL_APPLY);
-        k_apply<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(a);
-        apms_status st = launch_check(c, "k_apply");
+        st = launch_apply(c);
         if (st != APMS_OK) return st;
     }
     c->m_is_fp32 = false;      // from now on the momentum is the server's message
@@ -1464,7 +1491,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
-    c->steps = 0; c->has_sched = false;
+    c->steps = 0; c->has_sched = false; c->substep = 0;
     c->fine_run = kFineRunDefault;
     if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
@@ -1554,12 +1581,73 @@ apms_status apms_compressed_step_typed(apms_ctx* c, const void* const* grads_dev
 {
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step needs the COMPRESSED phase (call apms_freeze_v first)");
+    if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "a phase-wise step is in progress (finish it with apms_apply_phase)");
     GradPtrs G;
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
     st = launch_worker(c, G, (int)type, 0, c->L.n);
     if (st != APMS_OK) return st;
     return launch_server_and_apply(c);
+}
+
+apms_status apms_worker_phase(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_worker_phase needs the COMPRESSED phase (call apms_freeze_v first)");
+    if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "the previous phase-wise step is not finished (apms_apply_phase)");
+    GradPtrs G;
+    apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
+    if (st != APMS_OK) return st;
+    st = launch_worker(c, G, (int)type, 0, c->L.n);
+    if (st == APMS_OK) c->substep = 1;
+    return st;
+}
+
+apms_status apms_get_message(apms_ctx* c, int worker, uint32_t** bits_dev, float** scales_dev)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (worker < -1 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range (-1 = the server's message)");
+    apms_status st = ensure_workspace(c);
+    if (st != APMS_OK) return st;
+    if (bits_dev) *bits_dev = worker < 0 ? c->Bbar() : c->B(worker);
+    if (scales_dev) *scales_dev = worker < 0 ? c->Sbar() : c->s(worker);
+    return APMS_OK;
+}
+
+apms_status apms_server_phase(apms_ctx* c, const uint32_t* bits_rows_dev, int64_t row_words, const float* scale_rows_dev,
+                              int64_t row_scales, int rows, int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase needs the COMPRESSED phase");
+    if (c->substep < 1) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase follows apms_worker_phase");
+    if (!bits_rows_dev || !scale_rows_dev) return fail(c, APMS_ERR_INVALID_ARG, "a message pointer is NULL");
+    if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    const int64_t first_elem = chunk_begin * c->L.chunk;
+    const int64_t last_elem = chunk_end * c->L.chunk < c->L.d ? chunk_end * c->L.chunk : c->L.d;
+    const int64_t need_words = (last_elem - first_elem + 31) / 32;
+    // the staged kernel copies sign words in 16-byte pieces: rows must hold the range rounded up to 4 words
+    if (row_words < (need_words + 3) / 4 * 4 || row_words % 4 != 0 || row_scales < chunk_end - chunk_begin)
+        return fail(c, APMS_ERR_INVALID_ARG, "rows too short: row_words must be a multiple of 4 that covers the range's sign words rounded up to 4, row_scales its chunks");
+    if (((uintptr_t)bits_rows_dev & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "bits_rows_dev is not 16-byte aligned");
+    // kernels index by absolute word / chunk: shift the shard's pointers back to where index 0 would be
+    const ServerSource src = {bits_rows_dev - first_elem / 32, row_words, scale_rows_dev - chunk_begin, row_scales, rows};
+    bool applied = false;
+    apms_status st = launch_server(c, src, chunk_begin, chunk_end, false, &applied);
+    if (st == APMS_OK) c->substep = 2;
+    return st;
+}
+
+apms_status apms_apply_phase(apms_ctx* c)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_apply_phase needs the COMPRESSED phase");
+    if (c->substep != 2) return fail(c, APMS_ERR_BAD_STATE, "apms_apply_phase follows apms_server_phase");
+    apms_status st = launch_apply(c);
+    if (st != APMS_OK) return st;
+    c->m_is_fp32 = false;
+    c->substep = 0;
+    return APMS_OK;
 }
 
 apms_status apms_compressed_step_host(apms_ctx* c, const float* const* grads_host, float* x_out_host)
@@ -1571,6 +1659,7 @@ apms_status apms_compressed_step_host_typed(apms_ctx* c, const void* const* grad
 {
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_compressed_step_host needs the COMPRESSED phase (call apms_freeze_v first)");
+    if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "a phase-wise step is in progress (finish it with apms_apply_phase)");
     if (!valid_grad_type((int)type)) return fail(c, APMS_ERR_INVALID_ARG, "unknown gradient type");
     if (!grads_host) return fail(c, APMS_ERR_INVALID_ARG, "gradient pointer array is NULL");
     for (int i = 0; i < c->L.n; ++i)

@@ -1,0 +1,139 @@
+"""A compression-phase step across several processes, one GPU each.
+
+The paper runs its workers on separate GPUs and moves the 1-bit messages with a Gather-Scatter
+AllReduce (Figure 1; Section 3.3 steps 3 and 5): every worker sends the k-th part of its
+compressed momentum to worker k, worker k averages and recompresses what it received, and sends
+the result back to everybody.  `ShardedStep` does exactly that between the phases of the
+library's phase-wise step (apms_worker_phase / apms_server_phase / apms_apply_phase): process r
+holds `n_local` workers and serves a contiguous range of chunks; exchange 1 is a set of
+point-to-point transfers of (sign words, scales) shards, exchange 2 an all-gather of the server
+shards.  Only packed sign words and chunk scales cross the wire (d/8 + 4 C bytes per worker and
+direction instead of 4 d).
+
+The arithmetic stays in the library: this module only slices, sends and receives.  The rows a
+server averages are ordered by global worker index (rank * n_local + i), so P processes with
+n_local workers each give bit for bit the result of one context with P * n_local workers.
+
+`backend` is anything with the attributes d, n, chunk, C, W and the methods worker_phase(grads),
+message(i) -> (sign-word tensor, scale tensor) views (i = -1: the server's message),
+server_phase(bits_rows, scale_rows, chunk_begin, chunk_end) and apply_phase(): a
+`binding.Context` on a GPU, or a CPU stand-in in the tests of the exchange logic.
+"""
+from __future__ import annotations
+
+from typing import List, Sequence, Tuple
+
+
+def chunk_ranges(n_chunks: int, world: int) -> List[Tuple[int, int]]:
+    """Contiguous, near-equal ranges of chunks, one per process (the paper's 'k-th chunk to worker k')."""
+    return [(r * n_chunks // world, (r + 1) * n_chunks // world) for r in range(world)]
+
+
+def word_range(chunk_begin: int, chunk_end: int, chunk: int, d: int) -> Tuple[int, int]:
+    """Sign words [w0, w1) that hold the elements of chunks [chunk_begin, chunk_end)."""
+    first = chunk_begin * chunk
+    last = min(chunk_end * chunk, d)
+    return first // 32, (last + 31) // 32
+
+
+def _round4(words: int) -> int:
+    return (words + 3) // 4 * 4
+
+
+class ShardedStep:
+    def __init__(self, backend, group=None):
+        import torch.distributed as dist
+
+        self.b = backend
+        self.dist = dist
+        self.group = group
+        self.rank = dist.get_rank(group)
+        self.world = dist.get_world_size(group)
+        if backend.C < self.world:
+            raise ValueError(f"{backend.C} chunks cannot be served by {self.world} processes")
+        self.ranges = chunk_ranges(backend.C, self.world)
+        self.words = [word_range(cb, ce, backend.chunk, backend.d) for cb, ce in self.ranges]
+        self.row_words = [_round4(w1 - w0) for w0, w1 in self.words]
+        self.row_scales = [ce - cb for cb, ce in self.ranges]
+        self._buffers = None
+
+    # ------------------------------------------------------------------ buffers (made once)
+    def _make_buffers(self, like_bits, like_scales):
+        import torch
+
+        n, me = self.b.n, self.rank
+        dev = like_bits.device
+        mk = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+        self._buffers = {
+            "send_bits": [mk((n, self.row_words[k]), like_bits.dtype) for k in range(self.world)],
+            "send_scales": [mk((n, self.row_scales[k]), like_scales.dtype) for k in range(self.world)],
+            "recv_bits": mk((self.world * n, self.row_words[me]), like_bits.dtype),
+            "recv_scales": mk((self.world * n, self.row_scales[me]), like_scales.dtype),
+            "gather_bits": mk((self.world, max(self.row_words)), like_bits.dtype),
+            "gather_scales": mk((self.world, max(self.row_scales)), like_scales.dtype),
+            "mine_bits": mk((max(self.row_words),), like_bits.dtype),
+            "mine_scales": mk((max(self.row_scales),), like_scales.dtype),
+        }
+
+    def global_rank(self, k: int) -> int:
+        return k if self.group is None else self.dist.get_global_rank(self.group, k)
+
+    # ------------------------------------------------------------------ the step
+    def step(self, grads: Sequence) -> None:
+        """Section 3.3 steps 1-6 for this process's workers; `grads`: its n_local gradients."""
+        b, dist, n, me = self.b, self.dist, self.b.n, self.rank
+        b.worker_phase(grads)                                                   # steps 1-2
+        msgs = [b.message(i) for i in range(n)]
+        if self._buffers is None:
+            self._make_buffers(msgs[0][0], msgs[0][1])
+        buf = self._buffers
+
+        # step 3 (exchange 1): the part of every local message that process k serves goes to process k
+        for k in range(self.world):
+            (w0, w1), (cb, ce) = self.words[k], self.ranges[k]
+            for i, (bits, scales) in enumerate(msgs):
+                buf["send_bits"][k][i, :w1 - w0].copy_(bits[w0:w1])
+                buf["send_scales"][k][i].copy_(scales[cb:ce])
+        ops = []
+        for k in range(self.world):
+            rows = slice(k * n, (k + 1) * n)
+            if k == me:
+                buf["recv_bits"][rows].copy_(buf["send_bits"][k])
+                buf["recv_scales"][rows].copy_(buf["send_scales"][k])
+                continue
+            peer = self.global_rank(k)
+            ops.append(dist.P2POp(dist.isend, buf["send_bits"][k], peer, self.group))
+            ops.append(dist.P2POp(dist.isend, buf["send_scales"][k], peer, self.group))
+            ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][rows], peer, self.group))
+            ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][rows], peer, self.group))
+        if ops:
+            for req in dist.batch_isend_irecv(ops):
+                req.wait()
+
+        # step 4: average and recompress the chunks this process serves
+        cb, ce = self.ranges[me]
+        b.server_phase(buf["recv_bits"], buf["recv_scales"], cb, ce)
+
+        # step 5 (exchange 2): every process's range of the server message goes to everybody
+        sbits, sscales = b.message(-1)
+        w0, w1 = self.words[me]
+        buf["mine_bits"][:w1 - w0].copy_(sbits[w0:w1])
+        buf["mine_scales"][:ce - cb].copy_(sscales[cb:ce])
+        if self.world > 1:
+            dist.all_gather_into_tensor(buf["gather_bits"].view(-1), buf["mine_bits"], group=self.group)
+            dist.all_gather_into_tensor(buf["gather_scales"].view(-1), buf["mine_scales"], group=self.group)
+            for k in range(self.world):
+                if k == me:
+                    continue
+                (v0, v1), (kb, ke) = self.words[k], self.ranges[k]
+                sbits[v0:v1].copy_(buf["gather_bits"][k, :v1 - v0])
+                sscales[kb:ke].copy_(buf["gather_scales"][k, :ke - kb])
+
+        b.apply_phase()                                                         # steps 5-6
+
+    def wire_bytes_per_step(self) -> int:
+        """Bytes this process sends per step (both exchanges), for comparison with 4 d per worker."""
+        n, me = self.b.n, self.rank
+        ex1 = sum(4 * n * (self.row_words[k] + self.row_scales[k]) for k in range(self.world) if k != me)
+        ex2 = (self.world - 1) * 4 * (self.row_words[me] + self.row_scales[me])
+        return ex1 + ex2

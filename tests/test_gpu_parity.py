@@ -158,6 +158,79 @@ def test_error_norms_match_the_oracle_state():
     assert fresh.error_norms() == ([0.0] * w.n, 0.0)
 
 
+# ------------------------------------------------------------------ phase-wise step (the multi-process form)
+
+@pytest.mark.parametrize("d,n,chunk,cuts", [(9 * 2048 + 300, 4, 2048, (0, 3, 10)), (5 * 4096 + 1, 3, 4096, (0, 1, 5, 6)),
+                                            (7 * 96 + 5, 5, 96, (0, 4, 8)), (3 * 70016, 2, 70016, (0, 2, 3)),
+                                            (6 * 32768, 16, 32768, (0, 6))])
+def test_phase_wise_step_equals_the_whole_step(d, n, chunk, cuts):
+    """worker phase, the server phase range by range from COPIES of the messages laid out as a receiver would
+    hold them (rows = senders, word 0 = first word of the range), apply phase: bit-identical to apms_compressed_step."""
+    import torch
+
+    w = tiny(d, n, chunk, cfg_id=140)
+    a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    for c in (a, b):
+        c.set_params(wl.initial_params(w))
+        c.warmup_step(H.upload(wl.host_gradients(w, 0)))
+        c.freeze_v()
+    assert cuts[-1] == a.C
+    for step in range(1, 5):
+        gs = H.upload(wl.host_gradients(w, step))
+        a.compressed_step(gs)
+        b.worker_phase(gs)
+        msgs = [b.message(i) for i in range(n)]
+        for cb, ce in zip(cuts, cuts[1:]):
+            w0, w1 = cb * chunk // 32, (min(d, ce * chunk) + 31) // 32
+            row_words = (w1 - w0 + 3) // 4 * 4
+            bits_rows = torch.zeros((n, row_words), dtype=torch.int32, device="cuda")
+            scale_rows = torch.zeros((n, ce - cb), dtype=torch.float32, device="cuda")
+            for i, (bits, scales) in enumerate(msgs):
+                bits_rows[i, :w1 - w0] = bits[w0:w1]
+                scale_rows[i] = scales[cb:ce]
+            b.server_phase(bits_rows, scale_rows, cb, ce)
+        with pytest.raises(B.ApmsError) as e:
+            b.compressed_step(gs)                              # a phase-wise step is in progress
+        assert e.value.status == B.ERR_BAD_STATE
+        b.apply_phase()
+        for k in range(9):
+            for i in (range(n) if k in (3, 4, 5) else [0]):
+                assert np.array_equal(a.get_state(k, i).view(np.uint32), b.get_state(k, i).view(np.uint32)), (step, k, i)
+    with pytest.raises(B.ApmsError) as e:
+        b.apply_phase()                                        # nothing to apply
+    assert e.value.status == B.ERR_BAD_STATE
+
+
+def test_sharded_step_with_one_process_equals_the_whole_step():
+    import socket
+
+    import torch.distributed as dist
+
+    from paper_2008_11343_b200 import sharded
+
+    w = tiny(11 * 2048 + 77, 4, 2048, cfg_id=141)
+    a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    for c in (a, b):
+        c.set_params(wl.initial_params(w))
+        c.freeze_v()
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    try:
+        step = sharded.ShardedStep(b)
+        for k in range(3):
+            gs = H.upload(wl.host_gradients(w, k))
+            a.compressed_step(gs)
+            step.step(gs)
+        for k in (B.STATE_X, B.STATE_M, B.STATE_SERVER_ERR, B.STATE_SERVER_BITS, B.STATE_SERVER_SCALES):
+            assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32))
+    finally:
+        dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------ the benchmark's small configurations
 
 def test_config0_free_running_10_steps():

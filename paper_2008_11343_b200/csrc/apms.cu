@@ -1387,6 +1387,8 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
             sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
             const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
             sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
+            const int64_t fill = count / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
+            if (sa.span > 1 && fill < sa.span) sa.span = fill < 1 ? 1 : (int)fill;
             const int64_t ctas = (count + sa.span - 1) / sa.span;
             cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)ctas, smem, c->stream)
                                   : launch_staged_n<false>(sa, (unsigned)ctas, smem, c->stream);

@@ -100,6 +100,16 @@ typedef enum {
     APMS_GRAD_F16 = 2     /* IEEE binary16 */
 } apms_grad_type;
 
+/* The "magnitude" in the scaling factor of Section 5.1.  The default reads it as the paper's norm:
+ * scale = ||z||_2 / sqrt(L), so that the decompressed chunk has the l2 norm of the compensated one.
+ * The other common reading, the mean of |z| (the least-squares scale of a sign vector), is offered as
+ * a switch; it applies to the worker and the server compressor of the following steps (and runs on
+ * the library's general kernels, not on the forms tuned for the default). */
+typedef enum {
+    APMS_SCALE_L2 = 0,
+    APMS_SCALE_L1_MEAN = 1
+} apms_scale_kind;
+
 /* How threads are grouped on a tile of a chunk in the worker and server kernels. */
 typedef enum {
     APMS_TEAM_AUTO = 0,   /* the library's choice for the shape (the forms below, per kernel)      */
@@ -268,6 +278,9 @@ apms_status apms_error_norms(apms_ctx* ctx, double* worker_sq_host, double* serv
 
 apms_phase  apms_get_phase(const apms_ctx* ctx);
 int         apms_get_t(const apms_ctx* ctx);
+
+/* Choose the scale definition (see apms_scale_kind); any phase, takes effect from the next step. */
+apms_status apms_set_scale_kind(apms_ctx* ctx, apms_scale_kind kind);
 
 /* Launch-shape override (tuning and tests); results do not depend on it except for the order
  * of the binary64 additions inside a chunk's sum of squares. */

@@ -25,6 +25,7 @@ KERNEL_WARMUP_ADAM, KERNEL_WORKER, KERNEL_SERVER, KERNEL_APPLY = range(4)
 KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
 TEAM_AUTO, TEAM_CTA, TEAM_WARP, TEAM_STAGED = range(4)
 GRAD_F32, GRAD_BF16, GRAD_F16 = range(3)
+SCALE_L2, SCALE_L1_MEAN = range(2)
 MAX_WORKERS = 64
 NOALLOC_MAX_TILES = 16384
 
@@ -62,6 +63,7 @@ SIGNATURES = {
     "apms_error_norms": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "apms_get_phase": (C.c_int, [C.c_void_p]),
     "apms_get_t": (C.c_int, [C.c_void_p]),
+    "apms_set_scale_kind": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
@@ -235,6 +237,10 @@ def apms_get_phase(h) -> int:
 
 def apms_get_t(h) -> int:
     return int(load().apms_get_t(h))
+
+
+def apms_set_scale_kind(h, kind: int):
+    _check(h, load().apms_set_scale_kind(h, kind))
 
 
 def apms_set_team_mode(h, mode: int):
@@ -438,6 +444,9 @@ class Context:
     @property
     def t(self) -> int:
         return apms_get_t(self._h)
+
+    def set_scale_kind(self, kind: int):
+        apms_set_scale_kind(self._h, kind)
 
     def set_team_mode(self, mode: int):
         apms_set_team_mode(self._h, mode)

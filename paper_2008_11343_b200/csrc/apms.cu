@@ -134,6 +134,19 @@ __device__ __forceinline__ float apply_elem(float x, float v, float q, float lr,
     return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));
 }
 
+// One element's contribution to a chunk's scale, and the scale from the sum.  The scale is the
+// l2 norm of the chunk over sqrt(L) (Section 5.1 read with the paper's norm); the other reading
+// of "magnitude", the mean of |z|, is kept as a switch: |z| = z * (+-1) is added by the same fma.
+__device__ __forceinline__ void scale_accumulate(double& acc, float z, bool l1)
+{
+    const double zd = (double)z;
+    acc = fma(zd, l1 ? copysign(1.0, zd) : zd, acc);
+}
+__device__ __forceinline__ float scale_from_sum(double total, double L, bool l1)
+{
+    return l1 ? (float)(total / L) : (float)sqrt(total / L);
+}
+
 // The compression error implied by a stored compensated value and its chunk's scale.
 __device__ __forceinline__ float implied_error(float z, float s) { return __fsub_rn(z, signed_scale(z, s)); }
 
@@ -239,6 +252,7 @@ struct Tiling {
     int64_t d, chunk, tile;   // tile == chunk when P == 1
     int P;                    // tiles per chunk
     int64_t Pp;               // row stride of the partial-sum arrays (>= C * P)
+    int l1 = 0;               // scale = mean |z| instead of ||z||_2 / sqrt(L)
 };
 
 struct Item { int64_t c; int p; int64_t base; int L; int Lc; };
@@ -285,7 +299,7 @@ struct WorkerArgs {
 template <bool M32, bool CHECKED>
 __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __restrict__ z, uint32_t* __restrict__ obits,
                                              int grp, int lane, int L, float s_old, float Sbar,
-                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc)
+                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc, bool l1)
 {
     const int k = grp * kGroup + lane * 4;
     float mm[4];
@@ -307,8 +321,7 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
         zn[e] = __fadd_rn(mi, err);                                             // compensated
         const bool valid = !CHECKED || (k + e < L);
         if (valid) {
-            const double zd = (double)zn[e];
-            acc = fma(zd, zd, acc);
+            scale_accumulate(acc, zn[e], l1);
             nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
         }
     }
@@ -363,7 +376,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 #pragma unroll
         for (int u = 0; u < U; ++u)
             worker_group<M32, false>(a.beta1, a.omb1, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
-                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc);
+                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc, a.t.l1 != 0);
     }
     // remainder: one group at a time, bounds-checked
     for (; g0 < ngroups; g0 += WPC) {
@@ -374,12 +387,12 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         uint32_t mw = 0;
         if (M32) mv = ld4_checked(m32, k, L, false);
         else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
-        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc);
+        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc, a.t.l1 != 0);
     }
 
     const double total = team_sum<WPC>(acc, red);
     if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
-        if (a.t.P == 1) *sptr = (float)sqrt(total / (double)it.Lc);          // ||z||_2 / sqrt(L)
+        if (a.t.P == 1) *sptr = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);    // ||z||_2 / sqrt(L)
         else a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p] = total;
     }
 }
@@ -479,7 +492,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
             const float4 zv = ld4_checked(z, k, L, true);
             const uint32_t mw = (k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
             worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
-                                      make_float4(0, 0, 0, 0), mw, acc);
+                                      make_float4(0, 0, 0, 0), mw, acc, false);
         }
     }
     acc = warp_sum(acc);
@@ -515,7 +528,7 @@ __global__ void k_finalize_scales(const double* __restrict__ partial, float* __r
     const int64_t Lc = (t.d - cbeg < t.chunk) ? t.d - cbeg : t.chunk;
     double total = 0.0;
     for (int p = 0; p < t.P; ++p) total += partial[(int64_t)r * t.Pp + c * t.P + p];
-    scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+    scales[(int64_t)r * Cp + c] = scale_from_sum(total, (double)Lc, t.l1 != 0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -581,8 +594,7 @@ __device__ __forceinline__ void server_groups(const ServerArgs& a, const float* 
             zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
             const bool valid = !CHECKED || (k + e < L);
             if (valid) {
-                const double zd = (double)zn[e];
-                acc = fma(zd, zd, acc);
+                scale_accumulate(acc, zn[e], a.t.l1 != 0);
                 nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
             }
         }
@@ -630,7 +642,7 @@ k_server(const ServerArgs a)
         server_groups<1, true>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
     const double total = team_sum<WPC>(acc, red);
     if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
-        if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+        if (a.t.P == 1) a.Sbar[it.c] = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);
         else a.partial[it.c * a.t.P + it.p] = total;
     }
 }
@@ -1243,6 +1255,7 @@ apms_status device_status_check(apms_ctx* c)
 bool use_staged_server(const apms_ctx* c)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
+    if (c->L.t.l1) return false;             // the mean-|z| scale exists in the register-staged kernels only
     return c->L.chunk % kSlab == 0;
 }
 
@@ -1264,6 +1277,7 @@ apms_status launch_finalize(apms_ctx* c, int first_row, int rows, float* scales)
 bool use_fine_worker(const apms_ctx* c)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
+    if (c->L.t.l1) return false;             // see use_staged_server
     return !c->m_is_fp32 && c->L.fine_tiles > 0;
 }
 
@@ -1885,6 +1899,14 @@ apms_status apms_error_norms(apms_ctx* c, double* worker_sq_host, double* server
 
 apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }
 int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
+
+apms_status apms_set_scale_kind(apms_ctx* c, apms_scale_kind kind)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (kind != APMS_SCALE_L2 && kind != APMS_SCALE_L1_MEAN) return fail(c, APMS_ERR_INVALID_ARG, "unknown scale kind");
+    c->L.t.l1 = kind == APMS_SCALE_L1_MEAN ? 1 : 0;
+    return APMS_OK;
+}
 
 apms_status apms_set_team_mode(apms_ctx* c, apms_team_mode mode)
 {

@@ -113,6 +113,28 @@ def test_sixteen_bit_host_gradients_and_alignment():
     assert e.value.status == B.ERR_INVALID_ARG
 
 
+# ------------------------------------------------------------------ the other reading of the scale
+
+@pytest.mark.parametrize("team", [B.TEAM_AUTO, B.TEAM_CTA, B.TEAM_WARP], ids=["auto", "cta-per-tile", "warp-per-tile"])
+@pytest.mark.parametrize("d,n,chunk", [(5 * 4096 + 1234, 3, 4096), (3 * 1024 + 5, 4, 96), (3 * 70016, 2, 70016),
+                                       (2 * 32768 + 23552, 16, 32768), (9 * 512 + 3, 2, 512)])
+def test_mean_absolute_scale_matches_the_oracle_switch(d, n, chunk, team):
+    """scale = mean |z| on both sides (the oracle's switch, the library's apms_set_scale_kind): bit-identical state."""
+    w = tiny(d, n, chunk, cfg_id=150, warmup_steps=1, compressed_steps=4)
+    ctx, orc = H.make_pair(w, team_mode=team)
+    ctx.set_scale_kind(B.SCALE_L1_MEAN)
+    orc.set_scale_kind(ao.SCALE_L1_MEAN)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(1, 5):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        H.compare_state(ctx, orc, w, exact=True)
+    z = np.abs(orc.m[:min(chunk, d)].astype(np.float64) + orc.server_err[:min(chunk, d)])    # |zbar| of chunk 0
+    assert abs(float(ctx.get_state(B.STATE_SERVER_SCALES)[0]) - z.mean()) <= 1e-6 * z.mean()
+
+
 # ------------------------------------------------------------------ phase driver and error monitor
 
 def test_scheduled_steps_follow_algorithm_1():

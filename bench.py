@@ -38,7 +38,7 @@ UNIT = "worker-elements/s"
 # DRAM traffic of the worker kernel measured once with ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum per launch) on a smaller case of the same kernel, in bytes per
 # worker-element; scaled by n*d for the benchmarked launch.  Source: profiles/*.md.
-NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT = 11.95    # k_worker_fine, profiles/k_worker_fine_small_case.md
+NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT = 11.96    # k_worker_fine, profiles/k_worker_fine_small_case.md
 
 
 def algorithmic_bytes(d: int, n: int, chunk: int, grad_bytes: int = 4) -> dict:

@@ -499,21 +499,25 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     if (lane == 0) *slot = acc;
 }
 
-// Scales from the fine form's partial sums (one per 512 elements): a chunk's slots added in
-// element order, then sqrt(sum / L).
-__global__ void k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
-                                int rows, int64_t C, int64_t d, int64_t chunk)
+// Scales from the fine form's partial sums (one per 512 elements): one warp per (row, chunk) adds
+// the chunk's slots in a fixed order (lane l takes slots l, l + 32, ..., then the shuffle tree)
+// and takes sqrt(sum / L).
+__global__ void __launch_bounds__(kThreads)
+k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
+                int rows, int64_t C, int64_t d, int64_t chunk)
 {
-    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (int64_t)rows * C) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t idx = (int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (idx >= (int64_t)rows * C) return;                        // whole warps
     const int r = (int)(idx / C);
     const int64_t c = idx % C;
     const int64_t cbeg = c * chunk;
     const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
     const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
     double total = 0.0;
-    for (int64_t q = q0; q < q1; ++q) total += partial[(int64_t)r * Pp + q];
-    scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+    for (int64_t q = q0 + lane; q < q1; q += 32) total += partial[(int64_t)r * Pp + q];
+    total = warp_sum(total);
+    if (lane == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
 // Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).
@@ -1302,7 +1306,7 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
         apms_status st = launch_check(c, "k_worker_fine");
         if (st != APMS_OK) return st;
         const int64_t total = (int64_t)ni * c->L.C;
-        k_finalize_fine<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0),
+        k_finalize_fine<<<(unsigned)((total + kWarps - 1) / kWarps), kThreads, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0),
                                                                              c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk);
         st = launch_check(c, "k_finalize_fine");
         if (st != APMS_OK) return st;

@@ -33,6 +33,9 @@
  *   - The compressed-phase denominator is sqrt(v_Tw) + eps with the raw
  *     (not bias-corrected) frozen v; eps plays the role of Adam's constant.
  *   - The average is over all n workers, summed in worker order, divided by n.
+ *   - The gradient variant (Section 5.3, item 4) is described in one sentence; read as: workers
+ *     send C[g_i + delta_i], servers average and recompress as in the method, and every worker
+ *     forms m <- b1 m + (1-b1) g^ from the received g^ and updates the model with that m.
  *   - Arithmetic: IEEE binary32, every named operation rounded once, no
  *     contraction other than the fmaf written; sums of squares are accumulated
  *     in binary64 in element order and rounded to binary32 after the sqrt.
@@ -54,6 +57,12 @@
 
 enum { ORACLE_COMPRESSOR_ONEBIT = 0, ORACLE_COMPRESSOR_IDENTITY = 1 };
 enum { ORACLE_SCALE_L2 = 0, ORACLE_SCALE_L1_MEAN = 1 };
+/* What the workers compress and send.  MOMENTUM is the method (Section 3.3).  GRADIENT is the
+ * "APGSqueeze" variant of Section 5.3 (Implementations and setups, item 4): the error-compensated
+ * compression is applied to the gradient g_t instead of the momentum; what comes back from the
+ * servers is then a compressed averaged gradient, from which every worker updates the (uncompressed,
+ * identical) momentum m <- b1 m + (1-b1) g^ before the model update with the frozen variance. */
+enum { ORACLE_VARIANT_MOMENTUM = 0, ORACLE_VARIANT_GRADIENT = 1 };
 
 typedef struct apms_oracle {
     int64_t d;          /* parameters */
@@ -66,6 +75,7 @@ typedef struct apms_oracle {
     int   frozen;       /* 0 = warmup phase, 1 = compression phase */
     int   compressor;   /* ORACLE_COMPRESSOR_* */
     int   scale_kind;   /* ORACLE_SCALE_* */
+    int   variant;      /* ORACLE_VARIANT_* */
     int   threads;      /* OpenMP threads over chunks (chunks are independent) */
     float *x, *m, *v;   /* d each */
     float *ebar;        /* server error, d */
@@ -146,6 +156,7 @@ void apms_oracle_set_params(apms_oracle *o, const float *x0)
 void apms_oracle_set_lr(apms_oracle *o, float lr) { o->lr = lr; }
 void apms_oracle_set_compressor(apms_oracle *o, int c) { o->compressor = c; }
 void apms_oracle_set_scale_kind(apms_oracle *o, int k) { o->scale_kind = k; }
+void apms_oracle_set_variant(apms_oracle *o, int v) { o->variant = v; }
 void apms_oracle_set_threads(apms_oracle *o, int t) { o->threads = t < 1 ? 1 : t; }
 int  apms_oracle_max_threads(void)
 {
@@ -222,7 +233,9 @@ static void compressed_step_chunk(apms_oracle *o, const float *const *g, int64_t
         float *e = o->e + (size_t)i * (size_t)o->d + lo;
         float *qi = q + (size_t)i * (size_t)L;
         for (int64_t j = 0; j < L; ++j) {
-            const float mi = fmaf(o->beta1, o->m[lo + j], omb1 * g[i][lo + j]);
+            const float mi = (o->variant == ORACLE_VARIANT_GRADIENT)
+                                 ? g[i][lo + j]                                      /* the gradient itself is sent */
+                                 : fmaf(o->beta1, o->m[lo + j], omb1 * g[i][lo + j]);
             z[j] = mi + e[j];
         }
         if (o->compressor == ORACLE_COMPRESSOR_IDENTITY) {
@@ -251,10 +264,12 @@ static void compressed_step_chunk(apms_oracle *o, const float *const *g, int64_t
     for (int64_t j = 0; j < L; ++j) o->ebar[lo + j] = z[j] - qb[j];
 
     /* Steps 5-6 on every worker (all identical): the received chunk replaces the
-     * momentum; model update preconditioned by the frozen variance. */
+     * momentum (gradient variant: it is the gradient the momentum is updated with);
+     * model update preconditioned by the frozen variance. */
     for (int64_t j = 0; j < L; ++j) {
-        o->m[lo + j] = qb[j];
-        o->x[lo + j] = o->x[lo + j] - (o->lr * qb[j]) / (sqrtf(o->v[lo + j]) + o->eps);
+        if (o->variant == ORACLE_VARIANT_GRADIENT) o->m[lo + j] = fmaf(o->beta1, o->m[lo + j], omb1 * qb[j]);
+        else                                       o->m[lo + j] = qb[j];
+        o->x[lo + j] = o->x[lo + j] - (o->lr * o->m[lo + j]) / (sqrtf(o->v[lo + j]) + o->eps);
     }
     free(z); free(q); free(qb);
 }

@@ -13,6 +13,7 @@ import numpy as np
 from . import build as _build
 
 ONEBIT, IDENTITY = 0, 1
+VARIANT_MOMENTUM, VARIANT_GRADIENT = 0, 1
 SCALE_L2, SCALE_L1_MEAN = 0, 1
 
 _F = C.POINTER(C.c_float)
@@ -37,7 +38,7 @@ def _declare(L: C.CDLL) -> C.CDLL:
     L.apms_oracle_destroy.argtypes = [vp]
     L.apms_oracle_set_params.argtypes = [vp, _F]
     L.apms_oracle_set_lr.argtypes = [vp, C.c_float]
-    for f in ("set_compressor", "set_scale_kind", "set_threads"):
+    for f in ("set_compressor", "set_scale_kind", "set_threads", "set_variant"):
         getattr(L, "apms_oracle_" + f).argtypes = [vp, C.c_int]
     L.apms_oracle_max_threads.restype = C.c_int
     for f in ("x", "m", "v", "server_err", "server_scales"):
@@ -118,6 +119,9 @@ class Oracle:
 
     def set_compressor(self, kind: int):
         self._L.apms_oracle_set_compressor(self._h, kind)
+
+    def set_variant(self, variant: int):
+        self._L.apms_oracle_set_variant(self._h, variant)
 
     def set_scale_kind(self, kind: int):
         self._L.apms_oracle_set_scale_kind(self._h, kind)

@@ -302,6 +302,91 @@ def check_identity_compressor_closed_form(lib):
     np.testing.assert_allclose(o.x, x, rtol=0, atol=1e-6 * np.abs(x).max())
 
 
+# ------------------------------------------------------------------ the gradient-compressing variant
+
+def check_gradient_variant_worked_example(lib):
+    """Hand-derived step of the gradient-compressing variant (Section 5.3, item 4) in exact dyadic numbers."""
+    f = read_fixture("gradient_variant_worked_example.txt")
+    o = ao.Oracle(4, 2, f["beta1"][0], 0.999, f["eps"][0], f["lr"][0], 32, library=lib)
+    o.set_params(np.zeros(4, dtype=np.float32))
+    o.freeze_v()
+    o.set_variant(ao.VARIANT_GRADIENT)
+    o.m[:], o.v[:], o.x[:] = f["m"], f["v"], f["x"]
+    o.worker_err(0)[:], o.worker_err(1)[:], o.server_err[:] = f["e0"], f["e1"], f["ebar"]
+    o.compressed_step([np.array(f["g0"], np.float32), np.array(f["g1"], np.float32)])
+    assert o.worker_scales(0)[0] == f["expect_scale0"][0] and o.worker_scales(1)[0] == f["expect_scale1"][0]
+    assert int(o.worker_bits(0)[0]) == int(f["expect_bits0"][0]) and int(o.worker_bits(1)[0]) == int(f["expect_bits1"][0])
+    assert np.array_equal(o.worker_err(0), np.array(f["expect_e0"], np.float32))
+    assert np.array_equal(o.worker_err(1), np.array(f["expect_e1"], np.float32))
+    assert o.server_scales[0] == f["expect_Sbar"][0] and int(o.server_bits[0]) == int(f["expect_Bbar"][0])
+    assert np.array_equal(o.server_err, np.array(f["expect_ebar"], np.float32))
+    assert np.array_equal(o.m, np.array(f["expect_m"], np.float32))
+    assert np.array_equal(o.x, np.array(f["expect_x"], np.float32))
+
+
+def check_gradient_variant_identity_is_momentum_sgd(lib):
+    """Gradient variant with C = identity: nothing is lost, so the run is momentum SGD on the averaged
+    gradient with the frozen preconditioner - checked against torch.optim.SGD (momentum = dampening =
+    beta1, binary64) fed with the preconditioned gradient gbar/(sqrt v + eps)."""
+    import torch
+
+    rng = np.random.default_rng(23)
+    d, n, chunk, steps = 150, 3, 64, 10
+    beta, lr, eps = (float(np.float32(h)) for h in (0.9, 1e-2, 1e-8))
+    o = _frozen(lib, d, n, chunk, beta1=beta, lr=lr, eps=eps)
+    o.set_compressor(ao.IDENTITY)
+    o.set_variant(ao.VARIANT_GRADIENT)
+    _rand_state(o, rng, err_scale=0.0)
+    pre = 1.0 / (np.sqrt(o.v.astype(np.float64)) + eps)
+    p = torch.nn.Parameter(torch.tensor(o.x.astype(np.float64)))
+    opt = torch.optim.SGD([p], lr=lr, momentum=beta, dampening=float(np.float32(beta)))
+    # dampening must be beta1 as binary32 rounds 1 - beta1: use the oracle's own (1 - beta1)
+    opt.param_groups[0]["dampening"] = 1.0 - float(np.float32(1) - np.float32(beta))
+    opt.state[p]["momentum_buffer"] = torch.tensor(o.m.astype(np.float64) * pre)     # m/(sqrt v + eps) evolves linearly
+    x0 = o.x.astype(np.float64).copy()
+    for _ in range(steps):
+        gs = [(rng.standard_normal(d) * 1e-2).astype(np.float32) for _ in range(n)]
+        o.compressed_step(gs)
+        p.grad = torch.tensor(np.mean(np.stack(gs).astype(np.float64), axis=0) * pre)
+        opt.step()
+        assert not o.server_err.any() and not any(o.worker_err(i).any() for i in range(n))
+    ref = p.detach().numpy()
+    assert np.abs(o.x - ref).max() <= 2e-6 * np.abs(ref - x0).max() + 1e-7 * np.abs(ref).max()
+    np.testing.assert_allclose(o.m * pre, opt.state[p]["momentum_buffer"].numpy(), rtol=0,
+                               atol=2e-6 * np.abs(o.m * pre).max())
+
+
+def check_gradient_variant_invariants(lib):
+    """Gradient variant, 1-bit compressor: ghat_t + dbar_t = gbar_t + dbar_{t-1} (the telescoping of
+    Supplement A written for the gradient), m_t = beta m_{t-1} + (1-beta) ghat_t with ghat_t the
+    decompressed server message, and x moves by -lr m_t/(sqrt v + eps) with the NEW momentum."""
+    rng = np.random.default_rng(29)
+    d, n, chunk, steps = 3 * 96 + 20, 4, 96, 8
+    beta, lr, eps = 0.9, 2e-3, 1e-6
+    b, omb = float(np.float32(beta)), float(np.float32(1) - np.float32(beta))
+    o = _frozen(lib, d, n, chunk, beta1=beta, lr=lr, eps=eps)
+    o.set_variant(ao.VARIANT_GRADIENT)
+    _rand_state(o, rng)
+    pre = float(np.float32(lr)) / (np.sqrt(o.v.astype(np.float64)) + float(np.float32(eps)))
+
+    def dbar():
+        return sum(o.worker_err(i).astype(np.float64) for i in range(n)) / n + o.server_err
+
+    for _ in range(steps):
+        m_prev, x_prev, dbar_prev = o.m.astype(np.float64), o.x.astype(np.float64), dbar()
+        gs = [(rng.standard_normal(d) * 2e-3).astype(np.float32) for _ in range(n)]
+        gbar = np.mean(np.stack(gs).astype(np.float64), axis=0)
+        o.compressed_step(gs)
+        ghat = np.concatenate([ao.decompress_1bit(o.server_bits[c * chunk // 32:], o.server_scales[c],
+                                                  min(d, (c + 1) * chunk) - c * chunk, library=lib)
+                               for c in range(o.C)]).astype(np.float64)
+        rhs = gbar + dbar_prev
+        np.testing.assert_allclose(ghat + dbar(), rhs, rtol=0, atol=1e-6 * np.abs(rhs).max())
+        np.testing.assert_allclose(o.m, b * m_prev + omb * ghat, rtol=0, atol=2e-7 * np.abs(ghat).max())
+        step = pre * o.m.astype(np.float64)
+        np.testing.assert_allclose(x_prev - o.x, step, rtol=0, atol=1e-6 * np.abs(step).max() + 2e-7 * np.abs(x_prev).max())
+
+
 def check_phase_switch(lib):
     """After warmup: v stays fixed, raw m carries over, all errors start at zero (Algorithm 1
     initialisation; Section 3.3 first paragraph)."""
@@ -457,4 +542,7 @@ ALL_CHECKS = [
     check_phase_switch,
     check_metamorphic,
     check_bruteforce_exact,
+    check_gradient_variant_worked_example,
+    check_gradient_variant_identity_is_momentum_sgd,
+    check_gradient_variant_invariants,
 ]

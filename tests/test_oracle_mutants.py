@@ -23,7 +23,7 @@ MUTANTS = [
     ("server_error_not_updated", "o->ebar[lo + j] = z[j] - qb[j];", "o->ebar[lo + j] = z[j];"),
     ("momentum_not_replaced", "o->m[lo + j] = qb[j];", "o->m[lo + j] = z[j];"),
     ("precondition_without_sqrt", "(sqrtf(o->v[lo + j]) + o->eps)", "(o->v[lo + j] + o->eps)"),
-    ("update_sign", "o->x[lo + j] - (o->lr * qb[j])", "o->x[lo + j] + (o->lr * qb[j])"),
+    ("update_sign", "o->x[lo + j] - (o->lr * o->m[lo + j])", "o->x[lo + j] + (o->lr * o->m[lo + j])"),
     ("beta_swapped", "fmaf(o->beta1, o->m[lo + j], omb1 * g[i][lo + j])",
      "fmaf(omb1, o->m[lo + j], o->beta1 * g[i][lo + j])"),
     ("all_workers_use_gradient_0", "omb1 * g[i][lo + j]", "omb1 * g[0][lo + j]"),
@@ -34,8 +34,14 @@ MUTANTS = [
     ("adam_gradient_not_averaged", "const float gbar = gs / (float)o->n;", "const float gbar = gs;"),
     ("adam_v_not_squared", "omb2 * (gbar * gbar)", "omb2 * gbar"),
     ("adam_bc2_uses_beta1", "pow((double)o->beta2, (double)o->t)", "pow((double)o->beta1, (double)o->t)"),
-    ("v_keeps_updating", "o->x[lo + j] = o->x[lo + j] - (o->lr * qb[j])",
-     "o->v[lo + j] = 0.999f * o->v[lo + j]; o->x[lo + j] = o->x[lo + j] - (o->lr * qb[j])"),
+    ("v_keeps_updating", "o->x[lo + j] = o->x[lo + j] - (o->lr * o->m[lo + j])",
+     "o->v[lo + j] = 0.999f * o->v[lo + j]; o->x[lo + j] = o->x[lo + j] - (o->lr * o->m[lo + j])"),
+    ("gradient_variant_sends_momentum", "? g[i][lo + j]                                      /* the gradient itself is sent */",
+     "? fmaf(o->beta1, o->m[lo + j], omb1 * g[i][lo + j])"),
+    ("gradient_variant_momentum_replaced", "o->m[lo + j] = fmaf(o->beta1, o->m[lo + j], omb1 * qb[j]);", "o->m[lo + j] = qb[j];"),
+    ("gradient_variant_betas_swapped", "fmaf(o->beta1, o->m[lo + j], omb1 * qb[j])", "fmaf(omb1, o->m[lo + j], o->beta1 * qb[j])"),
+    ("gradient_variant_update_uses_gradient", "else                                       o->m[lo + j] = qb[j];",
+     "else                                       o->m[lo + j] = qb[j];\n        if (o->variant == ORACLE_VARIANT_GRADIENT) { o->x[lo + j] = o->x[lo + j] - (o->lr * qb[j]) / (sqrtf(o->v[lo + j]) + o->eps); continue; }"),
     ("server_uses_last_worker_only", "acc += q[(size_t)i * (size_t)L + j];",
      "acc = q[(size_t)i * (size_t)L + j] * (float)n;"),
 ]

@@ -110,6 +110,18 @@ typedef enum {
     APMS_SCALE_L1_MEAN = 1
 } apms_scale_kind;
 
+/* What the workers compress.  MOMENTUM is the method (Section 3.3).  GRADIENT is the comparison variant
+ * "APGSqueeze" of Section 5.3 (Implementations and setups, item 4): error-compensated compression of the
+ * gradient g_t instead of the momentum; per chunk
+ *   worker i:  z_i = g_i + delta_i ;  s_i, bits_i, delta_i as in apms_compressed_step
+ *   server:    as in apms_compressed_step; its message is a gradient ghat = +-S
+ *   workers:   m <- b1 m + (1-b1) ghat  (binary32, never compressed) ;  x <- x - (lr m) / (sqrt(v) + eps)
+ * All step functions of the compression phase follow the context's variant. */
+typedef enum {
+    APMS_VARIANT_MOMENTUM = 0,
+    APMS_VARIANT_GRADIENT = 1
+} apms_variant;
+
 /* How threads are grouped on a tile of a chunk in the worker and server kernels. */
 typedef enum {
     APMS_TEAM_AUTO = 0,   /* the library's choice for the shape (the forms below, per kernel)      */
@@ -278,6 +290,16 @@ apms_status apms_error_norms(apms_ctx* ctx, double* worker_sq_host, double* serv
 
 apms_phase  apms_get_phase(const apms_ctx* ctx);
 int         apms_get_t(const apms_ctx* ctx);
+
+/* Choose the variant (see apms_variant); allowed until the first compression-phase step has run. */
+apms_status apms_set_variant(apms_ctx* ctx, apms_variant variant);
+
+/* "APMSqueeze (Uncompressed)" of Section 5.3 (item 3): a step with v frozen and nothing compressed,
+ *   m <- (1/n) sum_i (b1 m + (1-b1) g_i)  (worker order) ;  x <- x - (lr m) / (sqrt(v) + eps).
+ * Phase must be COMPRESSED.  Compression errors are neither read nor changed; if the momentum is held
+ * as a server message it is first written out in binary32.  Counted under APMS_KERNEL_WARMUP_ADAM by
+ * apms_kernel_time.  Same gradient contract as the *_typed functions. */
+apms_status apms_uncompressed_step_typed(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
 
 /* Choose the scale definition (see apms_scale_kind); any phase, takes effect from the next step. */
 apms_status apms_set_scale_kind(apms_ctx* ctx, apms_scale_kind kind);

@@ -26,6 +26,7 @@ KERNEL_NAMES = ("warmup_adam", "worker", "server", "apply")
 TEAM_AUTO, TEAM_CTA, TEAM_WARP, TEAM_STAGED = range(4)
 GRAD_F32, GRAD_BF16, GRAD_F16 = range(3)
 SCALE_L2, SCALE_L1_MEAN = range(2)
+VARIANT_MOMENTUM, VARIANT_GRADIENT = range(2)
 MAX_WORKERS = 64
 NOALLOC_MAX_TILES = 16384
 
@@ -64,6 +65,8 @@ SIGNATURES = {
     "apms_get_phase": (C.c_int, [C.c_void_p]),
     "apms_get_t": (C.c_int, [C.c_void_p]),
     "apms_set_scale_kind": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_set_variant": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_uncompressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
@@ -237,6 +240,14 @@ def apms_get_phase(h) -> int:
 
 def apms_get_t(h) -> int:
     return int(load().apms_get_t(h))
+
+
+def apms_set_variant(h, variant: int):
+    _check(h, load().apms_set_variant(h, variant))
+
+
+def apms_uncompressed_step_typed(h, grad_ptrs: Sequence[int], grad_type: int):
+    _check(h, load().apms_uncompressed_step_typed(h, _ptr_array(grad_ptrs), grad_type))
 
 
 def apms_set_scale_kind(h, kind: int):
@@ -444,6 +455,14 @@ class Context:
     @property
     def t(self) -> int:
         return apms_get_t(self._h)
+
+    def set_variant(self, variant: int):
+        apms_set_variant(self._h, variant)
+
+    def uncompressed_step(self, grads):
+        """v frozen, nothing compressed ("APMSqueeze (Uncompressed)")."""
+        assert len(grads) == self.n
+        apms_uncompressed_step_typed(self._h, self._dev_ptrs(grads), self._grad_type(grads))
 
     def set_scale_kind(self, kind: int):
         apms_set_scale_kind(self._h, kind)

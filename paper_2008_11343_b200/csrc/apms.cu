@@ -294,12 +294,14 @@ struct WorkerArgs {
     int64_t items;                // C * P * ni
     int i0, ni;                   // this launch covers workers i0 .. i0+ni-1
     float beta1, omb1;
+    int send_gradient;            // gradient-compressing variant: z = g_i + delta_i, the momentum is not read
 };
 
 template <bool M32, bool CHECKED>
 __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __restrict__ z, uint32_t* __restrict__ obits,
                                              int grp, int lane, int L, float s_old, float Sbar,
-                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc, bool l1)
+                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc, bool l1,
+                                             bool send_gradient = false)
 {
     const int k = grp * kGroup + lane * 4;
     float mm[4];
@@ -316,7 +318,8 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
     uint32_t nibble = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const float mi = __fmaf_rn(beta1, mm[e], __fmul_rn(omb1, gg[e]));       // local momentum
+        const float mi = send_gradient ? gg[e]                                 // gradient variant: g_i itself is compensated
+                                       : __fmaf_rn(beta1, mm[e], __fmul_rn(omb1, gg[e]));   // local momentum
         const float err = implied_error(zo[e], s_old);                          // delta_i (old)
         zn[e] = __fadd_rn(mi, err);                                             // compensated
         const bool valid = !CHECKED || (k + e < L);
@@ -376,7 +379,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 #pragma unroll
         for (int u = 0; u < U; ++u)
             worker_group<M32, false>(a.beta1, a.omb1, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
-                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc, a.t.l1 != 0);
+                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc, a.t.l1 != 0, a.send_gradient != 0);
     }
     // remainder: one group at a time, bounds-checked
     for (; g0 < ngroups; g0 += WPC) {
@@ -387,7 +390,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
         uint32_t mw = 0;
         if (M32) mv = ld4_checked(m32, k, L, false);
         else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
-        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc, a.t.l1 != 0);
+        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc, a.t.l1 != 0, a.send_gradient != 0);
     }
 
     const double total = team_sum<WPC>(acc, red);
@@ -425,7 +428,7 @@ struct WorkerFineArgs {
     float beta1, omb1;
 };
 
-template <int GT>
+template <int GT, bool SENDG>          // SENDG: the gradient-compressing variant (no momentum is read)
 __global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
@@ -460,7 +463,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
             gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
             zv[u] = ld_stream4(z + u * kGroup + lane * 4);
         }
-        const uint32_t mine = (lane < 4 * kFineU) ? mbits[lane] : 0u;
+        const uint32_t mine = (!SENDG && lane < 4 * kFineU) ? mbits[lane] : 0u;
         uint32_t outw = 0;
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
@@ -472,7 +475,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
-                const float mi = __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
+                const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
                 zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
                 const double zd = (double)zn[e];
                 acc = fma(zd, zd, acc);
@@ -490,9 +493,9 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
             const int k = grp * kGroup + lane * 4;
             const float4 gv = ld_grad4_checked<GT>(g, k, L);
             const float4 zv = ld4_checked(z, k, L, true);
-            const uint32_t mw = (k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
+            const uint32_t mw = (!SENDG && k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
             worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
-                                      make_float4(0, 0, 0, 0), mw, acc, false);
+                                      make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
         }
     }
     acc = warp_sum(acc);
@@ -1010,6 +1013,98 @@ k_apply(const ApplyArgs a)
     }
 }
 
+// Steps 5-6 of the gradient-compressing variant (Section 5.3, item 4): the received chunk is a
+// gradient ghat = +-Sbar; m <- b1 m + (1-b1) ghat stays binary32, the model moves with the new m.
+struct ApplyGradArgs {
+    const uint32_t* Bbar; const float* Sbar; const float* v; float* x; float* m;
+    int64_t d; int64_t chunk; float lr, eps, beta1, omb1;
+};
+
+__global__ void __launch_bounds__(kThreads)
+k_apply_gradient(const ApplyGradArgs a)
+{
+    const int64_t base = (int64_t)blockIdx.x * kApplyTile;
+    const int64_t left = a.d - base;
+    const int L = (int)(left < kApplyTile ? left : kApplyTile);
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const int64_t j = base + k;
+        const float S = a.Sbar[j / a.chunk];                       // chunks are multiples of 32: one scale per 4 elements
+        const uint32_t nib = a.Bbar[j >> 5] >> (j & 31);
+        if (k + 3 < L) {
+            const float4 vv = ld_stream4(a.v + j);
+            float4 xx = ld_stream4(a.x + j);
+            float4 mm = ld_stream4(a.m + j);
+            mm.x = __fmaf_rn(a.beta1, mm.x, __fmul_rn(a.omb1, bit_scale(nib & 1u, S)));
+            mm.y = __fmaf_rn(a.beta1, mm.y, __fmul_rn(a.omb1, bit_scale(nib & 2u, S)));
+            mm.z = __fmaf_rn(a.beta1, mm.z, __fmul_rn(a.omb1, bit_scale(nib & 4u, S)));
+            mm.w = __fmaf_rn(a.beta1, mm.w, __fmul_rn(a.omb1, bit_scale(nib & 8u, S)));
+            xx.x = apply_elem(xx.x, vv.x, mm.x, a.lr, a.eps);
+            xx.y = apply_elem(xx.y, vv.y, mm.y, a.lr, a.eps);
+            xx.z = apply_elem(xx.z, vv.z, mm.z, a.lr, a.eps);
+            xx.w = apply_elem(xx.w, vv.w, mm.w, a.lr, a.eps);
+            st_stream4(a.m + j, mm);
+            st_stream4(a.x + j, xx);
+        } else {
+            for (int e = 0; e < 4 && k + e < L; ++e) {
+                const float mn = __fmaf_rn(a.beta1, a.m[j + e], __fmul_rn(a.omb1, bit_scale((nib >> e) & 1u, S)));
+                a.m[j + e] = mn;
+                a.x[j + e] = apply_elem(a.x[j + e], a.v[j + e], mn, a.lr, a.eps);
+            }
+        }
+    }
+}
+
+// "APMSqueeze (Uncompressed)" of Section 5.3 (item 3): v frozen, nothing compressed.  Every worker forms
+// its local momentum, the momenta are averaged in worker order, the average is the new momentum:
+//   m <- (1/n) sum_i (b1 m + (1-b1) g_i) ;  x <- x - lr m / (sqrt(v) + eps).
+// The additions of +0 stand for the (zero) compression errors of the general step, so that a negative
+// zero behaves as it does there.
+struct UncompressedArgs {
+    float* x; float* m; const float* v;
+    int64_t d; int n;
+    float beta1, omb1, lr, eps, nf;
+};
+
+__device__ __forceinline__ void uncompressed_elem(const UncompressedArgs& a, float acc, float& m, float v, float& x)
+{
+    m = __fadd_rn(__fdiv_rn(acc, a.nf), 0.0f);
+    x = apply_elem(x, v, m, a.lr, a.eps);
+}
+
+template <int GT>
+__global__ void __launch_bounds__(kThreads)
+k_uncompressed(const __grid_constant__ GradPtrs G, const UncompressedArgs a)
+{
+    const int64_t j = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
+    if (j + 3 < a.d) {
+        float4 m = ld_stream4(a.m + j);
+        const float4 v = ld_stream4(a.v + j);
+        float4 x = ld_stream4(a.x + j);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int i = 0; i < a.n; ++i) {
+            const float4 g = Grad<GT>::ld4(Grad<GT>::at(G.p[i], j), 0);
+            acc.x = __fadd_rn(acc.x, __fadd_rn(__fmaf_rn(a.beta1, m.x, __fmul_rn(a.omb1, g.x)), 0.0f));
+            acc.y = __fadd_rn(acc.y, __fadd_rn(__fmaf_rn(a.beta1, m.y, __fmul_rn(a.omb1, g.y)), 0.0f));
+            acc.z = __fadd_rn(acc.z, __fadd_rn(__fmaf_rn(a.beta1, m.z, __fmul_rn(a.omb1, g.z)), 0.0f));
+            acc.w = __fadd_rn(acc.w, __fadd_rn(__fmaf_rn(a.beta1, m.w, __fmul_rn(a.omb1, g.w)), 0.0f));
+        }
+        uncompressed_elem(a, acc.x, m.x, v.x, x.x); uncompressed_elem(a, acc.y, m.y, v.y, x.y);
+        uncompressed_elem(a, acc.z, m.z, v.z, x.z); uncompressed_elem(a, acc.w, m.w, v.w, x.w);
+        st_stream4(a.m + j, m);
+        st_stream4(a.x + j, x);
+    } else {
+        for (int64_t e = j; e < a.d; ++e) {
+            float acc = 0.f;
+            float m = a.m[e], x = a.x[e];
+            for (int i = 0; i < a.n; ++i)
+                acc = __fadd_rn(acc, __fadd_rn(__fmaf_rn(a.beta1, m, __fmul_rn(a.omb1, Grad<GT>::ld1(G.p[i], e))), 0.0f));
+            uncompressed_elem(a, acc, m, a.v[e], x);
+            a.m[e] = m; a.x[e] = x;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // State materialisation (parity, checkpoints): delta = z - (+-scale), m = +-Sbar.
 
@@ -1130,6 +1225,8 @@ struct apms_ctx {
     float beta1, beta2, eps, lr;
     int t;
     int64_t steps;           // steps taken through apms_step (warmup and compressed)
+    int variant;             // APMS_VARIANT_*: what the workers compress
+    int64_t csteps;          // compression-phase steps taken (the variant is fixed once one has run)
     int substep;             // phase-wise step: 0 = between steps, 1 = worker phase done, 2 = a server phase done
     apms_schedule sched; bool has_sched;
     apms_phase phase;
@@ -1282,7 +1379,7 @@ bool use_fine_worker(const apms_ctx* c)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
     if (c->L.t.l1) return false;             // see use_staged_server
-    return !c->m_is_fp32 && c->L.fine_tiles > 0;
+    return (!c->m_is_fp32 || c->variant == APMS_VARIANT_GRADIENT) && c->L.fine_tiles > 0;
 }
 
 apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
@@ -1302,7 +1399,8 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
     {
         Timed t(c, APMS_KERNEL_WORKER);
-        APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+        if (c->variant == APMS_VARIANT_GRADIENT) APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+        else                                     APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
         apms_status st = launch_check(c, "k_worker_fine");
         if (st != APMS_OK) return st;
         const int64_t total = (int64_t)ni * c->L.C;
@@ -1326,13 +1424,14 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int
     a.t = c->L.t; a.i0 = i0; a.ni = ni;
     a.items = c->L.C * c->L.t.P * ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
+    a.send_gradient = c->variant == APMS_VARIANT_GRADIENT;
     const bool warp_teams = use_warp_teams(c, a.items);
     const int64_t blocks = warp_teams ? (a.items + kWarps - 1) / kWarps : a.items;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
     {
         Timed t(c, APMS_KERNEL_WORKER);
         const unsigned gridx = (unsigned)blocks;
-        if (c->m_is_fp32) {
+        if (c->m_is_fp32 && !a.send_gradient) {
             if (warp_teams) APMS_DISPATCH_GRAD(gtype, k_worker<GT, true, 2, 1><<<gridx, kThreads, 0, c->stream>>>(G, a));
             else            APMS_DISPATCH_GRAD(gtype, k_worker<GT, true, 4, kWarps><<<gridx, kThreads, 0, c->stream>>>(G, a));
         } else {
@@ -1436,6 +1535,14 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
 // Section 3.3 steps 5-6 over the whole vector, from the server message held in Bbar / Sbar.
 apms_status launch_apply(apms_ctx* c)
 {
+    if (c->variant == APMS_VARIANT_GRADIENT) {
+        ApplyGradArgs g;
+        g.Bbar = c->Bbar(); g.Sbar = c->Sbar(); g.v = c->v(); g.x = c->x(); g.m = c->m();
+        g.d = c->L.d; g.chunk = c->L.chunk; g.lr = c->lr; g.eps = c->eps; g.beta1 = c->beta1; g.omb1 = 1.0f - c->beta1;
+        Timed t(c, APMS_KERNEL_APPLY);
+        k_apply_gradient<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(g);
+        return launch_check(c, "k_apply_gradient");
+    }
     ApplyArgs a;
     a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
     a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
@@ -1448,13 +1555,15 @@ apms_status launch_server_and_apply(apms_ctx* c)
 {
     const ServerSource own = {c->B(0), c->L.Wp, c->s(0), c->L.Cp, c->L.n};
     bool applied = false;      // steps 5-6 already done by the fused server kernel
-    apms_status st = launch_server(c, own, 0, c->L.C, true, &applied);
+    const bool gradient = c->variant == APMS_VARIANT_GRADIENT;      // its apply differs: never fused
+    apms_status st = launch_server(c, own, 0, c->L.C, !gradient, &applied);
     if (st != APMS_OK) return st;
     if (!applied) {
         st = launch_apply(c);
         if (st != APMS_OK) return st;
     }
-    c->m_is_fp32 = false;      // from now on the momentum is the server's message
+    c->m_is_fp32 = gradient;   // momentum variant: from now on the momentum is the server's message
+    c->csteps += 1;
     return APMS_OK;
 }
 
@@ -1511,7 +1620,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
-    c->steps = 0; c->has_sched = false; c->substep = 0;
+    c->steps = 0; c->has_sched = false; c->substep = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
     c->fine_run = kFineRunDefault;
     if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
@@ -1543,7 +1652,7 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
-    c->t = 0; c->steps = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
+    c->t = 0; c->steps = 0; c->csteps = 0; c->substep = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
     return APMS_OK;
 }
 
@@ -1665,7 +1774,8 @@ apms_status apms_apply_phase(apms_ctx* c)
     if (c->substep != 2) return fail(c, APMS_ERR_BAD_STATE, "apms_apply_phase follows apms_server_phase");
     apms_status st = launch_apply(c);
     if (st != APMS_OK) return st;
-    c->m_is_fp32 = false;
+    c->m_is_fp32 = c->variant == APMS_VARIANT_GRADIENT;
+    c->csteps += 1;
     c->substep = 0;
     return APMS_OK;
 }
@@ -1903,6 +2013,40 @@ apms_status apms_error_norms(apms_ctx* c, double* worker_sq_host, double* server
 
 apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }
 int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
+
+apms_status apms_set_variant(apms_ctx* c, apms_variant variant)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (variant != APMS_VARIANT_MOMENTUM && variant != APMS_VARIANT_GRADIENT) return fail(c, APMS_ERR_INVALID_ARG, "unknown variant");
+    if (c->csteps > 0 && (int)variant != c->variant)
+        return fail(c, APMS_ERR_BAD_STATE, "the variant cannot change once a compression-phase step has run");
+    c->variant = (int)variant;
+    return APMS_OK;
+}
+
+apms_status apms_uncompressed_step_typed(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_uncompressed_step needs v frozen (call apms_freeze_v first)");
+    if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "a phase-wise step is in progress (finish it with apms_apply_phase)");
+    GradPtrs G;
+    apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
+    if (st != APMS_OK) return st;
+    if (!c->m_is_fp32) {       // the momentum lives in the server's message: spell it out in binary32 first
+        k_materialise_momentum<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->m(), 0, c->L.d, c->L.chunk);
+        st = launch_check(c, "k_materialise_momentum");
+        if (st != APMS_OK) return st;
+        c->m_is_fp32 = true;
+    }
+    UncompressedArgs a;
+    a.x = c->x(); a.m = c->m(); a.v = c->v(); a.d = c->L.d; a.n = c->L.n;
+    a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1; a.lr = c->lr; a.eps = c->eps; a.nf = (float)c->L.n;
+    const int64_t blocks = (c->L.d + (int64_t)kThreads * 4 - 1) / ((int64_t)kThreads * 4);
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "d too large for one launch");
+    Timed t(c, APMS_KERNEL_WARMUP_ADAM);
+    APMS_DISPATCH_GRAD((int)type, k_uncompressed<GT><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+    return launch_check(c, "k_uncompressed");
+}
 
 apms_status apms_set_scale_kind(apms_ctx* c, apms_scale_kind kind)
 {

@@ -135,6 +135,76 @@ def test_mean_absolute_scale_matches_the_oracle_switch(d, n, chunk, team):
     assert abs(float(ctx.get_state(B.STATE_SERVER_SCALES)[0]) - z.mean()) <= 1e-6 * z.mean()
 
 
+# ------------------------------------------------------------------ the comparison variants of Section 5.3
+
+@pytest.mark.parametrize("team", [B.TEAM_AUTO, B.TEAM_CTA, B.TEAM_WARP], ids=["auto", "cta-per-tile", "warp-per-tile"])
+@pytest.mark.parametrize("d,n,chunk", [(5 * 4096 + 1234, 3, 4096), (3 * 1024 + 5, 4, 96), (3 * 70016, 2, 70016),
+                                       (2 * 32768 + 23552, 16, 32768), (9 * 512 + 3, 2, 512), (1, 1, 32)])
+def test_gradient_variant_bit_identical(d, n, chunk, team):
+    """Error-compensated compression of the gradient instead of the momentum: every state array bit-identical
+    to the oracle's variant, step by step (the momentum stays binary32 and is updated from the received gradient)."""
+    w = tiny(d, n, chunk, cfg_id=160, warmup_steps=2, compressed_steps=4)
+    ctx, orc = H.make_pair(w, team_mode=team)
+    ctx.set_variant(B.VARIANT_GRADIENT)
+    orc.set_variant(ao.VARIANT_GRADIENT)
+    for step in range(2):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(2, 6):
+        gs = wl.host_gradients(w, step)
+        if step == 4:
+            import torch
+            ctx.compressed_step_host([torch.from_numpy(g).pin_memory() for g in gs])      # the host-gradient path too
+        else:
+            ctx.compressed_step(H.upload(gs))
+        orc.compressed_step(gs)
+        for which, ref in ((B.STATE_X, orc.x), (B.STATE_M, orc.m), (B.STATE_V, orc.v), (B.STATE_SERVER_ERR, orc.server_err),
+                           (B.STATE_SERVER_BITS, orc.server_bits), (B.STATE_SERVER_SCALES, orc.server_scales)):
+            assert np.array_equal(ctx.get_state(which).view(np.uint32), ref.view(np.uint32)), (step, which)
+        for i in range(n):
+            assert np.array_equal(ctx.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), orc.worker_err(i).view(np.uint32))
+            assert np.array_equal(ctx.get_state(B.STATE_WORKER_BITS, i), orc.worker_bits(i))
+    with pytest.raises(B.ApmsError) as e:
+        ctx.set_variant(B.VARIANT_MOMENTUM)                    # fixed once a compression-phase step has run
+    assert e.value.status == B.ERR_BAD_STATE
+
+
+@pytest.mark.parametrize("d,n,chunk", [(4 * 1024 + 3, 4, 1024), (70001, 3, 4096), (2, 2, 32)])
+def test_uncompressed_step_equals_the_identity_compressor(d, n, chunk):
+    """v frozen, nothing compressed: the oracle with the identity compressor, bit for bit; then a compressed
+    step after it still agrees (the momentum was handed over in binary32)."""
+    w = tiny(d, n, chunk, cfg_id=161)
+    ctx, orc = H.make_pair(w)
+    for step in range(2):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    orc.set_compressor(ao.IDENTITY)
+    for step in range(2, 6):
+        gs = wl.host_gradients(w, step)
+        ctx.uncompressed_step(H.upload(gs)); orc.compressed_step(gs)
+        for which, ref in ((B.STATE_X, orc.x), (B.STATE_M, orc.m)):
+            assert np.array_equal(ctx.get_state(which).view(np.uint32), ref.view(np.uint32)), (step, which)
+    orc.set_compressor(ao.ONEBIT)
+    for step in range(6, 9):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        if step == 7:                                          # and back: the momentum is spelled out from the message
+            gs = wl.host_gradients(w, 100)
+            orc.set_compressor(ao.IDENTITY)
+            saved = [orc.worker_err(i).copy() for i in range(n)], orc.server_err.copy()
+            for i in range(n):
+                orc.worker_err(i)[:] = 0                       # the library's uncompressed step leaves the errors alone
+            orc.server_err[:] = 0
+            ctx.uncompressed_step(H.upload(gs)); orc.compressed_step(gs)
+            for i in range(n):
+                orc.worker_err(i)[:] = saved[0][i]
+            orc.server_err[:] = saved[1]
+            orc.set_compressor(ao.ONEBIT)
+    H.compare_state(ctx, orc, w, exact=True)
+
+
 # ------------------------------------------------------------------ phase driver and error monitor
 
 def test_scheduled_steps_follow_algorithm_1():

@@ -314,6 +314,15 @@ apms_status apms_set_team_mode(apms_ctx* ctx, apms_team_mode mode);
 apms_status apms_set_timing(apms_ctx* ctx, int enabled);
 apms_status apms_kernel_time(apms_ctx* ctx, apms_kernel_id which, double* total_ms, int64_t* launches);
 
+/* Self-test of the report path of bounded device-side waits.  Every wait inside the library's kernels
+ * (they wait only for their own asynchronous copies) gives up after about a second, records that in a
+ * status word and ends its CTA; the next synchronising call then returns APMS_ERR_TIMEOUT.  This call
+ * runs a one-CTA kernel that waits, with a bound of about a millisecond, for a barrier that nothing
+ * completes, and checks that the status word reads "gave up": APMS_OK if so.  With leave_reported != 0
+ * the word stays set, so that the next synchronising call returns APMS_ERR_TIMEOUT (apms_set_params
+ * clears it); otherwise it is cleared again.  Synchronises.  Harmless: no fault, no hang, no state touched. */
+apms_status apms_selftest_wait_report(apms_ctx* ctx, int leave_reported);
+
 /* Kernels launched by this context since creation. */
 int64_t     apms_launch_count(const apms_ctx* ctx);
 

@@ -70,6 +70,7 @@ SIGNATURES = {
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "apms_selftest_wait_report": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_launch_count": (C.c_int64, [C.c_void_p]),
     "apms_last_error": (C.c_char_p, [C.c_void_p]),
     "apms_destroy": (None, [C.c_void_p]),
@@ -266,6 +267,10 @@ def apms_kernel_time(h, which: int):
     ms, cnt = C.c_double(0.0), C.c_int64(0)
     _check(h, load().apms_kernel_time(h, which, C.byref(ms), C.byref(cnt)))
     return ms.value, cnt.value
+
+
+def apms_selftest_wait_report(h, leave_reported: bool = False):
+    _check(h, load().apms_selftest_wait_report(h, int(leave_reported)))
 
 
 def apms_launch_count(h) -> int:

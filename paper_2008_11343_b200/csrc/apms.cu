@@ -700,8 +700,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
                  : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return done != 0;
 }
-// Bounded wait: false when the phase did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+// Bounded wait: false when the phase did not complete within `limit` SM clocks.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -709,8 +709,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
 #pragma unroll 1
         for (int k = 0; k < 32; ++k)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
+}
+
+// Self-test of the give-up path: a barrier that nothing ever completes, waited for with a short bound.
+// No copy is in flight and nothing else is touched, so the CTA simply reports and ends.
+__global__ void k_selftest_wait(int* status, long long limit)
+{
+    __shared__ uint64_t never;
+    if (threadIdx.x == 0) { mbar_init(&never, 1); mbar_fence_init(); }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(&never, 0, limit)) atomicExch(status, DEVICE_WAIT_TIMEOUT);
 }
 // Global -> this CTA's shared memory; 16-byte aligned addresses, size a multiple of 16 bytes.
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
@@ -2013,6 +2023,21 @@ apms_status apms_error_norms(apms_ctx* c, double* worker_sq_host, double* server
 
 apms_phase apms_get_phase(const apms_ctx* c) { return c ? c->phase : APMS_PHASE_CREATED; }
 int apms_get_t(const apms_ctx* c) { return c ? c->t : -1; }
+
+apms_status apms_selftest_wait_report(apms_ctx* c, int leave_reported)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    k_selftest_wait<<<1, 32, 0, c->stream>>>(c->status(), 2000000ll);          // about a millisecond
+    apms_status st = launch_check(c, "k_selftest_wait");
+    if (st != APMS_OK) return st;
+    int seen = 0;
+    APMS_CUDA(c, cudaMemcpyAsync(&seen, c->status(), sizeof seen, cudaMemcpyDeviceToHost, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (!leave_reported) APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, sizeof(int), c->stream));
+    if (seen != DEVICE_WAIT_TIMEOUT) return fail(c, APMS_ERR_BAD_STATE, "the bounded wait did not report that it gave up");
+    return APMS_OK;
+}
 
 apms_status apms_set_variant(apms_ctx* c, apms_variant variant)
 {

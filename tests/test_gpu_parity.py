@@ -511,6 +511,25 @@ def test_phase_and_argument_errors_are_status_codes():
     assert ctx.launch_count == 1 + 3
 
 
+def test_a_wait_that_gives_up_is_reported_and_the_context_survives():
+    """A bounded wait that runs out (a barrier nothing completes, bound of a millisecond) sets the status word;
+    the next synchronising call returns APMS_ERR_TIMEOUT; after apms_set_params the context works again."""
+    w = tiny(3 * 2048 + 5, 2, 2048, cfg_id=170)
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    x0 = wl.initial_params(w)
+    ctx.set_params(x0)
+    B.apms_selftest_wait_report(ctx._h)                       # reported and cleared
+    assert np.array_equal(ctx.get_params(), x0)
+    B.apms_selftest_wait_report(ctx._h, leave_reported=True)
+    with pytest.raises(B.ApmsError) as e:
+        ctx.get_params()
+    assert e.value.status == B.ERR_TIMEOUT
+    ctx.set_params(x0)                                        # clears the word
+    ctx.freeze_v()
+    ctx.compressed_step(H.upload(wl.host_gradients(w, 0)))
+    assert np.isfinite(ctx.get_params()).all()
+
+
 def test_library_owned_workspace_and_default_stream():
     """apms_create without apms_bind: the library allocates its own workspace."""
     import torch

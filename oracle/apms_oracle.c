@@ -33,6 +33,9 @@
  *   - The compressed-phase denominator is sqrt(v_Tw) + eps with the raw
  *     (not bias-corrected) frozen v; eps plays the role of Adam's constant.
  *   - The average is over all n workers, summed in worker order, divided by n.
+ *   - Top-k compression (Section 5.1, second item) keeps "the top k% elements ... sorted by absolute
+ *     magnitude": per chunk K = ceil(k L) elements (at least one), equal magnitudes resolved in favour
+ *     of the lower index, the others are sent as nothing and decompress to 0.
  *   - The gradient variant (Section 5.3, item 4) is described in one sentence; read as: workers
  *     send C[g_i + delta_i], servers average and recompress as in the method, and every worker
  *     forms m <- b1 m + (1-b1) g^ from the received g^ and updates the model with that m.
@@ -55,7 +58,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_COMPRESSOR_ONEBIT = 0, ORACLE_COMPRESSOR_IDENTITY = 1 };
+enum { ORACLE_COMPRESSOR_ONEBIT = 0, ORACLE_COMPRESSOR_IDENTITY = 1, ORACLE_COMPRESSOR_TOPK = 2 };
 enum { ORACLE_SCALE_L2 = 0, ORACLE_SCALE_L1_MEAN = 1 };
 /* What the workers compress and send.  MOMENTUM is the method (Section 3.3).  GRADIENT is the
  * "APGSqueeze" variant of Section 5.3 (Implementations and setups, item 4): the error-compensated
@@ -76,6 +79,9 @@ typedef struct apms_oracle {
     int   compressor;   /* ORACLE_COMPRESSOR_* */
     int   scale_kind;   /* ORACLE_SCALE_* */
     int   variant;      /* ORACLE_VARIANT_* */
+    double topk_frac;   /* top-k compressor: fraction of a chunk's elements that is kept */
+    uint8_t *sel;       /* top-k: 1 where worker i kept element j last step, n x d */
+    uint8_t *selbar;    /* top-k: the same for the server, d */
     int   threads;      /* OpenMP threads over chunks (chunks are independent) */
     float *x, *m, *v;   /* d each */
     float *ebar;        /* server error, d */
@@ -104,6 +110,42 @@ void apms_oracle_compress_1bit(const float *z, int64_t L, int scale_kind,
     for (int64_t w = 0; w < (L + 31) / 32; ++w) bits[w] = 0u;
     for (int64_t j = 0; j < L; ++j)
         if (z[j] >= 0.0f) bits[j / 32] |= (uint32_t)1 << (j % 32);
+}
+
+/* Top-k compressor of Section 5.1 on one chunk: keep the K elements of largest absolute value,
+ * send nothing for the others (they decompress to 0).  Equal magnitudes: the lower index wins,
+ * so that the choice is unique.  Magnitudes are compared through the bit pattern of |z| (for
+ * finite values the same order; a NaN ranks above everything).  q receives C[z]; sel (may be
+ * NULL) the 0/1 mask of the kept elements. */
+typedef struct { uint32_t key; int64_t idx; } topk_item;
+static int topk_cmp(const void *a, const void *b)
+{
+    const topk_item *x = (const topk_item *)a, *y = (const topk_item *)b;
+    if (x->key != y->key) return x->key > y->key ? -1 : 1;      /* larger magnitude first */
+    return x->idx < y->idx ? -1 : (x->idx > y->idx ? 1 : 0);    /* then lower index       */
+}
+void apms_oracle_compress_topk(const float *z, int64_t L, int64_t K, float *q, uint8_t *sel)
+{
+    topk_item *items = (topk_item *)malloc((size_t)L * sizeof *items);
+    for (int64_t j = 0; j < L; ++j) {
+        uint32_t bits;
+        memcpy(&bits, &z[j], sizeof bits);
+        items[j].key = bits & 0x7fffffffu;
+        items[j].idx = j;
+    }
+    qsort(items, (size_t)L, sizeof *items, topk_cmp);
+    for (int64_t j = 0; j < L; ++j) { q[j] = 0.0f; if (sel) sel[j] = 0; }
+    for (int64_t r = 0; r < K && r < L; ++r) { q[items[r].idx] = z[items[r].idx]; if (sel) sel[items[r].idx] = 1; }
+    free(items);
+}
+
+/* "top k% elements" of a chunk of L elements: K = ceil(frac * L), at least 1, at most L. */
+int64_t apms_oracle_topk_count(double frac, int64_t L)
+{
+    int64_t K = (int64_t)ceil(frac * (double)L);
+    if (K < 1) K = 1;
+    if (K > L) K = L;
+    return K;
 }
 
 /* Decompression: scale * sign vector. */
@@ -135,6 +177,9 @@ apms_oracle *apms_oracle_create(int64_t d, int n, float beta1, float beta2, floa
     o->Sbar = (float *)calloc((size_t)o->C, sizeof(float));
     o->B = (uint32_t *)calloc((size_t)o->W * (size_t)n, sizeof(uint32_t));
     o->Bbar = (uint32_t *)calloc((size_t)o->W, sizeof(uint32_t));
+    o->sel = (uint8_t *)calloc((size_t)d * (size_t)n, 1);
+    o->selbar = (uint8_t *)calloc((size_t)d, 1);
+    o->topk_frac = 0.01;
     return o;
 }
 
@@ -142,7 +187,7 @@ void apms_oracle_destroy(apms_oracle *o)
 {
     if (!o) return;
     free(o->x); free(o->m); free(o->v); free(o->ebar); free(o->e);
-    free(o->s); free(o->Sbar); free(o->B); free(o->Bbar); free(o);
+    free(o->s); free(o->Sbar); free(o->B); free(o->Bbar); free(o->sel); free(o->selbar); free(o);
 }
 
 void apms_oracle_set_params(apms_oracle *o, const float *x0)
@@ -157,6 +202,9 @@ void apms_oracle_set_lr(apms_oracle *o, float lr) { o->lr = lr; }
 void apms_oracle_set_compressor(apms_oracle *o, int c) { o->compressor = c; }
 void apms_oracle_set_scale_kind(apms_oracle *o, int k) { o->scale_kind = k; }
 void apms_oracle_set_variant(apms_oracle *o, int v) { o->variant = v; }
+void apms_oracle_set_topk_fraction(apms_oracle *o, double f) { o->topk_frac = f; }
+uint8_t *apms_oracle_worker_selected(apms_oracle *o, int i) { return o->sel + (size_t)i * (size_t)o->d; }
+uint8_t *apms_oracle_server_selected(apms_oracle *o) { return o->selbar; }
 void apms_oracle_set_threads(apms_oracle *o, int t) { o->threads = t < 1 ? 1 : t; }
 int  apms_oracle_max_threads(void)
 {
@@ -240,6 +288,9 @@ static void compressed_step_chunk(apms_oracle *o, const float *const *g, int64_t
         }
         if (o->compressor == ORACLE_COMPRESSOR_IDENTITY) {
             memcpy(qi, z, (size_t)L * sizeof(float));
+        } else if (o->compressor == ORACLE_COMPRESSOR_TOPK) {
+            apms_oracle_compress_topk(z, L, apms_oracle_topk_count(o->topk_frac, L), qi,
+                                      o->sel + (size_t)i * (size_t)o->d + lo);
         } else {
             uint32_t *bits = o->B + (size_t)i * (size_t)o->W + lo / 32;
             float *scale = o->s + (size_t)i * (size_t)o->C + c;
@@ -257,6 +308,8 @@ static void compressed_step_chunk(apms_oracle *o, const float *const *g, int64_t
     }
     if (o->compressor == ORACLE_COMPRESSOR_IDENTITY) {
         memcpy(qb, z, (size_t)L * sizeof(float));
+    } else if (o->compressor == ORACLE_COMPRESSOR_TOPK) {
+        apms_oracle_compress_topk(z, L, apms_oracle_topk_count(o->topk_frac, L), qb, o->selbar + lo);
     } else {
         apms_oracle_compress_1bit(z, L, o->scale_kind, o->Bbar + lo / 32, o->Sbar + c);
         apms_oracle_decompress_1bit(o->Bbar + lo / 32, o->Sbar[c], L, qb);

@@ -12,7 +12,7 @@ import numpy as np
 
 from . import build as _build
 
-ONEBIT, IDENTITY = 0, 1
+ONEBIT, IDENTITY, TOPK = 0, 1, 2
 VARIANT_MOMENTUM, VARIANT_GRADIENT = 0, 1
 SCALE_L2, SCALE_L1_MEAN = 0, 1
 
@@ -59,6 +59,14 @@ def _declare(L: C.CDLL) -> C.CDLL:
     L.apms_oracle_t.restype = C.c_int
     L.apms_oracle_t.argtypes = [vp]
     L.apms_oracle_compress_1bit.argtypes = [_F, C.c_int64, C.c_int, _U, _F]
+    L.apms_oracle_compress_topk.argtypes = [_F, C.c_int64, C.c_int64, _F, C.POINTER(C.c_uint8)]
+    L.apms_oracle_topk_count.restype = C.c_int64
+    L.apms_oracle_topk_count.argtypes = [C.c_double, C.c_int64]
+    L.apms_oracle_set_topk_fraction.argtypes = [vp, C.c_double]
+    L.apms_oracle_worker_selected.restype = C.POINTER(C.c_uint8)
+    L.apms_oracle_worker_selected.argtypes = [vp, C.c_int]
+    L.apms_oracle_server_selected.restype = C.POINTER(C.c_uint8)
+    L.apms_oracle_server_selected.argtypes = [vp]
     L.apms_oracle_decompress_1bit.argtypes = [_U, C.c_float, C.c_int64, _F]
     return L
 
@@ -76,6 +84,21 @@ def compress_1bit(z: np.ndarray, scale_kind: int = SCALE_L2, library: C.CDLL | N
     L.apms_oracle_compress_1bit(z.ctypes.data_as(_F), z.size, scale_kind,
                                 bits.ctypes.data_as(_U), C.byref(scale))
     return bits, np.float32(scale.value)
+
+
+def compress_topk(z: np.ndarray, K: int, library: C.CDLL | None = None):
+    """Top-k C[z] on one chunk: (decompressed vector float32[L], mask of kept elements uint8[L])."""
+    L = library or lib()
+    z = np.ascontiguousarray(z, dtype=np.float32)
+    q = np.empty(z.size, dtype=np.float32)
+    sel = np.empty(z.size, dtype=np.uint8)
+    L.apms_oracle_compress_topk(z.ctypes.data_as(_F), z.size, K, q.ctypes.data_as(_F),
+                                sel.ctypes.data_as(C.POINTER(C.c_uint8)))
+    return q, sel
+
+
+def topk_count(frac: float, length: int, library: C.CDLL | None = None) -> int:
+    return int((library or lib()).apms_oracle_topk_count(frac, length))
 
 
 def decompress_1bit(bits: np.ndarray, scale, length: int, library: C.CDLL | None = None) -> np.ndarray:
@@ -119,6 +142,16 @@ class Oracle:
 
     def set_compressor(self, kind: int):
         self._L.apms_oracle_set_compressor(self._h, kind)
+
+    def set_topk_fraction(self, frac: float):
+        self._L.apms_oracle_set_topk_fraction(self._h, frac)
+
+    def worker_selected(self, i: int):
+        return _view(self._L.apms_oracle_worker_selected(self._h, i), self.d, np.uint8)
+
+    @property
+    def server_selected(self):
+        return _view(self._L.apms_oracle_server_selected(self._h), self.d, np.uint8)
 
     def set_variant(self, variant: int):
         self._L.apms_oracle_set_variant(self._h, variant)

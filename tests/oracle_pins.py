@@ -387,6 +387,98 @@ def check_gradient_variant_invariants(lib):
         np.testing.assert_allclose(x_prev - o.x, step, rtol=0, atol=1e-6 * np.abs(step).max() + 2e-7 * np.abs(x_prev).max())
 
 
+# ------------------------------------------------------------------ the top-k compressor
+
+def check_topk_compressor_against_a_library_sort(lib):
+    """Kept set = the first K of a stable sort by descending |z| (numpy), ties to the lower index."""
+    rng = np.random.default_rng(31)
+    for L, K in [(1, 1), (8, 2), (33, 5), (100, 100), (257, 1), (1000, 10), (4096, 41)]:
+        z = (rng.standard_normal(L) * 10.0 ** rng.uniform(-3, 1)).astype(np.float32)
+        z[rng.random(L) < 0.2] = 0.0
+        if L >= 8:
+            z[3], z[5], z[6] = z[1], -z[1], z[1]                  # equal magnitudes of both signs
+            z[7] = -0.0
+        q, sel = ao.compress_topk(z, K, library=lib)
+        order = np.argsort(-np.abs(z.astype(np.float64)), kind="stable")      # stable: lower index first among equals
+        expect = np.zeros(L, bool)
+        expect[order[:K]] = True
+        assert np.array_equal(sel.astype(bool), expect), (L, K)
+        assert np.array_equal(q[expect], z[expect]) and not q[~expect].any()
+        assert int(sel.sum()) == K
+    assert ao.topk_count(0.01, 32768, library=lib) == 328 and ao.topk_count(0.5, 7, library=lib) == 4
+    assert ao.topk_count(1e-9, 100, library=lib) == 1 and ao.topk_count(1.0, 100, library=lib) == 100
+
+
+def check_topk_worked_step(lib):
+    """Hand-derived step with the top-k compressor (Section 5.1 + Section 3.3), exact dyadic numbers."""
+    f = read_fixture("topk_step_worked_example.txt")
+    o = ao.Oracle(8, 2, f["beta1"][0], 0.999, f["eps"][0], f["lr"][0], 32, library=lib)
+    o.set_params(np.zeros(8, dtype=np.float32))
+    o.freeze_v()
+    o.set_compressor(ao.TOPK)
+    o.set_topk_fraction(f["frac"][0])
+    o.m[:], o.v[:], o.x[:] = f["m"], f["v"], f["x"]
+    o.worker_err(0)[:], o.worker_err(1)[:], o.server_err[:] = f["e0"], f["e1"], f["ebar"]
+    o.compressed_step([np.array(f["g0"], np.float32), np.array(f["g1"], np.float32)])
+    assert np.array_equal(o.worker_selected(0), np.array(f["expect_sel0"], np.uint8))
+    assert np.array_equal(o.worker_selected(1), np.array(f["expect_sel1"], np.uint8))
+    assert np.array_equal(o.worker_err(0), np.array(f["expect_e0"], np.float32))
+    assert np.array_equal(o.worker_err(1), np.array(f["expect_e1"], np.float32))
+    assert np.array_equal(o.server_selected, np.array(f["expect_selbar"], np.uint8))
+    assert np.array_equal(o.server_err, np.array(f["expect_ebar"], np.float32))
+    assert np.array_equal(o.m, np.array(f["expect_m"], np.float32))
+    assert np.array_equal(o.x, np.array(f["expect_x"], np.float32))
+
+
+def check_topk_invariants_and_full_fraction(lib):
+    """Top-k steps on a ragged multi-chunk problem: K elements kept per chunk and message, the error is
+    zero on them and the whole compensated value elsewhere, no dropped magnitude exceeds a kept one, the
+    telescoping identity of Supplement A holds (it needs nothing of the compressor), the momentum is the
+    server's sparse message.  With k = 100 % the compressor is the identity: same run, bit for bit."""
+    rng = np.random.default_rng(37)
+    d, n, chunk, frac = 4 * 96 + 37, 3, 96, 0.1
+    b, omb = float(np.float32(0.9)), float(np.float32(1) - np.float32(0.9))
+    o = _frozen(lib, d, n, chunk, beta1=0.9, lr=1e-3)
+    o.set_compressor(ao.TOPK)
+    o.set_topk_fraction(frac)
+    _rand_state(o, rng)
+
+    def dbar():
+        return sum(o.worker_err(i).astype(np.float64) for i in range(n)) / n + o.server_err
+
+    for _ in range(5):
+        m_prev, dbar_prev, x_prev = o.m.astype(np.float64), dbar(), o.x.copy()
+        e_prev = [o.worker_err(i).copy() for i in range(n)]
+        gs = [(rng.standard_normal(d) * 3e-3).astype(np.float32) for _ in range(n)]
+        o.compressed_step(gs)
+        for c in range(o.C):
+            sl = slice(c * chunk, min(d, (c + 1) * chunk))
+            K = ao.topk_count(frac, sl.stop - sl.start, library=lib)
+            for i in range(n):
+                sel = o.worker_selected(i)[sl].astype(bool)
+                z = (b * m_prev[sl] + omb * gs[i][sl].astype(np.float64)) + e_prev[i][sl]       # binary64 view of z
+                assert int(sel.sum()) == K and not o.worker_err(i)[sl][sel].any()
+                np.testing.assert_allclose(o.worker_err(i)[sl][~sel], z[~sel], rtol=0, atol=4e-7 * np.abs(z).max())
+                assert np.abs(z[sel]).min() >= np.abs(z[~sel]).max() - 4e-7 * np.abs(z).max()
+            sel = o.server_selected[sl].astype(bool)
+            assert int(sel.sum()) == K and not o.server_err[sl][sel].any() and not o.m[sl][~sel].any()
+            assert np.array_equal(o.x[sl][~sel], x_prev[sl][~sel])          # nothing received, nothing moves
+        rhs = b * m_prev + omb * np.mean(np.stack(gs).astype(np.float64), axis=0) + dbar_prev
+        np.testing.assert_allclose(o.m.astype(np.float64) + dbar(), rhs, rtol=0, atol=1e-6 * np.abs(rhs).max())
+
+    a1 = _frozen(lib, d, n, chunk, beta1=0.9, lr=1e-3)
+    a2 = _frozen(lib, d, n, chunk, beta1=0.9, lr=1e-3)
+    a1.set_compressor(ao.TOPK); a1.set_topk_fraction(1.0)
+    a2.set_compressor(ao.IDENTITY)
+    rng2 = np.random.default_rng(41)
+    _rand_state(a1, rng2, err_scale=0.0)
+    a2.x[:], a2.m[:], a2.v[:] = a1.x, a1.m, a1.v
+    for _ in range(4):
+        gs = [(rng2.standard_normal(d) * 3e-3).astype(np.float32) for _ in range(n)]
+        a1.compressed_step(gs); a2.compressed_step(gs)
+        assert np.array_equal(a1.x.view(np.uint32), a2.x.view(np.uint32)) and np.array_equal(a1.m.view(np.uint32), a2.m.view(np.uint32))
+
+
 def check_phase_switch(lib):
     """After warmup: v stays fixed, raw m carries over, all errors start at zero (Algorithm 1
     initialisation; Section 3.3 first paragraph)."""
@@ -545,4 +637,7 @@ ALL_CHECKS = [
     check_gradient_variant_worked_example,
     check_gradient_variant_identity_is_momentum_sgd,
     check_gradient_variant_invariants,
+    check_topk_compressor_against_a_library_sort,
+    check_topk_worked_step,
+    check_topk_invariants_and_full_fraction,
 ]

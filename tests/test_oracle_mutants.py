@@ -42,6 +42,13 @@ MUTANTS = [
     ("gradient_variant_betas_swapped", "fmaf(o->beta1, o->m[lo + j], omb1 * qb[j])", "fmaf(omb1, o->m[lo + j], o->beta1 * qb[j])"),
     ("gradient_variant_update_uses_gradient", "else                                       o->m[lo + j] = qb[j];",
      "else                                       o->m[lo + j] = qb[j];\n        if (o->variant == ORACLE_VARIANT_GRADIENT) { o->x[lo + j] = o->x[lo + j] - (o->lr * qb[j]) / (sqrtf(o->v[lo + j]) + o->eps); continue; }"),
+    ("topk_keeps_smallest", "if (x->key != y->key) return x->key > y->key ? -1 : 1;", "if (x->key != y->key) return x->key < y->key ? -1 : 1;"),
+    ("topk_ties_to_higher_index", "return x->idx < y->idx ? -1 : (x->idx > y->idx ? 1 : 0);", "return x->idx > y->idx ? -1 : (x->idx < y->idx ? 1 : 0);"),
+    ("topk_signed_comparison", "items[j].key = bits & 0x7fffffffu;", "items[j].key = bits;"),
+    ("topk_one_too_many", "for (int64_t r = 0; r < K && r < L; ++r)", "for (int64_t r = 0; r <= K && r < L; ++r)"),
+    ("topk_count_floor", "int64_t K = (int64_t)ceil(frac * (double)L);", "int64_t K = (int64_t)floor(frac * (double)L);"),
+    ("topk_server_not_compressed", "apms_oracle_compress_topk(z, L, apms_oracle_topk_count(o->topk_frac, L), qb, o->selbar + lo);",
+     "memcpy(qb, z, (size_t)L * sizeof(float));"),
     ("server_uses_last_worker_only", "acc += q[(size_t)i * (size_t)L + j];",
      "acc = q[(size_t)i * (size_t)L + j] * (float)n;"),
 ]

@@ -110,6 +110,19 @@ typedef enum {
     APMS_SCALE_L1_MEAN = 1
 } apms_scale_kind;
 
+/* The compression operator C (Section 5.1 describes two).  ONEBIT is the default and the one all of the
+ * above describes.  TOPK keeps, per chunk of L elements, the K = ceil(fraction * L) elements (at least one)
+ * of largest absolute value and sends nothing for the others, which decompress to 0; equal magnitudes are
+ * resolved in favour of the lower index; magnitudes are compared through the bit pattern of |z|.
+ * In TOPK mode the context keeps, in place of the sign words, a selection mask per worker and for the
+ * server (APMS_STATE_*_BITS return it: bit j = element j was sent), no scales (they read 0), and the
+ * momentum in binary32.  Chosen with apms_set_compressor until the first compression-phase step has run;
+ * TOPK works with the momentum variant, the l2 scale setting and the whole-step functions. */
+typedef enum {
+    APMS_COMPRESSOR_ONEBIT = 0,
+    APMS_COMPRESSOR_TOPK = 1
+} apms_compressor;
+
 /* What the workers compress.  MOMENTUM is the method (Section 3.3).  GRADIENT is the comparison variant
  * "APGSqueeze" of Section 5.3 (Implementations and setups, item 4): error-compensated compression of the
  * gradient g_t instead of the momentum; per chunk
@@ -290,6 +303,9 @@ apms_status apms_error_norms(apms_ctx* ctx, double* worker_sq_host, double* serv
 
 apms_phase  apms_get_phase(const apms_ctx* ctx);
 int         apms_get_t(const apms_ctx* ctx);
+
+/* Choose the compressor (see apms_compressor); topk_fraction in (0, 1] is used for TOPK only. */
+apms_status apms_set_compressor(apms_ctx* ctx, apms_compressor kind, double topk_fraction);
 
 /* Choose the variant (see apms_variant); allowed until the first compression-phase step has run. */
 apms_status apms_set_variant(apms_ctx* ctx, apms_variant variant);

@@ -27,6 +27,7 @@ TEAM_AUTO, TEAM_CTA, TEAM_WARP, TEAM_STAGED = range(4)
 GRAD_F32, GRAD_BF16, GRAD_F16 = range(3)
 SCALE_L2, SCALE_L1_MEAN = range(2)
 VARIANT_MOMENTUM, VARIANT_GRADIENT = range(2)
+COMPRESSOR_ONEBIT, COMPRESSOR_TOPK = range(2)
 MAX_WORKERS = 64
 NOALLOC_MAX_TILES = 16384
 
@@ -66,6 +67,7 @@ SIGNATURES = {
     "apms_get_t": (C.c_int, [C.c_void_p]),
     "apms_set_scale_kind": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_variant": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_set_compressor": (C.c_int, [C.c_void_p, C.c_int, C.c_double]),
     "apms_uncompressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
@@ -241,6 +243,10 @@ def apms_get_phase(h) -> int:
 
 def apms_get_t(h) -> int:
     return int(load().apms_get_t(h))
+
+
+def apms_set_compressor(h, kind: int, topk_fraction: float = 0.01):
+    _check(h, load().apms_set_compressor(h, kind, topk_fraction))
 
 
 def apms_set_variant(h, variant: int):
@@ -460,6 +466,9 @@ class Context:
     @property
     def t(self) -> int:
         return apms_get_t(self._h)
+
+    def set_compressor(self, kind: int, topk_fraction: float = 0.01):
+        apms_set_compressor(self._h, kind, topk_fraction)
 
     def set_variant(self, variant: int):
         apms_set_variant(self._h, variant)

@@ -1135,6 +1135,247 @@ __global__ void k_materialise_momentum(const uint32_t* __restrict__ bits, const 
 }
 
 // ------------------------------------------------------------------------------------------
+// Top-k compressor (Section 5.1, second item): per chunk the K = ceil(k L) elements of largest |z| are
+// sent, the others decompress to 0; equal magnitudes go to the lower index.  State in this mode: the
+// compensated vectors z as before, and in place of the sign words a SELECTION MASK (bit j = element j
+// was sent), from which  C[z] = mask ? z : 0  and  delta = z - C[z]  follow exactly; the momentum is
+// kept in binary32.  One CTA per (chunk, worker) / per chunk; a chunk's z is written once and re-read
+// from L2 by the selection passes.
+//
+// Selection: the K-th largest magnitude is found by a three-level radix select over the bit pattern of
+// |z| (11 + 11 + 9 bits, shared-memory histograms), giving the threshold key tau and the number of
+// elements equal to tau that are still to be kept; a last pass in index order marks  key > tau, and the
+// first `ties` elements with key == tau.
+
+constexpr int kTopkBins = 2048;
+
+__device__ __forceinline__ uint32_t mag_key(float z) { return __float_as_uint(z) & 0x7fffffffu; }
+
+// C[z] and the error it leaves, from a stored compensated value and its selection bit (the subtraction is
+// the one the method performs, so that non-finite values behave as they do there).
+__device__ __forceinline__ float topk_error(float z, uint32_t selected) { return __fsub_rn(z, selected ? z : 0.0f); }
+
+// hist[0..nbins) are counts; K >= 1 is the rank wanted, counted from the top bin.  Returns (to all threads)
+// the bin that holds the K-th key and reduces K to the rank inside that bin.  Ends with a barrier.
+__device__ __forceinline__ int topk_find_bin(const uint32_t* hist, int nbins, uint32_t& K, uint32_t* sh)
+{
+    __syncthreads();                                   // the histogram is complete
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x, per = nbins / 32;
+        const int hi = nbins - lane * per, lo = hi - per;             // lane 0 owns the top bins
+        uint32_t mine = 0;
+        for (int b = lo; b < hi; ++b) mine += hist[b];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const uint32_t excl = incl - mine;
+        if (excl < K && K <= incl) {                   // exactly one lane
+            uint32_t k = K - excl;
+            int b = hi - 1;
+            for (; b > lo; --b) { if (k <= hist[b]) break; k -= hist[b]; }
+            sh[0] = (uint32_t)b; sh[1] = k;
+        }
+    }
+    __syncthreads();
+    K = sh[1];
+    return (int)sh[0];
+}
+
+// Threshold of the K largest magnitudes of zc[0..L) (global memory, written by this CTA).  hist must hold
+// the level-0 histogram (key >> 20) already.  Out: tau and the number of elements equal to tau to keep.
+__device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t K, uint32_t* hist, uint32_t* sh,
+                                               uint32_t& tau, uint32_t& ties)
+{
+    const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < L; j += kThreads) {
+        const uint32_t key = mag_key(zc[j]);
+        if ((key >> 20) == b0) atomicAdd(&hist[(key >> 9) & 0x7ffu], 1u);
+    }
+    const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    const uint32_t top = (b0 << 11) | b1;
+    for (int j = threadIdx.x; j < L; j += kThreads) {
+        const uint32_t key = mag_key(zc[j]);
+        if ((key >> 9) == top) atomicAdd(&hist[key & 0x1ffu], 1u);
+    }
+    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 512, K, sh);
+    tau = (top << 9) | b2;
+    ties = K;
+}
+
+// One wave of the ordered pass: thread t looks at element j of the wave; returns whether it is selected.
+// `seen` counts the elements equal to tau in earlier positions (same value in every thread).
+__device__ __forceinline__ bool topk_select_wave(bool valid, uint32_t key, uint32_t tau, uint32_t ties, uint32_t& seen,
+                                                 uint32_t* warp_ties)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool tie = valid && key == tau;
+    const uint32_t ballot = __ballot_sync(0xffffffffu, tie);
+    if (lane == 0) warp_ties[warp] = __popc(ballot);
+    __syncthreads();
+    uint32_t before = seen, total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { const uint32_t c = warp_ties[w]; if (w < warp) before += c; total += c; }
+    before += __popc(ballot & ((1u << lane) - 1u));
+    seen += total;
+    __syncthreads();                                   // warp_ties may be rewritten by the next wave
+    return valid && (key > tau || (tie && before < ties));
+}
+
+struct TopkWorkerArgs {
+    float* z; int64_t dz;
+    uint32_t* B; int64_t Wp;          // selection masks
+    const float* m32;
+    int64_t d, chunk, C;
+    int i0, ni;
+    float beta1, omb1;
+    double frac;
+};
+
+__device__ __forceinline__ uint32_t topk_count(double frac, int L)
+{
+    long long K = (long long)ceil(frac * (double)L);
+    if (K < 1) K = 1;
+    if (K > L) K = L;
+    return (uint32_t)K;
+}
+
+template <int GT>
+__global__ void __launch_bounds__(kThreads)
+k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
+{
+    __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t sh[2];
+    __shared__ uint32_t warp_ties[kWarps];
+    const int ii = (int)(blockIdx.x % a.ni);
+    const int64_t c = blockIdx.x / a.ni;
+    const int i = a.i0 + ii;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
+    float* zc = a.z + (int64_t)i * a.dz + base;
+    uint32_t* maskw = a.B + (int64_t)i * a.Wp + base / 32;
+    const float* __restrict__ m = a.m32 + base;
+
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 gv = ld_grad4_checked<GT>(g, k, L);
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const float4 mv = ld4_checked(m, k, L, false);
+        const uint32_t nib = maskw[k >> 5] >> (k & 31);
+        const float gg[4] = {gv.x, gv.y, gv.z, gv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w}, mm[4] = {mv.x, mv.y, mv.z, mv.w};
+        float zn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
+            zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
+            if (k + e < L) atomicAdd(&hist[mag_key(zn[e]) >> 20], 1u);
+        }
+        if (k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
+    }
+    uint32_t tau, ties;
+    topk_threshold(zc, L, topk_count(a.frac, L), hist, sh, tau, ties);      // its first barrier also orders the z stores
+    // ordered pass: the selection mask, one word per warp and wave
+    uint32_t seen = 0;
+    for (int w0 = 0; w0 < L; w0 += kThreads) {
+        const int j = w0 + threadIdx.x;
+        const bool valid = j < L;
+        const uint32_t key = valid ? mag_key(zc[j]) : 0u;
+        const bool sel = topk_select_wave(valid, key, tau, ties, seen, warp_ties);
+        const uint32_t word = __ballot_sync(0xffffffffu, sel);
+        if ((threadIdx.x & 31) == 0 && w0 + (int)(threadIdx.x & ~31u) < L) maskw[(w0 + threadIdx.x) >> 5] = word;
+    }
+}
+
+struct TopkServerArgs {
+    const float* z; int64_t dz;       // the workers' compensated vectors
+    const uint32_t* B; int64_t Wp;    // and their masks
+    float* zbar; uint32_t* Bbar;      // the server's compensated vector and mask
+    float* m32;                       // accumulator during the step, the new momentum after it
+    const float* v; float* x;
+    int64_t d, chunk;
+    int n; float nf, lr, eps;
+    double frac;
+};
+
+__global__ void __launch_bounds__(kThreads)
+k_topk_server(const TopkServerArgs a)
+{
+    __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t sh[2];
+    __shared__ uint32_t warp_ties[kWarps];
+    const int64_t c = blockIdx.x;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const int nwords = (L + 31) / 32;
+    float* acc = a.m32 + base;
+    float* zb = a.zbar + base;
+    uint32_t* maskbar = a.Bbar + base / 32;
+
+    // sum of the n sparse messages, worker by worker (every element is touched by at most one thread per worker)
+    for (int j = threadIdx.x; j < L; j += kThreads) acc[j] = 0.0f;
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int i = 0; i < a.n; ++i) {
+        const uint32_t* mw = a.B + (int64_t)i * a.Wp + base / 32;
+        const float* zi = a.z + (int64_t)i * a.dz + base;
+        for (int w = threadIdx.x; w < nwords; w += kThreads) {
+            uint32_t word = mw[w];
+            while (word) {
+                const int j = w * 32 + (__ffs(word) - 1);
+                word &= word - 1;
+                if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+            }
+        }
+        __syncthreads();
+    }
+    // pass A: zbar = sum / n + dbar_old
+    for (int j = threadIdx.x; j < L; j += kThreads) {
+        const uint32_t old = (maskbar[j >> 5] >> (j & 31)) & 1u;
+        const float zn = __fadd_rn(__fdiv_rn(acc[j], a.nf), topk_error(zb[j], old));
+        atomicAdd(&hist[mag_key(zn) >> 20], 1u);
+        acc[j] = zn;                                   // staged here: zbar's old mask bits are still needed by other threads' words
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < L; j += kThreads) zb[j] = acc[j];
+    uint32_t tau, ties;
+    topk_threshold(zb, L, topk_count(a.frac, L), hist, sh, tau, ties);
+    // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
+    uint32_t seen = 0;
+    for (int w0 = 0; w0 < L; w0 += kThreads) {
+        const int j = w0 + threadIdx.x;
+        const bool valid = j < L;
+        const float zn = valid ? zb[j] : 0.0f;
+        const bool sel = topk_select_wave(valid, mag_key(zn), tau, ties, seen, warp_ties);
+        const uint32_t word = __ballot_sync(0xffffffffu, sel);
+        if ((threadIdx.x & 31) == 0 && w0 + (int)(threadIdx.x & ~31u) < L) maskbar[(w0 + threadIdx.x) >> 5] = word;
+        if (valid) {
+            const float mnew = sel ? zn : 0.0f;
+            acc[j] = mnew;
+            a.x[base + j] = apply_elem(a.x[base + j], a.v[base + j], mnew, a.lr, a.eps);
+        }
+    }
+}
+
+__global__ void k_materialise_error_topk(const float* __restrict__ z, const uint32_t* __restrict__ mask,
+                                         float* __restrict__ out, int64_t first, int64_t count)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = first + j;
+        out[j] = topk_error(z[e], (mask[e >> 5] >> (e & 31)) & 1u);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Error monitor: squared l2 norms of the compression errors (the quantities Assumption 1 bounds).
 // Row r < n is worker r (delta = z_r - (+-s_r)), row n the server.  One CTA per (row, 4096-element
 // tile) writes a binary64 partial sum; k_error_norm_rows adds a row's tiles in order.
@@ -1235,6 +1476,8 @@ struct apms_ctx {
     float beta1, beta2, eps, lr;
     int t;
     int64_t steps;           // steps taken through apms_step (warmup and compressed)
+    int compressor;          // APMS_COMPRESSOR_*
+    double topk_frac;        // top-k: fraction of a chunk that is sent
     int variant;             // APMS_VARIANT_*: what the workers compress
     int64_t csteps;          // compression-phase steps taken (the variant is fixed once one has run)
     int substep;             // phase-wise step: 0 = between steps, 1 = worker phase done, 2 = a server phase done
@@ -1422,8 +1665,22 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     return APMS_OK;
 }
 
+apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
+{
+    TopkWorkerArgs a;
+    a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp; a.m32 = c->m();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.C = c->L.C; a.i0 = i0; a.ni = ni;
+    a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1; a.frac = c->topk_frac;
+    const int64_t blocks = c->L.C * ni;
+    if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
+    Timed t(c, APMS_KERNEL_WORKER);
+    APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+    return launch_check(c, "k_topk_worker");
+}
+
 apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
 {
+    if (c->compressor == APMS_COMPRESSOR_TOPK) return launch_worker_topk(c, G, gtype, i0, ni);
     if (use_fine_worker(c)) return launch_worker_fine(c, G, gtype, i0, ni);
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
@@ -1563,6 +1820,21 @@ apms_status launch_apply(apms_ctx* c)
 
 apms_status launch_server_and_apply(apms_ctx* c)
 {
+    if (c->compressor == APMS_COMPRESSOR_TOPK) {       // one kernel: sparse average, recompression, momentum, model update
+        TopkServerArgs a;
+        a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp;
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.v = c->v(); a.x = c->x();
+        a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n; a.lr = c->lr; a.eps = c->eps;
+        a.frac = c->topk_frac;
+        if (c->L.C > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");
+        Timed t(c, APMS_KERNEL_SERVER);
+        k_topk_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
+        apms_status st = launch_check(c, "k_topk_server");
+        if (st != APMS_OK) return st;
+        c->m_is_fp32 = true;
+        c->csteps += 1;
+        return APMS_OK;
+    }
     const ServerSource own = {c->B(0), c->L.Wp, c->s(0), c->L.Cp, c->L.n};
     bool applied = false;      // steps 5-6 already done by the fused server kernel
     const bool gradient = c->variant == APMS_VARIANT_GRADIENT;      // its apply differs: never fused
@@ -1631,6 +1903,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
     c->steps = 0; c->has_sched = false; c->substep = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
+    c->compressor = APMS_COMPRESSOR_ONEBIT; c->topk_frac = 0.01;
     c->fine_run = kFineRunDefault;
     if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
@@ -1734,6 +2007,7 @@ apms_status apms_worker_phase(apms_ctx* c, const void* const* grads_dev, apms_gr
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_worker_phase needs the COMPRESSED phase (call apms_freeze_v first)");
     if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "the previous phase-wise step is not finished (apms_apply_phase)");
+    if (c->compressor != APMS_COMPRESSOR_ONEBIT) return fail(c, APMS_ERR_BAD_STATE, "the phase-wise step exists for the 1-bit compressor only");
     GradPtrs G;
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
@@ -1876,11 +2150,17 @@ apms_status apms_get_state_slice(apms_ctx* c, apms_state_id which, int worker, i
         }
         break;
     case APMS_STATE_WORKER_ERR:
-        k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->z(worker), c->s(worker), c->stage(0), first, count, c->L.chunk);
+        if (c->compressor == APMS_COMPRESSOR_TOPK)
+            k_materialise_error_topk<<<grid, kThreads, 0, c->stream>>>(c->z(worker), c->B(worker), c->stage(0), first, count);
+        else
+            k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->z(worker), c->s(worker), c->stage(0), first, count, c->L.chunk);
         staged = true;
         break;
     case APMS_STATE_SERVER_ERR:
-        k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->zbar(), c->Sbar(), c->stage(0), first, count, c->L.chunk);
+        if (c->compressor == APMS_COMPRESSOR_TOPK)
+            k_materialise_error_topk<<<grid, kThreads, 0, c->stream>>>(c->zbar(), c->Bbar(), c->stage(0), first, count);
+        else
+            k_materialise_error<<<grid, kThreads, 0, c->stream>>>(c->zbar(), c->Sbar(), c->stage(0), first, count, c->L.chunk);
         staged = true;
         break;
     case APMS_STATE_WORKER_BITS: src = (const char*)c->B(worker); break;
@@ -1921,6 +2201,8 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
         if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
         // delta = z - (+-0) = z: store the error as z with all scales of this worker zero
         APMS_CUDA(c, cudaMemsetAsync(c->s(worker), 0, (size_t)c->L.Cp * 4, c->stream));
+        if (c->compressor == APMS_COMPRESSOR_TOPK)      // top-k: delta = z - (mask ? z : 0) = z with an empty mask
+            APMS_CUDA(c, cudaMemsetAsync(c->B(worker), 0, (size_t)c->L.Wp * 4, c->stream));
         dst = c->z(worker);
         break;
     case APMS_STATE_SERVER_ERR:
@@ -1931,6 +2213,8 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
             c->m_is_fp32 = true;
         }
         APMS_CUDA(c, cudaMemsetAsync(c->Sbar(), 0, (size_t)c->L.Cp * 4, c->stream));
+        if (c->compressor == APMS_COMPRESSOR_TOPK)
+            APMS_CUDA(c, cudaMemsetAsync(c->Bbar(), 0, (size_t)c->L.Wp * 4, c->stream));
         dst = c->zbar();
         break;
     default: return fail(c, APMS_ERR_INVALID_ARG, "this state array cannot be set");
@@ -2039,10 +2323,27 @@ apms_status apms_selftest_wait_report(apms_ctx* c, int leave_reported)
     return APMS_OK;
 }
 
+apms_status apms_set_compressor(apms_ctx* c, apms_compressor kind, double topk_fraction)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (kind != APMS_COMPRESSOR_ONEBIT && kind != APMS_COMPRESSOR_TOPK) return fail(c, APMS_ERR_INVALID_ARG, "unknown compressor");
+    if (c->csteps > 0 && (int)kind != c->compressor)
+        return fail(c, APMS_ERR_BAD_STATE, "the compressor cannot change once a compression-phase step has run");
+    if (kind == APMS_COMPRESSOR_TOPK) {
+        if (!(topk_fraction > 0.0 && topk_fraction <= 1.0)) return fail(c, APMS_ERR_INVALID_ARG, "the top-k fraction must lie in (0, 1]");
+        if (c->variant != APMS_VARIANT_MOMENTUM || c->L.t.l1) return fail(c, APMS_ERR_BAD_STATE, "top-k runs with the momentum variant and has no scale");
+        c->topk_frac = topk_fraction;
+    }
+    c->compressor = (int)kind;
+    return APMS_OK;
+}
+
 apms_status apms_set_variant(apms_ctx* c, apms_variant variant)
 {
     if (!c) return APMS_ERR_INVALID_ARG;
     if (variant != APMS_VARIANT_MOMENTUM && variant != APMS_VARIANT_GRADIENT) return fail(c, APMS_ERR_INVALID_ARG, "unknown variant");
+    if (variant == APMS_VARIANT_GRADIENT && c->compressor == APMS_COMPRESSOR_TOPK)
+        return fail(c, APMS_ERR_BAD_STATE, "the gradient variant exists for the 1-bit compressor only");
     if (c->csteps > 0 && (int)variant != c->variant)
         return fail(c, APMS_ERR_BAD_STATE, "the variant cannot change once a compression-phase step has run");
     c->variant = (int)variant;

@@ -205,6 +205,77 @@ def test_uncompressed_step_equals_the_identity_compressor(d, n, chunk):
     H.compare_state(ctx, orc, w, exact=True)
 
 
+# ------------------------------------------------------------------ the top-k compressor
+
+def _topk_compare(ctx, orc, w, step):
+    d, n = w.d, w.n
+    idx = np.arange(d)
+    for which, ref in ((B.STATE_X, orc.x), (B.STATE_M, orc.m), (B.STATE_SERVER_ERR, orc.server_err)):
+        assert np.array_equal(ctx.get_state(which).view(np.uint32), ref.view(np.uint32)), (step, which)
+    mask = (ctx.get_state(B.STATE_SERVER_BITS)[idx // 32] >> (idx % 32).astype(np.uint32)) & 1
+    assert np.array_equal(mask.astype(np.uint8), orc.server_selected), (step, "server mask")
+    for i in range(n):
+        assert np.array_equal(ctx.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), orc.worker_err(i).view(np.uint32)), (step, i)
+        mask = (ctx.get_state(B.STATE_WORKER_BITS, i)[idx // 32] >> (idx % 32).astype(np.uint32)) & 1
+        assert np.array_equal(mask.astype(np.uint8), orc.worker_selected(i)), (step, i, "mask")
+
+
+@pytest.mark.parametrize("d,n,chunk,frac", [(5 * 4096 + 1234, 3, 4096, 0.01), (3 * 1024 + 5, 4, 96, 0.1), (2 * 32768 + 23552, 4, 32768, 0.01),
+                                            (70000, 16, 160, 0.05), (9 * 512 + 3, 2, 512, 0.5), (300, 2, 64, 1.0), (1, 1, 32, 0.3),
+                                            (3 * 65536 + 7, 2, 65536, 0.001)])
+def test_topk_compressor_bit_identical(d, n, chunk, frac):
+    """Top-k compression of the momentum: selection masks, errors, momentum and model bit-identical to the oracle,
+    through warmup, device-gradient steps, a host-gradient step and a bfloat16-gradient step."""
+    import torch
+
+    w = tiny(d, n, chunk, cfg_id=180)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, frac)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+    for step in range(2):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(2, 8):
+        gs = wl.host_gradients(w, step)
+        if step == 5:
+            ctx.compressed_step_host([torch.from_numpy(g).pin_memory() for g in gs])
+        elif step == 6:
+            g16 = [torch.from_numpy(g).to(torch.bfloat16) for g in gs]
+            gs = [g.to(torch.float32).numpy() for g in g16]
+            ctx.compressed_step([g.cuda() for g in g16])
+        else:
+            ctx.compressed_step(H.upload(gs))
+        orc.compressed_step(gs)
+        _topk_compare(ctx, orc, w, step)
+    with pytest.raises(B.ApmsError) as e:
+        ctx.set_compressor(B.COMPRESSOR_ONEBIT)               # fixed once a compression-phase step has run
+    assert e.value.status == B.ERR_BAD_STATE
+    with pytest.raises(B.ApmsError) as e:
+        ctx.worker_phase(H.upload(wl.host_gradients(w, 9)))
+    assert e.value.status == B.ERR_BAD_STATE
+
+
+def test_topk_ties_and_teacher_forced_errors():
+    """Many equal magnitudes (gradients drawn from three values) and errors forced from the oracle: the tie rule
+    (lower index first) and apms_set_state in top-k mode."""
+    w = tiny(4 * 256 + 40, 2, 256, cfg_id=181)
+    ctx, orc = H.make_pair(w, x0=np.zeros(w.d, np.float32))
+    ctx.set_compressor(B.COMPRESSOR_TOPK, 0.07)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(0.07)
+    ctx.freeze_v(); orc.freeze_v()
+    rng = np.random.default_rng(5)
+    for step in range(5):
+        gs = [rng.choice(np.array([-0.5, 0.25, 0.5], np.float32), size=w.d) for _ in range(w.n)]
+        if step == 3:
+            orc.server_err[:] = rng.choice(np.array([-0.125, 0.0, 0.125], np.float32), size=w.d)
+            for i in range(w.n):
+                orc.worker_err(i)[:] = rng.choice(np.array([-0.125, 0.0, 0.125], np.float32), size=w.d)
+            H.teacher_force(ctx, orc, w)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        _topk_compare(ctx, orc, w, step)
+
+
 # ------------------------------------------------------------------ phase driver and error monitor
 
 def test_scheduled_steps_follow_algorithm_1():

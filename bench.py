@@ -190,6 +190,8 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
 
     dev = torch.device("cuda", local_rank)
     ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}")
+    if args.compressor == "topk":
+        ctx.set_compressor(B.COMPRESSOR_TOPK, args.topk_fraction)
     x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)
     ctx.set_params(x0)
     del x0
@@ -302,6 +304,9 @@ def main(argv=None) -> int:
     ap.add_argument("--chunk", type=int, default=None, help="override the chunk length")
     ap.add_argument("--d", type=int, default=None, help="use only the first d elements of the parameter set")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--compressor", default="onebit", choices=["onebit", "topk"],
+                    help="the compression operator (the configurations of record use the 1-bit compressor)")
+    ap.add_argument("--topk-fraction", type=float, default=0.01)
     ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16", "float16"],
                     help="element type of the gradient arrays (the configurations of record use float32)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -328,6 +333,7 @@ def main(argv=None) -> int:
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": f"{w.name}: d={w.d}, n={w.n} simulated workers, chunk={w.chunk}, {w.dist} gradients",
               "d": w.d, "n_workers": w.n, "chunk": w.chunk, "gradient_dtype": args.grad_dtype,
+              "compressor": args.compressor if args.compressor == "onebit" else f"topk {args.topk_fraction}",
               "parallelism": f"replicas x{world}",
               "l2_policy": "inputs_exceed_l2" if 12 * w.d * w.n > (256 << 20) else "l2_resident",
               "gradient_ring": 2}
@@ -383,13 +389,21 @@ def main(argv=None) -> int:
     m = measure(w, args, rank, world, local_rank, dist, want_adam=args.adam, want_e2e=not args.no_e2e)
     ms_per_step, kernel_ms = m["ms_per_step"], m["kernel_ms"]
     ab = algorithmic_bytes(w.d, w.n, w.chunk, 4 if args.grad_dtype == "float32" else 2)
-    if "apply" not in kernel_ms:          # steps 4-6 ran as one kernel: it moves both kernels' bytes (Bbar is not re-read)
+    if args.compressor == "topk":
+        # g, z read, z write and both masks per worker, the binary32 momentum once; masks, the kept values,
+        # zbar read + write, new momentum, v, x read, x write, server mask
+        gb = 4 if args.grad_dtype == "float32" else 2
+        ab["worker"] = w.n * ((8 + gb) * w.d + w.d // 4) + 4 * w.d
+        ab["server"] = w.n * (w.d // 8 + int(4 * args.topk_fraction * w.d)) + (8 + 4 + 12) * w.d + w.d // 8
+        ab["step"] = ab["worker"] + ab["server"]
+    elif "apply" not in kernel_ms:          # steps 4-6 ran as one kernel: it moves both kernels' bytes (Bbar is not re-read)
         ab["server"] = ab["server"] + ab["apply"] - 4 * -(-w.d // 32)
         ab["step"] = ab["worker"] + ab["server"]
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
     step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * w.n
-               if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32" else None)
+               if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32"
+               and args.compressor == "onebit" else None)
     roofline = {"bound": "hbm", "kernel": "k_worker", "achieved": wk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": wk_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": traffic,
                 "algorithmic_bytes_per_launch": ab["worker"],

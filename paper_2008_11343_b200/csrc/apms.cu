@@ -1155,6 +1155,14 @@ __device__ __forceinline__ uint32_t mag_key(float z) { return __float_as_uint(z)
 // the one the method performs, so that non-finite values behave as they do there).
 __device__ __forceinline__ float topk_error(float z, uint32_t selected) { return __fsub_rn(z, selected ? z : 0.0f); }
 
+// hist[bin] += 1 for every lane with `on`, lanes with equal bins combined into one shared-memory atomic
+// (the magnitudes of a chunk crowd into a few bins of the top level; plain atomics would serialise there).
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool on, uint32_t bin)
+{
+    const uint32_t peers = __match_any_sync(0xffffffffu, on ? bin : 0xffffffffu);
+    if (on && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+}
+
 // hist[0..nbins) are counts; K >= 1 is the rank wanted, counted from the top bin.  Returns (to all threads)
 // the bin that holds the K-th key and reduces K to the rank inside that bin.  Ends with a barrier.
 __device__ __forceinline__ int topk_find_bin(const uint32_t* hist, int nbins, uint32_t& K, uint32_t* sh)
@@ -1192,40 +1200,66 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
     const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
     __syncthreads();
-    for (int j = threadIdx.x; j < L; j += kThreads) {
-        const uint32_t key = mag_key(zc[j]);
-        if ((key >> 20) == b0) atomicAdd(&hist[(key >> 9) & 0x7ffu], 1u);
+    // the lower levels spread over many bins: plain atomics (combining equal bins costs more than it saves there)
+#pragma unroll 4
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (k + e < L && (key[e] >> 20) == b0) atomicAdd(&hist[(key[e] >> 9) & 0x7ffu], 1u);
     }
     const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
     for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
     __syncthreads();
     const uint32_t top = (b0 << 11) | b1;
-    for (int j = threadIdx.x; j < L; j += kThreads) {
-        const uint32_t key = mag_key(zc[j]);
-        if ((key >> 9) == top) atomicAdd(&hist[key & 0x1ffu], 1u);
+#pragma unroll 4
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (k + e < L && (key[e] >> 9) == top) atomicAdd(&hist[key[e] & 0x1ffu], 1u);
     }
     const uint32_t b2 = (uint32_t)topk_find_bin(hist, 512, K, sh);
     tau = (top << 9) | b2;
     ties = K;
 }
 
-// One wave of the ordered pass: thread t looks at element j of the wave; returns whether it is selected.
-// `seen` counts the elements equal to tau in earlier positions (same value in every thread).
-__device__ __forceinline__ bool topk_select_wave(bool valid, uint32_t key, uint32_t tau, uint32_t ties, uint32_t& seen,
-                                                 uint32_t* warp_ties)
+// One wave (1024 elements) of the ordered pass: the thread holds the keys of 4 consecutive elements
+// (validmask: which of them exist) and gets back the nibble of its selected elements.  `seen` counts the
+// elements equal to tau in earlier positions (same value in every thread).
+__device__ __forceinline__ uint32_t topk_select_wave(const uint32_t key[4], uint32_t validmask, uint32_t tau, uint32_t ties,
+                                                     uint32_t& seen, uint32_t* warp_ties)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const bool tie = valid && key == tau;
-    const uint32_t ballot = __ballot_sync(0xffffffffu, tie);
-    if (lane == 0) warp_ties[warp] = __popc(ballot);
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) cnt += ((validmask >> e) & 1u) && key[e] == tau;
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) warp_ties[warp] = incl;
     __syncthreads();
     uint32_t before = seen, total = 0;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) { const uint32_t c = warp_ties[w]; if (w < warp) before += c; total += c; }
-    before += __popc(ballot & ((1u << lane) - 1u));
+    before += incl - cnt;
     seen += total;
     __syncthreads();                                   // warp_ties may be rewritten by the next wave
-    return valid && (key > tau || (tie && before < ties));
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if ((validmask >> e) & 1u) {
+            const bool tie = key[e] == tau;
+            if (key[e] > tau || (tie && before < ties)) nibble |= 1u << e;
+            before += tie;
+        }
+    }
+    return nibble;
 }
 
 struct TopkWorkerArgs {
@@ -1266,33 +1300,49 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
     __syncthreads();
     // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask
-    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
-        const float4 gv = ld_grad4_checked<GT>(g, k, L);
-        const float4 zv = ld4_checked(zc, k, L, false);
-        const float4 mv = ld4_checked(m, k, L, false);
-        const uint32_t nib = maskw[k >> 5] >> (k & 31);
-        const float gg[4] = {gv.x, gv.y, gv.z, gv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w}, mm[4] = {mv.x, mv.y, mv.z, mv.w};
-        float zn[4];
+    const int L128 = (L + 127) & ~127;                 // whole warps reach hist_add
+    constexpr int UA = 1;                              // iterations whose loads are issued together (more did not help: the pass is bound by the histogram updates)
+    for (int k0 = threadIdx.x * 4; k0 < L128; k0 += kThreads * 4 * UA) {
+        float4 gv[UA], zv[UA], mv[UA];
+        uint32_t nibs[UA];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
-            zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
-            if (k + e < L) atomicAdd(&hist[mag_key(zn[e]) >> 20], 1u);
+        for (int u = 0; u < UA; ++u) {
+            const int k = k0 + u * kThreads * 4;
+            gv[u] = ld_grad4_checked<GT>(g, k, L);
+            zv[u] = ld4_checked(zc, k, L, false);
+            mv[u] = ld4_checked(m, k, L, false);
+            nibs[u] = k < L ? maskw[k >> 5] >> (k & 31) : 0u;
         }
-        if (k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
-        else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
+#pragma unroll
+        for (int u = 0; u < UA; ++u) {
+            const int k = k0 + u * kThreads * 4;
+            if (k >= L128) break;                      // uniform in a warp
+            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w}, zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
+            const float mm[4] = {mv[u].x, mv[u].y, mv[u].z, mv[u].w};
+            float zn[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
+                zn[e] = __fadd_rn(mi, topk_error(zo[e], (nibs[u] >> e) & 1u));
+                hist_add(hist, k + e < L, mag_key(zn[e]) >> 20);
+            }
+            if (k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+            else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
+        }
     }
     uint32_t tau, ties;
     topk_threshold(zc, L, topk_count(a.frac, L), hist, sh, tau, ties);      // its first barrier also orders the z stores
     // ordered pass: the selection mask, one word per warp and wave
     uint32_t seen = 0;
-    for (int w0 = 0; w0 < L; w0 += kThreads) {
-        const int j = w0 + threadIdx.x;
-        const bool valid = j < L;
-        const uint32_t key = valid ? mag_key(zc[j]) : 0u;
-        const bool sel = topk_select_wave(valid, key, tau, ties, seen, warp_ties);
-        const uint32_t word = __ballot_sync(0xffffffffu, sel);
-        if ((threadIdx.x & 31) == 0 && w0 + (int)(threadIdx.x & ~31u) < L) maskw[(w0 + threadIdx.x) >> 5] = word;
+    const int lane = threadIdx.x & 31;
+    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+        const int k = w0 + threadIdx.x * 4;
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+        const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
+        const uint32_t nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+        if ((lane & 7) == 0 && k < L) maskw[k >> 5] = word;
     }
 }
 
@@ -1339,11 +1389,15 @@ k_topk_server(const TopkServerArgs a)
         __syncthreads();
     }
     // pass A: zbar = sum / n + dbar_old
-    for (int j = threadIdx.x; j < L; j += kThreads) {
-        const uint32_t old = (maskbar[j >> 5] >> (j & 31)) & 1u;
-        const float zn = __fadd_rn(__fdiv_rn(acc[j], a.nf), topk_error(zb[j], old));
-        atomicAdd(&hist[mag_key(zn) >> 20], 1u);
-        acc[j] = zn;                                   // staged here: zbar's old mask bits are still needed by other threads' words
+    const int Lr = (L + 31) & ~31;
+    for (int j = threadIdx.x; j < Lr; j += kThreads) {
+        float zn = 0.0f;
+        if (j < L) {
+            const uint32_t old = (maskbar[j >> 5] >> (j & 31)) & 1u;
+            zn = __fadd_rn(__fdiv_rn(acc[j], a.nf), topk_error(zb[j], old));
+            acc[j] = zn;                               // staged here: zbar's old mask bits are still needed by other threads' words
+        }
+        hist_add(hist, j < L, mag_key(zn) >> 20);
     }
     __syncthreads();
     for (int j = threadIdx.x; j < L; j += kThreads) zb[j] = acc[j];
@@ -1351,17 +1405,29 @@ k_topk_server(const TopkServerArgs a)
     topk_threshold(zb, L, topk_count(a.frac, L), hist, sh, tau, ties);
     // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
     uint32_t seen = 0;
-    for (int w0 = 0; w0 < L; w0 += kThreads) {
-        const int j = w0 + threadIdx.x;
-        const bool valid = j < L;
-        const float zn = valid ? zb[j] : 0.0f;
-        const bool sel = topk_select_wave(valid, mag_key(zn), tau, ties, seen, warp_ties);
-        const uint32_t word = __ballot_sync(0xffffffffu, sel);
-        if ((threadIdx.x & 31) == 0 && w0 + (int)(threadIdx.x & ~31u) < L) maskbar[(w0 + threadIdx.x) >> 5] = word;
-        if (valid) {
-            const float mnew = sel ? zn : 0.0f;
-            acc[j] = mnew;
-            a.x[base + j] = apply_elem(a.x[base + j], a.v[base + j], mnew, a.lr, a.eps);
+    const int lane = threadIdx.x & 31;
+    const float* __restrict__ v = a.v + base;
+    float* __restrict__ x = a.x + base;
+    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+        const int k = w0 + threadIdx.x * 4;
+        const float4 zv = ld4_checked(zb, k, L, false);
+        const float4 vv = ld4_checked(v, k, L, true);
+        const float4 xv = ld4_checked(x, k, L, true);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+        const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
+        const uint32_t nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+        if ((lane & 7) == 0 && k < L) maskbar[k >> 5] = word;
+        const float4 mn = make_float4((nibble & 1u) ? zv.x : 0.0f, (nibble & 2u) ? zv.y : 0.0f,
+                                      (nibble & 4u) ? zv.z : 0.0f, (nibble & 8u) ? zv.w : 0.0f);
+        const float4 xn = make_float4(apply_elem(xv.x, vv.x, mn.x, a.lr, a.eps), apply_elem(xv.y, vv.y, mn.y, a.lr, a.eps),
+                                      apply_elem(xv.z, vv.z, mn.z, a.lr, a.eps), apply_elem(xv.w, vv.w, mn.w, a.lr, a.eps));
+        if (k + 3 < L) {
+            *reinterpret_cast<float4*>(acc + k) = mn;
+            st_stream4(x + k, xn);
+        } else {
+            const float mm[4] = {mn.x, mn.y, mn.z, mn.w}, xx[4] = {xn.x, xn.y, xn.z, xn.w};
+            for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mm[e]; x[k + e] = xx[e]; }
         }
     }
 }

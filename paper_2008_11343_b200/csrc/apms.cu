@@ -1281,7 +1281,7 @@ __device__ __forceinline__ uint32_t topk_count(double frac, int L)
 }
 
 template <int GT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)     // latency-bound passes: eight resident CTAs beat fewer with more registers
 k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
@@ -1357,7 +1357,7 @@ struct TopkServerArgs {
     double frac;
 };
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)
 k_topk_server(const TopkServerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];

@@ -148,7 +148,8 @@ typedef enum {
 
 /* Bytes of device workspace a context of this shape needs (pure function; 0 if the shape
  * is invalid).  Covers x, v, m, the n worker and one server compensated vectors, all sign
- * words and scales, and two d-float staging buffers for the host-gradient entry point. */
+ * words and scales, two d-float staging buffers for the host-gradient entry point, and the
+ * kernels' scratch (partial sums of squares, the error monitor's sums, a status word). */
 size_t apms_workspace_bytes(int64_t d, int n, int64_t chunk);
 
 /* Create a context on the current CUDA device for d parameters and n simulated workers

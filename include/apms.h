@@ -115,8 +115,9 @@ typedef enum {
  * of largest absolute value and sends nothing for the others, which decompress to 0; equal magnitudes are
  * resolved in favour of the lower index; magnitudes are compared through the bit pattern of |z|.
  * In TOPK mode the context keeps, in place of the sign words, a selection mask per worker and for the
- * server (APMS_STATE_*_BITS return it: bit j = element j was sent), no scales (they read 0), and the
- * momentum in binary32.  Chosen with apms_set_compressor until the first compression-phase step has run;
+ * server (APMS_STATE_*_BITS return it: bit j = element j was sent), in place of the scales the magnitude
+ * of the K-th (smallest sent) element of each chunk (APMS_STATE_*_SCALES; the next step uses it to guess
+ * where its own threshold lies), and the momentum in binary32.  Chosen with apms_set_compressor until the first compression-phase step has run;
  * TOPK works with the momentum variant, the l2 scale setting and the whole-step functions. */
 typedef enum {
     APMS_COMPRESSOR_ONEBIT = 0,

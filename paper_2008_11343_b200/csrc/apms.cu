@@ -1155,14 +1155,6 @@ __device__ __forceinline__ uint32_t mag_key(float z) { return __float_as_uint(z)
 // the one the method performs, so that non-finite values behave as they do there).
 __device__ __forceinline__ float topk_error(float z, uint32_t selected) { return __fsub_rn(z, selected ? z : 0.0f); }
 
-// hist[bin] += 1 for every lane with `on`, lanes with equal bins combined into one shared-memory atomic
-// (the magnitudes of a chunk crowd into a few bins of the top level; plain atomics would serialise there).
-__device__ __forceinline__ void hist_add(uint32_t* hist, bool on, uint32_t bin)
-{
-    const uint32_t peers = __match_any_sync(0xffffffffu, on ? bin : 0xffffffffu);
-    if (on && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
-}
-
 // hist[0..nbins) are counts; K >= 1 is the rank wanted, counted from the top bin.  Returns (to all threads)
 // the bin that holds the K-th key and reduces K to the rank inside that bin.  Ends with a barrier.
 __device__ __forceinline__ int topk_find_bin(const uint32_t* hist, int nbins, uint32_t& K, uint32_t* sh)
@@ -1226,6 +1218,70 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
     ties = K;
 }
 
+// Last step's threshold of the same (worker, chunk) predicts this step's: only keys at or above a floor a
+// little below it (its mantissa lowered by a quarter: about 0.86 of its value) enter the top-level
+// histogram, which takes the shared-memory updates from one per element to a few per hundred.  If fewer
+// than K keys reach the floor the guess was wrong and the histogram is rebuilt from all keys (re-read from
+// L2).  The selection itself is exact either way.  A floor of 0 (first step) admits every key.
+constexpr uint32_t kTopkFloorDrop = 1u << 21;
+__device__ __forceinline__ uint32_t topk_floor(float last_threshold)
+{
+    const uint32_t key = mag_key(last_threshold);
+    return key > kTopkFloorDrop ? key - kTopkFloorDrop : 0u;
+}
+
+// The keys at or above the floor are few (a few per cent of a chunk): they are appended, with their
+// positions, to a list in shared memory, and the threshold is then selected from the list alone - no
+// further pass over the chunk.  kTopkList bounds the list; a chunk whose window overflows it, or holds
+// fewer than K keys, takes the general route (histograms over the whole chunk, re-read from L2).
+constexpr int kTopkList = 2048;
+// Resident CTAs per SM the top-k kernels are compiled for.  Their passes are latency-bound, so residency
+// matters more than registers, but at eight (32 registers) the spills cost more than the two CTAs give:
+// six measured fastest (worker 16.5 ms against 23.2 at eight and 17.9 at four, 16 workers, 335 M elements).
+constexpr int kTopkResident = 6;
+
+struct TopkList { uint32_t key[kTopkList]; uint32_t idx[kTopkList]; uint32_t count; };
+
+__device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_t idx)
+{
+    const uint32_t pos = atomicAdd(&l.count, 1u);
+    if (pos < (uint32_t)kTopkList) { l.key[pos] = key; l.idx[pos] = idx; }
+}
+
+// The same three-level select as topk_threshold, over the list's n keys.  Also returns how many keys
+// equal tau in all (ties_total); ties <= ties_total of them are to be kept.
+__device__ __forceinline__ void topk_threshold_list(const TopkList& l, int n, uint32_t K, uint32_t* hist, uint32_t* sh,
+                                                    uint32_t& tau, uint32_t& ties, uint32_t& ties_total)
+{
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int p = threadIdx.x; p < n; p += kThreads) atomicAdd(&hist[l.key[p] >> 20], 1u);
+    const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int p = threadIdx.x; p < n; p += kThreads)
+        if ((l.key[p] >> 20) == b0) atomicAdd(&hist[(l.key[p] >> 9) & 0x7ffu], 1u);
+    const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    const uint32_t top = (b0 << 11) | b1;
+    for (int p = threadIdx.x; p < n; p += kThreads)
+        if ((l.key[p] >> 9) == top) atomicAdd(&hist[l.key[p] & 0x1ffu], 1u);
+    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 512, K, sh);
+    tau = (top << 9) | b2;
+    ties = K;
+    ties_total = hist[b2];
+    __syncthreads();                                   // hist is reused by the caller
+}
+
+// Top-level histogram over the whole chunk (general route).
+__device__ __forceinline__ void topk_full_hist(const float* zc, int L, uint32_t* hist)
+{
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < L; j += kThreads) atomicAdd(&hist[mag_key(zc[j]) >> 20], 1u);
+}
+
 // One wave (1024 elements) of the ordered pass: the thread holds the keys of 4 consecutive elements
 // (validmask: which of them exist) and gets back the nibble of its selected elements.  `seen` counts the
 // elements equal to tau in earlier positions (same value in every thread).
@@ -1266,6 +1322,7 @@ struct TopkWorkerArgs {
     float* z; int64_t dz;
     uint32_t* B; int64_t Wp;          // selection masks
     const float* m32;
+    float* thr; int64_t Cp;           // per (worker, chunk): the magnitude of the K-th element of the last step
     int64_t d, chunk, C;
     int i0, ni;
     float beta1, omb1;
@@ -1281,12 +1338,13 @@ __device__ __forceinline__ uint32_t topk_count(double frac, int L)
 }
 
 template <int GT>
-__global__ void __launch_bounds__(kThreads, 8)     // latency-bound passes: eight resident CTAs beat fewer with more registers
+__global__ void __launch_bounds__(kThreads, kTopkResident)
 k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
     __shared__ uint32_t sh[2];
     __shared__ uint32_t warp_ties[kWarps];
+    __shared__ TopkList list;
     const int ii = (int)(blockIdx.x % a.ni);
     const int64_t c = blockIdx.x / a.ni;
     const int i = a.i0 + ii;
@@ -1296,43 +1354,72 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     float* zc = a.z + (int64_t)i * a.dz + base;
     uint32_t* maskw = a.B + (int64_t)i * a.Wp + base / 32;
     const float* __restrict__ m = a.m32 + base;
+    float* thr = a.thr + (int64_t)i * a.Cp + c;
+    const uint32_t K = topk_count(a.frac, L);
+    // a window from last step's threshold only pays while it is likely to fit the list
+    const uint32_t floor_key = 2 * K <= (uint32_t)kTopkList ? topk_floor(*thr) : 0u;
 
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    if (threadIdx.x == 0) list.count = 0;
     __syncthreads();
-    // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask
-    const int L128 = (L + 127) & ~127;                 // whole warps reach hist_add
-    constexpr int UA = 1;                              // iterations whose loads are issued together (more did not help: the pass is bound by the histogram updates)
-    for (int k0 = threadIdx.x * 4; k0 < L128; k0 += kThreads * 4 * UA) {
-        float4 gv[UA], zv[UA], mv[UA];
-        uint32_t nibs[UA];
+    // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask;
+    // whole 1024-element sweeps without bounds checks, two sweeps' loads in flight, then the ragged rest
+    const int Lfull = L & ~(kThreads * 4 - 1);
+    auto sweep = [&](int k, float4 gv, float4 zv, float4 mv, uint32_t nib, bool checked) {
+        const float gg[4] = {gv.x, gv.y, gv.z, gv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w}, mm[4] = {mv.x, mv.y, mv.z, mv.w};
+        float zn[4];
 #pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const int k = k0 + u * kThreads * 4;
-            gv[u] = ld_grad4_checked<GT>(g, k, L);
-            zv[u] = ld4_checked(zc, k, L, false);
-            mv[u] = ld4_checked(m, k, L, false);
-            nibs[u] = k < L ? maskw[k >> 5] >> (k & 31) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const int k = k0 + u * kThreads * 4;
-            if (k >= L128) break;                      // uniform in a warp
-            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w}, zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
-            const float mm[4] = {mv[u].x, mv[u].y, mv[u].z, mv[u].w};
-            float zn[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
-                zn[e] = __fadd_rn(mi, topk_error(zo[e], (nibs[u] >> e) & 1u));
-                hist_add(hist, k + e < L, mag_key(zn[e]) >> 20);
+        for (int e = 0; e < 4; ++e) {
+            const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
+            zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
+            if (!checked || k + e < L) {
+                const uint32_t key = mag_key(zn[e]);
+                if (floor_key == 0) atomicAdd(&hist[key >> 20], 1u);          // no guess yet: every key counts
+                else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
             }
-            if (k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
-            else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
         }
+        if (!checked || k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
+    };
+    int k = threadIdx.x * 4;
+    for (; k + kThreads * 4 < Lfull; k += 2 * kThreads * 4) {
+        const int k2 = k + kThreads * 4;
+        const float4 g0 = Grad<GT>::ld4(g, k), g1 = Grad<GT>::ld4(g, k2);
+        const float4 z0 = *reinterpret_cast<const float4*>(zc + k), z1 = *reinterpret_cast<const float4*>(zc + k2);
+        const float4 m0 = *reinterpret_cast<const float4*>(m + k), m1 = *reinterpret_cast<const float4*>(m + k2);
+        const uint32_t n0 = maskw[k >> 5] >> (k & 31), n1 = maskw[k2 >> 5] >> (k2 & 31);
+        sweep(k, g0, z0, m0, n0, false);
+        sweep(k2, g1, z1, m1, n1, false);
     }
+    for (; k < Lfull; k += kThreads * 4)
+        sweep(k, Grad<GT>::ld4(g, k), *reinterpret_cast<const float4*>(zc + k), *reinterpret_cast<const float4*>(m + k),
+              maskw[k >> 5] >> (k & 31), false);
+    for (; k < L; k += kThreads * 4)
+        sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), ld4_checked(m, k, L, false),
+              maskw[k >> 5] >> (k & 31), true);
+    __syncthreads();                                   // z stores, histogram and list are complete
+    const int nwords = (L + 31) / 32;
+    const uint32_t listed = list.count;
     uint32_t tau, ties;
-    topk_threshold(zc, L, topk_count(a.frac, L), hist, sh, tau, ties);      // its first barrier also orders the z stores
-    // ordered pass: the selection mask, one word per warp and wave
+    if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList && nwords <= kTopkBins) {
+        uint32_t ties_total;
+        topk_threshold_list(list, (int)listed, K, hist, sh, tau, ties, ties_total);
+        if (ties_total == ties) {                      // every key equal to tau is kept: the mask comes from the list
+            for (int w = threadIdx.x; w < nwords; w += kThreads) hist[w] = 0;
+            __syncthreads();
+            for (int p = threadIdx.x; p < (int)listed; p += kThreads)
+                if (list.key[p] >= tau) atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31));
+            __syncthreads();
+            for (int w = threadIdx.x; w < nwords; w += kThreads) maskw[w] = hist[w];
+            if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+            return;
+        }
+    } else {
+        if (floor_key != 0) topk_full_hist(zc, L, hist);
+        topk_threshold(zc, L, K, hist, sh, tau, ties);
+    }
+    if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+    // ordered pass over the chunk: the selection mask with the tie rule
     uint32_t seen = 0;
     const int lane = threadIdx.x & 31;
     for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
@@ -1351,18 +1438,20 @@ struct TopkServerArgs {
     const uint32_t* B; int64_t Wp;    // and their masks
     float* zbar; uint32_t* Bbar;      // the server's compensated vector and mask
     float* m32;                       // accumulator during the step, the new momentum after it
+    float* thr;                       // per chunk: the magnitude of the K-th element of the last step
     const float* v; float* x;
     int64_t d, chunk;
     int n; float nf, lr, eps;
     double frac;
 };
 
-__global__ void __launch_bounds__(kThreads, 8)
+__global__ void __launch_bounds__(kThreads, kTopkResident)
 k_topk_server(const TopkServerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
     __shared__ uint32_t sh[2];
     __shared__ uint32_t warp_ties[kWarps];
+    __shared__ TopkList list;
     const int64_t c = blockIdx.x;
     const int64_t base = c * a.chunk;
     const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
@@ -1371,38 +1460,68 @@ k_topk_server(const TopkServerArgs a)
     float* zb = a.zbar + base;
     uint32_t* maskbar = a.Bbar + base / 32;
 
-    // sum of the n sparse messages, worker by worker (every element is touched by at most one thread per worker)
-    for (int j = threadIdx.x; j < L; j += kThreads) acc[j] = 0.0f;
+    // sum of the n sparse messages in worker order.  A thread owns the same mask words for every worker, so
+    // an element is only ever updated by one thread and its program order is the worker order; the mask
+    // words of eight workers are fetched together.
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        if (k + 3 < L) *reinterpret_cast<float4*>(acc + k) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        else for (int e = 0; k + e < L; ++e) acc[k + e] = 0.0f;
+    }
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    if (threadIdx.x == 0) list.count = 0;
     __syncthreads();
-    for (int i = 0; i < a.n; ++i) {
-        const uint32_t* mw = a.B + (int64_t)i * a.Wp + base / 32;
-        const float* zi = a.z + (int64_t)i * a.dz + base;
-        for (int w = threadIdx.x; w < nwords; w += kThreads) {
-            uint32_t word = mw[w];
-            while (word) {
-                const int j = w * 32 + (__ffs(word) - 1);
-                word &= word - 1;
-                if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+    for (int w = threadIdx.x; w < nwords; w += kThreads) {
+        for (int i0 = 0; i0 < a.n; i0 += 8) {
+            uint32_t mw[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) mw[u] = i0 + u < a.n ? a.B[(int64_t)(i0 + u) * a.Wp + base / 32 + w] : 0u;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                uint32_t word = mw[u];
+                const float* zi = a.z + (int64_t)(i0 + u) * a.dz + base;
+                while (word) {
+                    const int j = w * 32 + (__ffs(word) - 1);
+                    word &= word - 1;
+                    if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+                }
             }
         }
-        __syncthreads();
-    }
-    // pass A: zbar = sum / n + dbar_old
-    const int Lr = (L + 31) & ~31;
-    for (int j = threadIdx.x; j < Lr; j += kThreads) {
-        float zn = 0.0f;
-        if (j < L) {
-            const uint32_t old = (maskbar[j >> 5] >> (j & 31)) & 1u;
-            zn = __fadd_rn(__fdiv_rn(acc[j], a.nf), topk_error(zb[j], old));
-            acc[j] = zn;                               // staged here: zbar's old mask bits are still needed by other threads' words
-        }
-        hist_add(hist, j < L, mag_key(zn) >> 20);
     }
     __syncthreads();
-    for (int j = threadIdx.x; j < L; j += kThreads) zb[j] = acc[j];
+    // pass A: zbar = sum / n + dbar_old
+    const uint32_t K = topk_count(a.frac, L);
+    const uint32_t floor_key = 2 * K <= (uint32_t)kTopkList ? topk_floor(a.thr[c]) : 0u;
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 av = ld4_checked(acc, k, L, false);
+        const float4 zv = ld4_checked(zb, k, L, false);
+        const uint32_t nib = maskbar[k >> 5] >> (k & 31);
+        const float aa[4] = {av.x, av.y, av.z, av.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
+        float zn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            zn[e] = __fadd_rn(__fdiv_rn(aa[e], a.nf), topk_error(zo[e], (nib >> e) & 1u));
+            if (k + e < L) {
+                const uint32_t key = mag_key(zn[e]);
+                if (floor_key == 0) atomicAdd(&hist[key >> 20], 1u);
+                else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
+            }
+        }
+        if (k + 3 < L) *reinterpret_cast<float4*>(zb + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        else for (int e = 0; k + e < L; ++e) zb[k + e] = zn[e];
+    }
+    __syncthreads();
+    const uint32_t listed = list.count;
     uint32_t tau, ties;
-    topk_threshold(zb, L, topk_count(a.frac, L), hist, sh, tau, ties);
+    bool keep_all_ties = false;                        // then "selected" is simply key >= tau
+    if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList) {
+        uint32_t ties_total;
+        topk_threshold_list(list, (int)listed, K, hist, sh, tau, ties, ties_total);
+        keep_all_ties = ties_total == ties;
+    } else {
+        if (floor_key != 0) topk_full_hist(zb, L, hist);
+        topk_threshold(zb, L, K, hist, sh, tau, ties);
+    }
+    if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
     // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
     uint32_t seen = 0;
     const int lane = threadIdx.x & 31;
@@ -1415,7 +1534,14 @@ k_topk_server(const TopkServerArgs a)
         const float4 xv = ld4_checked(x, k, L, true);
         const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
         const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
-        const uint32_t nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        uint32_t nibble;
+        if (keep_all_ties) {                           // uniform: no ranking, no barriers
+            nibble = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) nibble |= (((validmask >> e) & 1u) && key[e] >= tau) ? 1u << e : 0u;
+        } else {
+            nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        }
         const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
         if ((lane & 7) == 0 && k < L) maskbar[k >> 5] = word;
         const float4 mn = make_float4((nibble & 1u) ? zv.x : 0.0f, (nibble & 2u) ? zv.y : 0.0f,
@@ -1735,6 +1861,7 @@ apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0
 {
     TopkWorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp; a.m32 = c->m();
+    a.thr = c->s(0); a.Cp = c->L.Cp;
     a.d = c->L.d; a.chunk = c->L.chunk; a.C = c->L.C; a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1; a.frac = c->topk_frac;
     const int64_t blocks = c->L.C * ni;
@@ -1889,7 +2016,7 @@ apms_status launch_server_and_apply(apms_ctx* c)
     if (c->compressor == APMS_COMPRESSOR_TOPK) {       // one kernel: sparse average, recompression, momentum, model update
         TopkServerArgs a;
         a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp;
-        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.v = c->v(); a.x = c->x();
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n; a.lr = c->lr; a.eps = c->eps;
         a.frac = c->topk_frac;
         if (c->L.C > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");

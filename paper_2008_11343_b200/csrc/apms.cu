@@ -1218,60 +1218,80 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
     ties = K;
 }
 
-// Last step's threshold of the same (worker, chunk) predicts this step's: only keys at or above a floor a
-// little below it (its mantissa lowered by a quarter: about 0.86 of its value) enter the top-level
-// histogram, which takes the shared-memory updates from one per element to a few per hundred.  If fewer
-// than K keys reach the floor the guess was wrong and the histogram is rebuilt from all keys (re-read from
-// L2).  The selection itself is exact either way.  A floor of 0 (first step) admits every key.
-constexpr uint32_t kTopkFloorDrop = 1u << 21;
-__device__ __forceinline__ uint32_t topk_floor(float last_threshold)
+// Last step's threshold of the same (worker, chunk) predicts this step's: only the keys at or above a
+// floor a little below it (key lowered by 2^20, an eighth of an exponent step: 0.92 of the threshold) are
+// looked at for the selection, which is exact either way - a chunk whose window turns out to hold fewer
+// than K keys, or more than the list below can take, goes the general route (histograms over the whole
+// chunk, re-read from L2).  Error feedback piles the unsent elements up just under the threshold, and while
+// the errors still build up the threshold rises by 5 to 10 % a step, so the window holds several times K
+// keys (about 4 K on the benchmark's gradients at k = 1 %).  Hence a window only for K <= kTopkList / 6;
+// for larger K the first pass builds the top-level histogram of all keys itself.  A stored threshold of 0
+// (first step) also means no window.  The list is kept small on purpose: shared memory comes out of the L1
+// cache, which the first pass, the general route and the server's sparse sum live on (a list of 4096 entries
+// made the worker 45 % and the server 30 % slower).
+constexpr int kTopkList = 2048;
+constexpr uint32_t kTopkFloorDrop = 1u << 20;
+__device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K)
 {
     const uint32_t key = mag_key(last_threshold);
-    return key > kTopkFloorDrop ? key - kTopkFloorDrop : 0u;
+    return (6 * K <= (uint32_t)kTopkList && key > kTopkFloorDrop) ? key - kTopkFloorDrop : 0u;
 }
 
-// The keys at or above the floor are few (a few per cent of a chunk): they are appended, with their
-// positions, to a list in shared memory, and the threshold is then selected from the list alone - no
-// further pass over the chunk.  kTopkList bounds the list; a chunk whose window overflows it, or holds
-// fewer than K keys, takes the general route (histograms over the whole chunk, re-read from L2).
-constexpr int kTopkList = 2048;
+// The keys inside the window are appended, with their positions in the chunk (16 bits: the list is used
+// for chunks of up to 65536 elements), to a list in shared memory, and threshold and mask are then taken
+// from the list alone - no further pass over the chunk.
 // Resident CTAs per SM the top-k kernels are compiled for.  Their passes are latency-bound, so residency
 // matters more than registers, but at eight (32 registers) the spills cost more than the two CTAs give:
 // six measured fastest (worker 16.5 ms against 23.2 at eight and 17.9 at four, 16 workers, 335 M elements).
 constexpr int kTopkResident = 6;
 
-struct TopkList { uint32_t key[kTopkList]; uint32_t idx[kTopkList]; uint32_t count; };
+struct TopkList { uint32_t key[kTopkList]; uint16_t idx[kTopkList]; uint32_t count; };
 
 __device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_t idx)
 {
     const uint32_t pos = atomicAdd(&l.count, 1u);
-    if (pos < (uint32_t)kTopkList) { l.key[pos] = key; l.idx[pos] = idx; }
+    if (pos < (uint32_t)kTopkList) { l.key[pos] = key; l.idx[pos] = (uint16_t)idx; }
 }
 
-// The same three-level select as topk_threshold, over the list's n keys.  Also returns how many keys
-// equal tau in all (ties_total); ties <= ties_total of them are to be kept.
-__device__ __forceinline__ void topk_threshold_list(const TopkList& l, int n, uint32_t K, uint32_t* hist, uint32_t* sh,
+// Threshold of the K largest keys of the list (n >= K entries, all >= floor_key).  The keys lie in a
+// narrow band above the floor, so the select runs on rel = key - floor_key in three 8-bit levels (bits
+// 23..16, clipped at 255; 15..8; 7..0) with 256-bin histograms: one bin per thread to clear, eight per lane
+// to scan.  Returns false, with nothing decided, when the K-th key lies in the clipped bin (it is then
+// more than four times the floor).  Also returns how many keys equal tau in all (ties_total); ties <=
+// ties_total of them are to be kept.
+static_assert(kThreads == 256, "one histogram bin per thread");
+__device__ __forceinline__ bool topk_threshold_list(const TopkList& l, int n, uint32_t floor_key, uint32_t K,
+                                                    uint32_t* hist, uint32_t* sh,
                                                     uint32_t& tau, uint32_t& ties, uint32_t& ties_total)
 {
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    hist[threadIdx.x] = 0;
     __syncthreads();
-    for (int p = threadIdx.x; p < n; p += kThreads) atomicAdd(&hist[l.key[p] >> 20], 1u);
-    const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        atomicAdd(&hist[rel >> 16 < 255u ? rel >> 16 : 255u], 1u);
+    }
+    const uint32_t b0 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    if (b0 == 255u) return false;                      // the same value in every thread
+    hist[threadIdx.x] = 0;
     __syncthreads();
-    for (int p = threadIdx.x; p < n; p += kThreads)
-        if ((l.key[p] >> 20) == b0) atomicAdd(&hist[(l.key[p] >> 9) & 0x7ffu], 1u);
-    const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
-    for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        if (rel >> 16 == b0) atomicAdd(&hist[(rel >> 8) & 0xffu], 1u);
+    }
+    const uint32_t b1 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    hist[threadIdx.x] = 0;
     __syncthreads();
-    const uint32_t top = (b0 << 11) | b1;
-    for (int p = threadIdx.x; p < n; p += kThreads)
-        if ((l.key[p] >> 9) == top) atomicAdd(&hist[l.key[p] & 0x1ffu], 1u);
-    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 512, K, sh);
-    tau = (top << 9) | b2;
+    const uint32_t top = (b0 << 8) | b1;
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        if (rel >> 8 == top) atomicAdd(&hist[rel & 0xffu], 1u);
+    }
+    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    tau = floor_key + ((top << 8) | b2);
     ties = K;
     ties_total = hist[b2];
     __syncthreads();                                   // hist is reused by the caller
+    return true;
 }
 
 // Top-level histogram over the whole chunk (general route).
@@ -1356,8 +1376,7 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     const float* __restrict__ m = a.m32 + base;
     float* thr = a.thr + (int64_t)i * a.Cp + c;
     const uint32_t K = topk_count(a.frac, L);
-    // a window from last step's threshold only pays while it is likely to fit the list
-    const uint32_t floor_key = 2 * K <= (uint32_t)kTopkList ? topk_floor(*thr) : 0u;
+    const uint32_t floor_key = L <= 65536 ? topk_floor(*thr, K) : 0u;
 
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
     if (threadIdx.x == 0) list.count = 0;
@@ -1401,20 +1420,22 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     const int nwords = (L + 31) / 32;
     const uint32_t listed = list.count;
     uint32_t tau, ties;
+    bool have_tau = false;
     if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList && nwords <= kTopkBins) {
         uint32_t ties_total;
-        topk_threshold_list(list, (int)listed, K, hist, sh, tau, ties, ties_total);
-        if (ties_total == ties) {                      // every key equal to tau is kept: the mask comes from the list
+        have_tau = topk_threshold_list(list, (int)listed, floor_key, K, hist, sh, tau, ties, ties_total);
+        if (have_tau && ties_total == ties) {          // every key equal to tau is kept: the mask comes from the list
             for (int w = threadIdx.x; w < nwords; w += kThreads) hist[w] = 0;
             __syncthreads();
             for (int p = threadIdx.x; p < (int)listed; p += kThreads)
-                if (list.key[p] >= tau) atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31));
+                if (list.key[p] >= tau) atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31u));
             __syncthreads();
             for (int w = threadIdx.x; w < nwords; w += kThreads) maskw[w] = hist[w];
             if (threadIdx.x == 0) *thr = __uint_as_float(tau);
             return;
         }
-    } else {
+    }
+    if (!have_tau) {                                   // general route: histograms over the whole chunk
         if (floor_key != 0) topk_full_hist(zc, L, hist);
         topk_threshold(zc, L, K, hist, sh, tau, ties);
     }
@@ -1490,7 +1511,7 @@ k_topk_server(const TopkServerArgs a)
     __syncthreads();
     // pass A: zbar = sum / n + dbar_old
     const uint32_t K = topk_count(a.frac, L);
-    const uint32_t floor_key = 2 * K <= (uint32_t)kTopkList ? topk_floor(a.thr[c]) : 0u;
+    const uint32_t floor_key = L <= 65536 ? topk_floor(a.thr[c], K) : 0u;
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
         const float4 av = ld4_checked(acc, k, L, false);
         const float4 zv = ld4_checked(zb, k, L, false);
@@ -1513,11 +1534,13 @@ k_topk_server(const TopkServerArgs a)
     const uint32_t listed = list.count;
     uint32_t tau, ties;
     bool keep_all_ties = false;                        // then "selected" is simply key >= tau
+    bool have_tau = false;
     if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList) {
         uint32_t ties_total;
-        topk_threshold_list(list, (int)listed, K, hist, sh, tau, ties, ties_total);
-        keep_all_ties = ties_total == ties;
-    } else {
+        have_tau = topk_threshold_list(list, (int)listed, floor_key, K, hist, sh, tau, ties, ties_total);
+        keep_all_ties = have_tau && ties_total == ties;
+    }
+    if (!have_tau) {                                   // general route: histograms over the whole chunk
         if (floor_key != 0) topk_full_hist(zb, L, hist);
         topk_threshold(zb, L, K, hist, sh, tau, ties);
     }

@@ -276,6 +276,23 @@ def test_topk_ties_and_teacher_forced_errors():
         _topk_compare(ctx, orc, w, step)
 
 
+def test_topk_threshold_jumps():
+    """The kernels guess each chunk's threshold from the previous step's.  Gradients that grow and shrink by
+    large factors between steps make the guess useless in both directions (no key reaches the window; the
+    K-th key lies far above it): the selection must stay exact."""
+    w = tiny(3 * 8192 + 700, 3, 8192, cfg_id=182)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, 0.02)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(0.02)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step, factor in enumerate([1.0, 1.0, 4096.0, 1.0, 1.0 / 4096.0, 1.0 / 4096.0, 64.0, 1.0], start=1):
+        gs = [(g * np.float32(factor)).astype(np.float32) for g in wl.host_gradients(w, step)]
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        _topk_compare(ctx, orc, w, step)
+
+
 # ------------------------------------------------------------------ phase driver and error monitor
 
 def test_scheduled_steps_follow_algorithm_1():

@@ -1240,6 +1240,10 @@ __device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K)
 // The keys inside the window are appended, with their positions in the chunk (16 bits: the list is used
 // for chunks of up to 65536 elements), to a list in shared memory, and threshold and mask are then taken
 // from the list alone - no further pass over the chunk.
+// From this kept fraction on the server sums the workers' messages in registers (see k_topk_server): measured
+// on 16 workers, 335 M elements, the scattered form takes 2.7 / 3.7 / 5.9 / 12.4 ms at k = 0.1 / 1 / 3 / 10 %,
+// the register form 3.8 / 4.6 / 5.2 / 5.9 ms.
+constexpr double kTopkDenseSum = 0.02;
 // Resident CTAs per SM the top-k kernels are compiled for.  Their passes are latency-bound, so residency
 // matters more than registers, but at eight (32 registers) the spills cost more than the two CTAs give:
 // six measured fastest (worker 16.5 ms against 23.2 at eight and 17.9 at four, 16 workers, 335 M elements).
@@ -1261,7 +1265,7 @@ __device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_
 // ties_total of them are to be kept.
 static_assert(kThreads == 256, "one histogram bin per thread");
 __device__ __forceinline__ bool topk_threshold_list(const TopkList& l, int n, uint32_t floor_key, uint32_t K,
-                                                    uint32_t* hist, uint32_t* sh,
+                                                    uint32_t* hist /* 256 bins */, uint32_t* sh,
                                                     uint32_t& tau, uint32_t& ties, uint32_t& ties_total)
 {
     hist[threadIdx.x] = 0;
@@ -1290,8 +1294,40 @@ __device__ __forceinline__ bool topk_threshold_list(const TopkList& l, int n, ui
     tau = floor_key + ((top << 8) | b2);
     ties = K;
     ties_total = hist[b2];
-    __syncthreads();                                   // hist is reused by the caller
+    __syncthreads();                                   // the bins are reused by the caller
     return true;
+}
+
+// Is list entry p among the kept?  Keys above tau are; of the ties_total keys equal to tau the `ties` with
+// the lowest positions are (the ranking scans the list: only when not every tie is kept).
+__device__ __forceinline__ bool topk_list_selected(const TopkList& l, int n, int p, uint32_t tau, uint32_t ties, uint32_t ties_total)
+{
+    const uint32_t key = l.key[p];
+    if (key != tau) return key > tau;
+    if (ties == ties_total) return true;
+    const uint32_t idx = l.idx[p];
+    uint32_t before = 0;
+    for (int q = 0; q < n; ++q) before += (l.key[q] == tau && l.idx[q] < idx) ? 1u : 0u;
+    return before < ties;
+}
+
+// Without a window the first pass counts every key in 2048 bins of half the usual width (key >> 19: a
+// sixteenth of an exponent step), laid around the last threshold (64 exponent steps either way; around 1
+// when there is none yet), keys outside going to the end bins.  The bin of the K-th key then holds few
+// enough keys for the list (about 1000 of 32768 at k = 10 % on the benchmark's gradients), so that a second
+// pass settles the selection: keys in higher bins are kept, those of the bin itself go to the list, which
+// decides them.  Chunks of more than 65536 elements count key >> 20 from 0 (every key has its own bin) and
+// take the general route.
+__device__ __forceinline__ int topk_fine_base(float last_threshold)
+{
+    const int t = (int)(mag_key(last_threshold) >> 19);
+    if (t == 0) return 1024;
+    return t < 1024 ? 0 : (t > 3072 ? 2048 : t - 1024);
+}
+__device__ __forceinline__ int topk_bin(uint32_t key, int shift, int base)
+{
+    const int b = (int)(key >> shift) - base;
+    return b < 0 ? 0 : (b > kTopkBins - 1 ? kTopkBins - 1 : b);
 }
 
 // Top-level histogram over the whole chunk (general route).
@@ -1362,6 +1398,7 @@ __global__ void __launch_bounds__(kThreads, kTopkResident)
 k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t bins8[256];
     __shared__ uint32_t sh[2];
     __shared__ uint32_t warp_ties[kWarps];
     __shared__ TopkList list;
@@ -1376,7 +1413,10 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     const float* __restrict__ m = a.m32 + base;
     float* thr = a.thr + (int64_t)i * a.Cp + c;
     const uint32_t K = topk_count(a.frac, L);
-    const uint32_t floor_key = L <= 65536 ? topk_floor(*thr, K) : 0u;
+    const int nwords = (L + 31) / 32;
+    const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
+    const uint32_t floor_key = small ? topk_floor(*thr, K) : 0u;
+    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(*thr) : 0;
 
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
     if (threadIdx.x == 0) list.count = 0;
@@ -1393,7 +1433,7 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
             zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
             if (!checked || k + e < L) {
                 const uint32_t key = mag_key(zn[e]);
-                if (floor_key == 0) atomicAdd(&hist[key >> 20], 1u);          // no guess yet: every key counts
+                if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);     // no window: every key counts
                 else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
             }
         }
@@ -1417,32 +1457,59 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
         sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), ld4_checked(m, k, L, false),
               maskw[k >> 5] >> (k & 31), true);
     __syncthreads();                                   // z stores, histogram and list are complete
-    const int nwords = (L + 31) / 32;
-    const uint32_t listed = list.count;
+    const int lane = threadIdx.x & 31;
+    int n_list = 0;                                    // > 0: the list decides, hist[0..nwords) holds the mask so far
+    uint32_t K_list = K, floor_list = floor_key;
+    if (floor_key != 0) {                              // window route: the mask words are still all zero
+        const uint32_t listed = list.count;
+        if (listed >= K && listed <= (uint32_t)kTopkList) n_list = (int)listed;
+    } else if (small) {                                // two-pass route
+        uint32_t Kb = K;
+        const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
+        const uint32_t inbin = hist[b0];
+        __syncthreads();                               // everybody has read the histogram: its words become the mask
+        if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                const float4 zv = ld4_checked(zc, k, L, false);
+                const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+                uint32_t nibble = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (k + e < L) {
+                        const int b = topk_bin(key[e], 19, bin0);
+                        if (b > b0) nibble |= 1u << e;
+                        else if (b == b0) topk_list_add(list, key[e], (uint32_t)(k + e));
+                    }
+                }
+                const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
+                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+            }
+            __syncthreads();
+            n_list = (int)inbin; K_list = Kb; floor_list = (uint32_t)(b0 + bin0) << 19;
+        }
+    }
     uint32_t tau, ties;
     bool have_tau = false;
-    if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList && nwords <= kTopkBins) {
+    if (n_list > 0) {
         uint32_t ties_total;
-        have_tau = topk_threshold_list(list, (int)listed, floor_key, K, hist, sh, tau, ties, ties_total);
-        if (have_tau && ties_total == ties) {          // every key equal to tau is kept: the mask comes from the list
-            for (int w = threadIdx.x; w < nwords; w += kThreads) hist[w] = 0;
-            __syncthreads();
-            for (int p = threadIdx.x; p < (int)listed; p += kThreads)
-                if (list.key[p] >= tau) atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31u));
+        have_tau = topk_threshold_list(list, n_list, floor_list, K_list, bins8, sh, tau, ties, ties_total);
+        if (have_tau) {
+            for (int p = threadIdx.x; p < n_list; p += kThreads)
+                if (topk_list_selected(list, n_list, p, tau, ties, ties_total))
+                    atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31u));
             __syncthreads();
             for (int w = threadIdx.x; w < nwords; w += kThreads) maskw[w] = hist[w];
             if (threadIdx.x == 0) *thr = __uint_as_float(tau);
             return;
         }
     }
-    if (!have_tau) {                                   // general route: histograms over the whole chunk
-        if (floor_key != 0) topk_full_hist(zc, L, hist);
-        topk_threshold(zc, L, K, hist, sh, tau, ties);
-    }
+    // general route: histograms over the whole chunk
+    if (small) topk_full_hist(zc, L, hist);
+    topk_threshold(zc, L, K, hist, sh, tau, ties);
     if (threadIdx.x == 0) *thr = __uint_as_float(tau);
     // ordered pass over the chunk: the selection mask with the tie rule
     uint32_t seen = 0;
-    const int lane = threadIdx.x & 31;
     for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
         const int k = w0 + threadIdx.x * 4;
         const float4 zv = ld4_checked(zc, k, L, false);
@@ -1470,6 +1537,7 @@ __global__ void __launch_bounds__(kThreads, kTopkResident)
 k_topk_server(const TopkServerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t bins8[256];
     __shared__ uint32_t sh[2];
     __shared__ uint32_t warp_ties[kWarps];
     __shared__ TopkList list;
@@ -1481,49 +1549,79 @@ k_topk_server(const TopkServerArgs a)
     float* zb = a.zbar + base;
     uint32_t* maskbar = a.Bbar + base / 32;
 
-    // sum of the n sparse messages in worker order.  A thread owns the same mask words for every worker, so
-    // an element is only ever updated by one thread and its program order is the worker order; the mask
-    // words of eight workers are fetched together.
-    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
-        if (k + 3 < L) *reinterpret_cast<float4*>(acc + k) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        else for (int e = 0; k + e < L; ++e) acc[k + e] = 0.0f;
-    }
     for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
     if (threadIdx.x == 0) list.count = 0;
-    __syncthreads();
-    for (int w = threadIdx.x; w < nwords; w += kThreads) {
-        for (int i0 = 0; i0 < a.n; i0 += 8) {
-            uint32_t mw[8];
+    // The sum of the n sparse messages, in worker order, has two forms.  Few kept elements (k below
+    // kTopkDenseSum): scattered, through the momentum buffer - a thread owns the same mask words for every
+    // worker, so an element is only ever updated by one thread and its program order is the worker order;
+    // the mask words of eight workers are fetched together.  Many: in registers inside pass A (below).
+    const bool dense = a.frac >= kTopkDenseSum;
+    if (!dense) {
+        for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+            if (k + 3 < L) *reinterpret_cast<float4*>(acc + k) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            else for (int e = 0; k + e < L; ++e) acc[k + e] = 0.0f;
+        }
+        __syncthreads();
+        for (int w = threadIdx.x; w < nwords; w += kThreads) {
+            for (int i0 = 0; i0 < a.n; i0 += 8) {
+                uint32_t mw[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) mw[u] = i0 + u < a.n ? a.B[(int64_t)(i0 + u) * a.Wp + base / 32 + w] : 0u;
+                for (int u = 0; u < 8; ++u) mw[u] = i0 + u < a.n ? a.B[(int64_t)(i0 + u) * a.Wp + base / 32 + w] : 0u;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                uint32_t word = mw[u];
-                const float* zi = a.z + (int64_t)(i0 + u) * a.dz + base;
-                while (word) {
-                    const int j = w * 32 + (__ffs(word) - 1);
-                    word &= word - 1;
-                    if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+                for (int u = 0; u < 8; ++u) {
+                    uint32_t word = mw[u];
+                    const float* zi = a.z + (int64_t)(i0 + u) * a.dz + base;
+                    while (word) {
+                        const int j = w * 32 + (__ffs(word) - 1);
+                        word &= word - 1;
+                        if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+                    }
                 }
             }
         }
     }
     __syncthreads();
-    // pass A: zbar = sum / n + dbar_old
+    // pass A: zbar = sum / n + dbar_old.  In the dense form a thread sums its four elements here: it reads
+    // the four mask bits of every worker (four workers at a time) and loads a worker's values only where one
+    // of them is set.
     const uint32_t K = topk_count(a.frac, L);
-    const uint32_t floor_key = L <= 65536 ? topk_floor(a.thr[c], K) : 0u;
+    const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
+    const uint32_t floor_key = small ? topk_floor(a.thr[c], K) : 0u;
+    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(a.thr[c]) : 0;
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
-        const float4 av = ld4_checked(acc, k, L, false);
+        float aa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const uint32_t* mrow = a.B + base / 32 + (k >> 5);
+        const float* zrow = a.z + base;
+        if (!dense) {
+            const float4 av = ld4_checked(acc, k, L, false);
+            aa[0] = av.x; aa[1] = av.y; aa[2] = av.z; aa[3] = av.w;
+        }
+        for (int i0 = 0; dense && i0 < a.n; i0 += 4) {
+            uint32_t nb[4];
+            float4 zi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) nb[u] = i0 + u < a.n ? (mrow[(int64_t)(i0 + u) * a.Wp] >> (k & 31)) & 0xfu : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                zi[u] = nb[u] ? ld4_checked(zrow + (int64_t)(i0 + u) * a.dz, k, L, false) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (nb[u] & 1u) aa[0] = __fadd_rn(aa[0], zi[u].x);
+                if (nb[u] & 2u) aa[1] = __fadd_rn(aa[1], zi[u].y);
+                if (nb[u] & 4u) aa[2] = __fadd_rn(aa[2], zi[u].z);
+                if (nb[u] & 8u) aa[3] = __fadd_rn(aa[3], zi[u].w);
+            }
+        }
         const float4 zv = ld4_checked(zb, k, L, false);
         const uint32_t nib = maskbar[k >> 5] >> (k & 31);
-        const float aa[4] = {av.x, av.y, av.z, av.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
+        const float zo[4] = {zv.x, zv.y, zv.z, zv.w};
         float zn[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             zn[e] = __fadd_rn(__fdiv_rn(aa[e], a.nf), topk_error(zo[e], (nib >> e) & 1u));
             if (k + e < L) {
                 const uint32_t key = mag_key(zn[e]);
-                if (floor_key == 0) atomicAdd(&hist[key >> 20], 1u);
+                if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);
                 else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
             }
         }
@@ -1531,25 +1629,78 @@ k_topk_server(const TopkServerArgs a)
         else for (int e = 0; k + e < L; ++e) zb[k + e] = zn[e];
     }
     __syncthreads();
-    const uint32_t listed = list.count;
+    const int lane = threadIdx.x & 31;
+    const float* __restrict__ v = a.v + base;
+    float* __restrict__ x = a.x + base;
     uint32_t tau, ties;
-    bool keep_all_ties = false;                        // then "selected" is simply key >= tau
     bool have_tau = false;
-    if (floor_key != 0 && listed >= K && listed <= (uint32_t)kTopkList) {
-        uint32_t ties_total;
-        have_tau = topk_threshold_list(list, (int)listed, floor_key, K, hist, sh, tau, ties, ties_total);
-        keep_all_ties = have_tau && ties_total == ties;
+    bool keep_all_ties = false;                        // then "selected" is simply key >= tau
+    if (floor_key != 0) {                              // window route: threshold from the list, then one ordered pass
+        const uint32_t listed = list.count;
+        if (listed >= K && listed <= (uint32_t)kTopkList) {
+            uint32_t ties_total;
+            have_tau = topk_threshold_list(list, (int)listed, floor_key, K, bins8, sh, tau, ties, ties_total);
+            keep_all_ties = have_tau && ties_total == ties;
+        }
+    } else if (small) {                                // two-pass route
+        uint32_t Kb = K;
+        const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
+        const uint32_t inbin = hist[b0];
+        __syncthreads();                               // everybody has read the histogram: its words become the mask
+        if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            // second pass: momentum and model update for every element outside the bin of the K-th key (kept
+            // above it, dropped below); the elements of that bin go to the list, their x untouched
+            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                const float4 zv = ld4_checked(zb, k, L, false);
+                const float4 vv = ld4_checked(v, k, L, true);
+                const float4 xv = ld4_checked(x, k, L, true);
+                const float zz[4] = {zv.x, zv.y, zv.z, zv.w}, vs[4] = {vv.x, vv.y, vv.z, vv.w}, xs[4] = {xv.x, xv.y, xv.z, xv.w};
+                float mn[4], xn[4];
+                uint32_t nibble = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t key = mag_key(zz[e]);
+                    const int b = topk_bin(key, 19, bin0);
+                    const bool in_chunk = k + e < L;
+                    if (in_chunk && b > b0) nibble |= 1u << e;
+                    if (in_chunk && b == b0) topk_list_add(list, key, (uint32_t)(k + e));
+                    mn[e] = ((nibble >> e) & 1u) ? zz[e] : 0.0f;
+                    xn[e] = b == b0 ? xs[e] : apply_elem(xs[e], vs[e], mn[e], a.lr, a.eps);
+                }
+                const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
+                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+                if (k + 3 < L) {
+                    *reinterpret_cast<float4*>(acc + k) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+                    st_stream4(x + k, make_float4(xn[0], xn[1], xn[2], xn[3]));
+                } else {
+                    for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mn[e]; x[k + e] = xn[e]; }
+                }
+            }
+            __syncthreads();
+            uint32_t ties_total;
+            topk_threshold_list(list, (int)inbin, (uint32_t)(b0 + bin0) << 19, Kb, bins8, sh, tau, ties, ties_total);
+            for (int p = threadIdx.x; p < (int)inbin; p += kThreads) {          // the listed elements, one by one
+                const int j = (int)list.idx[p];
+                const bool kept = topk_list_selected(list, (int)inbin, p, tau, ties, ties_total);
+                const float mj = kept ? zb[j] : 0.0f;
+                acc[j] = mj;
+                x[j] = apply_elem(x[j], v[j], mj, a.lr, a.eps);
+                if (kept) atomicOr(&hist[j >> 5], 1u << (j & 31));
+            }
+            __syncthreads();
+            for (int w = threadIdx.x; w < nwords; w += kThreads) maskbar[w] = hist[w];
+            if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
+            return;
+        }
     }
     if (!have_tau) {                                   // general route: histograms over the whole chunk
-        if (floor_key != 0) topk_full_hist(zb, L, hist);
+        if (small) topk_full_hist(zb, L, hist);
         topk_threshold(zb, L, K, hist, sh, tau, ties);
     }
     if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
     // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
     uint32_t seen = 0;
-    const int lane = threadIdx.x & 31;
-    const float* __restrict__ v = a.v + base;
-    float* __restrict__ x = a.x + base;
     for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
         const int k = w0 + threadIdx.x * 4;
         const float4 zv = ld4_checked(zb, k, L, false);

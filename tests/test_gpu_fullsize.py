@@ -113,3 +113,62 @@ def test_sampled_chunks_at_full_size(cfg, samples):
     if w.d % 32:
         assert int(last) >> (w.d % 32) == 0
     assert np.isfinite(ctx.get_state_slice(B.STATE_SERVER_SCALES, 0, w.n_chunks)).all()
+
+
+@pytest.mark.parametrize("frac", [0.01, 0.05])
+def test_topk_sampled_chunks_at_full_size(frac):
+    """The top-k compressor at the benchmark's size and launch shape: sampled chunks replayed by the oracle from
+    the device state, over steps that take the kernels' first-step route and then their predicted-threshold
+    routes; masks, errors, momentum and model bit-identical."""
+    import torch
+
+    w = wl.config(3)
+    free, _ = torch.cuda.mem_get_info()
+    need = B.apms_workspace_bytes(w.d, w.n, w.chunk) + 4 * w.d * w.n + (2 << 30)
+    if free < need:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory, {free / 2**30:.0f} GiB free")
+    chunks = list(wl.sample_chunks(w, 6, seed_key=7))
+    assert chunks[-1] == w.n_chunks - 1
+    sl = _slices(w, chunks)
+    dsub = sum(cnt for _, cnt in sl)
+    # the sampled chunks keep their lengths in the oracle's small problem only if all but the last are whole
+    assert all(cnt == w.chunk for _, cnt in sl[:-1])
+
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, frac)
+    x0 = torch.empty(w.d, dtype=torch.float32, device="cuda").normal_(0.0, w.x0_std)
+    ctx.set_params(x0)
+    grads = [torch.empty(w.d, dtype=torch.float32, device="cuda") for _ in range(w.n)]
+
+    def draw(step):
+        for i in range(w.n):
+            wl.device_gradient(w, step, i, grads[i])
+        return [np.concatenate([g[lo:lo + cnt].cpu().numpy() for lo, cnt in sl]) for g in grads]
+
+    orc = ao.Oracle(dsub, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    orc.set_threads(orc.max_threads())
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+    orc.set_params(_gather(ctx, B.STATE_X, sl))
+    gsub = draw(0)
+    ctx.warmup_step(grads); orc.warmup_step(gsub)
+    ctx.freeze_v(); orc.freeze_v()
+    idx = np.arange(dsub)
+    for step in range(1, 5):
+        orc.x[:] = _gather(ctx, B.STATE_X, sl)
+        orc.m[:] = _gather(ctx, B.STATE_M, sl)
+        orc.server_err[:] = _gather(ctx, B.STATE_SERVER_ERR, sl)
+        for i in range(w.n):
+            orc.worker_err(i)[:] = _gather(ctx, B.STATE_WORKER_ERR, sl, worker=i)
+        gsub = draw(step)
+        ctx.compressed_step(grads)
+        orc.compressed_step(gsub)
+        for which, ref in ((B.STATE_X, orc.x), (B.STATE_M, orc.m), (B.STATE_SERVER_ERR, orc.server_err)):
+            assert np.array_equal(_gather(ctx, which, sl).view(np.uint32), ref.view(np.uint32)), (step, which)
+        words = _gather_words(ctx, B.STATE_SERVER_BITS, sl)
+        assert np.array_equal(((words[idx // 32] >> (idx % 32).astype(np.uint32)) & 1).astype(np.uint8), orc.server_selected), step
+        for i in range(w.n):
+            assert np.array_equal(_gather(ctx, B.STATE_WORKER_ERR, sl, worker=i).view(np.uint32),
+                                  orc.worker_err(i).view(np.uint32)), (step, i)
+            words = _gather_words(ctx, B.STATE_WORKER_BITS, sl, worker=i)
+            assert np.array_equal(((words[idx // 32] >> (idx % 32).astype(np.uint32)) & 1).astype(np.uint8),
+                                  orc.worker_selected(i)), (step, i, "mask")

@@ -222,7 +222,8 @@ def _topk_compare(ctx, orc, w, step):
 
 @pytest.mark.parametrize("d,n,chunk,frac", [(5 * 4096 + 1234, 3, 4096, 0.01), (3 * 1024 + 5, 4, 96, 0.1), (2 * 32768 + 23552, 4, 32768, 0.01),
                                             (70000, 16, 160, 0.05), (9 * 512 + 3, 2, 512, 0.5), (300, 2, 64, 1.0), (1, 1, 32, 0.3),
-                                            (3 * 65536 + 7, 2, 65536, 0.001)])
+                                            (3 * 65536 + 7, 2, 65536, 0.001),
+                                            (131072 + 5000, 2, 131072, 0.01), (2 * 32768 + 100, 3, 32768, 0.1)])
 def test_topk_compressor_bit_identical(d, n, chunk, frac):
     """Top-k compression of the momentum: selection masks, errors, momentum and model bit-identical to the oracle,
     through warmup, device-gradient steps, a host-gradient step and a bfloat16-gradient step."""

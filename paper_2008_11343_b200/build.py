@@ -7,7 +7,8 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SRC = os.path.join(HERE, "csrc", "apms.cu")
+CSRC = os.path.join(HERE, "csrc")
+SRC = os.path.join(CSRC, "apms.cu")                      # the one translation unit; it includes the .cuh files
 HDR = os.path.join(ROOT, "include", "apms.h")
 LIB = os.path.join(HERE, "libapms.so")
 NVCC_FLAGS = [
@@ -21,7 +22,8 @@ NVCC_FLAGS = [
 def is_stale(lib: str = LIB) -> bool:
     if not os.path.exists(lib):
         return True
-    return os.path.getmtime(lib) < max(os.path.getmtime(SRC), os.path.getmtime(HDR))
+    sources = [HDR] + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))]
+    return os.path.getmtime(lib) < max(os.path.getmtime(f) for f in sources)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

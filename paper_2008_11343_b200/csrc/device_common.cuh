@@ -1,0 +1,150 @@
+// Constants, tunables and the small device helpers every kernel uses (loads and stores,
+// the per-element arithmetic with its roundings pinned, sign-word packing, block sums).
+// Part of libapms.so: included by apms.cu, which is the only translation unit.
+#pragma once
+
+namespace {
+
+constexpr int kThreads = 256;            // threads per CTA in every kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kGroup = 128;              // elements one warp covers per 128-bit access (4 sign words)
+
+// Tunables (defaults chosen by measurement on B200; override with -D to re-tune).
+#ifndef APMS_WORKER_U
+#define APMS_WORKER_U 4                  // 128-element groups in flight per warp, worker kernel
+#endif
+#ifndef APMS_SERVER_U
+#define APMS_SERVER_U 2                  // the same for the server kernel
+#endif
+#ifndef APMS_WORKER_CTAS
+#define APMS_WORKER_CTAS 3               // resident CTAs per SM the worker kernel is compiled for
+#endif
+#ifndef APMS_SERVER_CTAS
+#define APMS_SERVER_CTAS 3
+#endif
+
+struct GradPtrs { const void* p[APMS_MAX_WORKERS]; };     // element type given by the kernel's GT template argument
+
+// ------------------------------------------------------------------------------------------
+// small device helpers
+
+__device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void st_stream4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+// Up to four consecutive floats starting at p[k]; elements at or past `len` read as 0.
+__device__ __forceinline__ float4 ld4_checked(const float* p, int k, int len, bool streaming) {
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k + 3 < len) {
+        r = streaming ? ld_stream4(p + k) : *reinterpret_cast<const float4*>(p + k);
+    } else {
+        if (k + 0 < len) r.x = p[k + 0];
+        if (k + 1 < len) r.y = p[k + 1];
+        if (k + 2 < len) r.z = p[k + 2];
+    }
+    return r;
+}
+__device__ __forceinline__ void st4_checked(float* p, int k, int len, float4 v) {
+    if (k + 3 < len) {
+        st_stream4(p + k, v);
+    } else {
+        if (k + 0 < len) p[k + 0] = v.x;
+        if (k + 1 < len) p[k + 1] = v.y;
+        if (k + 2 < len) p[k + 2] = v.z;
+    }
+}
+
+// Gradient element types (apms_grad_type): binary32, bfloat16, binary16.  A 16-bit gradient is
+// widened to binary32 exactly before its first use, so the arithmetic of a step does not change.
+template <int GT> struct Grad;
+template <> struct Grad<APMS_GRAD_F32> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const float*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return ((const float*)p)[e]; }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) { return ld_stream4((const float*)p + k); }
+};
+template <> struct Grad<APMS_GRAD_BF16> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const uint16_t*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __uint_as_float((uint32_t)((const uint16_t*)p)[e] << 16); }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const uint16_t*)p + k));
+        return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                           __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+    }
+};
+template <> struct Grad<APMS_GRAD_F16> {
+    static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const __half*)p + e; }
+    static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __half2float(((const __half*)p)[e]); }
+    static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const __half*)p + k));
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&r.y));
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+};
+// Up to four consecutive gradient elements starting at element k; elements at or past `len` read as 0.
+template <int GT>
+__device__ __forceinline__ float4 ld_grad4_checked(const void* p, int k, int len)
+{
+    if (k + 3 < len) return Grad<GT>::ld4(p, k);
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k + 0 < len) r.x = Grad<GT>::ld1(p, k + 0);
+    if (k + 1 < len) r.y = Grad<GT>::ld1(p, k + 1);
+    if (k + 2 < len) r.z = Grad<GT>::ld1(p, k + 2);
+    return r;
+}
+
+// +-s with the sign of the compressor: z >= 0 gives +s (so do +0 and -0), NaN gives -s.
+__device__ __forceinline__ float signed_scale(float z, float s) { return (z >= 0.0f) ? s : -s; }
+__device__ __forceinline__ float bit_scale(uint32_t bit, float s) { return bit ? s : -s; }
+
+// Model update of one element with the frozen variance (Section 3.3 step 6).
+__device__ __forceinline__ float apply_elem(float x, float v, float q, float lr, float eps) {
+    return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));
+}
+
+// One element's contribution to a chunk's scale, and the scale from the sum.  The scale is the
+// l2 norm of the chunk over sqrt(L) (Section 5.1 read with the paper's norm); the other reading
+// of "magnitude", the mean of |z|, is kept as a switch: |z| = z * (+-1) is added by the same fma.
+__device__ __forceinline__ void scale_accumulate(double& acc, float z, bool l1)
+{
+    const double zd = (double)z;
+    acc = fma(zd, l1 ? copysign(1.0, zd) : zd, acc);
+}
+__device__ __forceinline__ float scale_from_sum(double total, double L, bool l1)
+{
+    return l1 ? (float)(total / L) : (float)sqrt(total / L);
+}
+
+// The compression error implied by a stored compensated value and its chunk's scale.
+__device__ __forceinline__ float implied_error(float z, float s) { return __fsub_rn(z, signed_scale(z, s)); }
+
+// Lane l of a warp holds the four sign bits (nibble) of elements 4l..4l+3 of a 128-element
+// group.  Returns, in lanes 0, 8, 16, 24, the LSB-first sign word of elements 32*(l/8)...
+__device__ __forceinline__ uint32_t pack_group_words(uint32_t nibble, int lane) {
+    uint32_t w = nibble << (4 * (lane & 7));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    w |= __shfl_xor_sync(0xffffffffu, w, 2);
+    w |= __shfl_xor_sync(0xffffffffu, w, 4);
+    return w;
+}
+
+__device__ __forceinline__ double warp_sum(double a) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_down_sync(0xffffffffu, a, o);
+    return a;
+}
+
+// Fixed-order block sum (lane tree, then warps in order); result valid in thread 0.
+__device__ __forceinline__ double block_sum(double a, double* smem) {
+    a = warp_sum(a);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) smem[warp] = a;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += smem[w];
+    }
+    return t;
+}
+
+}  // namespace

@@ -1,0 +1,424 @@
+// Server side (Section 3.3 step 4): the register-staged kernel and the kernel that streams its
+// tiles through a shared-memory ring, optionally fused with the model update.
+// Part of libapms.so: included by apms.cu, which is the only translation unit.
+#pragma once
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Server side: average the n decompressed messages, add the server error, recompress
+// (Section 3.3 step 4).
+
+struct ServerArgs {
+    const uint32_t* B; int64_t Wp;
+    const float* s; int64_t Cp;
+    float* zbar; uint32_t* Bbar; float* Sbar;
+    double* partial;
+    Tiling t;
+    int64_t item0, items;         // items [item0, items) of the C * P chunk tiles
+    int n; float nf;
+};
+
+// U groups of one warp: the n sign words of every group are fetched worker by worker while
+// the running sums (sequential in worker order, as the average is defined) are updated.
+// +-s_i is formed by moving the complemented sign bit onto s_i's sign: no selects, no branches.
+template <int U, bool CHECKED>
+__device__ __forceinline__ void server_groups(const ServerArgs& a, const float* s_sh, const uint32_t* __restrict__ wb,
+                                              float* __restrict__ zb, uint32_t* __restrict__ ob,
+                                              int g0, int gstride, int lane, int L, float S_old, double& acc)
+{
+    const int sh = 4 * (lane & 7);
+    const int wl = lane >> 3;
+    float sum[U][4];
+    float4 zo4[U];
+    bool live[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int k = (g0 + gstride * u) * kGroup + lane * 4;
+        live[u] = !CHECKED || (k < L);
+        zo4[u] = CHECKED ? ld4_checked(zb, k, L, true) : ld_stream4(zb + k);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sum[u][e] = 0.0f;
+    }
+#pragma unroll 4
+    for (int i = 0; i < a.n; ++i) {
+        const uint32_t sbits = __float_as_uint(s_sh[i]);
+        uint32_t w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            w[u] = live[u] ? wb[(int64_t)i * a.Wp + (g0 + gstride * u) * 4 + wl] : 0u;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t neg = ~w[u] >> sh;            // bit e set: element e of this lane is negative
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                sum[u][e] = __fadd_rn(sum[u][e], __uint_as_float(sbits ^ ((neg << (31 - e)) & 0x80000000u)));
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int grp = g0 + gstride * u;
+        const int k = grp * kGroup + lane * 4;
+        const float zo[4] = {zo4[u].x, zo4[u].y, zo4[u].z, zo4[u].w};
+        float zn[4];
+        uint32_t nibble = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float avg = __fdiv_rn(sum[u][e], a.nf);
+            zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+            const bool valid = !CHECKED || (k + e < L);
+            if (valid) {
+                scale_accumulate(acc, zn[e], a.t.l1 != 0);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
+        }
+        const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        if (CHECKED) st4_checked(zb, k, L, out); else st_stream4(zb + k, out);
+        const uint32_t word = pack_group_words(nibble, lane);
+        const int wk = grp * 4 + wl;
+        if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) ob[wk] = word;
+    }
+}
+
+template <int U, int WPC>
+__global__ void __launch_bounds__(kThreads, APMS_SERVER_CTAS)
+k_server(const ServerArgs a)
+{
+    __shared__ double red[kWarps];
+    __shared__ float s_all[kWarps / WPC][APMS_MAX_WORKERS];
+    constexpr int TEAMS = kWarps / WPC;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int team = (WPC == 1) ? warp : 0;
+    const int64_t item = a.item0 + (int64_t)blockIdx.x * TEAMS + team;
+    if (item >= a.items) return;
+    const Item it = decode_item(a.t, item);
+    const int L = it.L;
+    float* s_sh = s_all[team];
+    const int tid_in_team = (WPC == 1) ? lane : (int)threadIdx.x;
+    for (int i = tid_in_team; i < a.n; i += WPC * 32) s_sh[i] = a.s[(int64_t)i * a.Cp + it.c];
+    const float S_old = a.Sbar[it.c];
+    if (WPC == 1) __syncwarp(); else __syncthreads();
+    const uint32_t* __restrict__ wb = a.B + it.base / 32;
+    float* __restrict__ zb = a.zbar + it.base;
+    uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+    const int full = L / kGroup;
+    const int ngroups = (L + kGroup - 1) / kGroup;
+    double acc = 0.0;
+    // Each warp takes a contiguous run of groups, so that the 128-byte line of sign words it
+    // fetches for a worker serves its next seven groups from L1.
+    const int per_warp = (WPC == 1) ? ngroups : (ngroups + WPC - 1) / WPC;
+    int g0 = (WPC == 1) ? 0 : warp * per_warp;
+    const int g_end = (g0 + per_warp < ngroups) ? g0 + per_warp : ngroups;
+    const int g_full = (full < g_end) ? full : g_end;
+    for (; g0 + (U - 1) < g_full; g0 += U)
+        server_groups<U, false>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+    for (; g0 < g_end; ++g0)
+        server_groups<1, true>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+    const double total = team_sum<WPC>(acc, red);
+    if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
+        if (a.t.P == 1) a.Sbar[it.c] = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);
+        else a.partial[it.c * a.t.P + it.p] = total;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Server side, staged form.  One CTA per chunk tile: a producer warp streams the tile through a
+// ring of shared-memory stages with bulk asynchronous copies (an mbarrier per stage counts the
+// arriving bytes, a second one collects the eight consumer warps' releases), so the bytes in
+// flight depend neither on registers nor on occupancy, and no CTA-wide barrier sits in the loop.
+// When the tile is the whole chunk, the CTA goes on to steps 5-6 for the same chunk (its new
+// scale is known once the eight consumer warps have met): v and x travel through the same ring
+// while other CTAs of the SM are still in their arithmetic-bound averaging phase.
+// Needs every slab of kSlab elements to start on a 16-byte boundary in all streams, i.e.
+// chunks that are multiples of kSlab; other shapes use k_server and k_apply.
+
+constexpr int kSlab = 2048;                      // elements per ring stage
+constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per consumer warp
+constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker and slab
+constexpr int kStages = 4;
+constexpr int64_t kStagedSpanElems = 32768;   // a CTA of the fused form walks enough chunks to stream about this many elements
+constexpr int kStagedThreads = kThreads + 32;    // eight consumer warps + one producer warp
+constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about a second of SM clocks
+
+enum { DEVICE_OK = 0, DEVICE_WAIT_TIMEOUT = 1 };
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 1000;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait: false when the phase did not complete within `limit` SM clocks.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int k = 0; k < 32; ++k)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > limit) return false;
+    }
+}
+
+// Self-test of the give-up path: a barrier that nothing ever completes, waited for with a short bound.
+// No copy is in flight and nothing else is touched, so the CTA simply reports and ends.
+__global__ void k_selftest_wait(int* status, long long limit)
+{
+    __shared__ uint64_t never;
+    if (threadIdx.x == 0) { mbar_init(&never, 1); mbar_fence_init(); }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(&never, 0, limit)) atomicExch(status, DEVICE_WAIT_TIMEOUT);
+}
+// Global -> this CTA's shared memory; 16-byte aligned addresses, size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Barrier among the 256 consumer threads only (the producer warp never joins it).
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+struct ServerStagedArgs {
+    ServerArgs a;
+    int* status;          // device status word: set when a bounded wait gave up
+    float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
+    const float* v; float* x; float lr, eps;     // steps 5-6, used by the fused form only
+    int span;             // chunks per CTA of the fused form
+};
+
+// Bytes of one ring stage: a slab of zbar plus n rows of sign words, or (fused form) a slab of v and of x.
+__host__ __device__ __forceinline__ size_t staged_stage_bytes(int n, bool fused)
+{
+    const size_t server = (size_t)kSlab * 4 + (size_t)n * kSlabWords * 4;
+    const size_t apply = (size_t)kSlab * 8;
+    return (fused && apply > server) ? apply : server;
+}
+
+// Sum over the workers, in worker order, of +-s_i for the lane's 2 x 4 elements of one slab.
+// NT > 0: the number of workers is the compile-time constant NT (fully unrolled).
+template <int NT>
+__device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r0, const uint32_t* __restrict__ r1,
+                                                  const uint32_t* __restrict__ neg_s, int n, int sh,
+                                                  float2& s01, float2& s23, float2& t01, float2& t23)
+{
+    const int nn = NT > 0 ? NT : n;
+#pragma unroll(NT > 0 ? NT : 4)
+    for (int i = 0; i < nn; ++i) {
+        const uint32_t ns = neg_s[i];
+        // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
+        const uint32_t y0 = r0[i * kSlabWords] << (28 - sh);
+        const uint32_t y1 = r1[i * kSlabWords] << (28 - sh);
+        float2 q;
+        q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns);
+        s01 = __fadd2_rn(s01, q);
+        q.x = __uint_as_float(((y0 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y0 & 0x80000000u) ^ ns);
+        s23 = __fadd2_rn(s23, q);
+        q.x = __uint_as_float(((y1 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y1 << 2) & 0x80000000u) ^ ns);
+        t01 = __fadd2_rn(t01, q);
+        q.x = __uint_as_float(((y1 << 1) & 0x80000000u) ^ ns); q.y = __uint_as_float((y1 & 0x80000000u) ^ ns);
+        t23 = __fadd2_rn(t23, q);
+    }
+}
+
+// A CTA of the fused form walks `span` consecutive chunks (short chunks are grouped so that a CTA
+// still streams about 32768 elements and the ring never drains between chunks); the unfused form
+// (chunks cut into tiles) handles one tile.  Jobs are numbered across the CTA's whole walk: per
+// chunk first its server slabs, then (fused) its slabs of v and x; job q uses stage q % kStages.
+template <int NT, bool FUSED, bool MULTI>
+__global__ void __launch_bounds__(kStagedThreads, 3)
+k_server_staged(const ServerStagedArgs sa)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const ServerArgs& a = sa.a;
+    __shared__ double red[kWarps];
+    __shared__ uint64_t full[kStages], empty[kStages];
+    __shared__ uint32_t neg_s[2][APMS_MAX_WORKERS];   // bit patterns of -s_i, double-buffered over the walk
+    __shared__ uint32_t nb[kTileMax / 32];            // the current tile's new sign words
+    __shared__ int failed;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = NT > 0 ? NT : a.n;
+    const size_t stage_bytes = staged_stage_bytes(n, FUSED);
+    const int span = MULTI ? sa.span : 1;                  // MULTI = false: one item, the walk's loops fold away
+    const int64_t item0 = a.item0 + (int64_t)blockIdx.x * span;
+    const int nitems = MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
+        failed = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == kWarps) {
+        // ---- producer warp: one lane feeds the ring (only whole 16-byte pieces that hold live elements)
+        if (lane == 0) {
+            int q = 0;
+            bool stop = false;
+            for (int w = 0; w < nitems && !stop; ++w) {
+                const Item it = decode_item(a.t, item0 + w);
+                const int L = it.L;
+                const int nslabs = (L + kSlab - 1) / kSlab;
+                const int njobs = FUSED ? 2 * nslabs : nslabs;
+                const float* __restrict__ zb_g = a.zbar + it.base;
+                const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
+                for (int r = 0; r < njobs; ++r, ++q) {
+                    const int st = q % kStages;
+                    if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; stop = true; break; }
+                    unsigned char* base = smem + (size_t)st * stage_bytes;
+                    const int j = r < nslabs ? r : r - nslabs;
+                    const int left = L - j * kSlab;
+                    const int live = left < kSlab ? left : kSlab;
+                    const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
+                    if (r < nslabs) {
+                        const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
+                        mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
+                        bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
+                        uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
+                        for (int i = 0; i < n; ++i)
+                            bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
+                    } else {
+                        mbar_arrive_expect_tx(&full[st], 2 * zbytes);
+                        bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                        bulk_load(base + (size_t)kSlab * 4, sa.x + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                    }
+                }
+            }
+            if (failed) {
+                // give the copies still in flight a bounded chance to land before shared memory is released
+                const int first = q > kStages ? q - kStages : 0;
+                for (int p = first; p < q; ++p) mbar_wait(&full[p % kStages], (uint32_t)(p / kStages) & 1u);
+            }
+        }
+    } else {
+        // ---- consumer warps: two 128-element groups of every slab each
+        const int sh = 4 * (lane & 7);
+        const int wl = lane >> 3;
+        const int g0 = warp, g1 = warp + kWarps;
+        // A warp whose wait gives up sets `failed`, skips the rest of its phase and still arrives at the next
+        // consumer barrier; after every barrier all consumers read `failed` and leave together.
+        int q = 0;
+        for (int w = 0; w < nitems; ++w) {
+            const Item it = decode_item(a.t, item0 + w);
+            const int L = it.L;
+            const int nslabs = (L + kSlab - 1) / kSlab;
+            uint32_t* negs = neg_s[w & 1];
+            for (int i = threadIdx.x; i < n; i += kThreads)
+                negs[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
+            const float S_old = a.Sbar[it.c];
+            consumer_barrier();                        // -s_i in place; everybody is done with the previous chunk
+            if (failed) break;
+            bool ok = true;
+            double acc = 0.0;
+            for (int j = 0; j < nslabs; ++j, ++q) {
+                const int st = q % kStages;
+                if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
+                const unsigned char* base = smem + (size_t)st * stage_bytes;
+                const float* zs = reinterpret_cast<const float*>(base);
+                const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
+                const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
+                const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
+                float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
+                signed_scale_sums<NT>(rows + g0 * 4 + wl, rows + g1 * 4 + wl, negs, n, sh, s01, s23, t01, t23);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int grp = j * kSlabGroups + (u ? g1 : g0);
+                    const int k = grp * kGroup + lane * 4;
+                    const float4 zo4 = u ? zo1 : zo0;
+                    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+                    const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
+                    float zn[4];
+                    uint32_t nibble = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
+                        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+                        if (k + e < L) {
+                            const double zd = (double)zn[e];
+                            acc = fma(zd, zd, acc);
+                            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                        }
+                    }
+                    st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                    const uint32_t word = pack_group_words(nibble, lane);
+                    if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
+                }
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) red[warp] = acc;
+            consumer_barrier();                        // partial sums and sign words of the tile are in shared memory
+            double total = 0.0;
+#pragma unroll
+            for (int r = 0; r < kWarps; ++r) total += red[r];
+            if (failed) break;
+            if (FUSED) {
+                // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
+                const float S_new = (float)sqrt(total / (double)it.Lc);
+                if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
+                for (int j = 0; ok && j < nslabs; ++j, ++q) {
+                    const int st = q % kStages;
+                    if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
+                    const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
+                    const float* xs = vs + kSlab;
+                    float4 vv[2], xx[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
+                        xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[st]);
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int grp = j * kSlabGroups + (u ? g1 : g0);
+                        const int k = grp * kGroup + lane * 4;
+                        const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                        xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib & 1u, S_new), sa.lr, sa.eps);
+                        xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib & 2u, S_new), sa.lr, sa.eps);
+                        xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib & 4u, S_new), sa.lr, sa.eps);
+                        xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib & 8u, S_new), sa.lr, sa.eps);
+                        st4_checked(sa.x + it.base, k, L, xx[u]);
+                    }
+                }
+            } else if (ok && threadIdx.x == 0) {
+                if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
+                else a.partial[it.c * a.t.P + it.p] = total;
+            }
+            // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
+            if (ok) {
+                uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
+                const int nwords = (L + 31) / 32;
+                for (int w4 = threadIdx.x * 4; w4 < nwords; w4 += kThreads * 4) {
+                    if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
+                    else for (int r = w4; r < nwords; ++r) ob[r] = nb[r];
+                }
+            }
+        }
+    }
+    __syncthreads();                                   // every warp has left its loops; shared memory may go
+    if (threadIdx.x == 0 && failed) atomicExch(sa.status, DEVICE_WAIT_TIMEOUT);
+}
+
+}  // namespace

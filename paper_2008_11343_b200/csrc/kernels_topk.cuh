@@ -1,0 +1,614 @@
+// Top-k compressor (Section 5.1, second item): worker and server kernels.
+// Part of libapms.so: included by apms.cu, which is the only translation unit.
+#pragma once
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Top-k compressor (Section 5.1, second item): per chunk the K = ceil(k L) elements of largest |z| are
+// sent, the others decompress to 0; equal magnitudes go to the lower index.  State in this mode: the
+// compensated vectors z as before, and in place of the sign words a SELECTION MASK (bit j = element j
+// was sent), from which  C[z] = mask ? z : 0  and  delta = z - C[z]  follow exactly; the momentum is
+// kept in binary32.  One CTA per (chunk, worker) / per chunk; a chunk's z is written once and re-read
+// from L2 by the selection passes.
+//
+// Selection: the K-th largest magnitude is found by a three-level radix select over the bit pattern of
+// |z| (11 + 11 + 9 bits, shared-memory histograms), giving the threshold key tau and the number of
+// elements equal to tau that are still to be kept; a last pass in index order marks  key > tau, and the
+// first `ties` elements with key == tau.
+
+constexpr int kTopkBins = 2048;
+
+__device__ __forceinline__ uint32_t mag_key(float z) { return __float_as_uint(z) & 0x7fffffffu; }
+
+// C[z] and the error it leaves, from a stored compensated value and its selection bit (the subtraction is
+// the one the method performs, so that non-finite values behave as they do there).
+__device__ __forceinline__ float topk_error(float z, uint32_t selected) { return __fsub_rn(z, selected ? z : 0.0f); }
+
+// hist[0..nbins) are counts; K >= 1 is the rank wanted, counted from the top bin.  Returns (to all threads)
+// the bin that holds the K-th key and reduces K to the rank inside that bin.  Ends with a barrier.
+__device__ __forceinline__ int topk_find_bin(const uint32_t* hist, int nbins, uint32_t& K, uint32_t* sh)
+{
+    __syncthreads();                                   // the histogram is complete
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x, per = nbins / 32;
+        const int hi = nbins - lane * per, lo = hi - per;             // lane 0 owns the top bins
+        uint32_t mine = 0;
+        for (int b = lo; b < hi; ++b) mine += hist[b];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const uint32_t excl = incl - mine;
+        if (excl < K && K <= incl) {                   // exactly one lane
+            uint32_t k = K - excl;
+            int b = hi - 1;
+            for (; b > lo; --b) { if (k <= hist[b]) break; k -= hist[b]; }
+            sh[0] = (uint32_t)b; sh[1] = k;
+        }
+    }
+    __syncthreads();
+    K = sh[1];
+    return (int)sh[0];
+}
+
+// Threshold of the K largest magnitudes of zc[0..L) (global memory, written by this CTA).  hist must hold
+// the level-0 histogram (key >> 20) already.  Out: tau and the number of elements equal to tau to keep.
+__device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t K, uint32_t* hist, uint32_t* sh,
+                                               uint32_t& tau, uint32_t& ties)
+{
+    const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    // the lower levels spread over many bins: plain atomics (combining equal bins costs more than it saves there)
+#pragma unroll 4
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (k + e < L && (key[e] >> 20) == b0) atomicAdd(&hist[(key[e] >> 9) & 0x7ffu], 1u);
+    }
+    const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
+    for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    const uint32_t top = (b0 << 11) | b1;
+#pragma unroll 4
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (k + e < L && (key[e] >> 9) == top) atomicAdd(&hist[key[e] & 0x1ffu], 1u);
+    }
+    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 512, K, sh);
+    tau = (top << 9) | b2;
+    ties = K;
+}
+
+// Last step's threshold of the same (worker, chunk) predicts this step's: only the keys at or above a
+// floor a little below it (key lowered by 2^20, an eighth of an exponent step: 0.92 of the threshold) are
+// looked at for the selection, which is exact either way - a chunk whose window turns out to hold fewer
+// than K keys, or more than the list below can take, goes the general route (histograms over the whole
+// chunk, re-read from L2).  Error feedback piles the unsent elements up just under the threshold, and while
+// the errors still build up the threshold rises by 5 to 10 % a step, so the window holds several times K
+// keys (about 4 K on the benchmark's gradients at k = 1 %).  Hence a window only for K <= kTopkList / 6;
+// for larger K the first pass builds the top-level histogram of all keys itself.  A stored threshold of 0
+// (first step) also means no window.  The list is kept small on purpose: shared memory comes out of the L1
+// cache, which the first pass, the general route and the server's sparse sum live on (a list of 4096 entries
+// made the worker 45 % and the server 30 % slower).
+constexpr int kTopkList = 2048;
+constexpr uint32_t kTopkFloorDrop = 1u << 20;
+__device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K)
+{
+    const uint32_t key = mag_key(last_threshold);
+    return (6 * K <= (uint32_t)kTopkList && key > kTopkFloorDrop) ? key - kTopkFloorDrop : 0u;
+}
+
+// The keys inside the window are appended, with their positions in the chunk (16 bits: the list is used
+// for chunks of up to 65536 elements), to a list in shared memory, and threshold and mask are then taken
+// from the list alone - no further pass over the chunk.
+// From this kept fraction on the server sums the workers' messages in registers (see k_topk_server): measured
+// on 16 workers, 335 M elements, the scattered form takes 2.7 / 3.7 / 5.9 / 12.4 ms at k = 0.1 / 1 / 3 / 10 %,
+// the register form 3.8 / 4.6 / 5.2 / 5.9 ms.
+constexpr double kTopkDenseSum = 0.02;
+// Resident CTAs per SM the top-k kernels are compiled for.  Their passes are latency-bound, so residency
+// matters more than registers, but at eight (32 registers) the spills cost more than the two CTAs give:
+// six measured fastest (worker 16.5 ms against 23.2 at eight and 17.9 at four, 16 workers, 335 M elements).
+constexpr int kTopkResident = 6;
+
+struct TopkList { uint32_t key[kTopkList]; uint16_t idx[kTopkList]; uint32_t count; };
+
+__device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_t idx)
+{
+    const uint32_t pos = atomicAdd(&l.count, 1u);
+    if (pos < (uint32_t)kTopkList) { l.key[pos] = key; l.idx[pos] = (uint16_t)idx; }
+}
+
+// Threshold of the K largest keys of the list (n >= K entries, all >= floor_key).  The keys lie in a
+// narrow band above the floor, so the select runs on rel = key - floor_key in three 8-bit levels (bits
+// 23..16, clipped at 255; 15..8; 7..0) with 256-bin histograms: one bin per thread to clear, eight per lane
+// to scan.  Returns false, with nothing decided, when the K-th key lies in the clipped bin (it is then
+// more than four times the floor).  Also returns how many keys equal tau in all (ties_total); ties <=
+// ties_total of them are to be kept.
+static_assert(kThreads == 256, "one histogram bin per thread");
+__device__ __forceinline__ bool topk_threshold_list(const TopkList& l, int n, uint32_t floor_key, uint32_t K,
+                                                    uint32_t* hist /* 256 bins */, uint32_t* sh,
+                                                    uint32_t& tau, uint32_t& ties, uint32_t& ties_total)
+{
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        atomicAdd(&hist[rel >> 16 < 255u ? rel >> 16 : 255u], 1u);
+    }
+    const uint32_t b0 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    if (b0 == 255u) return false;                      // the same value in every thread
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        if (rel >> 16 == b0) atomicAdd(&hist[(rel >> 8) & 0xffu], 1u);
+    }
+    const uint32_t b1 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t top = (b0 << 8) | b1;
+    for (int p = threadIdx.x; p < n; p += kThreads) {
+        const uint32_t rel = l.key[p] - floor_key;
+        if (rel >> 8 == top) atomicAdd(&hist[rel & 0xffu], 1u);
+    }
+    const uint32_t b2 = (uint32_t)topk_find_bin(hist, 256, K, sh);
+    tau = floor_key + ((top << 8) | b2);
+    ties = K;
+    ties_total = hist[b2];
+    __syncthreads();                                   // the bins are reused by the caller
+    return true;
+}
+
+// Is list entry p among the kept?  Keys above tau are; of the ties_total keys equal to tau the `ties` with
+// the lowest positions are (the ranking scans the list: only when not every tie is kept).
+__device__ __forceinline__ bool topk_list_selected(const TopkList& l, int n, int p, uint32_t tau, uint32_t ties, uint32_t ties_total)
+{
+    const uint32_t key = l.key[p];
+    if (key != tau) return key > tau;
+    if (ties == ties_total) return true;
+    const uint32_t idx = l.idx[p];
+    uint32_t before = 0;
+    for (int q = 0; q < n; ++q) before += (l.key[q] == tau && l.idx[q] < idx) ? 1u : 0u;
+    return before < ties;
+}
+
+// Without a window the first pass counts every key in 2048 bins of half the usual width (key >> 19: a
+// sixteenth of an exponent step), laid around the last threshold (64 exponent steps either way; around 1
+// when there is none yet), keys outside going to the end bins.  The bin of the K-th key then holds few
+// enough keys for the list (about 1000 of 32768 at k = 10 % on the benchmark's gradients), so that a second
+// pass settles the selection: keys in higher bins are kept, those of the bin itself go to the list, which
+// decides them.  Chunks of more than 65536 elements count key >> 20 from 0 (every key has its own bin) and
+// take the general route.
+__device__ __forceinline__ int topk_fine_base(float last_threshold)
+{
+    const int t = (int)(mag_key(last_threshold) >> 19);
+    if (t == 0) return 1024;
+    return t < 1024 ? 0 : (t > 3072 ? 2048 : t - 1024);
+}
+__device__ __forceinline__ int topk_bin(uint32_t key, int shift, int base)
+{
+    const int b = (int)(key >> shift) - base;
+    return b < 0 ? 0 : (b > kTopkBins - 1 ? kTopkBins - 1 : b);
+}
+
+// Top-level histogram over the whole chunk (general route).
+__device__ __forceinline__ void topk_full_hist(const float* zc, int L, uint32_t* hist)
+{
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < L; j += kThreads) atomicAdd(&hist[mag_key(zc[j]) >> 20], 1u);
+}
+
+// One wave (1024 elements) of the ordered pass: the thread holds the keys of 4 consecutive elements
+// (validmask: which of them exist) and gets back the nibble of its selected elements.  `seen` counts the
+// elements equal to tau in earlier positions (same value in every thread).
+__device__ __forceinline__ uint32_t topk_select_wave(const uint32_t key[4], uint32_t validmask, uint32_t tau, uint32_t ties,
+                                                     uint32_t& seen, uint32_t* warp_ties)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) cnt += ((validmask >> e) & 1u) && key[e] == tau;
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) warp_ties[warp] = incl;
+    __syncthreads();
+    uint32_t before = seen, total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { const uint32_t c = warp_ties[w]; if (w < warp) before += c; total += c; }
+    before += incl - cnt;
+    seen += total;
+    __syncthreads();                                   // warp_ties may be rewritten by the next wave
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if ((validmask >> e) & 1u) {
+            const bool tie = key[e] == tau;
+            if (key[e] > tau || (tie && before < ties)) nibble |= 1u << e;
+            before += tie;
+        }
+    }
+    return nibble;
+}
+
+struct TopkWorkerArgs {
+    float* z; int64_t dz;
+    uint32_t* B; int64_t Wp;          // selection masks
+    const float* m32;
+    float* thr; int64_t Cp;           // per (worker, chunk): the magnitude of the K-th element of the last step
+    int64_t d, chunk, C;
+    int i0, ni;
+    float beta1, omb1;
+    double frac;
+};
+
+__device__ __forceinline__ uint32_t topk_count(double frac, int L)
+{
+    long long K = (long long)ceil(frac * (double)L);
+    if (K < 1) K = 1;
+    if (K > L) K = L;
+    return (uint32_t)K;
+}
+
+template <int GT>
+__global__ void __launch_bounds__(kThreads, kTopkResident)
+k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
+{
+    __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t bins8[256];
+    __shared__ uint32_t sh[2];
+    __shared__ uint32_t warp_ties[kWarps];
+    __shared__ TopkList list;
+    const int ii = (int)(blockIdx.x % a.ni);
+    const int64_t c = blockIdx.x / a.ni;
+    const int i = a.i0 + ii;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
+    float* zc = a.z + (int64_t)i * a.dz + base;
+    uint32_t* maskw = a.B + (int64_t)i * a.Wp + base / 32;
+    const float* __restrict__ m = a.m32 + base;
+    float* thr = a.thr + (int64_t)i * a.Cp + c;
+    const uint32_t K = topk_count(a.frac, L);
+    const int nwords = (L + 31) / 32;
+    const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
+    const uint32_t floor_key = small ? topk_floor(*thr, K) : 0u;
+    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(*thr) : 0;
+
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    if (threadIdx.x == 0) list.count = 0;
+    __syncthreads();
+    // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask;
+    // whole 1024-element sweeps without bounds checks, two sweeps' loads in flight, then the ragged rest
+    const int Lfull = L & ~(kThreads * 4 - 1);
+    auto sweep = [&](int k, float4 gv, float4 zv, float4 mv, uint32_t nib, bool checked) {
+        const float gg[4] = {gv.x, gv.y, gv.z, gv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w}, mm[4] = {mv.x, mv.y, mv.z, mv.w};
+        float zn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
+            zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
+            if (!checked || k + e < L) {
+                const uint32_t key = mag_key(zn[e]);
+                if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);     // no window: every key counts
+                else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
+            }
+        }
+        if (!checked || k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
+    };
+    int k = threadIdx.x * 4;
+    for (; k + kThreads * 4 < Lfull; k += 2 * kThreads * 4) {
+        const int k2 = k + kThreads * 4;
+        const float4 g0 = Grad<GT>::ld4(g, k), g1 = Grad<GT>::ld4(g, k2);
+        const float4 z0 = *reinterpret_cast<const float4*>(zc + k), z1 = *reinterpret_cast<const float4*>(zc + k2);
+        const float4 m0 = *reinterpret_cast<const float4*>(m + k), m1 = *reinterpret_cast<const float4*>(m + k2);
+        const uint32_t n0 = maskw[k >> 5] >> (k & 31), n1 = maskw[k2 >> 5] >> (k2 & 31);
+        sweep(k, g0, z0, m0, n0, false);
+        sweep(k2, g1, z1, m1, n1, false);
+    }
+    for (; k < Lfull; k += kThreads * 4)
+        sweep(k, Grad<GT>::ld4(g, k), *reinterpret_cast<const float4*>(zc + k), *reinterpret_cast<const float4*>(m + k),
+              maskw[k >> 5] >> (k & 31), false);
+    for (; k < L; k += kThreads * 4)
+        sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), ld4_checked(m, k, L, false),
+              maskw[k >> 5] >> (k & 31), true);
+    __syncthreads();                                   // z stores, histogram and list are complete
+    const int lane = threadIdx.x & 31;
+    int n_list = 0;                                    // > 0: the list decides, hist[0..nwords) holds the mask so far
+    uint32_t K_list = K, floor_list = floor_key;
+    if (floor_key != 0) {                              // window route: the mask words are still all zero
+        const uint32_t listed = list.count;
+        if (listed >= K && listed <= (uint32_t)kTopkList) n_list = (int)listed;
+    } else if (small) {                                // two-pass route
+        uint32_t Kb = K;
+        const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
+        const uint32_t inbin = hist[b0];
+        __syncthreads();                               // everybody has read the histogram: its words become the mask
+        if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                const float4 zv = ld4_checked(zc, k, L, false);
+                const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+                uint32_t nibble = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (k + e < L) {
+                        const int b = topk_bin(key[e], 19, bin0);
+                        if (b > b0) nibble |= 1u << e;
+                        else if (b == b0) topk_list_add(list, key[e], (uint32_t)(k + e));
+                    }
+                }
+                const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
+                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+            }
+            __syncthreads();
+            n_list = (int)inbin; K_list = Kb; floor_list = (uint32_t)(b0 + bin0) << 19;
+        }
+    }
+    uint32_t tau, ties;
+    bool have_tau = false;
+    if (n_list > 0) {
+        uint32_t ties_total;
+        have_tau = topk_threshold_list(list, n_list, floor_list, K_list, bins8, sh, tau, ties, ties_total);
+        if (have_tau) {
+            for (int p = threadIdx.x; p < n_list; p += kThreads)
+                if (topk_list_selected(list, n_list, p, tau, ties, ties_total))
+                    atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31u));
+            __syncthreads();
+            for (int w = threadIdx.x; w < nwords; w += kThreads) maskw[w] = hist[w];
+            if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+            return;
+        }
+    }
+    // general route: histograms over the whole chunk
+    if (small) topk_full_hist(zc, L, hist);
+    topk_threshold(zc, L, K, hist, sh, tau, ties);
+    if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+    // ordered pass over the chunk: the selection mask with the tie rule
+    uint32_t seen = 0;
+    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+        const int k = w0 + threadIdx.x * 4;
+        const float4 zv = ld4_checked(zc, k, L, false);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+        const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
+        const uint32_t nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+        if ((lane & 7) == 0 && k < L) maskw[k >> 5] = word;
+    }
+}
+
+struct TopkServerArgs {
+    const float* z; int64_t dz;       // the workers' compensated vectors
+    const uint32_t* B; int64_t Wp;    // and their masks
+    float* zbar; uint32_t* Bbar;      // the server's compensated vector and mask
+    float* m32;                       // accumulator during the step, the new momentum after it
+    float* thr;                       // per chunk: the magnitude of the K-th element of the last step
+    const float* v; float* x;
+    int64_t d, chunk;
+    int n; float nf, lr, eps;
+    double frac;
+};
+
+__global__ void __launch_bounds__(kThreads, kTopkResident)
+k_topk_server(const TopkServerArgs a)
+{
+    __shared__ uint32_t hist[kTopkBins];
+    __shared__ uint32_t bins8[256];
+    __shared__ uint32_t sh[2];
+    __shared__ uint32_t warp_ties[kWarps];
+    __shared__ TopkList list;
+    const int64_t c = blockIdx.x;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const int nwords = (L + 31) / 32;
+    float* acc = a.m32 + base;
+    float* zb = a.zbar + base;
+    uint32_t* maskbar = a.Bbar + base / 32;
+
+    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    if (threadIdx.x == 0) list.count = 0;
+    // The sum of the n sparse messages, in worker order, has two forms.  Few kept elements (k below
+    // kTopkDenseSum): scattered, through the momentum buffer - a thread owns the same mask words for every
+    // worker, so an element is only ever updated by one thread and its program order is the worker order;
+    // the mask words of eight workers are fetched together.  Many: in registers inside pass A (below).
+    const bool dense = a.frac >= kTopkDenseSum;
+    if (!dense) {
+        for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+            if (k + 3 < L) *reinterpret_cast<float4*>(acc + k) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            else for (int e = 0; k + e < L; ++e) acc[k + e] = 0.0f;
+        }
+        __syncthreads();
+        for (int w = threadIdx.x; w < nwords; w += kThreads) {
+            for (int i0 = 0; i0 < a.n; i0 += 8) {
+                uint32_t mw[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) mw[u] = i0 + u < a.n ? a.B[(int64_t)(i0 + u) * a.Wp + base / 32 + w] : 0u;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    uint32_t word = mw[u];
+                    const float* zi = a.z + (int64_t)(i0 + u) * a.dz + base;
+                    while (word) {
+                        const int j = w * 32 + (__ffs(word) - 1);
+                        word &= word - 1;
+                        if (j < L) acc[j] = __fadd_rn(acc[j], zi[j]);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // pass A: zbar = sum / n + dbar_old.  In the dense form a thread sums its four elements here: it reads
+    // the four mask bits of every worker (four workers at a time) and loads a worker's values only where one
+    // of them is set.
+    const uint32_t K = topk_count(a.frac, L);
+    const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
+    const uint32_t floor_key = small ? topk_floor(a.thr[c], K) : 0u;
+    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(a.thr[c]) : 0;
+    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        float aa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const uint32_t* mrow = a.B + base / 32 + (k >> 5);
+        const float* zrow = a.z + base;
+        if (!dense) {
+            const float4 av = ld4_checked(acc, k, L, false);
+            aa[0] = av.x; aa[1] = av.y; aa[2] = av.z; aa[3] = av.w;
+        }
+        for (int i0 = 0; dense && i0 < a.n; i0 += 4) {
+            uint32_t nb[4];
+            float4 zi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) nb[u] = i0 + u < a.n ? (mrow[(int64_t)(i0 + u) * a.Wp] >> (k & 31)) & 0xfu : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                zi[u] = nb[u] ? ld4_checked(zrow + (int64_t)(i0 + u) * a.dz, k, L, false) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (nb[u] & 1u) aa[0] = __fadd_rn(aa[0], zi[u].x);
+                if (nb[u] & 2u) aa[1] = __fadd_rn(aa[1], zi[u].y);
+                if (nb[u] & 4u) aa[2] = __fadd_rn(aa[2], zi[u].z);
+                if (nb[u] & 8u) aa[3] = __fadd_rn(aa[3], zi[u].w);
+            }
+        }
+        const float4 zv = ld4_checked(zb, k, L, false);
+        const uint32_t nib = maskbar[k >> 5] >> (k & 31);
+        const float zo[4] = {zv.x, zv.y, zv.z, zv.w};
+        float zn[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            zn[e] = __fadd_rn(__fdiv_rn(aa[e], a.nf), topk_error(zo[e], (nib >> e) & 1u));
+            if (k + e < L) {
+                const uint32_t key = mag_key(zn[e]);
+                if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);
+                else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
+            }
+        }
+        if (k + 3 < L) *reinterpret_cast<float4*>(zb + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        else for (int e = 0; k + e < L; ++e) zb[k + e] = zn[e];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const float* __restrict__ v = a.v + base;
+    float* __restrict__ x = a.x + base;
+    uint32_t tau, ties;
+    bool have_tau = false;
+    bool keep_all_ties = false;                        // then "selected" is simply key >= tau
+    if (floor_key != 0) {                              // window route: threshold from the list, then one ordered pass
+        const uint32_t listed = list.count;
+        if (listed >= K && listed <= (uint32_t)kTopkList) {
+            uint32_t ties_total;
+            have_tau = topk_threshold_list(list, (int)listed, floor_key, K, bins8, sh, tau, ties, ties_total);
+            keep_all_ties = have_tau && ties_total == ties;
+        }
+    } else if (small) {                                // two-pass route
+        uint32_t Kb = K;
+        const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
+        const uint32_t inbin = hist[b0];
+        __syncthreads();                               // everybody has read the histogram: its words become the mask
+        if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            // second pass: momentum and model update for every element outside the bin of the K-th key (kept
+            // above it, dropped below); the elements of that bin go to the list, their x untouched
+            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                const float4 zv = ld4_checked(zb, k, L, false);
+                const float4 vv = ld4_checked(v, k, L, true);
+                const float4 xv = ld4_checked(x, k, L, true);
+                const float zz[4] = {zv.x, zv.y, zv.z, zv.w}, vs[4] = {vv.x, vv.y, vv.z, vv.w}, xs[4] = {xv.x, xv.y, xv.z, xv.w};
+                float mn[4], xn[4];
+                uint32_t nibble = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t key = mag_key(zz[e]);
+                    const int b = topk_bin(key, 19, bin0);
+                    const bool in_chunk = k + e < L;
+                    if (in_chunk && b > b0) nibble |= 1u << e;
+                    if (in_chunk && b == b0) topk_list_add(list, key, (uint32_t)(k + e));
+                    mn[e] = ((nibble >> e) & 1u) ? zz[e] : 0.0f;
+                    xn[e] = b == b0 ? xs[e] : apply_elem(xs[e], vs[e], mn[e], a.lr, a.eps);
+                }
+                const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
+                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+                if (k + 3 < L) {
+                    *reinterpret_cast<float4*>(acc + k) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+                    st_stream4(x + k, make_float4(xn[0], xn[1], xn[2], xn[3]));
+                } else {
+                    for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mn[e]; x[k + e] = xn[e]; }
+                }
+            }
+            __syncthreads();
+            uint32_t ties_total;
+            topk_threshold_list(list, (int)inbin, (uint32_t)(b0 + bin0) << 19, Kb, bins8, sh, tau, ties, ties_total);
+            for (int p = threadIdx.x; p < (int)inbin; p += kThreads) {          // the listed elements, one by one
+                const int j = (int)list.idx[p];
+                const bool kept = topk_list_selected(list, (int)inbin, p, tau, ties, ties_total);
+                const float mj = kept ? zb[j] : 0.0f;
+                acc[j] = mj;
+                x[j] = apply_elem(x[j], v[j], mj, a.lr, a.eps);
+                if (kept) atomicOr(&hist[j >> 5], 1u << (j & 31));
+            }
+            __syncthreads();
+            for (int w = threadIdx.x; w < nwords; w += kThreads) maskbar[w] = hist[w];
+            if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
+            return;
+        }
+    }
+    if (!have_tau) {                                   // general route: histograms over the whole chunk
+        if (small) topk_full_hist(zb, L, hist);
+        topk_threshold(zb, L, K, hist, sh, tau, ties);
+    }
+    if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
+    // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
+    uint32_t seen = 0;
+    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+        const int k = w0 + threadIdx.x * 4;
+        const float4 zv = ld4_checked(zb, k, L, false);
+        const float4 vv = ld4_checked(v, k, L, true);
+        const float4 xv = ld4_checked(x, k, L, true);
+        const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+        const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
+        uint32_t nibble;
+        if (keep_all_ties) {                           // uniform: no ranking, no barriers
+            nibble = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) nibble |= (((validmask >> e) & 1u) && key[e] >= tau) ? 1u << e : 0u;
+        } else {
+            nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
+        }
+        const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+        if ((lane & 7) == 0 && k < L) maskbar[k >> 5] = word;
+        const float4 mn = make_float4((nibble & 1u) ? zv.x : 0.0f, (nibble & 2u) ? zv.y : 0.0f,
+                                      (nibble & 4u) ? zv.z : 0.0f, (nibble & 8u) ? zv.w : 0.0f);
+        const float4 xn = make_float4(apply_elem(xv.x, vv.x, mn.x, a.lr, a.eps), apply_elem(xv.y, vv.y, mn.y, a.lr, a.eps),
+                                      apply_elem(xv.z, vv.z, mn.z, a.lr, a.eps), apply_elem(xv.w, vv.w, mn.w, a.lr, a.eps));
+        if (k + 3 < L) {
+            *reinterpret_cast<float4*>(acc + k) = mn;
+            st_stream4(x + k, xn);
+        } else {
+            const float mm[4] = {mn.x, mn.y, mn.z, mn.w}, xx[4] = {xn.x, xn.y, xn.z, xn.w};
+            for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mm[e]; x[k + e] = xx[e]; }
+        }
+    }
+}
+
+__global__ void k_materialise_error_topk(const float* __restrict__ z, const uint32_t* __restrict__ mask,
+                                         float* __restrict__ out, int64_t first, int64_t count)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = first + j;
+        out[j] = topk_error(z[e], (mask[e >> 5] >> (e & 31)) & 1u);
+    }
+}
+
+}  // namespace

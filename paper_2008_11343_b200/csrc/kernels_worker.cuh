@@ -1,0 +1,268 @@
+// Worker side of a compression-phase step (Section 3.3 steps 1-2): general and fine-tiled kernels,
+// and the kernels that finish the per-chunk scales.
+// Part of libapms.so: included by apms.cu, which is the only translation unit.
+#pragma once
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Worker side: local momentum + error-compensated 1-bit compression (Section 3.3 steps 1-2).
+// Items are ordered chunk-major, worker-minor, so that the n workers of one chunk run
+// together and share that chunk's momentum bits through L2.
+
+struct WorkerArgs {
+    float* z;  int64_t dz;        // n x d compensated vectors, stride dz
+    uint32_t* B; int64_t Wp;      // n x W sign words, stride Wp
+    float* s;  int64_t Cp;        // n x C scales, stride Cp
+    double* partial;              // n x Pp partial sums (only when P > 1)
+    const float* m32;             // binary32 momentum (first step / forced)
+    const uint32_t* Bbar; const float* Sbar;   // momentum as the server's last message
+    Tiling t;
+    int64_t items;                // C * P * ni
+    int i0, ni;                   // this launch covers workers i0 .. i0+ni-1
+    float beta1, omb1;
+    int send_gradient;            // gradient-compressing variant: z = g_i + delta_i, the momentum is not read
+};
+
+template <bool M32, bool CHECKED>
+__device__ __forceinline__ void worker_group(float beta1, float omb1, float* __restrict__ z, uint32_t* __restrict__ obits,
+                                             int grp, int lane, int L, float s_old, float Sbar,
+                                             float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc, bool l1,
+                                             bool send_gradient = false)
+{
+    const int k = grp * kGroup + lane * 4;
+    float mm[4];
+    if (M32) {
+        mm[0] = mv.x; mm[1] = mv.y; mm[2] = mv.z; mm[3] = mv.w;
+    } else {
+        const uint32_t nib = mw >> (4 * (lane & 7));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mm[e] = bit_scale((nib >> e) & 1u, Sbar);
+    }
+    const float gg[4] = {gv.x, gv.y, gv.z, gv.w};
+    const float zo[4] = {zv.x, zv.y, zv.z, zv.w};
+    float zn[4];
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float mi = send_gradient ? gg[e]                                 // gradient variant: g_i itself is compensated
+                                       : __fmaf_rn(beta1, mm[e], __fmul_rn(omb1, gg[e]));   // local momentum
+        const float err = implied_error(zo[e], s_old);                          // delta_i (old)
+        zn[e] = __fadd_rn(mi, err);                                             // compensated
+        const bool valid = !CHECKED || (k + e < L);
+        if (valid) {
+            scale_accumulate(acc, zn[e], l1);
+            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+        }
+    }
+    const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
+    if (CHECKED) st4_checked(z, k, L, out); else st_stream4(z + k, out);
+    const uint32_t word = pack_group_words(nibble, lane);
+    if ((lane & 7) == 0) {
+        const int wk = grp * 4 + (lane >> 3);
+        if (!CHECKED || wk * 32 < L) __stcs(obits + wk, word);     // streaming: a plain store here costs ~4 % of the kernel
+    }
+}
+
+template <int GT, bool M32, int U, int WPC>
+__global__ void __launch_bounds__(kThreads, APMS_WORKER_CTAS)
+k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
+{
+    __shared__ double red[kWarps];
+    constexpr int TEAMS = kWarps / WPC;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t item = (int64_t)blockIdx.x * TEAMS + (WPC == 1 ? warp : 0);
+    if (item >= a.items) return;                       // only in the last CTA of the WPC == 1 form
+    const int ii = (int)(item % a.ni);
+    const Item it = decode_item(a.t, item / a.ni);
+    const int i = a.i0 + ii;
+    const int L = it.L;
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], it.base);
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + it.base;
+    const float* __restrict__ m32 = a.m32 + it.base;
+    const uint32_t* __restrict__ mbits = a.Bbar + it.base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + it.base / 32;
+    float* sptr = a.s + (int64_t)i * a.Cp + it.c;
+    const float s_old = *sptr;
+    const float Sbar = M32 ? 0.0f : a.Sbar[it.c];
+    const int full = L / kGroup;                  // groups with all 128 elements present
+    const int ngroups = (L + kGroup - 1) / kGroup;
+    double acc = 0.0;
+
+    int g0 = (WPC == 1) ? 0 : warp;
+    // fast path: U groups per warp per iteration, all loads issued before any use
+    for (; g0 + WPC * (U - 1) < full; g0 += WPC * U) {
+        float4 gv[U], zv[U], mv[U];
+        uint32_t mw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int grp = g0 + WPC * u;
+            const int k = grp * kGroup + lane * 4;
+            gv[u] = Grad<GT>::ld4(g, k);
+            zv[u] = ld_stream4(z + k);
+            if (M32) mv[u] = *reinterpret_cast<const float4*>(m32 + k);
+            else     mw[u] = mbits[grp * 4 + (lane >> 3)];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            worker_group<M32, false>(a.beta1, a.omb1, z, obits, g0 + WPC * u, lane, L, s_old, Sbar,
+                                     gv[u], zv[u], M32 ? mv[u] : make_float4(0, 0, 0, 0), M32 ? 0u : mw[u], acc, a.t.l1 != 0, a.send_gradient != 0);
+    }
+    // remainder: one group at a time, bounds-checked
+    for (; g0 < ngroups; g0 += WPC) {
+        const int k = g0 * kGroup + lane * 4;
+        const float4 gv = ld_grad4_checked<GT>(g, k, L);
+        const float4 zv = ld4_checked(z, k, L, true);
+        float4 mv = make_float4(0, 0, 0, 0);
+        uint32_t mw = 0;
+        if (M32) mv = ld4_checked(m32, k, L, false);
+        else if (k < L) mw = mbits[g0 * 4 + (lane >> 3)];
+        worker_group<M32, true>(a.beta1, a.omb1, z, obits, g0, lane, L, s_old, Sbar, gv, zv, mv, mw, acc, a.t.l1 != 0, a.send_gradient != 0);
+    }
+
+    const double total = team_sum<WPC>(acc, red);
+    if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
+        if (a.t.P == 1) *sptr = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);    // ||z||_2 / sqrt(L)
+        else a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p] = total;
+    }
+}
+
+// Worker side, fine-tiled form (steady state, chunk a multiple of kFineSub): one CTA per
+// (worker, 4096-element tile), every load of the tile issued before the first use.  Short-lived
+// CTAs that each touch 16 KiB of every stream once keep DRAM pages and the memory pipeline busier
+// than long-running warps that each follow their own stream.
+// Warp w owns the tile's groups 4w..4w+3 (kFineSub = 512 consecutive elements, all of one chunk),
+// so its 16 momentum words are one 64-byte load handed round by shuffles, its 16 new sign words
+// one 64-byte store, and its binary64 sum of squares one slot of a partial-sum array that
+// k_finalize_fine adds up per chunk in element order: the kernel has no barrier at all.
+// Launch order: runs of `run` consecutive tiles of one worker, then the same tiles of the next
+// worker: every stream is read in long sequential pieces (measured: the longer the better for
+// DRAM), while the momentum bits of a run (run * 512 bytes) stay in L2 for the other workers.
+
+constexpr int kFineTile = 4096;           // 256 threads x 4 x (4 floats)
+constexpr int kFineU = kFineTile / (kThreads * 4);
+constexpr int kFineSub = kFineTile / kWarps;      // elements per warp = per partial sum
+constexpr int kFineRunDefault = 4096;
+
+struct WorkerFineArgs {
+    float* z; int64_t dz;
+    uint32_t* B; int64_t Wp;
+    const float* s; int64_t Cp;       // the scales of the previous step (read only here)
+    double* partial; int64_t Pp;      // ni rows of tiles * kWarps partial sums, row stride Pp
+    const uint32_t* Bbar; const float* Sbar;
+    int64_t d, chunk, tiles;
+    int i0, ni, run;
+    float beta1, omb1;
+};
+
+template <int GT, bool SENDG>          // SENDG: the gradient-compressing variant (no momentum is read)
+__global__ void __launch_bounds__(kThreads, 4)
+k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t per_stretch = (int64_t)a.ni * a.run;
+    const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
+    const int rem = (int)((int64_t)blockIdx.x - stretch * per_stretch);
+    const int ii = rem / a.run;
+    const int64_t t = stretch * a.run + (rem - ii * a.run);
+    if (t >= a.tiles) return;                                  // whole CTA: the last stretch may be short
+    const int i = a.i0 + ii;
+    const int64_t base = t * kFineTile + (int64_t)warp * kFineSub;     // this warp's 512 elements
+    double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + t * kWarps + warp;
+    const int64_t left = a.d - base;
+    if (left <= 0) {                                           // past the end of the vector
+        if (lane == 0) *slot = 0.0;
+        return;
+    }
+    const int L = (int)(left < kFineSub ? left : kFineSub);
+    const int64_t c = base / a.chunk;
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
+    const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
+    const float s_old = a.s[(int64_t)i * a.Cp + c];
+    const float Sbar = a.Sbar[c];
+    double acc = 0.0;
+    if (L == kFineSub) {
+        float4 gv[kFineU], zv[kFineU];
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
+            zv[u] = ld_stream4(z + u * kGroup + lane * 4);
+        }
+        const uint32_t mine = (!SENDG && lane < 4 * kFineU) ? mbits[lane] : 0u;
+        uint32_t outw = 0;
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
+            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+            const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
+            float zn[4];
+            uint32_t nibble = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
+                const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
+                zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
+                const double zd = (double)zn[e];
+                acc = fma(zd, zd, acc);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
+            st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+            const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
+            if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
+        }
+        if (lane < 4 * kFineU) __stcs(obits + lane, outw);
+    } else {
+        const int ngroups = (L + kGroup - 1) / kGroup;
+        for (int grp = 0; grp < ngroups; ++grp) {
+            const int k = grp * kGroup + lane * 4;
+            const float4 gv = ld_grad4_checked<GT>(g, k, L);
+            const float4 zv = ld4_checked(z, k, L, true);
+            const uint32_t mw = (!SENDG && k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
+            worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
+                                      make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
+        }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) *slot = acc;
+}
+
+// Scales from the fine form's partial sums (one per 512 elements): one warp per (row, chunk) adds
+// the chunk's slots in a fixed order (lane l takes slots l, l + 32, ..., then the shuffle tree)
+// and takes sqrt(sum / L).
+__global__ void __launch_bounds__(kThreads)
+k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
+                int rows, int64_t C, int64_t d, int64_t chunk)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t idx = (int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (idx >= (int64_t)rows * C) return;                        // whole warps
+    const int r = (int)(idx / C);
+    const int64_t c = idx % C;
+    const int64_t cbeg = c * chunk;
+    const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
+    const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
+    double total = 0.0;
+    for (int64_t q = q0 + lane; q < q1; q += 32) total += partial[(int64_t)r * Pp + q];
+    total = warp_sum(total);
+    if (lane == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+}
+
+// Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).
+__global__ void k_finalize_scales(const double* __restrict__ partial, float* __restrict__ scales,
+                                  int rows, int64_t C, int64_t Cp, Tiling t)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)rows * C) return;
+    const int r = (int)(idx / C);
+    const int64_t c = idx % C;
+    const int64_t cbeg = c * t.chunk;
+    const int64_t Lc = (t.d - cbeg < t.chunk) ? t.d - cbeg : t.chunk;
+    double total = 0.0;
+    for (int p = 0; p < t.P; ++p) total += partial[(int64_t)r * t.Pp + c * t.P + p];
+    scales[(int64_t)r * Cp + c] = scale_from_sum(total, (double)Lc, t.l1 != 0);
+}
+
+}  // namespace

@@ -167,7 +167,8 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
  * and a CUDA stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
  * The caller keeps ownership and must keep both alive until apms_destroy().  If never
  * called, the context allocates its own workspace with cudaMalloc on first use and works
- * on the default stream.  Must be called before apms_set_params(). */
+ * on the default stream; workspace_dev == NULL with bytes == 0 sets the stream alone and
+ * leaves the workspace to the library.  Must be called before apms_set_params(). */
 apms_status apms_bind(apms_ctx* ctx, void* workspace_dev, size_t bytes, void* cuda_stream);
 
 /* x <- x0, m <- 0, v <- 0, t <- 0 (Algorithm 1 initialisation); phase becomes WARMUP.
@@ -245,6 +246,42 @@ apms_status apms_server_phase(apms_ctx* ctx, const uint32_t* bits_rows_dev, int6
                               const float* scale_rows_dev, int64_t row_scales, int rows,
                               int64_t chunk_begin, int64_t chunk_end);
 apms_status apms_apply_phase(apms_ctx* ctx);
+
+/* The same step with the exchanges done by the GPUs themselves, for processes on one node whose
+ * GPUs reach each other's memory (NVLink / NVSwitch peers): every process maps its peers' workspaces
+ * (apms_ipc_export / apms_ipc_open), and
+ *
+ *   exchange 1 is the server kernel reading: apms_server_phase_rows takes one pair of device
+ *     pointers per sender - bits_rows[j] the address of row j's sign word of the first element of
+ *     chunk chunk_begin (inside a message buffer whose word 0 is 16-byte aligned, as the
+ *     library's are), scale_rows[j] the address of its scale of chunk chunk_begin - and loads
+ *     the rows where they lie, this GPU's memory or a mapped peer's.  A
+ *     peer worker's row is (mapped base of its process) + apms_message_offsets(worker) + the range's
+ *     offset; contexts created with the same d, n, chunk have the same offsets.  Both arrays are
+ *     HOST arrays of `rows` pointers, read during the call.  Rows are averaged in array order.
+ *   exchange 2 is a store: apms_put_server_range copies chunks [chunk_begin, chunk_end) of this
+ *     context's server message into a peer's server-message buffers (dst_* = the START of the
+ *     peer's sign-word / scale buffers, i.e. mapped base + apms_message_offsets(-1)), on the
+ *     context's stream.
+ *
+ * The caller orders the phases across processes (the library has no device-side waits on other
+ * GPUs): all workers' messages must be complete before any server phase reads them, and all
+ * server ranges stored before any apply phase - a stream synchronisation and a host barrier at
+ * each of the two points.  The paper's description of the exchanges: Section 3.3 steps 3 and 5,
+ * Figure 1.  apms_ipc_export: writes APMS_IPC_HANDLE_BYTES bytes naming this context's workspace,
+ * which must be the library's own allocation (no apms_bind); APMS_ERR_BAD_STATE otherwise.
+ * apms_ipc_open: maps the workspace named by a handle made in ANOTHER process and returns its base
+ * address in this process; apms_ipc_close unmaps it.  These two take no context; on failure
+ * apms_last_error(NULL) describes why. */
+#define APMS_IPC_HANDLE_BYTES 64
+apms_status apms_server_phase_rows(apms_ctx* ctx, const uint32_t* const* bits_rows, const float* const* scale_rows,
+                                   int rows, int64_t chunk_begin, int64_t chunk_end);
+apms_status apms_put_server_range(apms_ctx* ctx, uint32_t* dst_bits_dev, float* dst_scales_dev,
+                                  int64_t chunk_begin, int64_t chunk_end);
+apms_status apms_message_offsets(apms_ctx* ctx, int worker, size_t* bits_offset, size_t* scales_offset);
+apms_status apms_ipc_export(apms_ctx* ctx, void* handle_out);
+apms_status apms_ipc_open(const void* handle, void** base_dev);
+apms_status apms_ipc_close(void* base_dev);
 
 /* Copy x (d floats) to dst: device memory if dst_is_device != 0 (stream-ordered), else
  * host memory (synchronises the stream). */
@@ -345,7 +382,7 @@ apms_status apms_selftest_wait_report(apms_ctx* ctx, int leave_reported);
 int64_t     apms_launch_count(const apms_ctx* ctx);
 
 /* Message of the last failure on this context (ctx == NULL: of the last failed
- * apms_create on this thread).  Never NULL. */
+ * apms_create, apms_ipc_open or apms_ipc_close on this thread).  Never NULL. */
 const char* apms_last_error(const apms_ctx* ctx);
 
 /* Free the context (and its workspace if it allocated one).  NULL is ignored. */

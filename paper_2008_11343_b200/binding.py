@@ -53,6 +53,12 @@ SIGNATURES = {
     "apms_get_message": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
     "apms_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64]),
     "apms_apply_phase": (C.c_int, [C.c_void_p]),
+    "apms_server_phase_rows": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64]),
+    "apms_put_server_range": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64]),
+    "apms_message_offsets": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "apms_ipc_export": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "apms_ipc_open": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p)]),
+    "apms_ipc_close": (C.c_int, [C.c_void_p]),
     "apms_get_params": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
     "apms_get_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "apms_get_state_slice": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
@@ -187,6 +193,48 @@ def apms_apply_phase(h):
     _check(h, load().apms_apply_phase(h))
 
 
+def apms_server_phase_rows(h, bits_row_ptrs: Sequence[int], scale_row_ptrs: Sequence[int], chunk_begin: int, chunk_end: int):
+    rows = len(bits_row_ptrs)
+    assert len(scale_row_ptrs) == rows
+    barr = (C.c_void_p * rows)(*bits_row_ptrs)
+    sarr = (C.c_void_p * rows)(*scale_row_ptrs)
+    _check(h, load().apms_server_phase_rows(h, barr, sarr, rows, chunk_begin, chunk_end))
+
+
+def apms_put_server_range(h, dst_bits_ptr: int, dst_scales_ptr: int, chunk_begin: int, chunk_end: int):
+    _check(h, load().apms_put_server_range(h, dst_bits_ptr, dst_scales_ptr, chunk_begin, chunk_end))
+
+
+def apms_message_offsets(h, worker: int):
+    b, s = C.c_size_t(), C.c_size_t()
+    _check(h, load().apms_message_offsets(h, worker, C.byref(b), C.byref(s)))
+    return int(b.value), int(s.value)
+
+
+IPC_HANDLE_BYTES = 64
+
+
+def apms_ipc_export(h) -> bytes:
+    buf = C.create_string_buffer(IPC_HANDLE_BYTES)
+    _check(h, load().apms_ipc_export(h, buf))
+    return buf.raw
+
+
+def apms_ipc_open(handle: bytes) -> int:
+    assert len(handle) == IPC_HANDLE_BYTES
+    base = C.c_void_p()
+    st = load().apms_ipc_open(C.c_char_p(handle), C.byref(base))
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(None).decode())
+    return int(base.value)
+
+
+def apms_ipc_close(base: int):
+    st = load().apms_ipc_close(C.c_void_p(base))
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(None).decode())
+
+
 def apms_get_params(h, dst_ptr: int, dst_is_device: bool):
     _check(h, load().apms_get_params(h, dst_ptr, int(dst_is_device)))
 
@@ -305,10 +353,12 @@ def apms_compress_noalloc(z_ptr: int, d: int, chunk: int, bits_ptr: int, scales_
 # --- convenience wrapper: handle + torch workspace + stream ---------------------------------
 
 class Context:
-    """An apms context whose workspace is a torch CUDA tensor and whose stream is torch's."""
+    """An apms context whose workspace is a torch CUDA tensor and whose stream is torch's.
+    With library_workspace=True the library allocates the workspace itself (cudaMalloc): the form that
+    apms_ipc_export needs, without the tensor views of message()."""
 
     def __init__(self, d: int, n: int, beta1: float, beta2: float, eps: float, lr: float, chunk: int,
-                 device: str = "cuda:0", stream=None):
+                 device: str = "cuda:0", stream=None, library_workspace: bool = False):
         import torch
 
         if not torch.cuda.is_available():
@@ -320,9 +370,13 @@ class Context:
         torch.cuda.set_device(self.device)
         self._h = apms_create(d, n, beta1, beta2, eps, lr, chunk)
         nbytes = apms_workspace_bytes(d, n, chunk)
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
-        apms_bind(self._h, self.workspace.data_ptr(), nbytes, self.stream.cuda_stream)
+        if library_workspace:
+            self.workspace = None
+            apms_bind(self._h, None, 0, self.stream.cuda_stream)
+        else:
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            apms_bind(self._h, self.workspace.data_ptr(), nbytes, self.stream.cuda_stream)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -425,6 +479,8 @@ class Context:
         workspace (-1: the server's message).  No copy: the library writes these buffers."""
         import torch
 
+        if self.workspace is None:
+            raise RuntimeError("message() views need the torch workspace; use message_ptrs() with a library workspace")
         bits_ptr, scales_ptr = apms_get_message(self._h, worker)
         base = self.workspace.data_ptr()
         b0, s0 = bits_ptr - base, scales_ptr - base
@@ -440,6 +496,27 @@ class Context:
 
     def apply_phase(self):
         apms_apply_phase(self._h)
+
+    def message_ptrs(self, worker: int):
+        """Device addresses (sign words, scales) of worker `worker`'s message (-1: the server's)."""
+        return apms_get_message(self._h, worker)
+
+    def message_offsets(self, worker: int):
+        """Byte offsets of that message inside the workspace (equal for contexts of equal shape)."""
+        return apms_message_offsets(self._h, worker)
+
+    def server_phase_rows(self, bits_row_ptrs, scale_row_ptrs, chunk_begin: int, chunk_end: int):
+        """One device address per sender and array: where its sign words / scales of chunk_begin lie."""
+        apms_server_phase_rows(self._h, bits_row_ptrs, scale_row_ptrs, chunk_begin, chunk_end)
+
+    def put_server_range(self, dst_bits_ptr: int, dst_scales_ptr: int, chunk_begin: int, chunk_end: int):
+        apms_put_server_range(self._h, dst_bits_ptr, dst_scales_ptr, chunk_begin, chunk_end)
+
+    def ipc_export(self) -> bytes:
+        return apms_ipc_export(self._h)
+
+    def synchronize(self):
+        self.stream.synchronize()
 
     def set_schedule(self, schedule: Optional[Schedule]):
         apms_set_schedule(self._h, schedule)

@@ -375,7 +375,22 @@ cudaError_t launch_staged_n(const ServerStagedArgs& sa, unsigned blocks, size_t 
 
 // Where the server finds the workers' messages: `rows` senders, row j holding sign words and scales
 // addressed by ABSOLUTE word / chunk index (a pointer into a shard is shifted back by the caller).
-struct ServerSource { const uint32_t* B; int64_t Wp; const float* s; int64_t Cp; int rows; };
+struct ServerSource {
+    const uint32_t* B[APMS_MAX_WORKERS];
+    const float* s[APMS_MAX_WORKERS];
+    int rows;
+    // rows at a fixed stride from a base
+    static ServerSource strided(const uint32_t* B0, int64_t Wp, const float* s0, int64_t Cp, int rows)
+    {
+        ServerSource src;
+        for (int j = 0; j < APMS_MAX_WORKERS; ++j) {
+            src.B[j] = j < rows ? B0 + (int64_t)j * Wp : nullptr;
+            src.s[j] = j < rows ? s0 + (int64_t)j * Cp : nullptr;
+        }
+        src.rows = rows;
+        return src;
+    }
+};
 
 // Section 3.3 step 4 for chunks [cb, ce).  With may_fuse and a shape that allows it, steps 5-6 for
 // the same chunks run in the same kernel (*applied = true).
@@ -383,7 +398,7 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
 {
     *applied = false;
     ServerArgs a;
-    a.B = src.B; a.Wp = src.Wp; a.s = src.s; a.Cp = src.Cp;
+    for (int j = 0; j < APMS_MAX_WORKERS; ++j) { a.Brow[j] = src.B[j]; a.srow[j] = src.s[j]; }
     a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
     a.partial = c->partial(c->L.n);
     a.t = c->L.t; a.item0 = cb * c->L.t.P; a.items = ce * c->L.t.P; a.n = src.rows; a.nf = (float)src.rows;
@@ -467,7 +482,7 @@ apms_status launch_server_and_apply(apms_ctx* c)
         c->csteps += 1;
         return APMS_OK;
     }
-    const ServerSource own = {c->B(0), c->L.Wp, c->s(0), c->L.Cp, c->L.n};
+    const ServerSource own = ServerSource::strided(c->B(0), c->L.Wp, c->s(0), c->L.Cp, c->L.n);
     bool applied = false;      // steps 5-6 already done by the fused server kernel
     const bool gradient = c->variant == APMS_VARIANT_GRADIENT;      // its apply differs: never fused
     apms_status st = launch_server(c, own, 0, c->L.C, !gradient, &applied);
@@ -548,6 +563,10 @@ apms_status apms_bind(apms_ctx* c, void* workspace_dev, size_t bytes, void* cuda
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "apms_bind must precede apms_set_params");
     if (c->ws) return fail(c, APMS_ERR_BAD_STATE, "a workspace is already attached");
+    if (!workspace_dev && bytes == 0) {                // the stream only: the library allocates the workspace itself
+        c->stream = (cudaStream_t)cuda_stream;
+        return APMS_OK;
+    }
     if (!workspace_dev || ((uintptr_t)workspace_dev & 255u)) return fail(c, APMS_ERR_INVALID_ARG, "workspace must be non-NULL and 256-byte aligned");
     if (bytes < c->L.total) return fail(c, APMS_ERR_OOM, "workspace smaller than apms_workspace_bytes()");
     c->ws = (char*)workspace_dev; c->ws_bytes = bytes; c->owns_ws = false;
@@ -676,11 +695,106 @@ apms_status apms_server_phase(apms_ctx* c, const uint32_t* bits_rows_dev, int64_
         return fail(c, APMS_ERR_INVALID_ARG, "rows too short: row_words must be a multiple of 4 that covers the range's sign words rounded up to 4, row_scales its chunks");
     if (((uintptr_t)bits_rows_dev & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "bits_rows_dev is not 16-byte aligned");
     // kernels index by absolute word / chunk: shift the shard's pointers back to where index 0 would be
-    const ServerSource src = {bits_rows_dev - first_elem / 32, row_words, scale_rows_dev - chunk_begin, row_scales, rows};
+    const ServerSource src = ServerSource::strided(bits_rows_dev - first_elem / 32, row_words, scale_rows_dev - chunk_begin, row_scales, rows);
     bool applied = false;
     apms_status st = launch_server(c, src, chunk_begin, chunk_end, false, &applied);
     if (st == APMS_OK) c->substep = 2;
     return st;
+}
+
+apms_status apms_server_phase_rows(apms_ctx* c, const uint32_t* const* bits_rows, const float* const* scale_rows, int rows,
+                                   int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows needs the COMPRESSED phase");
+    if (c->substep < 1) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows follows apms_worker_phase");
+    if (!bits_rows || !scale_rows) return fail(c, APMS_ERR_INVALID_ARG, "a pointer array is NULL");
+    if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    const int64_t first_elem = chunk_begin * c->L.chunk;
+    ServerSource src;
+    for (int j = 0; j < APMS_MAX_WORKERS; ++j) { src.B[j] = nullptr; src.s[j] = nullptr; }
+    for (int j = 0; j < rows; ++j) {
+        if (!bits_rows[j] || !scale_rows[j]) return fail(c, APMS_ERR_INVALID_ARG, "a message pointer is NULL");
+        // kernels index by absolute word / chunk: shift the row's pointers back to where index 0 would be
+        src.B[j] = bits_rows[j] - first_elem / 32;
+        src.s[j] = scale_rows[j] - chunk_begin;
+        if (((uintptr_t)src.B[j] & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "a sign-word row does not belong to a 16-byte aligned message buffer");
+    }
+    src.rows = rows;
+    bool applied = false;
+    apms_status st = launch_server(c, src, chunk_begin, chunk_end, false, &applied);
+    if (st == APMS_OK) c->substep = 2;
+    return st;
+}
+
+apms_status apms_put_server_range(apms_ctx* c, uint32_t* dst_bits_dev, float* dst_scales_dev, int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase != APMS_PHASE_COMPRESSED || c->substep != 2) return fail(c, APMS_ERR_BAD_STATE, "apms_put_server_range follows the server phase of a phase-wise step");
+    if (!dst_bits_dev || !dst_scales_dev) return fail(c, APMS_ERR_INVALID_ARG, "a destination pointer is NULL");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (chunk_begin == chunk_end) return APMS_OK;
+    const int64_t first_elem = chunk_begin * c->L.chunk;
+    const int64_t last_elem = chunk_end * c->L.chunk < c->L.d ? chunk_end * c->L.chunk : c->L.d;
+    const int64_t w0 = first_elem / 32, w1 = (last_elem + 31) / 32;
+    APMS_CUDA(c, cudaMemcpyAsync(dst_bits_dev + w0, c->Bbar() + w0, (size_t)(w1 - w0) * 4, cudaMemcpyDefault, c->stream));
+    APMS_CUDA(c, cudaMemcpyAsync(dst_scales_dev + chunk_begin, c->Sbar() + chunk_begin, (size_t)(chunk_end - chunk_begin) * 4,
+                                 cudaMemcpyDefault, c->stream));
+    return APMS_OK;
+}
+
+apms_status apms_message_offsets(apms_ctx* c, int worker, size_t* bits_offset, size_t* scales_offset)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (worker < -1 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range (-1 = the server's message)");
+    apms_status st = ensure_workspace(c);
+    if (st != APMS_OK) return st;
+    if (bits_offset) *bits_offset = (size_t)((char*)(worker < 0 ? c->Bbar() : c->B(worker)) - c->ws);
+    if (scales_offset) *scales_offset = (size_t)((char*)(worker < 0 ? c->Sbar() : c->s(worker)) - c->ws);
+    return APMS_OK;
+}
+
+apms_status apms_ipc_export(apms_ctx* c, void* handle_out)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!handle_out) return fail(c, APMS_ERR_INVALID_ARG, "handle_out is NULL");
+    apms_status st = ensure_workspace(c);
+    if (st != APMS_OK) return st;
+    if (!c->owns_ws) return fail(c, APMS_ERR_BAD_STATE, "only a workspace the library allocated itself can be exported (do not call apms_bind)");
+    static_assert(sizeof(cudaIpcMemHandle_t) == APMS_IPC_HANDLE_BYTES, "handle size");
+    cudaIpcMemHandle_t h;
+    APMS_CUDA(c, cudaIpcGetMemHandle(&h, c->ws));
+    memcpy(handle_out, &h, sizeof h);
+    return APMS_OK;
+}
+
+apms_status apms_ipc_open(const void* handle, void** base_dev)
+{
+    if (!handle || !base_dev) return APMS_ERR_INVALID_ARG;
+    cudaIpcMemHandle_t h;
+    memcpy(&h, handle, sizeof h);
+    void* p = nullptr;
+    const cudaError_t e = cudaIpcOpenMemHandle(&p, h, cudaIpcMemLazyEnablePeerAccess);
+    if (e != cudaSuccess) {
+        snprintf(g_create_error, sizeof g_create_error, "cudaIpcOpenMemHandle failed: %s", cudaGetErrorString(e));
+        (void)cudaGetLastError();
+        return APMS_ERR_CUDA;
+    }
+    *base_dev = p;
+    return APMS_OK;
+}
+
+apms_status apms_ipc_close(void* base_dev)
+{
+    if (!base_dev) return APMS_ERR_INVALID_ARG;
+    const cudaError_t e = cudaIpcCloseMemHandle(base_dev);
+    if (e != cudaSuccess) {
+        snprintf(g_create_error, sizeof g_create_error, "cudaIpcCloseMemHandle failed: %s", cudaGetErrorString(e));
+        (void)cudaGetLastError();
+        return APMS_ERR_CUDA;
+    }
+    return APMS_OK;
 }
 
 apms_status apms_apply_phase(apms_ctx* c)

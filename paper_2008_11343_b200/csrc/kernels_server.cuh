@@ -9,9 +9,12 @@ namespace {
 // Server side: average the n decompressed messages, add the server error, recompress
 // (Section 3.3 step 4).
 
+// The messages the server averages: row j (one sender) is addressed by ABSOLUTE word / chunk index through
+// its own pair of pointers, so that the rows may lie anywhere - this context's workers, a buffer of received
+// rows, or the mapped workspaces of other processes' GPUs (plain and bulk loads only).
 struct ServerArgs {
-    const uint32_t* B; int64_t Wp;
-    const float* s; int64_t Cp;
+    const uint32_t* Brow[APMS_MAX_WORKERS];
+    const float* srow[APMS_MAX_WORKERS];
     float* zbar; uint32_t* Bbar; float* Sbar;
     double* partial;
     Tiling t;
@@ -23,7 +26,7 @@ struct ServerArgs {
 // the running sums (sequential in worker order, as the average is defined) are updated.
 // +-s_i is formed by moving the complemented sign bit onto s_i's sign: no selects, no branches.
 template <int U, bool CHECKED>
-__device__ __forceinline__ void server_groups(const ServerArgs& a, const float* s_sh, const uint32_t* __restrict__ wb,
+__device__ __forceinline__ void server_groups(const ServerArgs& a, const float* s_sh, int64_t wofs,
                                               float* __restrict__ zb, uint32_t* __restrict__ ob,
                                               int g0, int gstride, int lane, int L, float S_old, double& acc)
 {
@@ -46,7 +49,7 @@ __device__ __forceinline__ void server_groups(const ServerArgs& a, const float* 
         uint32_t w[U];
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            w[u] = live[u] ? wb[(int64_t)i * a.Wp + (g0 + gstride * u) * 4 + wl] : 0u;
+            w[u] = live[u] ? a.Brow[i][wofs + (g0 + gstride * u) * 4 + wl] : 0u;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint32_t neg = ~w[u] >> sh;            // bit e set: element e of this lane is negative
@@ -95,10 +98,10 @@ k_server(const ServerArgs a)
     const int L = it.L;
     float* s_sh = s_all[team];
     const int tid_in_team = (WPC == 1) ? lane : (int)threadIdx.x;
-    for (int i = tid_in_team; i < a.n; i += WPC * 32) s_sh[i] = a.s[(int64_t)i * a.Cp + it.c];
+    for (int i = tid_in_team; i < a.n; i += WPC * 32) s_sh[i] = a.srow[i][it.c];
     const float S_old = a.Sbar[it.c];
     if (WPC == 1) __syncwarp(); else __syncthreads();
-    const uint32_t* __restrict__ wb = a.B + it.base / 32;
+    const int64_t wofs = it.base / 32;
     float* __restrict__ zb = a.zbar + it.base;
     uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
     const int full = L / kGroup;
@@ -111,9 +114,9 @@ k_server(const ServerArgs a)
     const int g_end = (g0 + per_warp < ngroups) ? g0 + per_warp : ngroups;
     const int g_full = (full < g_end) ? full : g_end;
     for (; g0 + (U - 1) < g_full; g0 += U)
-        server_groups<U, false>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+        server_groups<U, false>(a, s_sh, wofs, zb, ob, g0, 1, lane, L, S_old, acc);
     for (; g0 < g_end; ++g0)
-        server_groups<1, true>(a, s_sh, wb, zb, ob, g0, 1, lane, L, S_old, acc);
+        server_groups<1, true>(a, s_sh, wofs, zb, ob, g0, 1, lane, L, S_old, acc);
     const double total = team_sum<WPC>(acc, red);
     if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
         if (a.t.P == 1) a.Sbar[it.c] = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);
@@ -281,7 +284,7 @@ k_server_staged(const ServerStagedArgs sa)
                 const int nslabs = (L + kSlab - 1) / kSlab;
                 const int njobs = FUSED ? 2 * nslabs : nslabs;
                 const float* __restrict__ zb_g = a.zbar + it.base;
-                const uint32_t* __restrict__ wb_g = a.B + it.base / 32;
+                const int64_t wofs = it.base / 32;
                 for (int r = 0; r < njobs; ++r, ++q) {
                     const int st = q % kStages;
                     if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; stop = true; break; }
@@ -296,7 +299,7 @@ k_server_staged(const ServerStagedArgs sa)
                         bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
                         uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
                         for (int i = 0; i < n; ++i)
-                            bulk_load(rows + i * kSlabWords, wb_g + (int64_t)i * a.Wp + (size_t)j * kSlabWords, wbytes, &full[st]);
+                            bulk_load(rows + i * kSlabWords, a.Brow[i] + wofs + (size_t)j * kSlabWords, wbytes, &full[st]);
                     } else {
                         mbar_arrive_expect_tx(&full[st], 2 * zbytes);
                         bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
@@ -324,7 +327,7 @@ k_server_staged(const ServerStagedArgs sa)
             const int nslabs = (L + kSlab - 1) / kSlab;
             uint32_t* negs = neg_s[w & 1];
             for (int i = threadIdx.x; i < n; i += kThreads)
-                negs[i] = __float_as_uint(a.s[(int64_t)i * a.Cp + it.c]) | 0x80000000u;
+                negs[i] = __float_as_uint(a.srow[i][it.c]) | 0x80000000u;
             const float S_old = a.Sbar[it.c];
             consumer_barrier();                        // -s_i in place; everybody is done with the previous chunk
             if (failed) break;

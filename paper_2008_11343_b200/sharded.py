@@ -18,6 +18,13 @@ n_local workers each give bit for bit the result of one context with P * n_local
 message(i) -> (sign-word tensor, scale tensor) views (i = -1: the server's message),
 server_phase(bits_rows, scale_rows, chunk_begin, chunk_end) and apply_phase(): a
 `binding.Context` on a GPU, or a CPU stand-in in the tests of the exchange logic.
+
+`PeerShardedStep` is the one-node form in which the GPUs move the messages themselves: every process
+maps its peers' workspaces once (CUDA IPC), the server kernel then loads its rows straight from the
+workers' message buffers wherever they lie (exchange 1 costs no copy and no staging buffer: the
+transfer is the kernel's own loads over NVLink), and each process stores its range of the server
+message into every peer's buffer (exchange 2).  `torch.distributed` carries only the handles and
+two host barriers per step.
 """
 from __future__ import annotations
 
@@ -137,3 +144,74 @@ class ShardedStep:
         ex1 = sum(4 * n * (self.row_words[k] + self.row_scales[k]) for k in range(self.world) if k != me)
         ex2 = (self.world - 1) * 4 * (self.row_words[me] + self.row_scales[me])
         return ex1 + ex2
+
+
+class PeerShardedStep:
+    """Section 3.3 steps 1-6 across processes of one node, the exchanges done by peer loads and stores.
+
+    `backend`: a `binding.Context` made with library_workspace=True (its workspace must be exportable);
+    `peers`: what opens and closes a handle - by default the binding's apms_ipc_open / apms_ipc_close.
+    The two barriers are host barriers after a stream synchronisation: no kernel waits on another GPU.
+    """
+
+    def __init__(self, backend, group=None, peers=None):
+        import torch.distributed as dist
+
+        self.b, self.dist, self.group = backend, dist, group
+        self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
+        if backend.C < self.world:
+            raise ValueError(f"{backend.C} chunks cannot be served by {self.world} processes")
+        if peers is None:
+            from . import binding as peers
+        self._peers = peers
+        self.ranges = chunk_ranges(backend.C, self.world)
+        n = backend.n
+        self.off = {i: backend.message_offsets(i) for i in range(-1, n)}
+        mine = (backend.ipc_export(), (backend.d, n, backend.chunk), tuple(sorted(self.off.items())))
+        everyone = [None] * self.world
+        dist.all_gather_object(everyone, mine, group=group)
+        for r, (_, shape, off) in enumerate(everyone):
+            if shape != mine[1] or off != mine[2]:
+                raise ValueError(f"process {r} holds a context of another shape: {shape} against {mine[1]}")
+        own_base = backend.message_ptrs(0)[0] - self.off[0][0]
+        self.base = [own_base if r == self.rank else peers.apms_ipc_open(h) for r, (h, _, _) in enumerate(everyone)]
+        dist.barrier(group=group)
+
+    def row_pointers(self):
+        """(sign-word addresses, scale addresses) of all world * n senders' rows for this process's chunk range,
+        in global worker order."""
+        cb, ce = self.ranges[self.rank]
+        w0, _ = word_range(cb, ce, self.b.chunk, self.b.d)
+        bits = [self.base[r] + self.off[i][0] + 4 * w0 for r in range(self.world) for i in range(self.b.n)]
+        scales = [self.base[r] + self.off[i][1] + 4 * cb for r in range(self.world) for i in range(self.b.n)]
+        return bits, scales
+
+    def step(self, grads: Sequence) -> None:
+        b, me = self.b, self.rank
+        b.worker_phase(grads)                                                   # steps 1-2
+        b.synchronize()
+        self.dist.barrier(group=self.group)                                     # every worker's message is complete
+        cb, ce = self.ranges[me]
+        bits, scales = self.row_pointers()
+        b.server_phase_rows(bits, scales, cb, ce)                               # steps 3-4: the kernel loads the rows
+        for r in range(self.world):                                             # step 5: my range to every peer
+            if r != me:
+                b.put_server_range(self.base[r] + self.off[-1][0], self.base[r] + self.off[-1][1], cb, ce)
+        b.synchronize()
+        self.dist.barrier(group=self.group)                                     # every range is stored everywhere
+        b.apply_phase()                                                         # steps 5-6
+
+    def close(self):
+        self.dist.barrier(group=self.group)                                     # nobody reads a mapping that goes away
+        for r, base in enumerate(self.base):
+            if r != self.rank and base is not None:
+                self._peers.apms_ipc_close(base)
+        self.base = []
+
+    def wire_bytes_per_step(self) -> int:
+        """Bytes that cross between GPUs per step because of this process: the rows it loads from peers and the
+        range it stores to them."""
+        cb, ce = self.ranges[self.rank]
+        w0, w1 = word_range(cb, ce, self.b.chunk, self.b.d)
+        per_row = 4 * (w1 - w0) + 4 * (ce - cb)
+        return (self.world - 1) * self.b.n * per_row + (self.world - 1) * per_row

@@ -294,6 +294,24 @@ def test_topk_threshold_jumps():
         _topk_compare(ctx, orc, w, step)
 
 
+@pytest.mark.parametrize("frac", [0.01, 0.1])
+def test_topk_long_free_run(frac):
+    """60 free-running top-k steps: the predicted-threshold routes run on thresholds that drift as the errors
+    build up; masks, errors, momentum and model stay bit-identical."""
+    w = tiny(6 * 8192 + 500, 3, 8192, cfg_id=183)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, frac)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(1, 61):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        if step % 10 == 0:
+            _topk_compare(ctx, orc, w, step)
+
+
 # ------------------------------------------------------------------ phase driver and error monitor
 
 def test_scheduled_steps_follow_algorithm_1():
@@ -419,6 +437,15 @@ def test_config0_free_running_10_steps():
     bit-exact (ties aside), scales / errors / parameters within 1e-5 after 10 steps."""
     w = wl.config(0)
     _, _, reports = H.run_both(w, check_every_step=False)
+    assert reports[-1]["server_tie_elems"] == 0
+
+
+def test_long_free_run_does_not_drift():
+    """150 compression-phase steps without any correction from the oracle, on a set that spans several chunk
+    shapes' kernels (fine worker + fused staged server): the state stays bit-identical, i.e. nothing in the
+    stored-z form, the 1-bit momentum or the error feedback accumulates a difference."""
+    w = tiny(24 * 4096 + 1000, 4, 4096, cfg_id=150)
+    ctx, orc, reports = H.run_both(w, warmup=3, compressed=150, check_every_step=False, exact=True)
     assert reports[-1]["server_tie_elems"] == 0
 
 

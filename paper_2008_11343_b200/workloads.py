@@ -100,7 +100,7 @@ def _log_uniform_partition(total: int, parts: int, lo: int, hi: int, cfg_id: int
 
 
 def config(idx: int) -> Workload:
-    """The benchmark configurations, indexed as in the build's baseline description.
+    """The benchmark configurations.
 
     0: one flat tensor, d = 2^20, n = 4, chunk = 4096 (fits in L2; parity-sized).
     1: d = 2^24 in 64 tensors of log-uniform size, 20 % zero gradients, n = 8.

@@ -114,7 +114,8 @@ struct apms_ctx {
     int substep;             // phase-wise step: 0 = between steps, 1 = worker phase done, 2 = a server phase done
     apms_schedule sched; bool has_sched;
     apms_phase phase;
-    bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar)
+    bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar; top-k: in zbar under the mask Bbar)
+    bool v_checked, v_plain; // top-k: has v been looked at since it last changed, and is every entry >= 0 (not NaN)
     char* ws; size_t ws_bytes; bool owns_ws;
     cudaStream_t stream;
     cudaStream_t copy_stream; cudaEvent_t ev_copied[2], ev_used[2]; bool host_path_ready;
@@ -300,13 +301,15 @@ apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0
 {
     TopkWorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp; a.m32 = c->m();
+    a.zbar = c->zbar(); a.Bbar = c->Bbar();
     a.thr = c->s(0); a.Cp = c->L.Cp;
     a.d = c->L.d; a.chunk = c->L.chunk; a.C = c->L.C; a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1; a.frac = c->topk_frac;
     const int64_t blocks = c->L.C * ni;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
     Timed t(c, APMS_KERNEL_WORKER);
-    APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+    if (c->m_is_fp32) APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+    else              APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
     return launch_check(c, "k_topk_worker");
 }
 
@@ -465,10 +468,50 @@ apms_status launch_apply(apms_ctx* c)
     return launch_check(c, "k_apply");
 }
 
+int grid_for(const apms_ctx* c, int64_t items, int per_sm);
+
+// Top-k: may the server leave the elements it does not keep alone?  Their momentum is +0, and
+// x - (lr * 0) / (sqrt(v) + eps) returns x itself iff lr is not negative (nor -0), eps > 0 and v is neither
+// negative nor NaN.  v is looked at once after it last changed (one pass and a synchronisation).
+apms_status topk_sparse_update_allowed(apms_ctx* c, bool* allowed)
+{
+    *allowed = false;
+    if (!(c->eps > 0.0f) || signbit(c->lr)) return APMS_OK;
+    if (!c->v_checked) {
+        int* flag = c->status() + 1;
+        int host_flag = 0;
+        APMS_CUDA(c, cudaMemsetAsync(flag, 0, sizeof(int), c->stream));
+        k_any_negative_or_nan<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->v(), c->L.d, flag);
+        apms_status st = launch_check(c, "k_any_negative_or_nan");
+        if (st != APMS_OK) return st;
+        APMS_CUDA(c, cudaMemcpyAsync(&host_flag, flag, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+        APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+        c->v_plain = host_flag == 0;
+        c->v_checked = true;
+    }
+    *allowed = c->v_plain;
+    return APMS_OK;
+}
+
+// The momentum, spelled out in binary32 into out[0..count) from where it lives when !m_is_fp32.
+apms_status launch_materialise_momentum(apms_ctx* c, float* out, int64_t first, int64_t count)
+{
+    const int grid = grid_for(c, count, 8);
+    if (c->compressor == APMS_COMPRESSOR_TOPK)
+        k_materialise_momentum_topk<<<grid, kThreads, 0, c->stream>>>(c->zbar(), c->Bbar(), out, first, count);
+    else
+        k_materialise_momentum<<<grid, kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), out, first, count, c->L.chunk);
+    return launch_check(c, "k_materialise_momentum");
+}
+
 apms_status launch_server_and_apply(apms_ctx* c)
 {
     if (c->compressor == APMS_COMPRESSOR_TOPK) {       // one kernel: sparse average, recompression, momentum, model update
+        bool sparse = false;
+        apms_status sst = topk_sparse_update_allowed(c, &sparse);
+        if (sst != APMS_OK) return sst;
         TopkServerArgs a;
+        a.sparse = sparse ? 1 : 0;
         a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp;
         a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n; a.lr = c->lr; a.eps = c->eps;
@@ -478,7 +521,7 @@ apms_status launch_server_and_apply(apms_ctx* c)
         k_topk_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
         apms_status st = launch_check(c, "k_topk_server");
         if (st != APMS_OK) return st;
-        c->m_is_fp32 = true;
+        c->m_is_fp32 = !sparse;    // sparse update: the momentum stays implicit in (zbar, Bbar)
         c->csteps += 1;
         return APMS_OK;
     }
@@ -544,7 +587,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     apms_ctx* c = new (std::nothrow) apms_ctx();
     if (!c) { snprintf(g_create_error, sizeof g_create_error, "host allocation failed"); return APMS_ERR_OOM; }
     c->L = L; c->beta1 = beta1; c->beta2 = beta2; c->eps = eps; c->lr = lr;
-    c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true;
+    c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true; c->v_checked = false; c->v_plain = false;
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
@@ -632,6 +675,7 @@ apms_status apms_freeze_v(apms_ctx* c)
     APMS_CUDA(c, cudaMemsetAsync(c->ws + c->L.off_zbar, 0, c->L.off_part - c->L.off_zbar, c->stream));
     c->phase = APMS_PHASE_COMPRESSED;
     c->m_is_fp32 = true;
+    c->v_checked = false;
     return APMS_OK;
 }
 
@@ -891,7 +935,8 @@ apms_status apms_get_state_slice(apms_ctx* c, apms_state_id which, int worker, i
     case APMS_STATE_M:
         if (c->m_is_fp32) src = (const char*)c->m();
         else {
-            k_materialise_momentum<<<grid, kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->stage(0), first, count, c->L.chunk);
+            apms_status mst = launch_materialise_momentum(c, c->stage(0), first, count);
+            if (mst != APMS_OK) return mst;
             staged = true;
         }
         break;
@@ -940,7 +985,7 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
     float* dst = nullptr;
     switch (which) {
     case APMS_STATE_X: dst = c->x(); break;
-    case APMS_STATE_V: dst = c->v(); break;
+    case APMS_STATE_V: dst = c->v(); c->v_checked = false; break;
     case APMS_STATE_M: dst = c->m(); c->m_is_fp32 = true; break;
     case APMS_STATE_WORKER_ERR:
         if (worker < 0 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range");
@@ -953,9 +998,9 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
         break;
     case APMS_STATE_SERVER_ERR:
         if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
-        if (!c->m_is_fp32) {   // Sbar is about to be zeroed: move the momentum it encodes to binary32 first
-            k_materialise_momentum<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->m(), 0, c->L.d, c->L.chunk);
-            APMS_CUDA(c, cudaGetLastError());
+        if (!c->m_is_fp32) {   // Sbar (top-k: the mask) is about to be zeroed: move the momentum it encodes to binary32 first
+            apms_status mst = launch_materialise_momentum(c, c->m(), 0, c->L.d);
+            if (mst != APMS_OK) return mst;
             c->m_is_fp32 = true;
         }
         APMS_CUDA(c, cudaMemsetAsync(c->Sbar(), 0, (size_t)c->L.Cp * 4, c->stream));
@@ -1105,8 +1150,7 @@ apms_status apms_uncompressed_step_typed(apms_ctx* c, const void* const* grads_d
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
     if (!c->m_is_fp32) {       // the momentum lives in the server's message: spell it out in binary32 first
-        k_materialise_momentum<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->Bbar(), c->Sbar(), c->m(), 0, c->L.d, c->L.chunk);
-        st = launch_check(c, "k_materialise_momentum");
+        st = launch_materialise_momentum(c, c->m(), 0, c->L.d);
         if (st != APMS_OK) return st;
         c->m_is_fp32 = true;
     }

@@ -247,7 +247,8 @@ __device__ __forceinline__ uint32_t topk_select_wave(const uint32_t key[4], uint
 struct TopkWorkerArgs {
     float* z; int64_t dz;
     uint32_t* B; int64_t Wp;          // selection masks
-    const float* m32;
+    const float* m32;                 // the momentum in binary32 (M32 form of the kernel) ...
+    const float* zbar; const uint32_t* Bbar;   // ... or as the server left it: m = C[zbar] = mask ? zbar : 0
     float* thr; int64_t Cp;           // per (worker, chunk): the magnitude of the K-th element of the last step
     int64_t d, chunk, C;
     int i0, ni;
@@ -263,7 +264,10 @@ __device__ __forceinline__ uint32_t topk_count(double frac, int L)
     return (uint32_t)K;
 }
 
-template <int GT>
+// M32: the momentum is read from the binary32 buffer (first step of the phase, after a state upload, or
+// when the server applies densely); otherwise it is taken from the server's compensated vector where the
+// server's mask has a bit, so that the server need not write a momentum vector at all.
+template <int GT, bool M32>
 __global__ void __launch_bounds__(kThreads, kTopkResident)
 k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
 {
@@ -280,7 +284,8 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
     float* zc = a.z + (int64_t)i * a.dz + base;
     uint32_t* maskw = a.B + (int64_t)i * a.Wp + base / 32;
-    const float* __restrict__ m = a.m32 + base;
+    const float* __restrict__ m = (M32 ? a.m32 : a.zbar) + base;
+    const uint32_t* __restrict__ mbar = a.Bbar + base / 32;
     float* thr = a.thr + (int64_t)i * a.Cp + c;
     const uint32_t K = topk_count(a.frac, L);
     const int nwords = (L + 31) / 32;
@@ -310,21 +315,29 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
         if (!checked || k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
         else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
     };
+    // the momentum of elements k..k+3
+    auto momentum = [&](int k, bool checked) -> float4 {
+        if (M32) return checked ? ld4_checked(m, k, L, false) : *reinterpret_cast<const float4*>(m + k);
+        const uint32_t nb = (mbar[k >> 5] >> (k & 31)) & 0xfu;
+        // loaded whether or not a bit is set: a load that waits for the mask word costs more than it saves
+        const float4 zb = checked ? ld4_checked(m, k, L, false) : *reinterpret_cast<const float4*>(m + k);
+        return make_float4((nb & 1u) ? zb.x : 0.0f, (nb & 2u) ? zb.y : 0.0f, (nb & 4u) ? zb.z : 0.0f, (nb & 8u) ? zb.w : 0.0f);
+    };
     int k = threadIdx.x * 4;
     for (; k + kThreads * 4 < Lfull; k += 2 * kThreads * 4) {
         const int k2 = k + kThreads * 4;
         const float4 g0 = Grad<GT>::ld4(g, k), g1 = Grad<GT>::ld4(g, k2);
         const float4 z0 = *reinterpret_cast<const float4*>(zc + k), z1 = *reinterpret_cast<const float4*>(zc + k2);
-        const float4 m0 = *reinterpret_cast<const float4*>(m + k), m1 = *reinterpret_cast<const float4*>(m + k2);
+        const float4 m0 = momentum(k, false), m1 = momentum(k2, false);
         const uint32_t n0 = maskw[k >> 5] >> (k & 31), n1 = maskw[k2 >> 5] >> (k2 & 31);
         sweep(k, g0, z0, m0, n0, false);
         sweep(k2, g1, z1, m1, n1, false);
     }
     for (; k < Lfull; k += kThreads * 4)
-        sweep(k, Grad<GT>::ld4(g, k), *reinterpret_cast<const float4*>(zc + k), *reinterpret_cast<const float4*>(m + k),
+        sweep(k, Grad<GT>::ld4(g, k), *reinterpret_cast<const float4*>(zc + k), momentum(k, false),
               maskw[k >> 5] >> (k & 31), false);
     for (; k < L; k += kThreads * 4)
-        sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), ld4_checked(m, k, L, false),
+        sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), momentum(k, true),
               maskw[k >> 5] >> (k & 31), true);
     __syncthreads();                                   // z stores, histogram and list are complete
     const int lane = threadIdx.x & 31;
@@ -395,12 +408,18 @@ struct TopkServerArgs {
     const float* z; int64_t dz;       // the workers' compensated vectors
     const uint32_t* B; int64_t Wp;    // and their masks
     float* zbar; uint32_t* Bbar;      // the server's compensated vector and mask
-    float* m32;                       // accumulator during the step, the new momentum after it
+    float* m32;                       // accumulator during the step; the new momentum after it where the chunk was applied densely
     float* thr;                       // per chunk: the magnitude of the K-th element of the last step
     const float* v; float* x;
     int64_t d, chunk;
     int n; float nf, lr, eps;
     double frac;
+    // An element that is not kept has m = +0, and x - (lr * 0) / (sqrt(v) + eps) is x itself whenever
+    // lr >= +0, eps > 0 and v is neither negative nor NaN (the host checks all three).  Then only the
+    // kept elements are touched (sparse != 0): the momentum stays implicit in (zbar, mask), v and x are read
+    // and x written for K elements per chunk instead of all.  Otherwise every chunk takes the general
+    // route, whose ordered pass updates every element and writes the momentum out.
+    int sparse;
 };
 
 __global__ void __launch_bounds__(kThreads, kTopkResident)
@@ -455,7 +474,7 @@ k_topk_server(const TopkServerArgs a)
     // the four mask bits of every worker (four workers at a time) and loads a worker's values only where one
     // of them is set.
     const uint32_t K = topk_count(a.frac, L);
-    const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
+    const bool small = nwords <= kTopkBins && a.sparse != 0;      // list routes: the mask fits the shared-memory words, sparse update allowed
     const uint32_t floor_key = small ? topk_floor(a.thr[c], K) : 0u;
     const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(a.thr[c]) : 0;
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
@@ -503,60 +522,54 @@ k_topk_server(const TopkServerArgs a)
     const float* __restrict__ v = a.v + base;
     float* __restrict__ x = a.x + base;
     uint32_t tau, ties;
-    bool have_tau = false;
-    bool keep_all_ties = false;                        // then "selected" is simply key >= tau
-    if (floor_key != 0) {                              // window route: threshold from the list, then one ordered pass
+    int n_list = 0;                                    // > 0: the list decides, hist[0..nwords) holds the mask so far
+    uint32_t K_list = K, floor_list = floor_key;
+    if (floor_key != 0) {                              // window route: the mask words are still all zero
         const uint32_t listed = list.count;
-        if (listed >= K && listed <= (uint32_t)kTopkList) {
-            uint32_t ties_total;
-            have_tau = topk_threshold_list(list, (int)listed, floor_key, K, bins8, sh, tau, ties, ties_total);
-            keep_all_ties = have_tau && ties_total == ties;
-        }
+        if (listed >= K && listed <= (uint32_t)kTopkList) n_list = (int)listed;
     } else if (small) {                                // two-pass route
         uint32_t Kb = K;
         const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
         const uint32_t inbin = hist[b0];
         __syncthreads();                               // everybody has read the histogram: its words become the mask
         if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
-            // second pass: momentum and model update for every element outside the bin of the K-th key (kept
-            // above it, dropped below); the elements of that bin go to the list, their x untouched
+            // second pass: the elements above the bin of the K-th key are kept - mask bit, model update
+            // (Section 3.3 steps 5-6) - and those of that bin go to the list
             for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
                 const int k = w0 + threadIdx.x * 4;
                 const float4 zv = ld4_checked(zb, k, L, false);
-                const float4 vv = ld4_checked(v, k, L, true);
-                const float4 xv = ld4_checked(x, k, L, true);
-                const float zz[4] = {zv.x, zv.y, zv.z, zv.w}, vs[4] = {vv.x, vv.y, vv.z, vv.w}, xs[4] = {xv.x, xv.y, xv.z, xv.w};
-                float mn[4], xn[4];
+                const float zz[4] = {zv.x, zv.y, zv.z, zv.w};
                 uint32_t nibble = 0;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const uint32_t key = mag_key(zz[e]);
-                    const int b = topk_bin(key, 19, bin0);
-                    const bool in_chunk = k + e < L;
-                    if (in_chunk && b > b0) nibble |= 1u << e;
-                    if (in_chunk && b == b0) topk_list_add(list, key, (uint32_t)(k + e));
-                    mn[e] = ((nibble >> e) & 1u) ? zz[e] : 0.0f;
-                    xn[e] = b == b0 ? xs[e] : apply_elem(xs[e], vs[e], mn[e], a.lr, a.eps);
+                    if (k + e < L) {
+                        const uint32_t key = mag_key(zz[e]);
+                        const int b = topk_bin(key, 19, bin0);
+                        if (b > b0) {
+                            nibble |= 1u << e;
+                            x[k + e] = apply_elem(x[k + e], v[k + e], zz[e], a.lr, a.eps);
+                        } else if (b == b0) {
+                            topk_list_add(list, key, (uint32_t)(k + e));
+                        }
+                    }
                 }
                 const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
                 if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
-                if (k + 3 < L) {
-                    *reinterpret_cast<float4*>(acc + k) = make_float4(mn[0], mn[1], mn[2], mn[3]);
-                    st_stream4(x + k, make_float4(xn[0], xn[1], xn[2], xn[3]));
-                } else {
-                    for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mn[e]; x[k + e] = xn[e]; }
-                }
             }
             __syncthreads();
-            uint32_t ties_total;
-            topk_threshold_list(list, (int)inbin, (uint32_t)(b0 + bin0) << 19, Kb, bins8, sh, tau, ties, ties_total);
-            for (int p = threadIdx.x; p < (int)inbin; p += kThreads) {          // the listed elements, one by one
+            n_list = (int)inbin; K_list = Kb; floor_list = (uint32_t)(b0 + bin0) << 19;
+        }
+    }
+    bool have_tau = false;
+    if (n_list > 0) {
+        uint32_t ties_total;
+        have_tau = topk_threshold_list(list, n_list, floor_list, K_list, bins8, sh, tau, ties, ties_total);
+        if (have_tau) {
+            for (int p = threadIdx.x; p < n_list; p += kThreads) {              // the listed elements, one by one
+                if (!topk_list_selected(list, n_list, p, tau, ties, ties_total)) continue;
                 const int j = (int)list.idx[p];
-                const bool kept = topk_list_selected(list, (int)inbin, p, tau, ties, ties_total);
-                const float mj = kept ? zb[j] : 0.0f;
-                acc[j] = mj;
-                x[j] = apply_elem(x[j], v[j], mj, a.lr, a.eps);
-                if (kept) atomicOr(&hist[j >> 5], 1u << (j & 31));
+                x[j] = apply_elem(x[j], v[j], zb[j], a.lr, a.eps);
+                atomicOr(&hist[j >> 5], 1u << (j & 31));
             }
             __syncthreads();
             for (int w = threadIdx.x; w < nwords; w += kThreads) maskbar[w] = hist[w];
@@ -564,12 +577,11 @@ k_topk_server(const TopkServerArgs a)
             return;
         }
     }
-    if (!have_tau) {                                   // general route: histograms over the whole chunk
-        if (small) topk_full_hist(zb, L, hist);
-        topk_threshold(zb, L, K, hist, sh, tau, ties);
-    }
+    // general route: histograms over the whole chunk
+    if (small) topk_full_hist(zb, L, hist);
+    topk_threshold(zb, L, K, hist, sh, tau, ties);
     if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
-    // ordered pass: mask, momentum m = C[zbar], model update (Section 3.3 steps 5-6)
+    // ordered pass: mask, momentum m = C[zbar] written out, model update (Section 3.3 steps 5-6) of every element
     uint32_t seen = 0;
     for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
         const int k = w0 + threadIdx.x * 4;
@@ -578,14 +590,7 @@ k_topk_server(const TopkServerArgs a)
         const float4 xv = ld4_checked(x, k, L, true);
         const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
         const uint32_t validmask = k + 3 < L ? 0xfu : (k < L ? (1u << (L - k)) - 1u : 0u);
-        uint32_t nibble;
-        if (keep_all_ties) {                           // uniform: no ranking, no barriers
-            nibble = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) nibble |= (((validmask >> e) & 1u) && key[e] >= tau) ? 1u << e : 0u;
-        } else {
-            nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
-        }
+        const uint32_t nibble = topk_select_wave(key, validmask, tau, ties, seen, warp_ties);
         const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
         if ((lane & 7) == 0 && k < L) maskbar[k >> 5] = word;
         const float4 mn = make_float4((nibble & 1u) ? zv.x : 0.0f, (nibble & 2u) ? zv.y : 0.0f,
@@ -599,6 +604,24 @@ k_topk_server(const TopkServerArgs a)
             const float mm[4] = {mn.x, mn.y, mn.z, mn.w}, xx[4] = {xn.x, xn.y, xn.z, xn.w};
             for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mm[e]; x[k + e] = xx[e]; }
         }
+    }
+}
+
+// Sets *flag if any v[j] is negative or NaN (v >= 0 fails); -0 and +inf pass.
+__global__ void k_any_negative_or_nan(const float* __restrict__ v, int64_t d, int* flag)
+{
+    bool found = false;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d; j += (int64_t)gridDim.x * blockDim.x)
+        found |= !(v[j] >= 0.0f);
+    if (found) *flag = 1;
+}
+
+__global__ void k_materialise_momentum_topk(const float* __restrict__ zbar, const uint32_t* __restrict__ mask,
+                                            float* __restrict__ out, int64_t first, int64_t count)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = first + j;
+        out[j] = ((mask[e >> 5] >> (e & 31)) & 1u) ? zbar[e] : 0.0f;
     }
 }
 

@@ -294,6 +294,24 @@ def test_topk_threshold_jumps():
         _topk_compare(ctx, orc, w, step)
 
 
+@pytest.mark.parametrize("lr,eps", [(-1e-3, 1e-8), (1e-3, 0.0)])
+def test_topk_updates_every_element_when_skipping_is_not_exact(lr, eps):
+    """With a negative learning rate or eps = 0 an element that is not kept need not come out of the update
+    unchanged, so the server must not skip it: same bit-identical comparison, on the route that updates all."""
+    w = tiny(5 * 4096 + 321, 3, 4096, cfg_id=184, lr=lr, eps=eps)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, 0.02)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(0.02)
+    for step in range(2):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(2, 8):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        _topk_compare(ctx, orc, w, step)
+
+
 @pytest.mark.parametrize("frac", [0.01, 0.1])
 def test_topk_long_free_run(frac):
     """60 free-running top-k steps: the predicted-threshold routes run on thresholds that drift as the errors

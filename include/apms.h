@@ -117,8 +117,12 @@ typedef enum {
  * In TOPK mode the context keeps, in place of the sign words, a selection mask per worker and for the
  * server (APMS_STATE_*_BITS return it: bit j = element j was sent), in place of the scales the magnitude
  * of the K-th (smallest sent) element of each chunk (APMS_STATE_*_SCALES; the next step uses it to guess
- * where its own threshold lies), and the momentum in binary32.  Chosen with apms_set_compressor until the first compression-phase step has run;
- * TOPK works with the momentum variant, the l2 scale setting and the whole-step functions. */
+ * where its own threshold lies).  The momentum m = C[zbar] is not stored separately while it can be read
+ * as (server mask ? server compensated vector : 0); APMS_STATE_M returns it spelled out.  An element
+ * that the server does not keep is left untouched by the model update when that is exact (lr >= +0,
+ * eps > 0, no negative or NaN entry in v); otherwise every element is updated.  Chosen with
+ * apms_set_compressor until the first compression-phase step has run; TOPK works with the momentum
+ * variant, the l2 scale setting and the whole-step functions. */
 typedef enum {
     APMS_COMPRESSOR_ONEBIT = 0,
     APMS_COMPRESSOR_TOPK = 1

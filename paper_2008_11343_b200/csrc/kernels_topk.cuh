@@ -352,21 +352,32 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
         const uint32_t inbin = hist[b0];
         __syncthreads();                               // everybody has read the histogram: its words become the mask
         if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
-            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
-                const int k = w0 + threadIdx.x * 4;
-                const float4 zv = ld4_checked(zc, k, L, false);
+            auto settle = [&](int k, float4 zv, bool checked) {
                 const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
                 uint32_t nibble = 0;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (k + e < L) {
+                    if (!checked || k + e < L) {
                         const int b = topk_bin(key[e], 19, bin0);
                         if (b > b0) nibble |= 1u << e;
                         else if (b == b0) topk_list_add(list, key[e], (uint32_t)(k + e));
                     }
                 }
                 const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
-                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+                if ((lane & 7) == 0 && (!checked || k < L)) hist[k >> 5] = word;
+            };
+            int w0 = 0;
+            for (; w0 + 4 * kThreads * 4 <= L; w0 += 4 * kThreads * 4) {      // four sweeps' loads in flight
+                const int k = w0 + threadIdx.x * 4;
+                float4 zv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zc + k + u * kThreads * 4);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) settle(k + u * kThreads * 4, zv[u], false);
+            }
+            for (; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                settle(k, ld4_checked(zc, k, L, false), true);
             }
             __syncthreads();
             n_list = (int)inbin; K_list = Kb; floor_list = (uint32_t)(b0 + bin0) << 19;
@@ -535,14 +546,12 @@ k_topk_server(const TopkServerArgs a)
         if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
             // second pass: the elements above the bin of the K-th key are kept - mask bit, model update
             // (Section 3.3 steps 5-6) - and those of that bin go to the list
-            for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
-                const int k = w0 + threadIdx.x * 4;
-                const float4 zv = ld4_checked(zb, k, L, false);
+            auto settle = [&](int k, float4 zv, bool checked) {
                 const float zz[4] = {zv.x, zv.y, zv.z, zv.w};
                 uint32_t nibble = 0;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (k + e < L) {
+                    if (!checked || k + e < L) {
                         const uint32_t key = mag_key(zz[e]);
                         const int b = topk_bin(key, 19, bin0);
                         if (b > b0) {
@@ -554,7 +563,20 @@ k_topk_server(const TopkServerArgs a)
                     }
                 }
                 const uint32_t word = pack_group_words(nibble, lane);   // valid in lanes 0, 8, 16, 24
-                if ((lane & 7) == 0 && k < L) hist[k >> 5] = word;
+                if ((lane & 7) == 0 && (!checked || k < L)) hist[k >> 5] = word;
+            };
+            int w0 = 0;
+            for (; w0 + 4 * kThreads * 4 <= L; w0 += 4 * kThreads * 4) {      // four sweeps' loads in flight
+                const int k = w0 + threadIdx.x * 4;
+                float4 zv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zb + k + u * kThreads * 4);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) settle(k + u * kThreads * 4, zv[u], false);
+            }
+            for (; w0 < L; w0 += kThreads * 4) {
+                const int k = w0 + threadIdx.x * 4;
+                settle(k, ld4_checked(zb, k, L, false), true);
             }
             __syncthreads();
             n_list = (int)inbin; K_list = Kb; floor_list = (uint32_t)(b0 + bin0) << 19;

@@ -289,8 +289,20 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
         apms_status st = launch_check(c, "k_worker_fine");
         if (st != APMS_OK) return st;
         const int64_t total = (int64_t)ni * c->L.C;
-        k_finalize_fine<<<(unsigned)((total + kWarps - 1) / kWarps), kThreads, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0),
-                                                                             c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk);
+        const int64_t slots = c->L.chunk / kFineSub;                 // partial sums of a whole chunk
+        int team = 1;
+        while (team < 32 && team < slots) team *= 2;
+        const int64_t per_cta = (int64_t)kWarps * (32 / team);
+        const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
+        const double* part = c->fine_partial(i0);
+        switch (team) {
+        case 1:  k_finalize_fine<1><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        case 2:  k_finalize_fine<2><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        case 4:  k_finalize_fine<4><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        case 8:  k_finalize_fine<8><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        case 16: k_finalize_fine<16><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        default: k_finalize_fine<32><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        }
         st = launch_check(c, "k_finalize_fine");
         if (st != APMS_OK) return st;
     }

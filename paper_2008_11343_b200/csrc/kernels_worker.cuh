@@ -229,25 +229,30 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     if (lane == 0) *slot = acc;
 }
 
-// Scales from the fine form's partial sums (one per 512 elements): one warp per (row, chunk) adds
-// the chunk's slots in a fixed order (lane l takes slots l, l + 32, ..., then the shuffle tree)
-// and takes sqrt(sum / L).
+// Scales from the fine form's partial sums (one per 512 elements): a team of T lanes per (row, chunk)
+// adds the chunk's slots in a fixed order (lane l of the team takes slots l, l + T, ..., then the shuffle
+// tree) and takes sqrt(sum / L).  T is the number of slots of a whole chunk rounded up to a power of two,
+// at most a warp; the sums are not negative, so a team's tree gives bit for bit what a whole warp's tree
+// with zeros in the other lanes gives, and short chunks do not leave most of a warp idle (chunk = 1024:
+// 16 chunks per warp; one warp per chunk took 1.2 ms longer at n = 16).
+template <int T>
 __global__ void __launch_bounds__(kThreads)
 k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
                 int rows, int64_t C, int64_t d, int64_t chunk)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t idx = (int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (idx >= (int64_t)rows * C) return;                        // whole warps
-    const int r = (int)(idx / C);
-    const int64_t c = idx % C;
+    const int lane = threadIdx.x & 31, sub = lane % T;
+    const int64_t idx = ((int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * (32 / T) + lane / T;
+    const bool live = idx < (int64_t)rows * C;                   // every lane stays for the shuffles
+    const int r = live ? (int)(idx / C) : 0;
+    const int64_t c = live ? idx % C : 0;
     const int64_t cbeg = c * chunk;
     const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
     const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
     double total = 0.0;
-    for (int64_t q = q0 + lane; q < q1; q += 32) total += partial[(int64_t)r * Pp + q];
-    total = warp_sum(total);
-    if (lane == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+    if (live) for (int64_t q = q0 + sub; q < q1; q += T) total += partial[(int64_t)r * Pp + q];
+#pragma unroll
+    for (int o = T / 2; o > 0; o >>= 1) total += __shfl_down_sync(0xffffffffu, total, o, T);
+    if (live && sub == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
 // Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).

@@ -202,11 +202,14 @@ class PeerShardedStep:
         b.apply_phase()                                                         # steps 5-6
 
     def close(self):
+        """Unmaps the peers' workspaces.  Collective: returns when every process has unmapped, so that each may
+        then free its own workspace."""
         self.dist.barrier(group=self.group)                                     # nobody reads a mapping that goes away
         for r, base in enumerate(self.base):
             if r != self.rank and base is not None:
                 self._peers.apms_ipc_close(base)
         self.base = []
+        self.dist.barrier(group=self.group)                                     # nobody frees memory that is still mapped
 
     def wire_bytes_per_step(self) -> int:
         """Bytes that cross between GPUs per step because of this process: the rows it loads from peers and the

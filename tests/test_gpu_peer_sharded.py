@@ -95,7 +95,14 @@ def test_rows_argument_errors_are_status_codes():
     assert ctx.message_offsets(0)[0] % 256 == 0 and ctx.message_offsets(-1)[1] % 256 == 0
 
 
-def _rank_main(rank, world, port, d, chunk, n_local, steps, out):
+def _report(outdir, rank, result):
+    import json
+
+    with open(os.path.join(outdir, f"rank{rank}.json"), "w") as f:
+        json.dump(result, f)
+
+
+def _rank_main(rank, world, port, d, chunk, n_local, steps, outdir):
     import torch
     import torch.distributed as dist
 
@@ -124,23 +131,24 @@ def _rank_main(rank, world, port, d, chunk, n_local, steps, out):
         wire = step.wire_bytes_per_step()
         step.close()
         ctx.close()
-        out[rank] = (ok, wire, "")
+        _report(outdir, rank, [ok, wire, ""])
         dist.destroy_process_group()
     except Exception as exc:                                        # reported to the parent, which fails the test
-        out[rank] = (False, 0, repr(exc))
+        _report(outdir, rank, [False, 0, repr(exc)])
         raise
 
 
-def test_two_processes_on_one_gpu_exchange_through_mapped_workspaces():
+def test_two_processes_on_one_gpu_exchange_through_mapped_workspaces(tmp_path):
+    import json
+
     import torch.multiprocessing as mp
 
     d, chunk, n_local, world = 9 * 2048 + 300, 2048, 2, 2
     with socket.socket() as sock:
         sock.bind(("127.0.0.1", 0))
         port = sock.getsockname()[1]
-    with mp.Manager() as mgr:
-        out = mgr.dict()
-        mp.spawn(_rank_main, args=(world, port, d, chunk, n_local, 3, out), nprocs=world, join=True)
-        res = dict(out)
+    # results come back through files: nothing is forked from this process, which holds a CUDA context
+    mp.spawn(_rank_main, args=(world, port, d, chunk, n_local, 3, str(tmp_path)), nprocs=world, join=True)
+    res = {r: json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)}
     assert res[0][0] and res[1][0], res
     assert max(res[0][1], res[1][1]) < 0.1 * 4 * d * n_local

@@ -8,14 +8,19 @@ namespace {
 // Top-k compressor (Section 5.1, second item): per chunk the K = ceil(k L) elements of largest |z| are
 // sent, the others decompress to 0; equal magnitudes go to the lower index.  State in this mode: the
 // compensated vectors z as before, and in place of the sign words a SELECTION MASK (bit j = element j
-// was sent), from which  C[z] = mask ? z : 0  and  delta = z - C[z]  follow exactly; the momentum is
-// kept in binary32.  One CTA per (chunk, worker) / per chunk; a chunk's z is written once and re-read
-// from L2 by the selection passes.
+// was sent), from which  C[z] = mask ? z : 0  and  delta = z - C[z]  follow exactly; in place of the
+// scales the chunk's last threshold.  The momentum C[zbar] is read as (server mask ? zbar : 0) unless it
+// was written out in binary32.  One CTA per (chunk, worker) / per chunk.
 //
-// Selection: the K-th largest magnitude is found by a three-level radix select over the bit pattern of
-// |z| (11 + 11 + 9 bits, shared-memory histograms), giving the threshold key tau and the number of
-// elements equal to tau that are still to be kept; a last pass in index order marks  key > tau, and the
-// first `ties` elements with key == tau.
+// Selection.  Keys are the bit patterns of |z|; the K-th largest key tau and the number of elements
+// equal to tau that are to be kept (`ties`, lowest positions first) define the mask.  Three routes, all
+// exact, in the order of their cost:
+//   window     small K: the first pass lists the keys at or above a floor a little below the chunk's last
+//              threshold; tau and the mask come from that list alone (topk_threshold_list);
+//   two passes the first pass counts all keys in fine bins around the last threshold; a second pass keeps
+//              what lies above the K-th key's bin and lists that bin, which the list settles;
+//   general    three-level radix select over the whole chunk (11 + 11 + 9 bits, topk_threshold) and a pass
+//              in index order that ranks equal keys across the block (topk_select_wave).
 
 constexpr int kTopkBins = 2048;
 

@@ -36,6 +36,11 @@
  *     failure is a status code and a message available from apms_last_error().
  *   - The library has no CPU fallback: without a CUDA device every device call fails with
  *     APMS_ERR_CUDA.
+ *   - The step functions that take device gradients enqueue kernels and nothing else, so a
+ *     step can be recorded by CUDA stream capture on the context's stream and replayed as a
+ *     graph (not the first step of the COMPRESSED phase, which differs from the later ones, and
+ *     not with timing on).  A replay repeats the device work only: the host-side counters
+ *     (apms_get_step, apms_launch_count) count the capture, not the replays.
  *   - One context must not be used from two host threads at once.
  */
 #ifndef APMS_H

@@ -448,6 +448,38 @@ def test_sharded_step_with_one_process_equals_the_whole_step():
         dist.destroy_process_group()
 
 
+def test_a_step_can_be_captured_in_a_cuda_graph_and_replayed():
+    """apms_compressed_step only enqueues kernels on the context's stream, so it can be captured once and
+    replayed (gradients refreshed in place between replays): the replayed steps equal eager steps bit for bit."""
+    import torch
+
+    w = tiny(6 * 4096 + 77, 3, 4096, cfg_id=151)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, stream=s)
+        b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, stream=s)
+        gs = [g.to("cuda") for g in map(torch.from_numpy, wl.host_gradients(w, 0))]
+        for c in (a, b):
+            c.set_params(wl.initial_params(w))
+            c.warmup_step(gs)
+            c.freeze_v()
+            c.compressed_step(gs)              # the first step of the phase differs (binary32 momentum): not the one to capture
+        s.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            b.compressed_step(gs)              # recorded, not run
+        for step in range(1, 6):
+            for g, h in zip(gs, wl.host_gradients(w, step)):
+                g.copy_(torch.from_numpy(h), non_blocking=False)
+            a.compressed_step(gs)
+            graph.replay()
+        s.synchronize()
+        for which in (B.STATE_X, B.STATE_SERVER_BITS, B.STATE_SERVER_SCALES, B.STATE_SERVER_ERR):
+            assert np.array_equal(a.get_state(which).view(np.uint32), b.get_state(which).view(np.uint32)), which
+        for i in range(w.n):
+            assert np.array_equal(a.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), b.get_state(B.STATE_WORKER_ERR, i).view(np.uint32))
+
+
 # ------------------------------------------------------------------ the benchmark's small configurations
 
 def test_config0_free_running_10_steps():

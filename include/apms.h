@@ -280,8 +280,9 @@ apms_status apms_apply_phase(apms_ctx* ctx);
  * Figure 1.  apms_ipc_export: writes APMS_IPC_HANDLE_BYTES bytes naming this context's workspace,
  * which must be the library's own allocation (no apms_bind); APMS_ERR_BAD_STATE otherwise.
  * apms_ipc_open: maps the workspace named by a handle made in ANOTHER process and returns its base
- * address in this process; apms_ipc_close unmaps it.  These two take no context; on failure
- * apms_last_error(NULL) describes why. */
+ * address in this process; apms_ipc_close unmaps it.  An exported context must outlive every
+ * mapping of it: destroy it only after all processes that opened its handle have closed it.
+ * apms_ipc_open and apms_ipc_close take no context; on failure apms_last_error(NULL) describes why. */
 #define APMS_IPC_HANDLE_BYTES 64
 apms_status apms_server_phase_rows(apms_ctx* ctx, const uint32_t* const* bits_rows, const float* const* scale_rows,
                                    int rows, int64_t chunk_begin, int64_t chunk_end);

@@ -226,9 +226,21 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
         adam = {"ms_per_step": ms / cnt, "achieved_gbs": ab / (ms / cnt * 1e-3) / 1e9,
                 "worker_elements_per_s": w.d * w.n / (ms / cnt * 1e-3)}
     ctx.freeze_v()
-    ctx.compressed_step(ring[0])             # reads the binary32 momentum once; not representative
+    if args.path == "phases":
+        # the step as a one-process-per-GPU run makes it (worker phase, server phase over rows given by address,
+        # apply phase), here with one process that serves every chunk from its own workers' messages
+        own_bits = [ctx.message_ptrs(i)[0] for i in range(w.n)]
+        own_scales = [ctx.message_ptrs(i)[1] for i in range(w.n)]
+
+        def step(gs):
+            ctx.worker_phase(gs)
+            ctx.server_phase_rows(own_bits, own_scales, 0, ctx.C)
+            ctx.apply_phase()
+    else:
+        step = ctx.compressed_step
+    step(ring[0])                            # reads the binary32 momentum once; not representative
     for k in range(args.warmup):
-        ctx.compressed_step(ring[(k + 1) % 2])
+        step(ring[(k + 1) % 2])
     torch.cuda.synchronize()
 
     # timed region: K steps between two events on the context's stream
@@ -243,7 +255,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
     with ClockSampler(local_rank) as clocks:
         e0.record(ctx.stream)
         for k in range(args.steps):
-            ctx.compressed_step(ring[k % 2])
+            step(ring[k % 2])
         e1.record(ctx.stream)
         torch.cuda.synchronize()
     if world > 1:
@@ -307,6 +319,9 @@ def main(argv=None) -> int:
     ap.add_argument("--compressor", default="onebit", choices=["onebit", "topk"],
                     help="the compression operator (the configurations of record use the 1-bit compressor)")
     ap.add_argument("--topk-fraction", type=float, default=0.01)
+    ap.add_argument("--path", default="whole", choices=["whole", "phases"],
+                    help="whole: apms_compressed_step (the configurations of record); phases: the same step through "
+                         "apms_worker_phase / apms_server_phase_rows / apms_apply_phase (1-bit compressor only)")
     ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16", "float16"],
                     help="element type of the gradient arrays (the configurations of record use float32)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -334,6 +349,7 @@ def main(argv=None) -> int:
     config = {"workload": f"{w.name}: d={w.d}, n={w.n} simulated workers, chunk={w.chunk}, {w.dist} gradients",
               "d": w.d, "n_workers": w.n, "chunk": w.chunk, "gradient_dtype": args.grad_dtype,
               "compressor": args.compressor if args.compressor == "onebit" else f"topk {args.topk_fraction}",
+              "path": args.path,
               "parallelism": f"replicas x{world}",
               "l2_policy": "inputs_exceed_l2" if 12 * w.d * w.n > (256 << 20) else "l2_resident",
               "gradient_ring": 2}

@@ -58,7 +58,7 @@ struct Layout {
     int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_status, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
 };
 
 bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
@@ -92,6 +92,7 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
     L->off_stage = take((size_t)L->dz * 4 * 2);
     L->off_mon = take(((size_t)(n + 1) * (size_t)((d + 4095) / 4096) + (size_t)(n + 1)) * 8);   // error monitor: tile sums + row sums
+    L->off_den = take((size_t)L->dz * 4);              // sqrt(v) + eps of the frozen v
     L->off_status = take(256);
     L->total = o;
     return true;
@@ -116,6 +117,7 @@ struct apms_ctx {
     apms_phase phase;
     bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar; top-k: in zbar under the mask Bbar)
     bool v_checked, v_plain; // top-k: has v been looked at since it last changed, and is every entry >= 0 (not NaN)
+    bool den_valid;          // den holds sqrt(v) + eps of the current v
     char* ws; size_t ws_bytes; bool owns_ws;
     cudaStream_t stream;
     cudaStream_t copy_stream; cudaEvent_t ev_copied[2], ev_used[2]; bool host_path_ready;
@@ -140,6 +142,7 @@ struct apms_ctx {
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
     int* status() { return (int*)(ws + L.off_status); }
+    float* den() { return (float*)(ws + L.off_den); }
     double* fine_partial(int row) { return (double*)(ws + L.off_fine) + (int64_t)row * L.fine_Pp; }
     double* partial(int row) { return (double*)(ws + L.off_part) + (int64_t)row * L.t.Pp; }   // row n = server
 };
@@ -388,6 +391,20 @@ cudaError_t launch_staged_n(const ServerStagedArgs& sa, unsigned blocks, size_t 
     }
 }
 
+int grid_for(const apms_ctx* c, int64_t items, int per_sm);
+
+// The denominator of the model update, sqrt(v) + eps, is the same in every step of the compression phase
+// (v is frozen): it is formed once - the same two rounded operations - and the update kernels of the 1-bit
+// path read it in place of v.
+apms_status ensure_den(apms_ctx* c)
+{
+    if (c->den_valid) return APMS_OK;
+    k_make_den<<<grid_for(c, c->L.d, 8), kThreads, 0, c->stream>>>(c->v(), c->den(), c->L.d, c->eps);
+    apms_status st = launch_check(c, "k_make_den");
+    if (st == APMS_OK) c->den_valid = true;
+    return st;
+}
+
 // Where the server finds the workers' messages: `rows` senders, row j holding sign words and scales
 // addressed by ABSOLUTE word / chunk index (a pointer into a shard is shifted back by the caller).
 struct ServerSource {
@@ -427,10 +444,14 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
         Timed t(c, APMS_KERNEL_SERVER);
         if (staged) {
             const bool fused = may_fuse && c->L.t.P == 1;   // the CTA sees the whole chunk, so it knows the new scale
+            if (fused) {
+                apms_status dst = ensure_den(c);
+                if (dst != APMS_OK) return dst;
+            }
             ServerStagedArgs sa;
             sa.a = a; sa.status = c->status();
             sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
-            sa.v = c->v(); sa.x = c->x(); sa.lr = c->lr; sa.eps = c->eps;
+            sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr;
             const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
             sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
             const int64_t fill = count / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
@@ -472,15 +493,15 @@ apms_status launch_apply(apms_ctx* c)
         k_apply_gradient<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(g);
         return launch_check(c, "k_apply_gradient");
     }
+    apms_status dst = ensure_den(c);
+    if (dst != APMS_OK) return dst;
     ApplyArgs a;
-    a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.v = c->v(); a.x = c->x();
-    a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr; a.eps = c->eps;
+    a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.den = c->den(); a.x = c->x();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr;
     Timed t(c, APMS_KERNEL_APPLY);
     k_apply<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(a);
     return launch_check(c, "k_apply");
 }
-
-int grid_for(const apms_ctx* c, int64_t items, int per_sm);
 
 // Top-k: may the server leave the elements it does not keep alone?  Their momentum is +0, and
 // x - (lr * 0) / (sqrt(v) + eps) returns x itself iff lr is not negative (nor -0), eps > 0 and v is neither
@@ -599,7 +620,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     apms_ctx* c = new (std::nothrow) apms_ctx();
     if (!c) { snprintf(g_create_error, sizeof g_create_error, "host allocation failed"); return APMS_ERR_OOM; }
     c->L = L; c->beta1 = beta1; c->beta2 = beta2; c->eps = eps; c->lr = lr;
-    c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true; c->v_checked = false; c->v_plain = false;
+    c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true; c->v_checked = false; c->v_plain = false; c->den_valid = false;
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
@@ -688,6 +709,7 @@ apms_status apms_freeze_v(apms_ctx* c)
     c->phase = APMS_PHASE_COMPRESSED;
     c->m_is_fp32 = true;
     c->v_checked = false;
+    c->den_valid = false;
     return APMS_OK;
 }
 
@@ -997,7 +1019,7 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
     float* dst = nullptr;
     switch (which) {
     case APMS_STATE_X: dst = c->x(); break;
-    case APMS_STATE_V: dst = c->v(); c->v_checked = false; break;
+    case APMS_STATE_V: dst = c->v(); c->v_checked = false; c->den_valid = false; break;
     case APMS_STATE_M: dst = c->m(); c->m_is_fp32 = true; break;
     case APMS_STATE_WORKER_ERR:
         if (worker < 0 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range");

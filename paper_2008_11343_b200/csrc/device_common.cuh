@@ -96,6 +96,12 @@ __device__ __forceinline__ float4 ld_grad4_checked(const void* p, int k, int len
 __device__ __forceinline__ float signed_scale(float z, float s) { return (z >= 0.0f) ? s : -s; }
 __device__ __forceinline__ float bit_scale(uint32_t bit, float s) { return bit ? s : -s; }
 
+// The same update from its stored pieces: den = sqrt(v) + eps (formed once while v is frozen) and
+// c = lr * S (once per chunk); lr * (+-S) = +-(lr * S) exactly, so this is apply_elem(x, v, +-S, lr, eps) bit for bit.
+__device__ __forceinline__ float apply_stored(float x, float den, uint32_t bit, float c) {
+    return __fsub_rn(x, __fdiv_rn(bit ? c : -c, den));
+}
+
 // Model update of one element with the frozen variance (Section 3.3 step 6).
 __device__ __forceinline__ float apply_elem(float x, float v, float q, float lr, float eps) {
     return __fsub_rn(x, __fdiv_rn(__fmul_rn(lr, q), __fadd_rn(__fsqrt_rn(v), eps)));

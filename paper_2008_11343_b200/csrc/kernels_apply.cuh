@@ -14,9 +14,16 @@ constexpr int kApplyTile = 4096;
 constexpr int kApplyU = kApplyTile / (kThreads * 4);
 
 struct ApplyArgs {
-    const uint32_t* Bbar; const float* Sbar; const float* v; float* x;
-    int64_t d; int64_t chunk; float lr, eps;
+    const uint32_t* Bbar; const float* Sbar; const float* den; float* x;     // den = sqrt(v) + eps, see k_make_den
+    int64_t d; int64_t chunk; float lr;
 };
+
+// den = sqrt(v) + eps, the denominator of the model update while v is frozen.
+__global__ void k_make_den(const float* __restrict__ v, float* __restrict__ den, int64_t d, float eps)
+{
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d; j += (int64_t)gridDim.x * blockDim.x)
+        den[j] = __fadd_rn(__fsqrt_rn(v[j]), eps);
+}
 
 __global__ void __launch_bounds__(kThreads)
 k_apply(const ApplyArgs a)
@@ -28,7 +35,7 @@ k_apply(const ApplyArgs a)
     const uint32_t off0 = (uint32_t)(base - c0 * a.chunk);
     const uint32_t chunk32 = (uint32_t)a.chunk;
     const uint32_t* __restrict__ bits = a.Bbar + base / 32;
-    const float* __restrict__ v = a.v + base;
+    const float* __restrict__ v = a.den + base;
     float* __restrict__ x = a.x + base;
     const float* __restrict__ Sb = a.Sbar + c0;
     if (L == kApplyTile) {
@@ -47,10 +54,11 @@ k_apply(const ApplyArgs a)
 #pragma unroll
         for (int u = 0; u < kApplyU; ++u) {
             const int k = (u * kThreads + threadIdx.x) * 4;
-            xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib[u] & 1u, S[u]), a.lr, a.eps);
-            xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib[u] & 2u, S[u]), a.lr, a.eps);
-            xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib[u] & 4u, S[u]), a.lr, a.eps);
-            xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib[u] & 8u, S[u]), a.lr, a.eps);
+            const float cc = __fmul_rn(a.lr, S[u]);
+            xx[u].x = apply_stored(xx[u].x, vv[u].x, nib[u] & 1u, cc);
+            xx[u].y = apply_stored(xx[u].y, vv[u].y, nib[u] & 2u, cc);
+            xx[u].z = apply_stored(xx[u].z, vv[u].z, nib[u] & 4u, cc);
+            xx[u].w = apply_stored(xx[u].w, vv[u].w, nib[u] & 8u, cc);
             st_stream4(x + k, xx[u]);
         }
         return;
@@ -59,17 +67,18 @@ k_apply(const ApplyArgs a)
         const uint32_t rel = off0 + (uint32_t)k;
         const float S = Sb[rel < chunk32 ? 0u : rel / chunk32];
         const uint32_t nib = bits[k >> 5] >> (k & 31);
+        const float cc = __fmul_rn(a.lr, S);
         if (k + 3 < L) {
             const float4 vv = ld_stream4(v + k);
             float4 xx = ld_stream4(x + k);
-            xx.x = apply_elem(xx.x, vv.x, bit_scale(nib & 1u, S), a.lr, a.eps);
-            xx.y = apply_elem(xx.y, vv.y, bit_scale(nib & 2u, S), a.lr, a.eps);
-            xx.z = apply_elem(xx.z, vv.z, bit_scale(nib & 4u, S), a.lr, a.eps);
-            xx.w = apply_elem(xx.w, vv.w, bit_scale(nib & 8u, S), a.lr, a.eps);
+            xx.x = apply_stored(xx.x, vv.x, nib & 1u, cc);
+            xx.y = apply_stored(xx.y, vv.y, nib & 2u, cc);
+            xx.z = apply_stored(xx.z, vv.z, nib & 4u, cc);
+            xx.w = apply_stored(xx.w, vv.w, nib & 8u, cc);
             st_stream4(x + k, xx);
         } else {
             for (int e = 0; e < 4 && k + e < L; ++e)
-                x[k + e] = apply_elem(x[k + e], v[k + e], bit_scale((nib >> e) & 1u, S), a.lr, a.eps);
+                x[k + e] = apply_stored(x[k + e], v[k + e], (nib >> e) & 1u, cc);
         }
     }
 }

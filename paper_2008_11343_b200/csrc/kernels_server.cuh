@@ -205,7 +205,7 @@ struct ServerStagedArgs {
     ServerArgs a;
     int* status;          // device status word: set when a bounded wait gave up
     float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
-    const float* v; float* x; float lr, eps;     // steps 5-6, used by the fused form only
+    const float* den; float* x; float lr;        // steps 5-6 (fused form only): den = sqrt(v) + eps, see k_make_den
     int span;             // chunks per CTA of the fused form
 };
 
@@ -302,7 +302,7 @@ k_server_staged(const ServerStagedArgs sa)
                             bulk_load(rows + i * kSlabWords, a.Brow[i] + wofs + (size_t)j * kSlabWords, wbytes, &full[st]);
                     } else {
                         mbar_arrive_expect_tx(&full[st], 2 * zbytes);
-                        bulk_load(base, sa.v + it.base + (size_t)j * kSlab, zbytes, &full[st]);
+                        bulk_load(base, sa.den + it.base + (size_t)j * kSlab, zbytes, &full[st]);
                         bulk_load(base + (size_t)kSlab * 4, sa.x + it.base + (size_t)j * kSlab, zbytes, &full[st]);
                     }
                 }
@@ -380,6 +380,7 @@ k_server_staged(const ServerStagedArgs sa)
                 // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
                 const float S_new = (float)sqrt(total / (double)it.Lc);
                 if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
+                const float c_new = __fmul_rn(sa.lr, S_new);        // lr * (+-S) = +-(lr * S)
                 for (int j = 0; ok && j < nslabs; ++j, ++q) {
                     const int st = q % kStages;
                     if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; break; }
@@ -398,10 +399,10 @@ k_server_staged(const ServerStagedArgs sa)
                         const int grp = j * kSlabGroups + (u ? g1 : g0);
                         const int k = grp * kGroup + lane * 4;
                         const uint32_t nib = nb[grp * 4 + wl] >> sh;
-                        xx[u].x = apply_elem(xx[u].x, vv[u].x, bit_scale(nib & 1u, S_new), sa.lr, sa.eps);
-                        xx[u].y = apply_elem(xx[u].y, vv[u].y, bit_scale(nib & 2u, S_new), sa.lr, sa.eps);
-                        xx[u].z = apply_elem(xx[u].z, vv[u].z, bit_scale(nib & 4u, S_new), sa.lr, sa.eps);
-                        xx[u].w = apply_elem(xx[u].w, vv[u].w, bit_scale(nib & 8u, S_new), sa.lr, sa.eps);
+                        xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, c_new);
+                        xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new);
+                        xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new);
+                        xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, c_new);
                         st4_checked(sa.x + it.base, k, L, xx[u]);
                     }
                 }

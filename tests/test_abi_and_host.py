@@ -39,7 +39,7 @@ def test_workspace_bytes_is_pure_and_covers_the_state(lib):
     d, n, chunk = 335_141_888, 16, 32768
     nbytes = B.apms_workspace_bytes(d, n, chunk)
     C, W = -(-d // chunk), -(-d // 32)
-    need = 4 * d * (n + 4 + 2) + 4 * W * (n + 1) + 4 * C * (n + 1)
+    need = 4 * d * (n + 4 + 2 + 1) + 4 * W * (n + 1) + 4 * C * (n + 1)   # x, v, m, zbar, n z, 2 staging, sqrt(v) + eps
     need += 8 * n * -(-d // 512)                     # one binary64 partial sum per worker and 512 elements
     assert need <= nbytes <= need * 1.001 + (1 << 20)
     assert B.apms_workspace_bytes(d, n, chunk) == nbytes

@@ -674,7 +674,7 @@ def test_phase_and_argument_errors_are_status_codes():
             B.apms_create(bad[0], bad[1], 0.9, 0.999, 1e-8, 1e-3, bad[2])
         assert B.apms_workspace_bytes(*bad) == 0
     ctx.compressed_step(g)                      # the context is still usable after all of the above
-    assert ctx.launch_count == 1 + 3
+    assert ctx.launch_count == 1 + 3 + 1            # the warmup step; worker, server, update; sqrt(v) + eps formed once
 
 
 def test_a_wait_that_gives_up_is_reported_and_the_context_survives():

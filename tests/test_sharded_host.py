@@ -155,3 +155,13 @@ def test_chunk_and_word_ranges_tile_the_vector():
     r = sharded.chunk_ranges(-(-d // chunk), 8)
     words = [sharded.word_range(b, e, chunk, d) for b, e in r]
     assert words[0][0] == 0 and words[-1][1] == -(-d // 32) and all(a[1] == b[0] for a, b in zip(words, words[1:]))
+
+
+def test_chunk_for_servers_gives_one_chunk_per_server():
+    from paper_2008_11343_b200 import sharded
+
+    for d, n in [(335_141_888, 16), (109_482_240, 8), (2049, 2), (4096, 2), (1, 1)]:
+        chunk = sharded.chunk_for_servers(d, n)
+        assert chunk % 2048 == 0 and -(-d // chunk) <= n and chunk * n >= d
+        assert chunk - 2048 < -(-d // n)                         # not rounded further than needed
+    assert -(-335_141_888 // sharded.chunk_for_servers(335_141_888, 16)) == 16

@@ -140,6 +140,17 @@ def sum_over_ranks(value: float, dist) -> float:
 
 # ------------------------------------------------------------------------------------------ CPU oracle leg
 
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def oracle_sample_workload(w, max_chunks: int = 48):
     from paper_2008_11343_b200 import workloads as wl
 
@@ -172,10 +183,22 @@ def time_oracle(w, steps: int, warmup: int, budget_s: float = 20.0) -> dict:
         if time.perf_counter() - t_begin > budget_s and len(times) >= 3:
             break
     per_step = sum(times) / len(times)
+    # the same sample on one thread (a few steps), for the per-core rate
+    orc.set_threads(1)
+    single = []
+    t_begin = time.perf_counter()
+    for k in range(3):
+        t0 = time.perf_counter()
+        orc.compressed_step(ring[k % 2])
+        single.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_begin > budget_s / 2:
+            break
+    per_step_1 = sum(single) / len(single)
     return {"value": ws.d * ws.n / per_step, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"{ws.name} (d={ws.d}, n={ws.n}, chunk={ws.chunk}), {len(times)} steps, "
                       f"{per_step * 1e3:.1f} ms/step, OpenMP over chunks",
-            "ms_per_step": per_step * 1e3, "steps": len(times)}
+            "ms_per_step": per_step * 1e3, "steps": len(times),
+            "single_thread_value": ws.d * ws.n / per_step_1, "cpu_model": cpu_model()}
 
 
 # ------------------------------------------------------------------------------------------ GPU leg
@@ -362,7 +385,7 @@ def main(argv=None) -> int:
                 "steps": r["steps"], "warmup": args.warmup, "ms_per_step": r["ms_per_step"],
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic", "config": config,
-                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "single_thread_value", "cpu_model")},
                 "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "gpu_launches": 0}
         print(json.dumps(line))
@@ -431,7 +454,7 @@ def main(argv=None) -> int:
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = time_oracle(w, steps=50, warmup=1, budget_s=15.0)
-        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "single_thread_value", "cpu_model")}
 
     if rank == 0:
         line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -276,14 +276,19 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
         dist.barrier()
     torch.cuda.synchronize()
     with ClockSampler(local_rank) as clocks:
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps - 1)]
         e0.record(ctx.stream)
         for k in range(args.steps):
             step(ring[k % 2])
+            if k < args.steps - 1:
+                marks[k].record(ctx.stream)          # per-step times (min, median); the value comes from e0..e1
         e1.record(ctx.stream)
         torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     seconds = max_over_ranks(e0.elapsed_time(e1) * 1e-3, group)
+    edges = [e0] + marks + [e1]
+    per_step_ms = sorted(a.elapsed_time(b) for a, b in zip(edges, edges[1:]))
     launches = ctx.launch_count - launches0
     kernel_ms = {}
     for kid, name in enumerate(B.KERNEL_NAMES):
@@ -292,6 +297,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
             kernel_ms[name] = ms / cnt
     ctx.set_timing(False)
     out = {"ms_per_step": seconds * 1e3 / args.steps, "value": world * w.d * w.n * args.steps / seconds,
+           "ms_per_step_min": per_step_ms[0], "ms_per_step_median": per_step_ms[len(per_step_ms) // 2],
            "kernel_ms": kernel_ms, "launches": launches, "clocks": clocks.summary(), "adam": adam, "e2e": None}
 
     # end to end through the host-gradient entry point: H2D of the n gradients and D2H of x
@@ -461,7 +467,8 @@ def main(argv=None) -> int:
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": m["e2e"], "gpu_launches": m["launches"],
-                "clocks": m["clocks"]}
+                "clocks": m["clocks"],
+                "ms_per_step_min": m["ms_per_step_min"], "ms_per_step_median": m["ms_per_step_median"]}
         if m["adam"]:
             line["warmup_adam"] = m["adam"]
         print(json.dumps(line))

@@ -313,7 +313,11 @@ apms_status apms_get_state_slice(apms_ctx* ctx, apms_state_id which, int worker,
  * Synchronises. */
 apms_status apms_set_state(apms_ctx* ctx, apms_state_id which, int worker, const void* src_host);
 
-/* Restore the step counter and phase of a checkpoint (t = Adam steps taken so far). */
+/* Restore the Adam step counter and phase of a checkpoint (t = Adam steps taken so far; it sets the
+ * bias correction of the next warmup step).  Going to COMPRESSED from WARMUP freezes v as apms_freeze_v
+ * does; going back to WARMUP while the momentum is held as a server message first writes it out in
+ * binary32, which is what the Adam step reads.  A phase-wise step in progress is abandoned.
+ * The schedule's step counter is restored separately with apms_set_step. */
 apms_status apms_restore(apms_ctx* ctx, int t, apms_phase phase);
 
 /* Algorithm 1 end to end: T_w Adam steps, then compression-phase steps, with the learning rate
@@ -344,10 +348,19 @@ apms_status apms_set_schedule(apms_ctx* ctx, const apms_schedule* schedule);
 apms_status apms_step(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
 int64_t     apms_get_step(const apms_ctx* ctx);
 
+/* Set the step counter of apms_step (what apms_get_step returned when a checkpoint was taken), so that
+ * a restored context continues the schedule - the learning-rate ramp and decay of Section 5.2 and the
+ * T_w warmup steps of Algorithm 1 - where the saved one stopped instead of from step 0.  Call it after
+ * apms_restore: in the COMPRESSED phase the steps beyond t count as compression-phase steps taken,
+ * which fixes the variant and the compressor as they do in an uninterrupted run. */
+apms_status apms_set_step(apms_ctx* ctx, int64_t steps);
+
 /* Monitor for Assumption 1 (the compression errors stay bounded): squared l2 norms of the n
  * worker errors delta^(i) (worker_sq_host, n doubles, may be NULL) and of the server error
  * delta-bar (server_sq_host, may be NULL), summed in binary64 in a fixed order.  Reads every
- * compensated vector once ((n+1) d floats) and synchronises.  Phase must be COMPRESSED.  Not part of a step; call it as often as wanted. */
+ * compensated vector once ((n+1) d floats) and synchronises.  Phase must be COMPRESSED.  Not part of
+ * a step; call it as often as wanted.  With the top-k compressor the error of an element is its
+ * compensated value where it was not sent and zero where it was. */
 apms_status apms_error_norms(apms_ctx* ctx, double* worker_sq_host, double* server_sq_host);
 
 apms_phase  apms_get_phase(const apms_ctx* ctx);

@@ -20,7 +20,7 @@
  *     plus one scaling factor  |compensated vector| / |sign vector|, so that the
  *     decompressed vector has the magnitude of the compensated one.
  *
- * Readings taken where the paper is silent (all stated again in the design notes)
+ * Readings taken where the paper is silent
  *   - "magnitude" is the l2 norm (the paper's ||.||), so the scale of a chunk of
  *     length L is ||z||_2 / sqrt(L).  A mean-|z| scale is available as a switch.
  *   - sign(0) = +1 (bit 1), so the sign vector always has norm sqrt(L);

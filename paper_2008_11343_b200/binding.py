@@ -68,6 +68,7 @@ SIGNATURES = {
     "apms_set_schedule": (C.c_int, [C.c_void_p, C.c_void_p]),
     "apms_step": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_get_step": (C.c_int64, [C.c_void_p]),
+    "apms_set_step": (C.c_int, [C.c_void_p, C.c_int64]),
     "apms_error_norms": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "apms_get_phase": (C.c_int, [C.c_void_p]),
     "apms_get_t": (C.c_int, [C.c_void_p]),
@@ -275,6 +276,10 @@ def apms_step(h, grad_ptrs: Sequence[int], grad_type: int):
 
 def apms_get_step(h) -> int:
     return int(load().apms_get_step(h))
+
+
+def apms_set_step(h, steps: int):
+    _check(h, load().apms_set_step(h, steps))
 
 
 def apms_error_norms(h, n: int):
@@ -533,8 +538,11 @@ class Context:
     def error_norms(self):
         return apms_error_norms(self._h, self.n)
 
-    def restore(self, t: int, phase: int):
+    def restore(self, t: int, phase: int, steps: Optional[int] = None):
+        """Counters of a checkpoint: Adam steps t, phase, and (if given) the schedule's step counter."""
         apms_restore(self._h, t, phase)
+        if steps is not None:
+            apms_set_step(self._h, steps)
 
     @property
     def phase(self) -> int:

@@ -628,7 +628,6 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->steps = 0; c->has_sched = false; c->substep = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
     c->compressor = APMS_COMPRESSOR_ONEBIT; c->topk_frac = 0.01;
     c->fine_run = kFineRunDefault;
-    if (const char* e = getenv("APMS_FINE_RUN")) { const int r = atoi(e); if (r >= 1 && r <= (1 << 24)) c->fine_run = r; }   // tuning knob
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
     *out = c;
     return APMS_OK;
@@ -1058,7 +1057,24 @@ apms_status apms_restore(apms_ctx* c, int t, apms_phase phase)
         apms_status st = apms_freeze_v(c);
         if (st != APMS_OK) return st;
     }
-    c->t = t; c->phase = phase;
+    if (phase == APMS_PHASE_WARMUP && !c->m_is_fp32) {
+        // Adam reads the binary32 momentum: spell out the one held as a server message first
+        apms_status st = launch_materialise_momentum(c, c->m(), 0, c->L.d);
+        if (st != APMS_OK) return st;
+        c->m_is_fp32 = true;
+    }
+    c->t = t; c->phase = phase; c->substep = 0;
+    return APMS_OK;
+}
+
+apms_status apms_set_step(apms_ctx* c, int64_t steps)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    if (steps < 0) return fail(c, APMS_ERR_INVALID_ARG, "the step count cannot be negative");
+    c->steps = steps;
+    // compression-phase steps among them: what fixes the variant and the compressor
+    c->csteps = (c->phase == APMS_PHASE_COMPRESSED && steps > (int64_t)c->t) ? steps - (int64_t)c->t : 0;
     return APMS_OK;
 }
 
@@ -1111,6 +1127,7 @@ apms_status apms_error_norms(apms_ctx* c, double* worker_sq_host, double* server
     const int rows = c->L.n + 1;
     ErrNormArgs a;
     a.z = c->z(0); a.dz = c->L.dz; a.s = c->s(0); a.Cp = c->L.Cp; a.zbar = c->zbar(); a.Sbar = c->Sbar();
+    a.B = c->B(0); a.Wp = c->L.Wp; a.Bbar = c->Bbar(); a.topk = c->compressor == APMS_COMPRESSOR_TOPK ? 1 : 0;
     a.tiles = (c->L.d + 4095) / 4096; a.n = c->L.n; a.d = c->L.d; a.chunk = c->L.chunk;
     a.partial = reinterpret_cast<double*>(c->ws + c->L.off_mon);
     double* out = a.partial + (size_t)rows * (size_t)a.tiles;

@@ -8,7 +8,7 @@ namespace {
 // ------------------------------------------------------------------------------------------
 // Worker side again: the received chunk replaces the momentum (it stays in its compressed
 // form) and the model moves with the frozen variance (Section 3.3 steps 5-6).
-// One CTA per 8192 consecutive elements, whatever the chunk length.
+// One CTA per kApplyTile (4096) consecutive elements, whatever the chunk length.
 
 constexpr int kApplyTile = 4096;
 constexpr int kApplyU = kApplyTile / (kThreads * 4);

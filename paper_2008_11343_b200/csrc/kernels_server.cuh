@@ -198,8 +198,16 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
-// Barrier among the 256 consumer threads only (the producer warp never joins it).
-__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barrier among the 256 consumer threads only (the producer warp never joins it) that also ORs a flag
+// over them: every consumer gets the same answer, so a decision to leave taken on it is uniform even
+// when the flag it is fed from changes while the threads arrive.
+__device__ __forceinline__ bool consumer_barrier_any(bool flag)
+{
+    uint32_t any;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(any) : "r"(flag ? 1u : 0u) : "memory");
+    return any != 0;
+}
 
 struct ServerStagedArgs {
     ServerArgs a;
@@ -319,7 +327,9 @@ k_server_staged(const ServerStagedArgs sa)
         const int wl = lane >> 3;
         const int g0 = warp, g1 = warp + kWarps;
         // A warp whose wait gives up sets `failed`, skips the rest of its phase and still arrives at the next
-        // consumer barrier; after every barrier all consumers read `failed` and leave together.
+        // consumer barrier.  Each thread hands its own reading of `failed` to that barrier, which ORs them:
+        // all consumers see the same result and leave together, whenever the producer may have set the flag.
+        const volatile int* vfailed = &failed;
         int q = 0;
         for (int w = 0; w < nitems; ++w) {
             const Item it = decode_item(a.t, item0 + w);
@@ -329,8 +339,7 @@ k_server_staged(const ServerStagedArgs sa)
             for (int i = threadIdx.x; i < n; i += kThreads)
                 negs[i] = __float_as_uint(a.srow[i][it.c]) | 0x80000000u;
             const float S_old = a.Sbar[it.c];
-            consumer_barrier();                        // -s_i in place; everybody is done with the previous chunk
-            if (failed) break;
+            if (consumer_barrier_any(*vfailed != 0)) break;      // -s_i in place; everybody is done with the previous chunk
             bool ok = true;
             double acc = 0.0;
             for (int j = 0; j < nslabs; ++j, ++q) {
@@ -371,11 +380,11 @@ k_server_staged(const ServerStagedArgs sa)
             }
             acc = warp_sum(acc);
             if (lane == 0) red[warp] = acc;
-            consumer_barrier();                        // partial sums and sign words of the tile are in shared memory
+            const bool leave = consumer_barrier_any(!ok || *vfailed != 0);   // partial sums and sign words of the tile are in shared memory
             double total = 0.0;
 #pragma unroll
             for (int r = 0; r < kWarps; ++r) total += red[r];
-            if (failed) break;
+            if (leave) break;
             if (FUSED) {
                 // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
                 const float S_new = (float)sqrt(total / (double)it.Lc);

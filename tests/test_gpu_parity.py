@@ -20,14 +20,17 @@ def tiny(d, n, chunk, cfg_id=100, **kw):
 EDGE = [(1, 1, 32), (31, 2, 32), (32, 2, 32), (33, 3, 32), (127, 4, 128), (128, 4, 128), (129, 4, 128),
         (4095, 2, 4096), (4096, 2, 4096), (4097, 2, 4096), (1000, 5, 96), (12345, 3, 1024),
         (5 * 8192 + 77, 2, 8192), (3 * 65536 + 1, 2, 65536), (70000, 16, 160), (2050, 64, 2048),
-        (300000, 2, 131104), (4 * 70016, 4, 70016), (5000, 3, 1024), (40000, 2, 4096)]
+        (300000, 2, 131104), (4 * 70016, 4, 70016), (5000, 3, 1024), (40000, 2, 4096),
+        (3000, 32, 96), (9000, 12, 1024), (7 * 1056 + 31, 8, 1056)]
 
 
 # shapes for the staged forms (chunk a multiple of 2048): one slab, many slabs, ragged last slab and chunk,
 # split chunks, n not a power of two (IEEE division instead of the exact multiplication by 1/n), n = 64
 STAGED = [(2048, 1, 2048), (10 * 2048 + 1, 5, 2048), (6144 * 3 + 33, 7, 6144), (3 * 131072 + 4099, 3, 131072),
           (8 * 32768 + 23552, 16, 32768), (2 * 4096 + 2047, 64, 4096), (65536 + 2049, 2, 65536),
-          (3 * 512 + 100, 3, 512), (7 * 1536 + 511, 2, 1536), (9 * 4096 + 513, 4, 1024)]
+          (3 * 512 + 100, 3, 512), (7 * 1536 + 511, 2, 1536), (9 * 4096 + 513, 4, 1024),
+          (5 * 4096 + 100, 32, 4096), (3 * 2048 + 7, 12, 2048), (2 * 32768 + 1000, 32, 32768), (6 * 8192 + 5, 8, 8192),
+          (65536 + 4097, 32, 65536), (11 * 1024 + 9, 32, 1024)]
 
 
 @pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP, B.TEAM_AUTO, B.TEAM_STAGED],
@@ -39,6 +42,15 @@ def test_free_running_edge_sizes_bit_identical(d, n, chunk, team):
     bit-identical (the binary64 sums differ only in the order of additions)."""
     w = tiny(d, n, chunk, warmup_steps=3, compressed_steps=4)
     H.run_both(w, exact=True, team_mode=team)
+
+
+@pytest.mark.parametrize("n", [32, 16, 12, 8])
+def test_many_short_chunks_per_cta_bit_identical(n):
+    """Enough chunks that every CTA of the fused server kernel walks several of them (1200 chunks of 4096 on
+    148 SMs), at the worker counts the benchmark's sweep uses (each its own unrolled instantiation) and at one
+    count that takes the generic loop: the whole state bit-identical after free-running steps."""
+    w = tiny(1200 * 4096 + 777, n, 4096, cfg_id=111, warmup_steps=1, compressed_steps=3)
+    H.run_both(w, exact=True, check_every_step=False)
 
 
 def test_teacher_forced_steps_bits_exact():
@@ -501,9 +513,22 @@ def test_long_free_run_does_not_drift():
 
 def test_config1_mixed_tensors_zero_gradients():
     """d = 2^24 in 64 tensors with per-tensor scales over three decades and 20 % zero gradient
-    entries, n = 8, chunk = 8192 (steps reduced to keep the oracle's share of the run short)."""
+    entries, n = 8, chunk = 8192, free-running for the configuration's own 10 warmup + 50 compressed steps;
+    compared after the warmup phase, after the 10th compressed step and at the end."""
     w = wl.config(1)
-    H.run_both(w, warmup=3, compressed=5, check_every_step=False)
+    assert (w.warmup_steps, w.compressed_steps) == (10, 50)
+    ctx, orc = H.make_pair(w)
+    for step in range(w.warmup_steps):
+        gs = wl.host_gradients(w, step)
+        ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    H.compare_state(ctx, orc, w, phase_compressed=False)
+    ctx.freeze_v(); orc.freeze_v()
+    for k in range(w.compressed_steps):
+        gs = wl.host_gradients(w, w.warmup_steps + k)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        if k + 1 in (10, w.compressed_steps):
+            report = H.compare_state(ctx, orc, w)
+            assert report["server_tie_elems"] == 0
 
 
 def test_structural_zero_gradients_stay_finite():
@@ -624,6 +649,87 @@ def test_checkpoint_restore_continues_bit_identically():
         assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32))
     for i in range(w.n):
         assert np.array_equal(a.get_state(B.STATE_WORKER_ERR, i), b.get_state(B.STATE_WORKER_ERR, i))
+
+
+@pytest.mark.parametrize("stop_at", [2, 5])
+def test_checkpoint_under_a_schedule_resumes_the_learning_rate_and_the_warmup_count(stop_at):
+    """A run driven by apms_step is checkpointed in the middle of the learning-rate ramp - once still in the
+    warmup phase, once in the compression phase - and resumed in a fresh context: the resumed run must be
+    bit-identical to the uninterrupted one (same learning rates, same number of Adam steps, same phase switch)."""
+    w = tiny(4 * 1024 + 17, 3, 1024, cfg_id=112)
+    sc = B.Schedule(3, 2e-3, 8, 0.5, 2)                      # T_w = 3; ramp over 8 steps; then halve every 2 steps
+    a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    a.set_params(wl.initial_params(w))
+    a.set_schedule(sc)
+    for k in range(stop_at):
+        a.step(H.upload(wl.host_gradients(w, k)))
+    compressed = a.phase == B.PHASE_COMPRESSED
+    assert compressed == (stop_at > 3)
+    saved = {k: a.get_state(k) for k in (B.STATE_X, B.STATE_V, B.STATE_M)}
+    if compressed:
+        saved[B.STATE_SERVER_ERR] = a.get_state(B.STATE_SERVER_ERR)
+        werr = [a.get_state(B.STATE_WORKER_ERR, i) for i in range(w.n)]
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b.set_params(np.zeros(w.d, np.float32))
+    b.set_schedule(sc)
+    b.restore(a.t, a.phase, steps=a.steps_taken)
+    for k, val in saved.items():
+        b.set_state(k, val)
+    if compressed:
+        for i in range(w.n):
+            b.set_state(B.STATE_WORKER_ERR, werr[i], worker=i)
+    assert (b.t, b.phase, b.steps_taken) == (a.t, a.phase, a.steps_taken)
+    for k in range(stop_at, 12):
+        gs = H.upload(wl.host_gradients(w, k))
+        a.step(gs)
+        b.step(gs)
+    assert (b.t, b.phase, b.steps_taken) == (a.t, a.phase, a.steps_taken) == (3, B.PHASE_COMPRESSED, 12)
+    for k in (B.STATE_X, B.STATE_M, B.STATE_V, B.STATE_SERVER_ERR, B.STATE_SERVER_BITS, B.STATE_SERVER_SCALES):
+        assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32)), k
+    for i in range(w.n):
+        assert np.array_equal(a.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), b.get_state(B.STATE_WORKER_ERR, i).view(np.uint32))
+    if compressed:
+        with pytest.raises(B.ApmsError) as e:
+            b.set_variant(B.VARIANT_GRADIENT)                  # compression-phase steps count as taken after the restore
+        assert e.value.status == B.ERR_BAD_STATE
+
+
+def test_restore_to_warmup_spells_out_a_momentum_held_as_a_message():
+    """After compression-phase steps the momentum lives in the server's message.  Going back to the WARMUP phase
+    must hand Adam that momentum in binary32: the next Adam step equals the oracle's from the same state."""
+    w = tiny(3 * 2048 + 40, 2, 2048, cfg_id=113)
+    ctx, orc, _ = H.run_both(w, warmup=2, compressed=3, check_every_step=False, exact=True)
+    ctx.restore(2, B.PHASE_WARMUP)
+    fresh = ao.Oracle(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    fresh.set_params(orc.x.copy())
+    gs = wl.host_gradients(w, 0)
+    fresh.warmup_step(gs); fresh.warmup_step(gs)               # brings its t to 2; its state is replaced next
+    fresh.x[:] = orc.x; fresh.m[:] = orc.m; fresh.v[:] = orc.v
+    gs = wl.host_gradients(w, 9)
+    ctx.warmup_step(H.upload(gs)); fresh.warmup_step(gs)
+    assert ctx.t == 3
+    for which, ref in ((B.STATE_X, fresh.x), (B.STATE_M, fresh.m), (B.STATE_V, fresh.v)):
+        assert np.array_equal(ctx.get_state(which).view(np.uint32), ref.view(np.uint32)), which
+
+
+def test_error_norms_with_the_topk_compressor():
+    """Top-k mode keeps masks where the 1-bit mode keeps scales: the monitor must use delta = z where not sent."""
+    w = tiny(5 * 4096 + 300, 3, 4096, cfg_id=114)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, 0.03)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(0.03)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(1, 4):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+    workers, server = ctx.error_norms()
+    for i in range(w.n):
+        ref = float(np.sum(orc.worker_err(i).astype(np.float64) ** 2))
+        assert ref > 0 and abs(workers[i] - ref) <= 1e-12 * ref
+    ref = float(np.sum(orc.server_err.astype(np.float64) ** 2))
+    assert ref > 0 and abs(server - ref) <= 1e-12 * ref
 
 
 def test_state_slices_agree_with_full_arrays():

@@ -1,11 +1,12 @@
-"""The allocation-free entry point, apms_compress_noalloc, against the ordinary path.
+"""The allocation-free entry point, apms_compress_noalloc, against the ordinary path and the CPU oracle.
 
 Some callers of this library cannot allocate device memory: a step function running inside a
 framework region where allocator calls are forbidden, a plugin that owns nothing but the buffers
 and the stream it was handed, a loop that cannot tolerate the device-wide synchronisation a
 cudaMalloc implies.  For them the library compresses a vector using only a fixed scratch array
 that is part of the library itself.  This test drives that entry point through the C ABI and
-requires the same sign words and scales as the context-based step produces for the same vector,
+requires the same sign words and scales as the context-based step produces for the same vector -
+and as the CPU oracle's compressor (Section 5.1) gives chunk by chunk -
 on two calls issued back to back (the second must not be disturbed by what the first left in
 the shared scratch array), and requires that oversize shapes are refused with a message.
 
@@ -17,6 +18,7 @@ import pytest
 
 pytestmark = pytest.mark.gpu
 
+from oracle import apms_oracle as ao
 from paper_2008_11343_b200 import binding as B
 
 REL = 1e-5      # the scale tolerance of the parity tests; sign words must be equal
@@ -35,6 +37,17 @@ def _reference(z: np.ndarray, chunk: int):
     bits, scales = ctx.get_state(B.STATE_WORKER_BITS, 0), ctx.get_state(B.STATE_WORKER_SCALES, 0)
     ctx.close()
     return bits, scales
+
+
+def _oracle(z: np.ndarray, chunk: int):
+    """Sign words and scales of z from the CPU oracle's 1-bit compressor, one chunk at a time."""
+    bits = np.zeros((z.size + 31) // 32, np.uint32)
+    scales = []
+    for lo in range(0, z.size, chunk):
+        b, s = ao.compress_1bit(z[lo:lo + chunk])
+        bits[lo // 32:lo // 32 + b.size] = b          # chunks are multiples of 32 elements: whole words
+        scales.append(s)
+    return bits, np.asarray(scales, np.float32)
 
 
 def _vector(d: int, seed: int) -> np.ndarray:
@@ -78,6 +91,9 @@ def test_two_calls_in_a_row_match_the_context_path():
         got_bits = bits.cpu().numpy().view(np.uint32)
         assert np.array_equal(got_bits, ref_bits), f"d={d} chunk={chunk}: sign words differ"
         np.testing.assert_allclose(scales.cpu().numpy(), ref_scales, rtol=REL, atol=0)
+        orc_bits, orc_scales = _oracle(z, chunk)
+        assert np.array_equal(got_bits, orc_bits), f"d={d} chunk={chunk}: sign words differ from the oracle's"
+        np.testing.assert_allclose(scales.cpu().numpy(), orc_scales, rtol=REL, atol=0)
         assert np.array_equal(zdev.cpu().numpy(), z)                       # the input is not modified
 
 

@@ -250,6 +250,14 @@ apms_status apms_compressed_step_host_typed(apms_ctx* ctx, const void* const* gr
  * apms_get_message: device addresses of worker i's message (worker = -1: the server's), valid
  * while the workspace lives; the buffers hold W words / C scales, rows padded to 256 bytes. */
 apms_status apms_worker_phase(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type);
+/* The worker phase over chunks [chunk_begin, chunk_end) only (Section 3.3 steps 1-2 are independent per
+ * chunk): after the call - in stream order - that part of every worker's message is final, so the caller
+ * can hand it to the process that serves those chunks while the rest of the vector is still being
+ * compressed (Section 3.3 step 3, Figure 1a).  One step's calls must cover every chunk exactly once, in any
+ * order, with the same gradients; the server phases may follow once they do.  apms_worker_phase is the
+ * call for [0, C). */
+apms_status apms_worker_phase_range(apms_ctx* ctx, const void* const* grads_dev, apms_grad_type type,
+                                    int64_t chunk_begin, int64_t chunk_end);
 apms_status apms_get_message(apms_ctx* ctx, int worker, uint32_t** bits_dev, float** scales_dev);
 apms_status apms_server_phase(apms_ctx* ctx, const uint32_t* bits_rows_dev, int64_t row_words,
                               const float* scale_rows_dev, int64_t row_scales, int rows,
@@ -262,8 +270,10 @@ apms_status apms_apply_phase(apms_ctx* ctx);
  *
  *   exchange 1 is the server kernel reading: apms_server_phase_rows takes one pair of device
  *     pointers per sender - bits_rows[j] the address of row j's sign word of the first element of
- *     chunk chunk_begin (inside a message buffer whose word 0 is 16-byte aligned, as the
- *     library's are), scale_rows[j] the address of its scale of chunk chunk_begin - and loads
+ *     chunk chunk_begin (inside a message buffer padded as the library's are; the kernel that
+ *     streams the rows with bulk copies runs when all rows lie at the same distance from a 16-byte
+ *     boundary, as rows of equally shaped contexts do), scale_rows[j] the address of its scale of
+ *     chunk chunk_begin - and loads
  *     the rows where they lie, this GPU's memory or a mapped peer's.  A
  *     peer worker's row is (mapped base of its process) + apms_message_offsets(worker) + the range's
  *     offset; contexts created with the same d, n, chunk have the same offsets.  Both arrays are

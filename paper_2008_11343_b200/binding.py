@@ -50,6 +50,7 @@ SIGNATURES = {
     "apms_compressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_compressed_step_host_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int, C.c_void_p]),
     "apms_worker_phase": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
+    "apms_worker_phase_range": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int, C.c_int64, C.c_int64]),
     "apms_get_message": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
     "apms_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64]),
     "apms_apply_phase": (C.c_int, [C.c_void_p]),
@@ -175,6 +176,10 @@ def apms_compressed_step_host_typed(h, grad_host_ptrs: Sequence[int], grad_type:
 
 def apms_worker_phase(h, grad_ptrs: Sequence[int], grad_type: int):
     _check(h, load().apms_worker_phase(h, _ptr_array(grad_ptrs), grad_type))
+
+
+def apms_worker_phase_range(h, grad_ptrs: Sequence[int], grad_type: int, chunk_begin: int, chunk_end: int):
+    _check(h, load().apms_worker_phase_range(h, _ptr_array(grad_ptrs), grad_type, chunk_begin, chunk_end))
 
 
 def apms_get_message(h, worker: int):
@@ -479,6 +484,11 @@ class Context:
         assert len(grads) == self.n
         apms_worker_phase(self._h, self._dev_ptrs(grads), self._grad_type(grads))
 
+    def worker_phase_range(self, grads, chunk_begin: int, chunk_end: int):
+        """Steps 1-2 for chunks [chunk_begin, chunk_end) only; one step's ranges must cover every chunk once."""
+        assert len(grads) == self.n
+        apms_worker_phase_range(self._h, self._dev_ptrs(grads), self._grad_type(grads), chunk_begin, chunk_end)
+
     def message(self, worker: int):
         """Torch views (int32 sign words [W], float32 scales [C]) onto worker `worker`'s message inside the
         workspace (-1: the server's message).  No copy: the library writes these buffers."""
@@ -522,6 +532,14 @@ class Context:
 
     def synchronize(self):
         self.stream.synchronize()
+
+    def record_event(self):
+        """A torch CUDA event recorded on the context's stream (its synchronize() waits for the work enqueued so far)."""
+        import torch
+
+        ev = torch.cuda.Event()
+        ev.record(self.stream)
+        return ev
 
     def set_schedule(self, schedule: Optional[Schedule]):
         apms_set_schedule(self._h, schedule)

@@ -56,6 +56,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
     int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
+    int fine_split;
     int n;
     Tiling t;
     size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
@@ -87,8 +88,9 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
     L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
-    L->fine_tiles = (chunk % kFineSub == 0) ? (d + kFineTile - 1) / kFineTile : 0;
-    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles * kWarps, 64);
+    L->fine_tiles = (chunk >= kFineSub) ? (d + kFineTile - 1) / kFineTile : 0;
+    L->fine_split = (chunk % kFineSub != 0) ? 1 : 0;     // a warp's 512 elements may lie in two chunks: two partial sums each
+    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles * kWarps * (size_t)(L->fine_split ? 2 : 1), 64);
     L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
     L->off_stage = take((size_t)L->dz * 4 * 2);
     L->off_mon = take(((size_t)(n + 1) * (size_t)((d + 4095) / 4096) + (size_t)(n + 1)) * 8);   // error monitor: tile sums + row sums
@@ -112,7 +114,8 @@ struct apms_ctx {
     double topk_frac;        // top-k: fraction of a chunk that is sent
     int variant;             // APMS_VARIANT_*: what the workers compress
     int64_t csteps;          // compression-phase steps taken (the variant is fixed once one has run)
-    int substep;             // phase-wise step: 0 = between steps, 1 = worker phase done, 2 = a server phase done
+    int substep;             // phase-wise step: 0 = between steps, 1 = in or past the worker phase, 2 = a server phase done
+    int64_t worker_chunks;   // phase-wise step: chunks the worker phase has covered so far
     apms_schedule sched; bool has_sched;
     apms_phase phase;
     bool m_is_fp32;          // momentum lives in the binary32 buffer (else in Bbar/Sbar; top-k: in zbar under the mask Bbar)
@@ -239,13 +242,20 @@ apms_status device_status_check(apms_ctx* c)
     return APMS_OK;
 }
 
-// The staged server kernel needs every 2048-element slab of a tile to start on a 16-byte boundary
-// in zbar and in the sign words, i.e. chunks that are multiples of 2048 elements.
+// The staged server kernel streams slabs of 2048 elements: chunks of at least one slab.
 bool use_staged_server(const apms_ctx* c)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
     if (c->L.t.l1) return false;             // the mean-|z| scale exists in the register-staged kernels only
-    return c->L.chunk % kSlab == 0;
+    return c->L.chunk >= kSlab;
+}
+
+// Chunks of 128, 256, 512 or 1024 elements: whole chunks per slab, the fused kernel k_server_packed.
+bool use_packed_server(const apms_ctx* c)
+{
+    if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
+    if (c->L.t.l1) return false;
+    return c->L.chunk >= kGroup && c->L.chunk < kSlab && kSlab % c->L.chunk == 0;
 }
 
 bool use_warp_teams(const apms_ctx* c, int64_t items)
@@ -255,22 +265,28 @@ bool use_warp_teams(const apms_ctx* c, int64_t items)
     return items / kWarps >= (int64_t)kWarpTeamMinCtasPerSm * c->sms;
 }
 
-apms_status launch_finalize(apms_ctx* c, int first_row, int rows, float* scales)
+// Scales of the split chunks [cb, ce) of `rows` workers from first_row on: the range as a vector of its own.
+apms_status launch_finalize(apms_ctx* c, int first_row, int rows, int64_t cb, int64_t ce)
 {
-    const int64_t total = (int64_t)rows * c->L.C;
-    k_finalize_scales<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->partial(first_row), scales, rows,
-                                                                            c->L.C, c->L.Cp, c->L.t);
+    const int64_t nchunks = ce - cb;
+    const int64_t total = (int64_t)rows * nchunks;
+    Tiling t = c->L.t;
+    t.d = c->L.d - cb * c->L.chunk;
+    k_finalize_scales<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->partial(first_row) + cb * c->L.t.P, c->s(first_row) + cb, rows,
+                                                                            nchunks, c->L.Cp, t);
     return launch_check(c, "k_finalize_scales");
 }
 
-bool use_fine_worker(const apms_ctx* c)
+bool use_fine_worker(const apms_ctx* c, bool whole_vector)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
     if (c->L.t.l1) return false;             // see use_staged_server
+    if (!whole_vector && c->L.fine_split) return false;      // a range of chunks must end between two warps' pieces
     return (!c->m_is_fp32 || c->variant == APMS_VARIANT_GRADIENT) && c->L.fine_tiles > 0;
 }
 
-apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
+// Workers i0 .. i0+ni-1 on chunks [cb, ce).
+apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni, int64_t cb, int64_t ce)
 {
     WorkerFineArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
@@ -278,33 +294,45 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     a.s = c->s(0); a.Cp = c->L.Cp;
     a.partial = c->fine_partial(i0); a.Pp = c->L.fine_Pp;
     a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
-    a.d = c->L.d; a.chunk = c->L.chunk; a.tiles = c->L.fine_tiles;
+    a.d = c->L.d; a.chunk = c->L.chunk;
+    a.e0 = cb * c->L.chunk; a.e1 = ce * c->L.chunk < c->L.d ? ce * c->L.chunk : c->L.d;
+    a.tile0 = a.e0 / kFineTile; a.tiles = (a.e1 + kFineTile - 1) / kFineTile - a.tile0;
     a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
     a.run = c->fine_run;
+    if ((int64_t)a.run > a.tiles) a.run = a.tiles < 1 ? 1 : (int)a.tiles;
     const int64_t stretches = (a.tiles + a.run - 1) / a.run;
     const int64_t blocks = stretches * a.run * ni;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
     {
         Timed t(c, APMS_KERNEL_WORKER);
-        if (c->variant == APMS_VARIANT_GRADIENT) APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
-        else                                     APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+        const bool sendg = c->variant == APMS_VARIANT_GRADIENT;
+        if (c->L.fine_split) {
+            if (sendg) APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, true, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+            else       APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, false, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+        } else {
+            if (sendg) APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, true, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+            else       APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, false, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+        }
         apms_status st = launch_check(c, "k_worker_fine");
         if (st != APMS_OK) return st;
-        const int64_t total = (int64_t)ni * c->L.C;
-        const int64_t slots = c->L.chunk / kFineSub;                 // partial sums of a whole chunk
+        const int64_t nchunks = ce - cb;
+        const int64_t total = (int64_t)ni * nchunks;
+        const int per = c->L.fine_split ? 2 : 1;
+        // 512-element pieces a whole chunk can touch: its own, plus one at each end that it shares
+        const int64_t slots = c->L.fine_split ? c->L.chunk / kFineSub + 2 : c->L.chunk / kFineSub;
         int team = 1;
         while (team < 32 && team < slots) team *= 2;
         const int64_t per_cta = (int64_t)kWarps * (32 / team);
         const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
         const double* part = c->fine_partial(i0);
         switch (team) {
-        case 1:  k_finalize_fine<1><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
-        case 2:  k_finalize_fine<2><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
-        case 4:  k_finalize_fine<4><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
-        case 8:  k_finalize_fine<8><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
-        case 16: k_finalize_fine<16><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
-        default: k_finalize_fine<32><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, c->L.C, c->L.d, c->L.chunk); break;
+        case 1:  k_finalize_fine<1><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
+        case 2:  k_finalize_fine<2><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
+        case 4:  k_finalize_fine<4><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
+        case 8:  k_finalize_fine<8><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
+        case 16: k_finalize_fine<16><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
+        default: k_finalize_fine<32><<<grid, kThreads, 0, c->stream>>>(part, c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks, c->L.d, c->L.chunk, per); break;
         }
         st = launch_check(c, "k_finalize_fine");
         if (st != APMS_OK) return st;
@@ -328,10 +356,13 @@ apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     return launch_check(c, "k_topk_worker");
 }
 
-apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
+// Section 3.3 steps 1-2 for workers i0 .. i0+ni-1 on chunks [cb, ce).
+apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni, int64_t cb, int64_t ce)
 {
-    if (c->compressor == APMS_COMPRESSOR_TOPK) return launch_worker_topk(c, G, gtype, i0, ni);
-    if (use_fine_worker(c)) return launch_worker_fine(c, G, gtype, i0, ni);
+    const bool whole = cb == 0 && ce == c->L.C;
+    if (c->compressor == APMS_COMPRESSOR_TOPK) return launch_worker_topk(c, G, gtype, i0, ni);      // whole vector only (checked by the callers)
+    if (ce <= cb) return APMS_OK;
+    if (use_fine_worker(c, whole)) return launch_worker_fine(c, G, gtype, i0, ni, cb, ce);
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
     a.B = c->B(0); a.Wp = c->L.Wp;
@@ -339,7 +370,8 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int
     a.partial = c->partial(0);
     a.m32 = c->m(); a.Bbar = c->Bbar(); a.Sbar = c->Sbar();
     a.t = c->L.t; a.i0 = i0; a.ni = ni;
-    a.items = c->L.C * c->L.t.P * ni;
+    a.tile0 = cb * c->L.t.P;
+    a.items = (ce - cb) * c->L.t.P * ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
     a.send_gradient = c->variant == APMS_VARIANT_GRADIENT;
     const bool warp_teams = use_warp_teams(c, a.items);
@@ -358,7 +390,7 @@ apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int
         apms_status st = launch_check(c, "k_worker");
         if (st != APMS_OK) return st;
     }
-    if (c->L.t.P > 1) return launch_finalize(c, i0, ni, c->s(i0));
+    if (c->L.t.P > 1) return launch_finalize(c, i0, ni, cb, ce);
     return APMS_OK;
 }
 
@@ -376,6 +408,27 @@ cudaError_t launch_staged(const ServerStagedArgs& sa, unsigned blocks, size_t sm
         k_server_staged<NT, FUSED, false><<<blocks, kStagedThreads, smem, stream>>>(sa);
     }
     return cudaSuccess;
+}
+
+template <int NT>
+cudaError_t launch_packed(const ServerStagedArgs& sa, unsigned blocks, size_t smem, cudaStream_t stream)
+{
+    cudaError_t e = cudaFuncSetAttribute(k_server_packed<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_server_packed<NT><<<blocks, kStagedThreads, smem, stream>>>(sa);
+    return cudaSuccess;
+}
+
+cudaError_t launch_packed_n(const ServerStagedArgs& sa, unsigned blocks, size_t smem, cudaStream_t stream)
+{
+    switch (sa.a.n) {
+    case 2:  return launch_packed<2>(sa, blocks, smem, stream);
+    case 4:  return launch_packed<4>(sa, blocks, smem, stream);
+    case 8:  return launch_packed<8>(sa, blocks, smem, stream);
+    case 16: return launch_packed<16>(sa, blocks, smem, stream);
+    case 32: return launch_packed<32>(sa, blocks, smem, stream);
+    default: return launch_packed<0>(sa, blocks, smem, stream);
+    }
 }
 
 template <bool FUSED>
@@ -411,6 +464,15 @@ struct ServerSource {
     const uint32_t* B[APMS_MAX_WORKERS];
     const float* s[APMS_MAX_WORKERS];
     int rows;
+    // Distance of every row's word 0 from a 16-byte boundary, in words, if all rows share it (what the staged
+    // kernel's bulk copies need); -1 otherwise.
+    int common_alignment() const
+    {
+        const int first = (int)(((uintptr_t)B[0] >> 2) & 3u);
+        for (int j = 1; j < rows; ++j)
+            if ((int)(((uintptr_t)B[j] >> 2) & 3u) != first) return -1;
+        return first;
+    }
     // rows at a fixed stride from a base
     static ServerSource strided(const uint32_t* B0, int64_t Wp, const float* s0, int64_t Cp, int rows)
     {
@@ -436,7 +498,32 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
     a.t = c->L.t; a.item0 = cb * c->L.t.P; a.items = ce * c->L.t.P; a.n = src.rows; a.nf = (float)src.rows;
     const int64_t count = a.items - a.item0;
     if (count <= 0) return APMS_OK;
-    const bool staged = use_staged_server(c);
+    const int row_align = src.common_alignment();
+    if (may_fuse && use_packed_server(c) && row_align >= 0 && cb == 0 && ce == c->L.C) {
+        // short chunks, several per slab: the fused kernel for them (items are slabs of the whole vector)
+        apms_status dst = ensure_den(c);
+        if (dst != APMS_OK) return dst;
+        ServerStagedArgs sa;
+        sa.a = a; sa.status = c->status();
+        sa.a.item0 = 0; sa.a.items = (c->L.d + kSlab - 1) / kSlab;
+        sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
+        sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr; sa.row_align = row_align;
+        const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, true);
+        sa.span = (int)(kStagedSpanElems / kSlab);
+        const int64_t fill = sa.a.items / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
+        if (fill < sa.span) sa.span = fill < 1 ? 1 : (int)fill;
+        const int64_t ctas = (sa.a.items + sa.span - 1) / sa.span;
+        if (ctas > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many slabs for one launch");
+        Timed t(c, APMS_KERNEL_SERVER);
+        cudaError_t e = launch_packed_n(sa, (unsigned)ctas, smem, c->stream);
+        if (e != cudaSuccess) {
+            snprintf(c->err, sizeof c->err, "setting up k_server_packed failed: %s", cudaGetErrorString(e));
+            return APMS_ERR_CUDA;
+        }
+        *applied = true;
+        return launch_check(c, "k_server_packed");
+    }
+    const bool staged = use_staged_server(c) && row_align >= 0;
     const bool warp_teams = !staged && use_warp_teams(c, count);
     const int64_t blocks = warp_teams ? (count + kWarps - 1) / kWarps : count;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
@@ -451,7 +538,7 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
             ServerStagedArgs sa;
             sa.a = a; sa.status = c->status();
             sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
-            sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr;
+            sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr; sa.row_align = row_align;
             const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
             sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
             const int64_t fill = count / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
@@ -625,7 +712,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
     c->team_mode = APMS_TEAM_AUTO;
-    c->steps = 0; c->has_sched = false; c->substep = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
+    c->steps = 0; c->has_sched = false; c->substep = 0; c->worker_chunks = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
     c->compressor = APMS_COMPRESSOR_ONEBIT; c->topk_frac = 0.01;
     c->fine_run = kFineRunDefault;
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
@@ -661,7 +748,7 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
-    c->t = 0; c->steps = 0; c->csteps = 0; c->substep = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
+    c->t = 0; c->steps = 0; c->csteps = 0; c->substep = 0; c->worker_chunks = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
     return APMS_OK;
 }
 
@@ -725,7 +812,7 @@ apms_status apms_compressed_step_typed(apms_ctx* c, const void* const* grads_dev
     GradPtrs G;
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
-    st = launch_worker(c, G, (int)type, 0, c->L.n);
+    st = launch_worker(c, G, (int)type, 0, c->L.n, 0, c->L.C);
     if (st != APMS_OK) return st;
     return launch_server_and_apply(c);
 }
@@ -733,15 +820,26 @@ apms_status apms_compressed_step_typed(apms_ctx* c, const void* const* grads_dev
 apms_status apms_worker_phase(apms_ctx* c, const void* const* grads_dev, apms_grad_type type)
 {
     if (!c) return APMS_ERR_INVALID_ARG;
+    return apms_worker_phase_range(c, grads_dev, type, 0, c->L.C);
+}
+
+apms_status apms_worker_phase_range(apms_ctx* c, const void* const* grads_dev, apms_grad_type type, int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_worker_phase needs the COMPRESSED phase (call apms_freeze_v first)");
-    if (c->substep != 0) return fail(c, APMS_ERR_BAD_STATE, "the previous phase-wise step is not finished (apms_apply_phase)");
+    if (c->substep > 1 || (c->substep == 1 && c->worker_chunks >= c->L.C))
+        return fail(c, APMS_ERR_BAD_STATE, "the worker phase of this step is complete (continue with the server and apply phases)");
     if (c->compressor != APMS_COMPRESSOR_ONEBIT) return fail(c, APMS_ERR_BAD_STATE, "the phase-wise step exists for the 1-bit compressor only");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (c->worker_chunks + (chunk_end - chunk_begin) > c->L.C) return fail(c, APMS_ERR_INVALID_ARG, "the ranges of one step's worker phase cover more chunks than there are");
     GradPtrs G;
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
     if (st != APMS_OK) return st;
-    st = launch_worker(c, G, (int)type, 0, c->L.n);
-    if (st == APMS_OK) c->substep = 1;
-    return st;
+    st = launch_worker(c, G, (int)type, 0, c->L.n, chunk_begin, chunk_end);
+    if (st != APMS_OK) return st;
+    c->worker_chunks += chunk_end - chunk_begin;
+    c->substep = 1;
+    return APMS_OK;
 }
 
 apms_status apms_get_message(apms_ctx* c, int worker, uint32_t** bits_dev, float** scales_dev)
@@ -760,7 +858,7 @@ apms_status apms_server_phase(apms_ctx* c, const uint32_t* bits_rows_dev, int64_
 {
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase needs the COMPRESSED phase");
-    if (c->substep < 1) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase follows apms_worker_phase");
+    if (c->substep < 1 || c->worker_chunks < c->L.C) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase follows a complete worker phase (every chunk once)");
     if (!bits_rows_dev || !scale_rows_dev) return fail(c, APMS_ERR_INVALID_ARG, "a message pointer is NULL");
     if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
     if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
@@ -784,7 +882,7 @@ apms_status apms_server_phase_rows(apms_ctx* c, const uint32_t* const* bits_rows
 {
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows needs the COMPRESSED phase");
-    if (c->substep < 1) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows follows apms_worker_phase");
+    if (c->substep < 1 || c->worker_chunks < c->L.C) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows follows a complete worker phase (every chunk once)");
     if (!bits_rows || !scale_rows) return fail(c, APMS_ERR_INVALID_ARG, "a pointer array is NULL");
     if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
     if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
@@ -796,7 +894,7 @@ apms_status apms_server_phase_rows(apms_ctx* c, const uint32_t* const* bits_rows
         // kernels index by absolute word / chunk: shift the row's pointers back to where index 0 would be
         src.B[j] = bits_rows[j] - first_elem / 32;
         src.s[j] = scale_rows[j] - chunk_begin;
-        if (((uintptr_t)src.B[j] & 15u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "a sign-word row does not belong to a 16-byte aligned message buffer");
+        if (((uintptr_t)src.B[j] & 3u) != 0) return fail(c, APMS_ERR_INVALID_ARG, "a sign-word row is not 4-byte aligned");
     }
     src.rows = rows;
     bool applied = false;
@@ -883,7 +981,7 @@ apms_status apms_apply_phase(apms_ctx* c)
     if (st != APMS_OK) return st;
     c->m_is_fp32 = c->variant == APMS_VARIANT_GRADIENT;
     c->csteps += 1;
-    c->substep = 0;
+    c->substep = 0; c->worker_chunks = 0;
     return APMS_OK;
 }
 
@@ -922,7 +1020,7 @@ apms_status apms_compressed_step_host_typed(apms_ctx* c, const void* const* grad
         APMS_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
         GradPtrs G;
         G.p[0] = c->stage(b);
-        apms_status st = launch_worker(c, G, (int)type, i, 1);
+        apms_status st = launch_worker(c, G, (int)type, i, 1, 0, c->L.C);
         if (st != APMS_OK) return st;
         APMS_CUDA(c, cudaEventRecord(c->ev_used[b], c->stream));
     }
@@ -1063,7 +1161,7 @@ apms_status apms_restore(apms_ctx* c, int t, apms_phase phase)
         if (st != APMS_OK) return st;
         c->m_is_fp32 = true;
     }
-    c->t = t; c->phase = phase; c->substep = 0;
+    c->t = t; c->phase = phase; c->substep = 0; c->worker_chunks = 0;
     return APMS_OK;
 }
 

@@ -132,12 +132,18 @@ k_server(const ServerArgs a)
 // When the tile is the whole chunk, the CTA goes on to steps 5-6 for the same chunk (its new
 // scale is known once the eight consumer warps have met): v and x travel through the same ring
 // while other CTAs of the SM are still in their arithmetic-bound averaging phase.
-// Needs every slab of kSlab elements to start on a 16-byte boundary in all streams, i.e.
-// chunks that are multiples of kSlab; other shapes use k_server and k_apply.
+// Bulk copies start on 16-byte boundaries.  Every slab of zbar, v and x does (chunks are multiples of
+// 32 elements); a chunk's first sign word need not.  The rows of sign words are therefore copied from
+// the 16-byte boundary at or below the slab's first word - up to three words early - and everything
+// held in shared memory as sign words (the rows and the tile's new words) is indexed by the distance
+// from that boundary, so that whole 16-byte pieces in shared memory are whole 16-byte pieces in global
+// memory.  All rows of a launch must share one alignment (`row_align`); chunks shorter than a slab use
+// k_server and k_apply.
 
 constexpr int kSlab = 2048;                      // elements per ring stage
 constexpr int kSlabGroups = kSlab / kGroup;      // 16 groups, two per consumer warp
 constexpr int kSlabWords = kSlab / 32;           // 64 sign words per worker and slab
+constexpr int kRowWords = kSlabWords + 4;        // a row in shared memory: up to three words before the slab's first, rounded to 16 bytes
 constexpr int kStages = 4;
 constexpr int64_t kStagedSpanElems = 32768;   // a CTA of the fused form walks enough chunks to stream about this many elements
 constexpr int kStagedThreads = kThreads + 32;    // eight consumer warps + one producer warp
@@ -215,12 +221,13 @@ struct ServerStagedArgs {
     float inv_n;          // 1/n when n is a power of two (then avg = sum * inv_n is the exact quotient), else 0
     const float* den; float* x; float lr;        // steps 5-6 (fused form only): den = sqrt(v) + eps, see k_make_den
     int span;             // chunks per CTA of the fused form
+    int row_align;        // (address of every row's word 0 / 4) mod 4: the rows' common distance from a 16-byte boundary, in words
 };
 
 // Bytes of one ring stage: a slab of zbar plus n rows of sign words, or (fused form) a slab of v and of x.
 __host__ __device__ __forceinline__ size_t staged_stage_bytes(int n, bool fused)
 {
-    const size_t server = (size_t)kSlab * 4 + (size_t)n * kSlabWords * 4;
+    const size_t server = (size_t)kSlab * 4 + (size_t)n * kRowWords * 4;
     const size_t apply = (size_t)kSlab * 8;
     return (fused && apply > server) ? apply : server;
 }
@@ -237,8 +244,8 @@ __device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r
     for (int i = 0; i < nn; ++i) {
         const uint32_t ns = neg_s[i];
         // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
-        const uint32_t y0 = r0[i * kSlabWords] << (28 - sh);
-        const uint32_t y1 = r1[i * kSlabWords] << (28 - sh);
+        const uint32_t y0 = r0[i * kRowWords] << (28 - sh);
+        const uint32_t y1 = r1[i * kRowWords] << (28 - sh);
         float2 q;
         q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns);
         s01 = __fadd2_rn(s01, q);
@@ -264,7 +271,7 @@ k_server_staged(const ServerStagedArgs sa)
     __shared__ double red[kWarps];
     __shared__ uint64_t full[kStages], empty[kStages];
     __shared__ uint32_t neg_s[2][APMS_MAX_WORKERS];   // bit patterns of -s_i, double-buffered over the walk
-    __shared__ uint32_t nb[kTileMax / 32];            // the current tile's new sign words
+    __shared__ __align__(16) uint32_t nb[kTileMax / 32 + 4];   // the current tile's new sign words, from the 16-byte boundary below the first
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -302,12 +309,13 @@ k_server_staged(const ServerStagedArgs sa)
                     const int live = left < kSlab ? left : kSlab;
                     const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
                     if (r < nslabs) {
-                        const uint32_t wbytes = (uint32_t)(((live + 31) / 32 + 3) / 4) * 16u;
+                        const int off_in = (int)((wofs + sa.row_align) & 3);       // words between the 16-byte boundary and the slab's first word
+                        const uint32_t wbytes = (uint32_t)((off_in + (live + 31) / 32 + 3) / 4) * 16u;
                         mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
                         bulk_load(base, zb_g + (size_t)j * kSlab, zbytes, &full[st]);
                         uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
                         for (int i = 0; i < n; ++i)
-                            bulk_load(rows + i * kSlabWords, a.Brow[i] + wofs + (size_t)j * kSlabWords, wbytes, &full[st]);
+                            bulk_load(rows + i * kRowWords, a.Brow[i] + (wofs - off_in) + (size_t)j * kSlabWords, wbytes, &full[st]);
                     } else {
                         mbar_arrive_expect_tx(&full[st], 2 * zbytes);
                         bulk_load(base, sa.den + it.base + (size_t)j * kSlab, zbytes, &full[st]);
@@ -335,6 +343,8 @@ k_server_staged(const ServerStagedArgs sa)
             const Item it = decode_item(a.t, item0 + w);
             const int L = it.L;
             const int nslabs = (L + kSlab - 1) / kSlab;
+            const int64_t wofs = it.base / 32;
+            const int off_in = (int)((wofs + sa.row_align) & 3), off_out = (int)(wofs & 3);
             uint32_t* negs = neg_s[w & 1];
             for (int i = threadIdx.x; i < n; i += kThreads)
                 negs[i] = __float_as_uint(a.srow[i][it.c]) | 0x80000000u;
@@ -351,7 +361,7 @@ k_server_staged(const ServerStagedArgs sa)
                 const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
                 const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
                 float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
-                signed_scale_sums<NT>(rows + g0 * 4 + wl, rows + g1 * 4 + wl, negs, n, sh, s01, s23, t01, t23);
+                signed_scale_sums<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl, negs, n, sh, s01, s23, t01, t23);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
 #pragma unroll
@@ -375,7 +385,7 @@ k_server_staged(const ServerStagedArgs sa)
                     }
                     st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
                     const uint32_t word = pack_group_words(nibble, lane);
-                    if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
+                    if ((lane & 7) == 0) nb[off_out + grp * 4 + wl] = word;   // words past L hold zeros and are never stored
                 }
             }
             acc = warp_sum(acc);
@@ -407,7 +417,7 @@ k_server_staged(const ServerStagedArgs sa)
                     for (int u = 0; u < 2; ++u) {
                         const int grp = j * kSlabGroups + (u ? g1 : g0);
                         const int k = grp * kGroup + lane * 4;
-                        const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                        const uint32_t nib = nb[off_out + grp * 4 + wl] >> sh;
                         xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, c_new);
                         xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new);
                         xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new);
@@ -421,12 +431,244 @@ k_server_staged(const ServerStagedArgs sa)
             }
             // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
             if (ok) {
-                uint32_t* __restrict__ ob = a.Bbar + it.base / 32;
-                const int nwords = (L + 31) / 32;
-                for (int w4 = threadIdx.x * 4; w4 < nwords; w4 += kThreads * 4) {
-                    if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
-                    else for (int r = w4; r < nwords; ++r) ob[r] = nb[r];
+                uint32_t* __restrict__ ob = a.Bbar + (wofs - off_out);          // 16-byte aligned; the tile's words are [off_out, wend)
+                const int wend = off_out + (L + 31) / 32;
+                for (int w4 = threadIdx.x * 4; w4 < wend; w4 += kThreads * 4) {
+                    if (w4 >= off_out && w4 + 3 < wend) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
+                    else for (int r = (w4 < off_out ? off_out : w4); r < w4 + 4 && r < wend; ++r) ob[r] = nb[r];
                 }
+            }
+        }
+    }
+    __syncthreads();                                   // every warp has left its loops; shared memory may go
+    if (threadIdx.x == 0 && failed) atomicExch(sa.status, DEVICE_WAIT_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------
+// Server side, staged and fused, for short chunks: 128, 256, 512 or 1024 elements, so that a slab of
+// kSlab elements holds K = kSlab / chunk whole chunks.  The ring, the producer and the split of a slab
+// over the consumer warps are those of k_server_staged (a slab is contiguous in every stream whatever
+// the chunk length); what differs is that a warp's two groups lie in two different chunks: each group
+// has its own set of -s_i, its own old and new server scale, and the sums of squares are kept per group
+// and added per chunk in group order.  A CTA walks `span` slabs; per slab one job for the server step and
+// one for steps 5-6.  Slabs start at multiples of kSlab elements, so the new sign words of a slab are
+// whole 16-byte pieces; the rows may still lie `row_align` words off a 16-byte boundary.
+
+constexpr int kPackedMaxChunks = kSlab / kGroup;         // 16 chunks of 128 elements
+
+template <int NT>
+__device__ __forceinline__ void signed_scale_sums2(const uint32_t* __restrict__ r0, const uint32_t* __restrict__ r1,
+                                                   const uint32_t* __restrict__ neg_s0, const uint32_t* __restrict__ neg_s1,
+                                                   int n, int sh, float2& s01, float2& s23, float2& t01, float2& t23)
+{
+    const int nn = NT > 0 ? NT : n;
+#pragma unroll(NT > 0 ? NT : 4)
+    for (int i = 0; i < nn; ++i) {
+        const uint32_t ns0 = neg_s0[i], ns1 = neg_s1[i];
+        const uint32_t y0 = r0[i * kRowWords] << (28 - sh);
+        const uint32_t y1 = r1[i * kRowWords] << (28 - sh);
+        float2 q;
+        q.x = __uint_as_float(((y0 << 3) & 0x80000000u) ^ ns0); q.y = __uint_as_float(((y0 << 2) & 0x80000000u) ^ ns0);
+        s01 = __fadd2_rn(s01, q);
+        q.x = __uint_as_float(((y0 << 1) & 0x80000000u) ^ ns0); q.y = __uint_as_float((y0 & 0x80000000u) ^ ns0);
+        s23 = __fadd2_rn(s23, q);
+        q.x = __uint_as_float(((y1 << 3) & 0x80000000u) ^ ns1); q.y = __uint_as_float(((y1 << 2) & 0x80000000u) ^ ns1);
+        t01 = __fadd2_rn(t01, q);
+        q.x = __uint_as_float(((y1 << 1) & 0x80000000u) ^ ns1); q.y = __uint_as_float((y1 & 0x80000000u) ^ ns1);
+        t23 = __fadd2_rn(t23, q);
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kStagedThreads, 3)
+k_server_packed(const ServerStagedArgs sa)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const ServerArgs& a = sa.a;
+    __shared__ double red[kPackedMaxChunks];                          // one sum of squares per group of the slab
+    __shared__ uint64_t full[kStages], empty[kStages];
+    __shared__ uint32_t neg_s[2][kPackedMaxChunks * APMS_MAX_WORKERS];   // -s_i per chunk of the slab, double-buffered over the walk
+    __shared__ float S_old_sh[2][kPackedMaxChunks];
+    __shared__ __align__(16) uint32_t nb[kSlabWords];                 // the slab's new sign words
+    __shared__ int failed;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = NT > 0 ? NT : a.n;
+    const size_t stage_bytes = staged_stage_bytes(n, true);
+    const int chunk = (int)a.t.chunk;                                  // 128 .. 1024, divides kSlab
+    const int gpc = chunk / kGroup;                                    // groups per chunk
+    const int64_t nslabs_all = (a.t.d + kSlab - 1) / kSlab;
+    const int64_t slab_first = a.item0 + (int64_t)blockIdx.x * sa.span;       // items are slabs here
+    const int nmine = (int)(a.items - slab_first < sa.span ? a.items - slab_first : sa.span);
+    (void)nslabs_all;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
+        failed = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == kWarps) {
+        if (lane == 0) {
+            int q = 0;
+            bool stop = false;
+            for (int w = 0; w < nmine && !stop; ++w) {
+                const int64_t base_e = (slab_first + w) * kSlab;
+                const int64_t left = a.t.d - base_e;
+                const int live = (int)(left < kSlab ? left : kSlab);
+                const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
+                const int64_t wofs = base_e / 32;
+                for (int r = 0; r < 2; ++r, ++q) {
+                    const int st = q % kStages;
+                    if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; stop = true; break; }
+                    unsigned char* base = smem + (size_t)st * stage_bytes;
+                    if (r == 0) {
+                        const int off_in = sa.row_align;                 // slabs start at multiples of 64 words
+                        const uint32_t wbytes = (uint32_t)((off_in + (live + 31) / 32 + 3) / 4) * 16u;
+                        mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
+                        bulk_load(base, a.zbar + base_e, zbytes, &full[st]);
+                        uint32_t* rows = reinterpret_cast<uint32_t*>(base + (size_t)kSlab * 4);
+                        for (int i = 0; i < n; ++i)
+                            bulk_load(rows + i * kRowWords, a.Brow[i] + (wofs - off_in), wbytes, &full[st]);
+                    } else {
+                        mbar_arrive_expect_tx(&full[st], 2 * zbytes);
+                        bulk_load(base, sa.den + base_e, zbytes, &full[st]);
+                        bulk_load(base + (size_t)kSlab * 4, sa.x + base_e, zbytes, &full[st]);
+                    }
+                }
+            }
+            if (failed) {
+                const int first = q > kStages ? q - kStages : 0;
+                for (int p = first; p < q; ++p) mbar_wait(&full[p % kStages], (uint32_t)(p / kStages) & 1u);
+            }
+        }
+    } else {
+        const int sh = 4 * (lane & 7);
+        const int wl = lane >> 3;
+        const int g0 = warp, g1 = warp + kWarps;
+        const int k0 = g0 / gpc, k1 = g1 / gpc;                          // the chunks (within the slab) of this warp's two groups
+        const volatile int* vfailed = &failed;
+        const int off_in = sa.row_align;
+        int q = 0;
+        for (int w = 0; w < nmine; ++w) {
+            const int64_t base_e = (slab_first + w) * kSlab;
+            const int64_t left = a.t.d - base_e;
+            const int L = (int)(left < kSlab ? left : kSlab);
+            const int64_t c0 = base_e / chunk;
+            const int nchunks = (L + chunk - 1) / chunk;
+            uint32_t* negs = neg_s[w & 1];
+            float* Sold = S_old_sh[w & 1];
+            for (int idx = threadIdx.x; idx < nchunks * n; idx += kThreads) {
+                const int kk = idx / n, i = idx - kk * n;
+                negs[kk * APMS_MAX_WORKERS + i] = __float_as_uint(a.srow[i][c0 + kk]) | 0x80000000u;
+            }
+            if (threadIdx.x < nchunks) Sold[threadIdx.x] = a.Sbar[c0 + threadIdx.x];
+            if (consumer_barrier_any(*vfailed != 0)) break;      // -s_i and old scales in place; everybody is done with the previous slab
+            bool ok = true;
+            double acc0 = 0.0, acc1 = 0.0;
+            {
+                const int st = q % kStages;
+                if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
+                if (ok) {
+                    const unsigned char* base = smem + (size_t)st * stage_bytes;
+                    const float* zs = reinterpret_cast<const float*>(base);
+                    const uint32_t* rows = reinterpret_cast<const uint32_t*>(base + (size_t)kSlab * 4);
+                    const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
+                    const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
+                    float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
+                    // a group past the end of the vector has no chunk: it reads the first chunk's values and is masked below
+                    const int kk0 = k0 < nchunks ? k0 : 0, kk1 = k1 < nchunks ? k1 : 0;
+                    signed_scale_sums2<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl,
+                                           negs + kk0 * APMS_MAX_WORKERS, negs + kk1 * APMS_MAX_WORKERS, n, sh, s01, s23, t01, t23);
+                    const float So0 = Sold[kk0], So1 = Sold[kk1];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int grp = u ? g1 : g0;
+                        const int k = grp * kGroup + lane * 4;
+                        const float4 zo4 = u ? zo1 : zo0;
+                        const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+                        const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
+                        const float S_old = u ? So1 : So0;
+                        float zn[4];
+                        uint32_t nibble = 0;
+                        double acc = 0.0;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
+                            zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+                            if (k + e < L) {
+                                const double zd = (double)zn[e];
+                                acc = fma(zd, zd, acc);
+                                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+                            }
+                        }
+                        if (u) acc1 = acc; else acc0 = acc;
+                        st4_checked(a.zbar + base_e, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                        const uint32_t word = pack_group_words(nibble, lane);
+                        if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
+                    }
+                }
+                ++q;
+            }
+            acc0 = warp_sum(acc0);
+            acc1 = warp_sum(acc1);
+            if (lane == 0) { red[g0] = acc0; red[g1] = acc1; }
+            const bool leave = consumer_barrier_any(!ok || *vfailed != 0);   // the groups' sums and the slab's sign words are in shared memory
+            if (leave) break;
+            // Section 3.3 steps 5-6 for this slab: every group with the new scale of its chunk
+            float c_new[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int kk = u ? k1 : k0;
+                float S_new = 0.0f;
+                if (kk < nchunks) {
+                    double total = 0.0;
+                    for (int r = 0; r < gpc; ++r) total += red[kk * gpc + r];          // group order
+                    const int64_t cbeg = (c0 + kk) * (int64_t)chunk;
+                    const int64_t Lc = (a.t.d - cbeg < chunk) ? a.t.d - cbeg : chunk;
+                    S_new = (float)sqrt(total / (double)Lc);
+                    if (lane == 0 && (u ? g1 : g0) == kk * gpc) a.Sbar[c0 + kk] = S_new;     // the warp that holds the chunk's first group
+                }
+                c_new[u] = __fmul_rn(sa.lr, S_new);                  // lr * (+-S) = +-(lr * S)
+            }
+            {
+                const int st = q % kStages;
+                if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
+                if (ok) {
+                    const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
+                    const float* xs = vs + kSlab;
+                    float4 vv[2], xx[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
+                        xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[st]);
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int grp = u ? g1 : g0;
+                        const int k = grp * kGroup + lane * 4;
+                        const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                        xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, c_new[u]);
+                        xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new[u]);
+                        xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new[u]);
+                        xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, c_new[u]);
+                        st4_checked(sa.x + base_e, k, L, xx[u]);
+                    }
+                }
+                ++q;
+            }
+            // the slab's sign words leave in whole 16-byte pieces
+            if (ok) {
+                uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
+                const int nwords = (L + 31) / 32;
+                const int w4 = threadIdx.x * 4;
+                if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
+                else for (int r = w4; r < nwords; ++r) ob[r] = nb[r];
             }
         }
     }

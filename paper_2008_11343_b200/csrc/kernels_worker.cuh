@@ -18,7 +18,8 @@ struct WorkerArgs {
     const float* m32;             // binary32 momentum (first step / forced)
     const uint32_t* Bbar; const float* Sbar;   // momentum as the server's last message
     Tiling t;
-    int64_t items;                // C * P * ni
+    int64_t items;                // chunk tiles of this launch * ni
+    int64_t tile0;                // first chunk tile of this launch (a launch may cover a range of chunks)
     int i0, ni;                   // this launch covers workers i0 .. i0+ni-1
     float beta1, omb1;
     int send_gradient;            // gradient-compressing variant: z = g_i + delta_i, the momentum is not read
@@ -74,7 +75,7 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
     const int64_t item = (int64_t)blockIdx.x * TEAMS + (WPC == 1 ? warp : 0);
     if (item >= a.items) return;                       // only in the last CTA of the WPC == 1 form
     const int ii = (int)(item % a.ni);
-    const Item it = decode_item(a.t, item / a.ni);
+    const Item it = decode_item(a.t, a.tile0 + item / a.ni);
     const int i = a.i0 + ii;
     const int L = it.L;
     const void* __restrict__ g = Grad<GT>::at(G.p[ii], it.base);
@@ -127,14 +128,19 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
     }
 }
 
-// Worker side, fine-tiled form (steady state, chunk a multiple of kFineSub): one CTA per
+// Worker side, fine-tiled form (steady state, chunks of at least kFineSub elements): one CTA per
 // (worker, 4096-element tile), every load of the tile issued before the first use.  Short-lived
 // CTAs that each touch 16 KiB of every stream once keep DRAM pages and the memory pipeline busier
 // than long-running warps that each follow their own stream.
-// Warp w owns the tile's groups 4w..4w+3 (kFineSub = 512 consecutive elements, all of one chunk),
-// so its 16 momentum words are one 64-byte load handed round by shuffles, its 16 new sign words
-// one 64-byte store, and its binary64 sum of squares one slot of a partial-sum array that
-// k_finalize_fine adds up per chunk in element order: the kernel has no barrier at all.
+// Warp w owns the tile's groups 4w..4w+3 (kFineSub = 512 consecutive elements), so its 16 momentum
+// words are one 64-byte load handed round by shuffles, its 16 new sign words one 64-byte store, and
+// its binary64 sum of squares one slot of a partial-sum array that k_finalize_fine adds up per chunk
+// in element order: the kernel has no barrier at all.
+// Chunks are multiples of 32 elements, so a chunk boundary inside a warp's 512 elements falls
+// between two sign words, i.e. between two 8-lane groups of one 128-element access, and there is at
+// most one of them (chunk >= 512).  With SPLIT (chunks that are not multiples of 512) a warp that
+// sees a boundary reads the scales of both chunks and keeps two sums; every warp then writes two
+// slots: [0] = its elements of the chunk its first element belongs to, [1] = those of the next chunk.
 // Launch order: runs of `run` consecutive tiles of one worker, then the same tiles of the next
 // worker: every stream is read in long sequential pieces (measured: the longer the better for
 // DRAM), while the momentum bits of a run (run * 512 bytes) stay in L2 for the other workers.
@@ -142,20 +148,22 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 constexpr int kFineTile = 4096;           // 256 threads x 4 x (4 floats)
 constexpr int kFineU = kFineTile / (kThreads * 4);
 constexpr int kFineSub = kFineTile / kWarps;      // elements per warp = per partial sum
+constexpr int kFineSubWords = kFineSub / 32;
 constexpr int kFineRunDefault = 4096;
 
 struct WorkerFineArgs {
     float* z; int64_t dz;
     uint32_t* B; int64_t Wp;
     const float* s; int64_t Cp;       // the scales of the previous step (read only here)
-    double* partial; int64_t Pp;      // ni rows of tiles * kWarps partial sums, row stride Pp
+    double* partial; int64_t Pp;      // ni rows of tiles * kWarps (* 2 with SPLIT) partial sums, row stride Pp
     const uint32_t* Bbar; const float* Sbar;
-    int64_t d, chunk, tiles;
+    int64_t d, chunk, tiles;          // tiles: 4096-element tiles of this launch, the first one being tile0
+    int64_t tile0, e0, e1;            // a launch may cover the elements [e0, e1) of whole chunks only (multiples of 512 without SPLIT)
     int i0, ni, run;
     float beta1, omb1;
 };
 
-template <int GT, bool SENDG>          // SENDG: the gradient-compressing variant (no momentum is read)
+template <int GT, bool SENDG, bool SPLIT>          // SENDG: the gradient-compressing variant (no momentum is read)
 __global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
@@ -164,14 +172,16 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
     const int rem = (int)((int64_t)blockIdx.x - stretch * per_stretch);
     const int ii = rem / a.run;
-    const int64_t t = stretch * a.run + (rem - ii * a.run);
-    if (t >= a.tiles) return;                                  // whole CTA: the last stretch may be short
+    const int64_t tl = stretch * a.run + (rem - ii * a.run);
+    if (tl >= a.tiles) return;                                 // whole CTA: the last stretch may be short
+    const int64_t t = a.tile0 + tl;
     const int i = a.i0 + ii;
     const int64_t base = t * kFineTile + (int64_t)warp * kFineSub;     // this warp's 512 elements
-    double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + t * kWarps + warp;
+    if (base < a.e0 || base >= a.e1) return;                   // a launch over a range of chunks: the tiles at its ends are shared
+    double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + (t * kWarps + warp) * (SPLIT ? 2 : 1);
     const int64_t left = a.d - base;
     if (left <= 0) {                                           // past the end of the vector
-        if (lane == 0) *slot = 0.0;
+        if (lane == 0) { slot[0] = 0.0; if (SPLIT) slot[1] = 0.0; }
         return;
     }
     const int L = (int)(left < kFineSub ? left : kFineSub);
@@ -180,9 +190,13 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
     const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
     uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
-    const float s_old = a.s[(int64_t)i * a.Cp + c];
-    const float Sbar = a.Sbar[c];
-    double acc = 0.0;
+    const float* __restrict__ srow = a.s + (int64_t)i * a.Cp;
+    // first sign word of this warp's elements that belongs to chunk c + 1 (>= kFineSubWords: none does)
+    const int bw = SPLIT ? (int)(((c + 1) * a.chunk - base) >> 5) : kFineSubWords;
+    const bool two = SPLIT && bw * 32 < L;
+    const float s_lo = srow[c], S_lo = a.Sbar[c];
+    const float s_hi = two ? srow[c + 1] : s_lo, S_hi = two ? a.Sbar[c + 1] : S_lo;
+    double acc = 0.0, acc_hi = 0.0;
     if (L == kFineSub) {
         float4 gv[kFineU], zv[kFineU];
 #pragma unroll
@@ -195,19 +209,24 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 #pragma unroll
         for (int u = 0; u < kFineU; ++u) {
             const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
+            const bool hi = SPLIT && (u * 4 + (lane >> 3) >= bw);      // this lane's word lies in chunk c + 1
+            const float s_old = hi ? s_hi : s_lo, Sbar = hi ? S_hi : S_lo;
             const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
             const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
             float zn[4];
             uint32_t nibble = 0;
+            double part = SPLIT ? 0.0 : acc;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
                 const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
                 zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
                 const double zd = (double)zn[e];
-                acc = fma(zd, zd, acc);
+                part = fma(zd, zd, part);
                 nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
             }
+            if (SPLIT) { acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0; }
+            else acc = part;
             st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
             const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
             const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
@@ -221,35 +240,47 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
             const float4 gv = ld_grad4_checked<GT>(g, k, L);
             const float4 zv = ld4_checked(z, k, L, true);
             const uint32_t mw = (!SENDG && k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
-            worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_old, Sbar, gv, zv,
-                                      make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
+            const bool hi = SPLIT && (grp * 4 + (lane >> 3) >= bw);
+            if (SPLIT) {
+                double part = 0.0;
+                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, hi ? s_hi : s_lo, hi ? S_hi : S_lo, gv, zv,
+                                          make_float4(0, 0, 0, 0), mw, part, false, SENDG);
+                acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0;
+            } else {
+                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_lo, S_lo, gv, zv,
+                                          make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
+            }
         }
     }
     acc = warp_sum(acc);
-    if (lane == 0) *slot = acc;
+    if (SPLIT) acc_hi = warp_sum(acc_hi);
+    if (lane == 0) { slot[0] = acc; if (SPLIT) slot[1] = acc_hi; }
 }
 
-// Scales from the fine form's partial sums (one per 512 elements): a team of T lanes per (row, chunk)
-// adds the chunk's slots in a fixed order (lane l of the team takes slots l, l + T, ..., then the shuffle
-// tree) and takes sqrt(sum / L).  T is the number of slots of a whole chunk rounded up to a power of two,
-// at most a warp; the sums are not negative, so a team's tree gives bit for bit what a whole warp's tree
+// Scales from the fine form's partial sums (one - or, with chunks that are not multiples of 512, two -
+// per 512 elements): a team of T lanes per (row, chunk) adds the chunk's slots in a fixed order (lane l
+// of the team takes the 512-element pieces l, l + T, ..., then the shuffle tree) and takes sqrt(sum / L).
+// With two slots per piece (`per` = 2) a chunk takes slot [1] of the piece it begins inside of and slot
+// [0] of all later ones.  T is the number of pieces a chunk can touch rounded up to a power of two, at
+// most a warp; the sums are not negative, so a team's tree gives bit for bit what a whole warp's tree
 // with zeros in the other lanes gives, and short chunks do not leave most of a warp idle (chunk = 1024:
 // 16 chunks per warp; one warp per chunk took 1.2 ms longer at n = 16).
 template <int T>
 __global__ void __launch_bounds__(kThreads)
 k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
-                int rows, int64_t C, int64_t d, int64_t chunk)
+                int rows, int64_t c_first, int64_t C, int64_t d, int64_t chunk, int per)
 {
     const int lane = threadIdx.x & 31, sub = lane % T;
     const int64_t idx = ((int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * (32 / T) + lane / T;
-    const bool live = idx < (int64_t)rows * C;                   // every lane stays for the shuffles
+    const bool live = idx < (int64_t)rows * C;                   // every lane stays for the shuffles; C chunks from c_first on
     const int r = live ? (int)(idx / C) : 0;
-    const int64_t c = live ? idx % C : 0;
+    const int64_t c = c_first + (live ? idx % C : 0);
     const int64_t cbeg = c * chunk;
     const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
     const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
     double total = 0.0;
-    if (live) for (int64_t q = q0 + sub; q < q1; q += T) total += partial[(int64_t)r * Pp + q];
+    if (live) for (int64_t q = q0 + sub; q < q1; q += T)
+        total += partial[(int64_t)r * Pp + q * per + ((per == 2 && q * kFineSub < cbeg) ? 1 : 0)];
 #pragma unroll
     for (int o = T / 2; o > 0; o >>= 1) total += __shfl_down_sync(0xffffffffu, total, o, T);
     if (live && sub == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);

@@ -36,13 +36,12 @@ def chunk_ranges(n_chunks: int, world: int) -> List[Tuple[int, int]]:
     return [(r * n_chunks // world, (r + 1) * n_chunks // world) for r in range(world)]
 
 
-def chunk_for_servers(d: int, servers: int, multiple: int = 2048) -> int:
+def chunk_for_servers(d: int, servers: int) -> int:
     """The paper's own layout has one chunk per worker-as-server (Section 3.3: the vector is cut into n
-    chunks).  This is that chunk length, d / servers, rounded up to a multiple of 2048 elements - the
-    granularity at which the library's tuned kernels apply (measured on the BERT-Large-shaped set with 16
-    workers: 11.0 ms per step against 12.2 ms with the unrounded d / 16); the last chunk is a little shorter."""
+    chunks).  This is that chunk length: d / servers rounded up to the next multiple of 32 elements (a
+    chunk holds whole sign words); the last chunk is shorter when d is not a multiple of it."""
     per = -(-d // servers)
-    return -(-per // multiple) * multiple
+    return -(-per // 32) * 32
 
 
 def word_range(chunk_begin: int, chunk_end: int, chunk: int, d: int) -> Tuple[int, int]:
@@ -72,6 +71,7 @@ class ShardedStep:
         self.row_words = [_round4(w1 - w0) for w0, w1 in self.words]
         self.row_scales = [ce - cb for cb, ce in self.ranges]
         self._buffers = None
+        self._sends = []
 
     # ------------------------------------------------------------------ buffers (made once)
     def _make_buffers(self, like_bits, like_scales):
@@ -96,35 +96,53 @@ class ShardedStep:
 
     # ------------------------------------------------------------------ the step
     def step(self, grads: Sequence) -> None:
-        """Section 3.3 steps 1-6 for this process's workers; `grads`: its n_local gradients."""
+        """Section 3.3 steps 1-6 for this process's workers; `grads`: its n_local gradients.
+
+        The worker phase runs range by range, in the order of the serving processes (the same order on every
+        process, so that the grouped transfers of a range pair up like one gather and cannot deadlock): as soon
+        as the kernels of range k are enqueued, this process's rows of that range are packed and handed to the
+        transfer to process k, which runs while the later ranges are still being compressed.  Transfers are
+        stream-ordered after the kernels (NCCL) - nothing waits on the host until the server phase needs the
+        received rows."""
         b, dist, n, me = self.b, self.dist, self.b.n, self.rank
-        b.worker_phase(grads)                                                   # steps 1-2
+        ranged = hasattr(b, "worker_phase_range")
+        if not ranged:
+            b.worker_phase(grads)                                               # steps 1-2, whole vector
         msgs = [b.message(i) for i in range(n)]
         if self._buffers is None:
             self._make_buffers(msgs[0][0], msgs[0][1])
         buf = self._buffers
-
-        # step 3 (exchange 1): the part of every local message that process k serves goes to process k
+        for req in self._sends:                                                 # the previous step's send buffers are free again
+            req.wait()
+        self._sends = []
+        recvs = []
         for k in range(self.world):
             (w0, w1), (cb, ce) = self.words[k], self.ranges[k]
+            if ranged:
+                b.worker_phase_range(grads, cb, ce)                             # steps 1-2 for the chunks process k serves
+            # step 3 (exchange 1): the part of every local message that process k serves goes to process k
             for i, (bits, scales) in enumerate(msgs):
                 buf["send_bits"][k][i, :w1 - w0].copy_(bits[w0:w1])
                 buf["send_scales"][k][i].copy_(scales[cb:ce])
-        ops = []
-        for k in range(self.world):
-            rows = slice(k * n, (k + 1) * n)
+            ops = []
             if k == me:
-                buf["recv_bits"][rows].copy_(buf["send_bits"][k])
-                buf["recv_scales"][rows].copy_(buf["send_scales"][k])
-                continue
-            peer = self.global_rank(k)
-            ops.append(dist.P2POp(dist.isend, buf["send_bits"][k], peer, self.group))
-            ops.append(dist.P2POp(dist.isend, buf["send_scales"][k], peer, self.group))
-            ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][rows], peer, self.group))
-            ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][rows], peer, self.group))
-        if ops:
-            for req in dist.batch_isend_irecv(ops):
-                req.wait()
+                for q in range(self.world):
+                    rows = slice(q * n, (q + 1) * n)
+                    if q == me:
+                        buf["recv_bits"][rows].copy_(buf["send_bits"][k])
+                        buf["recv_scales"][rows].copy_(buf["send_scales"][k])
+                        continue
+                    peer = self.global_rank(q)
+                    ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][rows], peer, self.group))
+                    ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][rows], peer, self.group))
+            else:
+                peer = self.global_rank(k)
+                ops.append(dist.P2POp(dist.isend, buf["send_bits"][k], peer, self.group))
+                ops.append(dist.P2POp(dist.isend, buf["send_scales"][k], peer, self.group))
+            if ops:
+                (recvs if k == me else self._sends).extend(dist.batch_isend_irecv(ops))
+        for req in recvs:
+            req.wait()
 
         # step 4: average and recompress the chunks this process serves
         cb, ce = self.ranges[me]
@@ -155,15 +173,64 @@ class ShardedStep:
         return ex1 + ex2
 
 
+class HostFlags:
+    """Step counters shared by the processes of one node (POSIX shared memory): flag [r, k] is the number of
+    the last step in which process r finished its part of stage k.  Processes tell each other on the host
+    how far they are - no kernel ever waits for another process.  A wait that lasts longer than `timeout_s`
+    raises: a peer that died or never joined shows up as an error on the host, with every GPU still usable."""
+
+    def __init__(self, dist, group, world: int, stages: int, timeout_s: float = 120.0):
+        import numpy as np
+        from multiprocessing import shared_memory
+
+        self.rank, self.world, self.timeout_s = dist.get_rank(group), world, timeout_s
+        name = [None]
+        if self.rank == 0:
+            self._shm = shared_memory.SharedMemory(create=True, size=8 * world * stages)
+            name[0] = self._shm.name
+        dist.broadcast_object_list(name, src=0 if group is None else dist.get_global_rank(group, 0), group=group)
+        if self.rank != 0:
+            self._shm = shared_memory.SharedMemory(name=name[0])
+        self.flags = np.ndarray((world, stages), dtype=np.int64, buffer=self._shm.buf)
+        if self.rank == 0:
+            self.flags[:] = 0
+        dist.barrier(group=group)
+
+    def post(self, stage: int, step: int) -> None:
+        self.flags[self.rank, stage] = step
+
+    def wait_all(self, stage: int, step: int) -> None:
+        import time
+
+        t0 = time.monotonic()
+        while True:
+            if (self.flags[:, stage] >= step).all():
+                return
+            if time.monotonic() - t0 > self.timeout_s:
+                late = [r for r in range(self.world) if self.flags[r, stage] < step]
+                raise RuntimeError(f"processes {late} did not reach stage {stage} of step {step} within {self.timeout_s} s")
+            time.sleep(0)
+
+    def close(self, dist, group) -> None:
+        self.flags = None
+        dist.barrier(group=group)
+        self._shm.close()
+        if self.rank == 0:
+            self._shm.unlink()
+
+
 class PeerShardedStep:
     """Section 3.3 steps 1-6 across processes of one node, the exchanges done by peer loads and stores.
 
     `backend`: a `binding.Context` made with library_workspace=True (its workspace must be exportable);
     `peers`: what opens and closes a handle - by default the binding's apms_ipc_open / apms_ipc_close.
-    The two barriers are host barriers after a stream synchronisation: no kernel waits on another GPU.
+    No kernel waits on another GPU: the processes tell each other on the host (`HostFlags`) which part of
+    their messages is complete.  The worker phase runs range by range, every process starting with the range
+    after its own, so the range a process serves is finished everywhere one range before the end of the
+    worker phase: its server phase does not wait for the slowest process's last kernel.
     """
 
-    def __init__(self, backend, group=None, peers=None):
+    def __init__(self, backend, group=None, peers=None, timeout_s: float = 120.0):
         import torch.distributed as dist
 
         self.b, self.dist, self.group = backend, dist, group
@@ -184,6 +251,10 @@ class PeerShardedStep:
                 raise ValueError(f"process {r} holds a context of another shape: {shape} against {mine[1]}")
         own_base = backend.message_ptrs(0)[0] - self.off[0][0]
         self.base = [own_base if r == self.rank else peers.apms_ipc_open(h) for r, (h, _, _) in enumerate(everyone)]
+        # stages 0 .. world-1: "my workers' messages for range k are complete"; stage world: "my server range is stored everywhere"
+        self.flags = HostFlags(dist, group, self.world, self.world + 1, timeout_s)
+        self.steps = 0
+        self.order = [(self.rank + 1 + j) % self.world for j in range(self.world)]      # own range last
         dist.barrier(group=group)
 
     def row_pointers(self):
@@ -196,10 +267,16 @@ class PeerShardedStep:
         return bits, scales
 
     def step(self, grads: Sequence) -> None:
-        b, me = self.b, self.rank
-        b.worker_phase(grads)                                                   # steps 1-2
-        b.synchronize()
-        self.dist.barrier(group=self.group)                                     # every worker's message is complete
+        b, me, flags = self.b, self.rank, self.flags
+        self.steps += 1
+        events = []
+        for k in self.order:                                                    # steps 1-2, range by range
+            b.worker_phase_range(grads, *self.ranges[k])
+            events.append((k, b.record_event()))
+        for k, ev in events:
+            ev.synchronize()
+            flags.post(k, self.steps)                                           # my rows of range k may be read
+        flags.wait_all(me, self.steps)                                          # every process's rows of my range are complete
         cb, ce = self.ranges[me]
         bits, scales = self.row_pointers()
         b.server_phase_rows(bits, scales, cb, ce)                               # steps 3-4: the kernel loads the rows
@@ -207,7 +284,8 @@ class PeerShardedStep:
             if r != me:
                 b.put_server_range(self.base[r] + self.off[-1][0], self.base[r] + self.off[-1][1], cb, ce)
         b.synchronize()
-        self.dist.barrier(group=self.group)                                     # every range is stored everywhere
+        flags.post(self.world, self.steps)
+        flags.wait_all(self.world, self.steps)                                  # every range is stored everywhere
         b.apply_phase()                                                         # steps 5-6
 
     def close(self):
@@ -218,6 +296,7 @@ class PeerShardedStep:
             if r != self.rank and base is not None:
                 self._peers.apms_ipc_close(base)
         self.base = []
+        self.flags.close(self.dist, self.group)
         self.dist.barrier(group=self.group)                                     # nobody frees memory that is still mapped
 
     def wire_bytes_per_step(self) -> int:

@@ -5,6 +5,8 @@ The oracle cannot run 335M x 16 elements in a test, but chunks are independent p
 (Supplement A: the algorithm equals a parameter-server step per chunk), so a sample of chunks -
 the first, the ragged last one and random ones - is run by the oracle as a small problem of its own,
 on the same gradients, and compared with the same chunks of the device state step by step."""
+import gc
+
 import numpy as np
 import pytest
 
@@ -49,6 +51,8 @@ def test_sampled_chunks_free_running_at_full_size(cfg, samples, n, chunk, steps)
         w = w.with_(n=n)
     if chunk is not None:
         w = w.with_(chunk=chunk)
+    gc.collect()
+    torch.cuda.empty_cache()                                 # memory cached for earlier tests counts as free
     free, _ = torch.cuda.mem_get_info()
     need = B.apms_workspace_bytes(w.d, w.n, w.chunk) + 4 * w.d * w.n + (2 << 30)
     if free < need:
@@ -136,6 +140,8 @@ def test_topk_sampled_chunks_at_full_size(frac):
     import torch
 
     w = wl.config(3)
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     need = B.apms_workspace_bytes(w.d, w.n, w.chunk) + 4 * w.d * w.n + (2 << 30)
     if free < need:

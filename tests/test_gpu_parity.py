@@ -30,7 +30,12 @@ STAGED = [(2048, 1, 2048), (10 * 2048 + 1, 5, 2048), (6144 * 3 + 33, 7, 6144), (
           (8 * 32768 + 23552, 16, 32768), (2 * 4096 + 2047, 64, 4096), (65536 + 2049, 2, 65536),
           (3 * 512 + 100, 3, 512), (7 * 1536 + 511, 2, 1536), (9 * 4096 + 513, 4, 1024),
           (5 * 4096 + 100, 32, 4096), (3 * 2048 + 7, 12, 2048), (2 * 32768 + 1000, 32, 32768), (6 * 8192 + 5, 8, 8192),
-          (65536 + 4097, 32, 65536), (11 * 1024 + 9, 32, 1024)]
+          (65536 + 4097, 32, 65536), (11 * 1024 + 9, 32, 1024),
+          # chunks that are not multiples of a slab, a tile or 512: sign-word rows off the 16-byte boundary, a chunk
+          # boundary inside a warp's 512 elements; short chunks packed several to a slab, any worker count
+          (5 * 2080 + 100, 3, 2080), (3 * 4128 + 33, 16, 4128), (2 * 20960 + 7000, 4, 20960), (3 * 66592 + 5, 2, 66592),
+          (7 * 2048 * 3 + 2016 * 5, 5, 2016 * 3), (3 * 2048 + 700, 5, 256), (9 * 2048 + 1500, 7, 512), (40 * 2048 + 130, 16, 128),
+          (6 * 1056 + 1000, 4, 1056), (5 * 544 + 17, 2, 544)]
 
 
 @pytest.mark.parametrize("team", [B.TEAM_CTA, B.TEAM_WARP, B.TEAM_AUTO, B.TEAM_STAGED],
@@ -391,7 +396,8 @@ def test_error_norms_match_the_oracle_state():
 
 @pytest.mark.parametrize("d,n,chunk,cuts", [(9 * 2048 + 300, 4, 2048, (0, 3, 10)), (5 * 4096 + 1, 3, 4096, (0, 1, 5, 6)),
                                             (7 * 96 + 5, 5, 96, (0, 4, 8)), (3 * 70016, 2, 70016, (0, 2, 3)),
-                                            (6 * 32768, 16, 32768, (0, 6))])
+                                            (6 * 32768, 16, 32768, (0, 6)), (9 * 4096 + 100, 4, 4096, (0, 2, 3, 7, 10)),
+                                            (5 * 2080 + 100, 3, 2080, (0, 2, 6)), (23 * 512 + 9, 2, 512, (0, 5, 6, 24))])
 def test_phase_wise_step_equals_the_whole_step(d, n, chunk, cuts):
     """worker phase, the server phase range by range from COPIES of the messages laid out as a receiver would
     hold them (rows = senders, word 0 = first word of the range), apply phase: bit-identical to apms_compressed_step."""
@@ -408,7 +414,20 @@ def test_phase_wise_step_equals_the_whole_step(d, n, chunk, cuts):
     for step in range(1, 5):
         gs = H.upload(wl.host_gradients(w, step))
         a.compressed_step(gs)
-        b.worker_phase(gs)
+        if step == 1:
+            b.worker_phase(gs)
+        else:                                                  # range by range, in another order every step
+            pieces = list(zip(cuts, cuts[1:]))
+            pieces = pieces[::-1] if step % 2 else pieces[1:] + pieces[:1]
+            for cb, ce in pieces[:-1]:
+                b.worker_phase_range(gs, cb, ce)
+            with pytest.raises(B.ApmsError) as e:              # the worker phase does not cover every chunk yet
+                b.server_phase_rows([b.message_ptrs(i)[0] for i in range(n)], [b.message_ptrs(i)[1] for i in range(n)], 0, b.C)
+            assert e.value.status == B.ERR_BAD_STATE
+            b.worker_phase_range(gs, *pieces[-1])
+            with pytest.raises(B.ApmsError) as e:
+                b.worker_phase_range(gs, 0, 1)                 # every chunk has been covered
+            assert e.value.status == B.ERR_BAD_STATE
         msgs = [b.message(i) for i in range(n)]
         for cb, ce in zip(cuts, cuts[1:]):
             w0, w1 = cb * chunk // 32, (min(d, ce * chunk) + 31) // 32

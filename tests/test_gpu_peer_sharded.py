@@ -79,7 +79,7 @@ def test_rows_argument_errors_are_status_codes():
     assert e.value.status == B.ERR_BAD_STATE
     ctx.worker_phase(gs)
     with pytest.raises(B.ApmsError) as e:
-        ctx.server_phase_rows([bits[0], bits[1] + 4], scales, 0, ctx.C)
+        ctx.server_phase_rows([bits[0], bits[1] + 2], scales, 0, ctx.C)     # not a word address
     assert e.value.status == B.ERR_INVALID_ARG
     with pytest.raises(B.ApmsError) as e:
         ctx.server_phase_rows(bits, scales, 0, ctx.C + 1)

@@ -125,6 +125,9 @@ def _rank_main(rank, world, port, out):
               and np.array_equal(backend.scales[-1].numpy(), ref.server_scales))
     for i in range(n_local):
         ok = ok and bool(np.array_equal(backend.err[i], ref.worker_err(rank * n_local + i)))
+    # the worker phase ran range by range, starting after the rank's own range and ending with it
+    own_last = [step.ranges[(rank + 1 + j) % world] for j in range(world)]
+    ok = ok and backend.ranges_seen == own_last * len(grads) and own_last[-1] == step.ranges[rank]
     wire = step.wire_bytes_per_step()
     step.close()
     ok = ok and peers.opened == [r for r in range(world) if r != rank] and sorted(peers.closed) == peers.opened
@@ -142,3 +145,33 @@ def test_two_ranks_exchange_by_peer_addresses_and_equal_one_four_worker_run():
         res = dict(out)
     assert res[0][0] and res[1][0]
     assert max(res[0][1], res[1][1]) < 0.1 * 4 * D * (N_TOTAL // world)
+
+
+def _flags_main(rank, world, port, out):
+    from paper_2008_11343_b200 import sharded
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    flags = sharded.HostFlags(dist, None, world, 2, timeout_s=0.5)
+    flags.post(0, 1)
+    flags.wait_all(0, 1)                                        # both ranks posted stage 0 of step 1
+    seen = ""
+    if rank == 0:
+        flags.post(1, 1)
+        try:
+            flags.wait_all(1, 1)                                # rank 1 never reports stage 1
+        except RuntimeError as exc:
+            seen = str(exc)
+    dist.barrier()
+    flags.close(dist, None)
+    out[rank] = seen
+    dist.destroy_process_group()
+
+
+def test_a_process_that_never_reports_is_an_error_on_the_host_not_a_hang():
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_flags_main, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    assert "processes [1] did not reach stage 1 of step 1" in res[0] and res[1] == ""

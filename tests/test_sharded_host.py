@@ -45,6 +45,7 @@ class OracleBackend:
         self.server_err = np.zeros(d, np.float32)
         self.bits = [torch.zeros(self.W, dtype=torch.int32) for _ in range(n + 1)]       # last = server
         self.scales = [torch.zeros(self.C, dtype=torch.float32) for _ in range(n + 1)]
+        self.ranges_seen = []
 
     def _chunks(self, cb, ce):
         for c in range(cb, ce):
@@ -54,10 +55,20 @@ class OracleBackend:
         return self.bits[i], self.scales[i]
 
     def worker_phase(self, grads):
+        self.worker_phase_range(grads, 0, self.C)
+
+    def record_event(self):
+        class Done:                                                # the stand-in works synchronously
+            def synchronize(self):
+                pass
+        return Done()
+
+    def worker_phase_range(self, grads, cb, ce):
+        self.ranges_seen.append((cb, ce))
         omb1 = np.float32(1.0) - np.float32(BETA1)
         for i, g in enumerate(grads):
             g = g.numpy()
-            for c, lo, hi in self._chunks(0, self.C):
+            for c, lo, hi in self._chunks(cb, ce):
                 z = _fma32(np.float32(BETA1), self.m[lo:hi], omb1 * g[lo:hi]) + self.err[i][lo:hi]
                 bits, s = self.ao.compress_1bit(z)
                 self.err[i][lo:hi] = z - self.ao.decompress_1bit(bits, s, hi - lo)
@@ -128,6 +139,8 @@ def _rank_main(rank, world, port, out):
     cb, ce = step.ranges[rank]
     lo, hi = cb * CHUNK, min(D, ce * CHUNK)
     ok = ok and bool(np.array_equal(backend.server_err[lo:hi], ref.server_err[lo:hi]))      # a rank owns only its range
+    # the worker phase ran range by range, in the order of the serving processes, on every rank alike
+    ok = ok and backend.ranges_seen == list(step.ranges) * len(grads)
     out[rank] = (ok, step.wire_bytes_per_step())
     dist.barrier()
     dist.destroy_process_group()
@@ -162,6 +175,7 @@ def test_chunk_for_servers_gives_one_chunk_per_server():
 
     for d, n in [(335_141_888, 16), (109_482_240, 8), (2049, 2), (4096, 2), (1, 1)]:
         chunk = sharded.chunk_for_servers(d, n)
-        assert chunk % 2048 == 0 and -(-d // chunk) <= n and chunk * n >= d
-        assert chunk - 2048 < -(-d // n)                         # not rounded further than needed
+        assert chunk % 32 == 0 and -(-d // chunk) <= n and chunk * n >= d
+        assert chunk - 32 < -(-d // n)                           # not rounded further than whole sign words need
+    assert sharded.chunk_for_servers(335_141_888, 16) == 335_141_888 // 16     # the headline set: exactly d / 16
     assert -(-335_141_888 // sharded.chunk_for_servers(335_141_888, 16)) == 16

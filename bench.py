@@ -11,8 +11,15 @@ resident in HBM before the timed region (a ring of two distinct sets); the worki
 step (~73 GB) is far larger than L2, so no flush is needed between steps.
 
 Prints ONE JSON line.  With --gpus N > 1 (launched by torchrun) every rank runs an independent
-replica of the same single-GPU job - the path has no cross-GPU exchange in this build - and the
+replica of the same single-GPU job - the measured path keeps all n workers on one GPU - and the
 value is the aggregate over ranks, timed as the maximum over ranks.
+
+--path sharded | peer (under torchrun) runs the paper's own layout instead: the workload's n workers
+are split over the processes, one GPU each, every process serves a range of chunks, and the 1-bit
+messages are exchanged (Section 3.3 steps 3 and 5) over torch.distributed (sharded) or by the server
+kernel's own loads from the peers' mapped workspaces (peer).  The total work is fixed ("scaling": "strong").
+--one-gpu puts every process on cuda:0 (peer form only; host flags over gloo): the code path of a
+one-process-per-GPU run where only one GPU is at hand.
 
 --impl reference times the CPU oracle (oracle/) on a bounded sample of the same workload on the
 host cores; it is a deliberately plain program, reported as a baseline.
@@ -212,7 +219,13 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
     from paper_2008_11343_b200 import workloads as wl
 
     dev = torch.device("cuda", local_rank)
-    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}")
+    split = args.path in ("sharded", "peer")          # the workload's workers are split over the processes
+    n_total = w.n
+    if split:
+        assert n_total % world == 0, "the worker count must be a multiple of the number of processes"
+        w = w.with_(n=n_total // world)
+    ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}",
+                    library_workspace=(args.path == "peer"))
     if args.compressor == "topk":
         ctx.set_compressor(B.COMPRESSOR_TOPK, args.topk_fraction)
     x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)
@@ -259,6 +272,11 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
             ctx.worker_phase(gs)
             ctx.server_phase_rows(own_bits, own_scales, 0, ctx.C)
             ctx.apply_phase()
+    elif split:
+        from paper_2008_11343_b200 import sharded
+
+        stepper = (sharded.PeerShardedStep if args.path == "peer" else sharded.ShardedStep)(ctx)
+        step = stepper.step
     else:
         step = ctx.compressed_step
     step(ring[0])                            # reads the binary32 momentum once; not representative
@@ -296,13 +314,17 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
         if cnt:
             kernel_ms[name] = ms / cnt
     ctx.set_timing(False)
-    out = {"ms_per_step": seconds * 1e3 / args.steps, "value": world * w.d * w.n * args.steps / seconds,
+    work = n_total if split else world * w.n          # worker vectors the whole job compresses per step
+    out = {"ms_per_step": seconds * 1e3 / args.steps, "value": work * w.d * args.steps / seconds,
            "ms_per_step_min": per_step_ms[0], "ms_per_step_median": per_step_ms[len(per_step_ms) // 2],
            "kernel_ms": kernel_ms, "launches": launches, "clocks": clocks.summary(), "adam": adam, "e2e": None}
 
     # end to end through the host-gradient entry point: H2D of the n gradients and D2H of x
     # inside the timed region, every step
-    if want_e2e:
+    if split:
+        out["wire_bytes_per_step"] = stepper.wire_bytes_per_step()
+        stepper.close() if args.path == "peer" else None
+    if want_e2e and not split:
         try:
             host = [torch.empty(w.d, dtype=gdt).pin_memory() for _ in range(w.n)]
             for i in range(w.n):
@@ -348,9 +370,11 @@ def main(argv=None) -> int:
     ap.add_argument("--compressor", default="onebit", choices=["onebit", "topk"],
                     help="the compression operator (the configurations of record use the 1-bit compressor)")
     ap.add_argument("--topk-fraction", type=float, default=0.01)
-    ap.add_argument("--path", default="whole", choices=["whole", "phases"],
+    ap.add_argument("--path", default="whole", choices=["whole", "phases", "sharded", "peer"],
                     help="whole: apms_compressed_step (the configurations of record); phases: the same step through "
-                         "apms_worker_phase / apms_server_phase_rows / apms_apply_phase (1-bit compressor only)")
+                         "apms_worker_phase / apms_server_phase_rows / apms_apply_phase (1-bit compressor only); "
+                         "sharded / peer: the workers split over the processes of a torchrun launch, messages exchanged")
+    ap.add_argument("--one-gpu", action="store_true", help="every process on cuda:0 (--path peer only)")
     ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16", "float16"],
                     help="element type of the gradient arrays (the configurations of record use float32)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -374,12 +398,16 @@ def main(argv=None) -> int:
         w = w.with_(chunk=args.chunk)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    local_rank = 0 if args.one_gpu else int(os.environ.get("LOCAL_RANK", "0"))
+    split = args.path in ("sharded", "peer")
+    if args.one_gpu and args.path != "peer":
+        raise SystemExit("--one-gpu exists for --path peer only (NCCL wants one GPU per process)")
     config = {"workload": f"{w.name}: d={w.d}, n={w.n} simulated workers, chunk={w.chunk}, {w.dist} gradients",
               "d": w.d, "n_workers": w.n, "chunk": w.chunk, "gradient_dtype": args.grad_dtype,
               "compressor": args.compressor if args.compressor == "onebit" else f"topk {args.topk_fraction}",
               "path": args.path,
-              "parallelism": f"replicas x{world}",
+              "parallelism": (f"{world} processes x {w.n // world} workers, {args.path} exchange"
+                              + (", all on one GPU" if args.one_gpu else "")) if split else f"replicas x{world}",
               "l2_policy": "inputs_exceed_l2" if 12 * w.d * w.n > (256 << 20) else "l2_resident",
               "gradient_ring": 2}
 
@@ -407,8 +435,18 @@ def main(argv=None) -> int:
     if libbuild.is_stale():
         libbuild.build()
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if world > 1 or split:
+        if args.one_gpu or world == 1:
+            if world == 1 and "MASTER_ADDR" not in os.environ:      # a plain `python bench.py --path sharded`
+                import socket
+
+                with socket.socket() as sock:
+                    sock.bind(("127.0.0.1", 0))
+                    port = sock.getsockname()[1]
+                os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK="0", WORLD_SIZE="1")
+            dist.init_process_group("gloo")           # handles and host flags only; every exchange is a load or a store
+        else:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks = measured_peaks()
 
     if args.sweep:
@@ -433,7 +471,12 @@ def main(argv=None) -> int:
 
     m = measure(w, args, rank, world, local_rank, dist, want_adam=args.adam, want_e2e=not args.no_e2e)
     ms_per_step, kernel_ms = m["ms_per_step"], m["kernel_ms"]
-    ab = algorithmic_bytes(w.d, w.n, w.chunk, 4 if args.grad_dtype == "float32" else 2)
+    n_local = w.n // world if split else w.n           # what one process's kernels move
+    ab = algorithmic_bytes(w.d, n_local, w.chunk, 4 if args.grad_dtype == "float32" else 2)
+    if split:                                          # a process serves 1 / world of the chunks, from all n workers' rows
+        full = algorithmic_bytes(w.d, w.n, w.chunk, 4 if args.grad_dtype == "float32" else 2)
+        ab["server"] = full["server"] // world
+        ab["step"] = ab["worker"] + ab["server"] + ab["apply"]
     if args.compressor == "topk":
         # g, z read, z write and both masks per worker, the binary32 momentum once; masks, the kept values,
         # zbar read + write, new momentum, v, x read, x write, server mask
@@ -446,7 +489,7 @@ def main(argv=None) -> int:
         ab["step"] = ab["worker"] + ab["server"]
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
     step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
-    traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * w.n
+    traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * n_local
                if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32"
                and args.compressor == "onebit" else None)
     roofline = {"bound": "hbm", "kernel": "k_worker", "achieved": wk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -464,15 +507,18 @@ def main(argv=None) -> int:
 
     if rank == 0:
         line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong" if split else "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": m["e2e"], "gpu_launches": m["launches"],
                 "clocks": m["clocks"],
                 "ms_per_step_min": m["ms_per_step_min"], "ms_per_step_median": m["ms_per_step_median"]}
         if m["adam"]:
             line["warmup_adam"] = m["adam"]
+        if "wire_bytes_per_step" in m:
+            line["wire_bytes_per_step_per_process"] = m["wire_bytes_per_step"]
         print(json.dumps(line))
-    if world > 1:
+    if dist.is_initialized():
         dist.destroy_process_group()
     return 0
 

@@ -63,7 +63,8 @@ typedef enum {
     APMS_ERR_OOM = 4,           /* workspace too small, or allocation failed               */
     APMS_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (reported by the next
                                    synchronising call; the context's state is then undefined) */
-    APMS_ERR_BOUNDS = 6         /* reserved: a checked build recorded an out-of-range index */
+    APMS_ERR_BOUNDS = 6         /* apms_check_guards found guard bytes overwritten: something wrote
+                                   outside an array of the workspace                        */
 } apms_status;
 
 /* Phases of Algorithm 1. */
@@ -395,6 +396,18 @@ apms_status apms_set_scale_kind(apms_ctx* ctx, apms_scale_kind kind);
 /* Launch-shape override (tuning and tests); results do not depend on it except for the order
  * of the binary64 additions inside a chunk's sum of squares. */
 apms_status apms_set_team_mode(apms_ctx* ctx, apms_team_mode mode);
+
+/* Guard bytes (a debugging aid that stands in for a memory checker).  apms_set_guard_bytes(b) is a
+ * process-wide switch read by apms_create and apms_workspace_bytes: contexts created while b > 0 (a multiple
+ * of 256, at most 1 MiB) lay out their workspace with at least b bytes that belong to no array behind every
+ * row of every array (each worker's compensated vector, sign words, scales, partial sums, ...) and before the
+ * first; apms_set_params and apms_freeze_v fill them with a fixed pattern.  apms_check_guards synchronises the
+ * stream, reads all guard bytes back and compares: APMS_OK if untouched, APMS_ERR_BOUNDS otherwise, with the
+ * workspace offset of the first changed byte in *bad_offset (may be NULL) and the array it follows named in
+ * apms_last_error.  Results of steps do not depend on the switch.  b = 0 restores the ordinary layout for
+ * contexts created afterwards. */
+apms_status apms_set_guard_bytes(size_t bytes);
+apms_status apms_check_guards(apms_ctx* ctx, int64_t* bad_offset);
 
 /* Kernel timing: when enabled, every kernel launch is bracketed by CUDA events on the
  * context's stream.  apms_kernel_time() synchronises the stream, returns the total time

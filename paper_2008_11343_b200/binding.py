@@ -78,6 +78,8 @@ SIGNATURES = {
     "apms_set_compressor": (C.c_int, [C.c_void_p, C.c_int, C.c_double]),
     "apms_uncompressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_set_guard_bytes": (C.c_int, [C.c_size_t]),
+    "apms_check_guards": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "apms_kernel_time": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "apms_selftest_wait_report": (C.c_int, [C.c_void_p, C.c_int]),
@@ -321,6 +323,23 @@ def apms_set_scale_kind(h, kind: int):
 
 def apms_set_team_mode(h, mode: int):
     _check(h, load().apms_set_team_mode(h, mode))
+
+
+def apms_set_guard_bytes(nbytes: int):
+    st = load().apms_set_guard_bytes(nbytes)
+    if st != OK:
+        raise ApmsError(st, load().apms_last_error(None).decode())
+
+
+def apms_check_guards(h) -> int:
+    """Raises ApmsError(ERR_BOUNDS) naming the array whose guard bytes changed; its .bad_offset is the workspace offset."""
+    bad = C.c_int64(-1)
+    st = load().apms_check_guards(h, C.byref(bad))
+    if st != OK:
+        err = ApmsError(st, load().apms_last_error(h).decode())
+        err.bad_offset = int(bad.value)
+        raise err
+    return int(bad.value)
 
 
 def apms_set_timing(h, enabled: bool):
@@ -589,6 +608,9 @@ class Context:
 
     def set_timing(self, enabled: bool):
         apms_set_timing(self._h, enabled)
+
+    def check_guards(self):
+        apms_check_guards(self._h)
 
     def kernel_time(self, which: int):
         return apms_kernel_time(self._h, which)

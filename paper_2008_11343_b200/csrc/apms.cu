@@ -53,6 +53,9 @@ namespace {
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// A guard region: bytes of the workspace that no kernel may write (see apms_set_guard_bytes).
+struct GuardRegion { size_t off, bytes; const char* what; };
+
 struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
     int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
@@ -60,42 +63,62 @@ struct Layout {
     int n;
     Tiling t;
     size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
+    size_t guard;                  // guard bytes behind every row of every array (0 = the ordinary layout)
 };
 
-bool make_layout(int64_t d, int n, int64_t chunk, Layout* L)
+size_t g_guard_bytes = 0;          // process-wide, read when a context is created
+
+// guard > 0: every row of every array is followed by at least `guard` bytes that belong to no array, and
+// so is the start of the workspace; `regions` (if given) receives them.
+bool make_layout(int64_t d, int n, int64_t chunk, Layout* L, size_t guard = 0, std::vector<GuardRegion>* regions = nullptr)
 {
     if (d < 1 || n < 1 || n > APMS_MAX_WORKERS || chunk < 32 || chunk % 32 != 0) return false;
     if (chunk > (int64_t)1 << 30) return false;
-    L->d = d; L->n = n; L->chunk = chunk;
+    L->d = d; L->n = n; L->chunk = chunk; L->guard = guard;
     L->C = (d + chunk - 1) / chunk;
     L->W = (d + 31) / 32;
-    L->dz = (int64_t)round_up((size_t)d, 64);
-    L->Wp = (int64_t)round_up((size_t)L->W, 64);
-    L->Cp = (int64_t)round_up((size_t)L->C, 64);
+    L->dz = (int64_t)round_up((size_t)d, 64) + (int64_t)(guard / 4);
+    L->Wp = (int64_t)round_up((size_t)L->W, 64) + (int64_t)(guard / 4);
+    L->Cp = (int64_t)round_up((size_t)L->C, 64) + (int64_t)(guard / 4);
     size_t o = 0;
-    auto take = [&](size_t bytes) { size_t at = o; o += round_up(bytes, 256); return at; };
-    L->off_x = take((size_t)L->dz * 4);
-    L->off_v = take((size_t)L->dz * 4);
-    L->off_m = take((size_t)L->dz * 4);
-    L->off_zbar = take((size_t)L->dz * 4);
-    L->off_z = take((size_t)L->dz * 4 * (size_t)n);
-    L->off_B = take((size_t)L->Wp * 4 * (size_t)n);
-    L->off_Bbar = take((size_t)L->Wp * 4);
-    L->off_s = take((size_t)L->Cp * 4 * (size_t)n);
-    L->off_Sbar = take((size_t)L->Cp * 4);
+    // `rows` rows of `stride` elements of `es` bytes, of which the first `used` are the array's own
+    auto take = [&](const char* what, size_t rows, size_t stride, size_t used, size_t es) {
+        const size_t at = o;
+        if (guard && regions)
+            for (size_t r = 0; r < rows; ++r)
+                if (stride > used) regions->push_back({at + (r * stride + used) * es, (stride - used) * es, what});
+        o += round_up(rows * stride * es, 256);
+        return at;
+    };
+    if (guard) {
+        if (regions) regions->push_back({0, guard, "the start of the workspace"});
+        o = guard;
+    }
+    const size_t ud = (size_t)d, un = (size_t)n;
+    L->off_x = take("x", 1, L->dz, ud, 4);
+    L->off_v = take("v", 1, L->dz, ud, 4);
+    L->off_m = take("m", 1, L->dz, ud, 4);
+    L->off_zbar = take("zbar", 1, L->dz, ud, 4);
+    L->off_z = take("z_i", un, L->dz, ud, 4);
+    L->off_B = take("B_i", un, L->Wp, L->W, 4);
+    L->off_Bbar = take("Bbar", 1, L->Wp, L->W, 4);
+    L->off_s = take("s_i", un, L->Cp, L->C, 4);
+    L->off_Sbar = take("Sbar", 1, L->Cp, L->C, 4);
     L->t.d = d; L->t.chunk = chunk;
     if (chunk <= kTileMax) { L->t.tile = chunk; L->t.P = 1; }
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
-    L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64);
-    L->off_part = take(L->t.P > 1 ? (size_t)L->t.Pp * 8 * (size_t)(n + 1) : 0);   // n worker rows + 1 server row
+    L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64) + (int64_t)(guard / 8);
+    L->off_part = take("partial sums of split chunks", L->t.P > 1 ? un + 1 : 0, L->t.Pp, (size_t)(L->C * L->t.P), 8);   // n worker rows + 1 server row
     L->fine_tiles = (chunk >= kFineSub) ? (d + kFineTile - 1) / kFineTile : 0;
     L->fine_split = (chunk % kFineSub != 0) ? 1 : 0;     // a warp's 512 elements may lie in two chunks: two partial sums each
-    L->fine_Pp = (int64_t)round_up((size_t)L->fine_tiles * kWarps * (size_t)(L->fine_split ? 2 : 1), 64);
-    L->off_fine = take((size_t)L->fine_Pp * 8 * (size_t)n);
-    L->off_stage = take((size_t)L->dz * 4 * 2);
-    L->off_mon = take(((size_t)(n + 1) * (size_t)((d + 4095) / 4096) + (size_t)(n + 1)) * 8);   // error monitor: tile sums + row sums
-    L->off_den = take((size_t)L->dz * 4);              // sqrt(v) + eps of the frozen v
-    L->off_status = take(256);
+    const size_t fine_used = (size_t)L->fine_tiles * kWarps * (size_t)(L->fine_split ? 2 : 1);
+    L->fine_Pp = (int64_t)round_up(fine_used, 64) + (int64_t)(guard / 8);
+    L->off_fine = take("partial sums of the fine worker form", un, L->fine_Pp, fine_used, 8);
+    L->off_stage = take("staging buffers", 2, L->dz, ud, 4);
+    const size_t mon_used = (un + 1) * (size_t)((d + 4095) / 4096) + (un + 1);
+    L->off_mon = take("error monitor sums", 1, round_up(mon_used, 32) + guard / 8, mon_used, 8);   // tile sums + row sums
+    L->off_den = take("den", 1, L->dz, ud, 4);              // sqrt(v) + eps of the frozen v
+    L->off_status = take("status", 1, 64 + guard / 4, 64, 4);
     L->total = o;
     return true;
 }
@@ -132,6 +155,7 @@ struct apms_ctx {
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
+    std::vector<GuardRegion> guards;   // empty in the ordinary layout
     char err[512];
 
     float* x() { return (float*)(ws + L.off_x); }
@@ -178,6 +202,15 @@ apms_status ensure_workspace(apms_ctx* c)
         return e == cudaErrorMemoryAllocation ? APMS_ERR_OOM : APMS_ERR_CUDA;
     }
     c->ws = (char*)p; c->ws_bytes = c->L.total; c->owns_ws = true;
+    return APMS_OK;            // guard regions are written by apms_set_params, the first call that touches the workspace
+}
+
+// Guard layout only: (re)writes the pattern into every guard region, on the context's stream.
+constexpr int kGuardByte = 0xA5;
+apms_status fill_guards(apms_ctx* c)
+{
+    for (const GuardRegion& g : c->guards)
+        APMS_CUDA(c, cudaMemsetAsync(c->ws + g.off, kGuardByte, g.bytes, c->stream));
     return APMS_OK;
 }
 
@@ -321,6 +354,12 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
         const int per = c->L.fine_split ? 2 : 1;
         // 512-element pieces a whole chunk can touch: its own, plus one at each end that it shares
         const int64_t slots = c->L.fine_split ? c->L.chunk / kFineSub + 2 : c->L.chunk / kFineSub;
+        if (slots > kFineLongSlots) {                 // long chunks: a CTA per (worker, chunk)
+            if (total > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) pairs for one launch");
+            k_finalize_fine_cta<<<(unsigned)total, kThreads, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0), c->L.Cp, ni, cb, nchunks,
+                                                                           c->L.d, c->L.chunk, per);
+            return launch_check(c, "k_finalize_fine_cta");
+        }
         int team = 1;
         while (team < 32 && team < slots) team *= 2;
         const int64_t per_cta = (int64_t)kWarps * (32 / team);
@@ -678,7 +717,7 @@ extern "C" {
 size_t apms_workspace_bytes(int64_t d, int n, int64_t chunk)
 {
     Layout L;
-    return make_layout(d, n, chunk, &L) ? L.total : 0;
+    return make_layout(d, n, chunk, &L, g_guard_bytes) ? L.total : 0;
 }
 
 apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float beta2, float eps,
@@ -687,7 +726,8 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     if (!out) { snprintf(g_create_error, sizeof g_create_error, "out is NULL"); return APMS_ERR_INVALID_ARG; }
     *out = nullptr;
     Layout L;
-    if (!make_layout(d, n, chunk, &L)) {
+    std::vector<GuardRegion> guards;
+    if (!make_layout(d, n, chunk, &L, g_guard_bytes, &guards)) {
         snprintf(g_create_error, sizeof g_create_error,
                  "invalid shape: need d >= 1, 1 <= n <= %d, chunk a positive multiple of 32 (got d=%lld n=%d chunk=%lld)",
                  APMS_MAX_WORKERS, (long long)d, n, (long long)chunk);
@@ -706,7 +746,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     }
     apms_ctx* c = new (std::nothrow) apms_ctx();
     if (!c) { snprintf(g_create_error, sizeof g_create_error, "host allocation failed"); return APMS_ERR_OOM; }
-    c->L = L; c->beta1 = beta1; c->beta2 = beta2; c->eps = eps; c->lr = lr;
+    c->L = L; c->guards.swap(guards); c->beta1 = beta1; c->beta2 = beta2; c->eps = eps; c->lr = lr;
     c->t = 0; c->phase = APMS_PHASE_CREATED; c->m_is_fp32 = true; c->v_checked = false; c->v_plain = false; c->den_valid = false;
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
@@ -744,9 +784,11 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     if (st != APMS_OK) return st;
     const size_t bytes = (size_t)c->L.d * 4;
     APMS_CUDA(c, cudaMemcpyAsync(c->x(), x0, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
-    APMS_CUDA(c, cudaMemsetAsync(c->m(), 0, (size_t)c->L.dz * 4, c->stream));
-    APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.dz * 4, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->m(), 0, (size_t)c->L.d * 4, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.d * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
+    st = fill_guards(c);
+    if (st != APMS_OK) return st;
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
     c->t = 0; c->steps = 0; c->csteps = 0; c->substep = 0; c->worker_chunks = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
     return APMS_OK;
@@ -792,6 +834,10 @@ apms_status apms_freeze_v(apms_ctx* c)
     if (c->phase != APMS_PHASE_WARMUP) return fail(c, APMS_ERR_BAD_STATE, "apms_freeze_v needs the WARMUP phase");
     // errors start at zero: z = 0 with scale 0 implies delta = 0 - (+0) = 0
     APMS_CUDA(c, cudaMemsetAsync(c->ws + c->L.off_zbar, 0, c->L.off_part - c->L.off_zbar, c->stream));
+    if (!c->guards.empty()) {                      // the one memset above ran over the guard regions in between
+        apms_status gst = fill_guards(c);
+        if (gst != APMS_OK) return gst;
+    }
     c->phase = APMS_PHASE_COMPRESSED;
     c->m_is_fp32 = true;
     c->v_checked = false;
@@ -1122,9 +1168,9 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
         if (worker < 0 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range");
         if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "errors exist only in the COMPRESSED phase");
         // delta = z - (+-0) = z: store the error as z with all scales of this worker zero
-        APMS_CUDA(c, cudaMemsetAsync(c->s(worker), 0, (size_t)c->L.Cp * 4, c->stream));
+        APMS_CUDA(c, cudaMemsetAsync(c->s(worker), 0, (size_t)c->L.C * 4, c->stream));
         if (c->compressor == APMS_COMPRESSOR_TOPK)      // top-k: delta = z - (mask ? z : 0) = z with an empty mask
-            APMS_CUDA(c, cudaMemsetAsync(c->B(worker), 0, (size_t)c->L.Wp * 4, c->stream));
+            APMS_CUDA(c, cudaMemsetAsync(c->B(worker), 0, (size_t)c->L.W * 4, c->stream));
         dst = c->z(worker);
         break;
     case APMS_STATE_SERVER_ERR:
@@ -1134,9 +1180,9 @@ apms_status apms_set_state(apms_ctx* c, apms_state_id which, int worker, const v
             if (mst != APMS_OK) return mst;
             c->m_is_fp32 = true;
         }
-        APMS_CUDA(c, cudaMemsetAsync(c->Sbar(), 0, (size_t)c->L.Cp * 4, c->stream));
+        APMS_CUDA(c, cudaMemsetAsync(c->Sbar(), 0, (size_t)c->L.C * 4, c->stream));
         if (c->compressor == APMS_COMPRESSOR_TOPK)
-            APMS_CUDA(c, cudaMemsetAsync(c->Bbar(), 0, (size_t)c->L.Wp * 4, c->stream));
+            APMS_CUDA(c, cudaMemsetAsync(c->Bbar(), 0, (size_t)c->L.W * 4, c->stream));
         dst = c->zbar();
         break;
     default: return fail(c, APMS_ERR_INVALID_ARG, "this state array cannot be set");
@@ -1319,6 +1365,39 @@ apms_status apms_set_scale_kind(apms_ctx* c, apms_scale_kind kind)
     if (kind != APMS_SCALE_L2 && kind != APMS_SCALE_L1_MEAN) return fail(c, APMS_ERR_INVALID_ARG, "unknown scale kind");
     c->L.t.l1 = kind == APMS_SCALE_L1_MEAN ? 1 : 0;
     return APMS_OK;
+}
+
+apms_status apms_set_guard_bytes(size_t bytes)
+{
+    if (bytes % 256 != 0 || bytes > ((size_t)1 << 20)) {
+        snprintf(g_create_error, sizeof g_create_error, "guard bytes must be a multiple of 256, at most 1 MiB");
+        return APMS_ERR_INVALID_ARG;
+    }
+    g_guard_bytes = bytes;
+    return APMS_OK;
+}
+
+apms_status apms_check_guards(apms_ctx* c, int64_t* bad_offset)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (bad_offset) *bad_offset = -1;
+    if (c->guards.empty()) return fail(c, APMS_ERR_BAD_STATE, "this context was created without guard bytes (apms_set_guard_bytes)");
+    if (c->phase == APMS_PHASE_CREATED || !c->ws) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    std::vector<unsigned char> host;
+    for (const GuardRegion& g : c->guards) {
+        host.resize(g.bytes);
+        APMS_CUDA(c, cudaMemcpy(host.data(), c->ws + g.off, g.bytes, cudaMemcpyDeviceToHost));
+        for (size_t k = 0; k < g.bytes; ++k) {
+            if (host[k] != (unsigned char)kGuardByte) {
+                if (bad_offset) *bad_offset = (int64_t)(g.off + k);
+                snprintf(c->err, sizeof c->err, "guard bytes behind %s were overwritten: workspace offset %zu (byte %zu of the %zu guard bytes there)",
+                         g.what, g.off + k, k, g.bytes);
+                return APMS_ERR_BOUNDS;
+            }
+        }
+    }
+    return device_status_check(c);
 }
 
 apms_status apms_set_team_mode(apms_ctx* c, apms_team_mode mode)

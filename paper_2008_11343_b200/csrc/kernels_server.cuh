@@ -339,6 +339,16 @@ k_server_staged(const ServerStagedArgs sa)
         // all consumers see the same result and leave together, whenever the producer may have set the flag.
         const volatile int* vfailed = &failed;
         int q = 0;
+        // The scales of a chunk are fetched from global memory while the chunk before it is being worked on
+        // (threads 0 .. n-1 one worker's scale each, every thread the server's old scale).
+        static_assert(APMS_MAX_WORKERS <= kThreads, "one scale per thread");
+        uint32_t pre_neg = 0u;
+        float pre_S = 0.0f;
+        {
+            const Item it0 = decode_item(a.t, item0);
+            if ((int)threadIdx.x < n) pre_neg = __float_as_uint(a.srow[threadIdx.x][it0.c]) | 0x80000000u;
+            pre_S = a.Sbar[it0.c];
+        }
         for (int w = 0; w < nitems; ++w) {
             const Item it = decode_item(a.t, item0 + w);
             const int L = it.L;
@@ -346,9 +356,13 @@ k_server_staged(const ServerStagedArgs sa)
             const int64_t wofs = it.base / 32;
             const int off_in = (int)((wofs + sa.row_align) & 3), off_out = (int)(wofs & 3);
             uint32_t* negs = neg_s[w & 1];
-            for (int i = threadIdx.x; i < n; i += kThreads)
-                negs[i] = __float_as_uint(a.srow[i][it.c]) | 0x80000000u;
-            const float S_old = a.Sbar[it.c];
+            if ((int)threadIdx.x < n) negs[threadIdx.x] = pre_neg;
+            const float S_old = pre_S;
+            if (MULTI && w + 1 < nitems) {
+                const Item nx = decode_item(a.t, item0 + w + 1);
+                if ((int)threadIdx.x < n) pre_neg = __float_as_uint(a.srow[threadIdx.x][nx.c]) | 0x80000000u;
+                pre_S = a.Sbar[nx.c];
+            }
             if (consumer_barrier_any(*vfailed != 0)) break;      // -s_i in place; everybody is done with the previous chunk
             bool ok = true;
             double acc = 0.0;
@@ -485,11 +499,13 @@ k_server_packed(const ServerStagedArgs sa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const ServerArgs& a = sa.a;
-    __shared__ double red[kPackedMaxChunks];                          // one sum of squares per group of the slab
+    // Everything the consumers hand to each other is double-buffered over the walk, so that one barrier per
+    // slab suffices: what slab w+1 writes, slab w-1 was the last to read, and two barriers lie in between.
+    __shared__ double red[2][kPackedMaxChunks];                          // one sum of squares per group of the slab
     __shared__ uint64_t full[kStages], empty[kStages];
-    __shared__ uint32_t neg_s[2][kPackedMaxChunks * APMS_MAX_WORKERS];   // -s_i per chunk of the slab, double-buffered over the walk
+    __shared__ uint32_t neg_s[2][kPackedMaxChunks * APMS_MAX_WORKERS];   // -s_i per chunk of the slab
     __shared__ float S_old_sh[2][kPackedMaxChunks];
-    __shared__ __align__(16) uint32_t nb[kSlabWords];                 // the slab's new sign words
+    __shared__ __align__(16) uint32_t nb[2][kSlabWords];                 // the slab's new sign words
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -497,10 +513,8 @@ k_server_packed(const ServerStagedArgs sa)
     const size_t stage_bytes = staged_stage_bytes(n, true);
     const int chunk = (int)a.t.chunk;                                  // 128 .. 1024, divides kSlab
     const int gpc = chunk / kGroup;                                    // groups per chunk
-    const int64_t nslabs_all = (a.t.d + kSlab - 1) / kSlab;
     const int64_t slab_first = a.item0 + (int64_t)blockIdx.x * sa.span;       // items are slabs here
     const int nmine = (int)(a.items - slab_first < sa.span ? a.items - slab_first : sa.span);
-    (void)nslabs_all;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
@@ -548,23 +562,57 @@ k_server_packed(const ServerStagedArgs sa)
         const int wl = lane >> 3;
         const int g0 = warp, g1 = warp + kWarps;
         const int k0 = g0 / gpc, k1 = g1 / gpc;                          // the chunks (within the slab) of this warp's two groups
+        const int kmax = kSlab / chunk;                                  // chunks per whole slab
         const volatile int* vfailed = &failed;
         const int off_in = sa.row_align;
-        int q = 0;
-        for (int w = 0; w < nmine; ++w) {
+        // this thread's share of a slab's scales: entry idx = kk * n + i for idx = threadIdx.x + 256 r
+        constexpr int kPre = kPackedMaxChunks * APMS_MAX_WORKERS / kThreads;
+        uint32_t pre[kPre];
+        float pre_S = 0.0f;
+        auto fetch_scales = [&](int w) {                                  // global loads only: issued long before they are stored
             const int64_t base_e = (slab_first + w) * kSlab;
             const int64_t left = a.t.d - base_e;
             const int L = (int)(left < kSlab ? left : kSlab);
             const int64_t c0 = base_e / chunk;
             const int nchunks = (L + chunk - 1) / chunk;
-            uint32_t* negs = neg_s[w & 1];
-            float* Sold = S_old_sh[w & 1];
-            for (int idx = threadIdx.x; idx < nchunks * n; idx += kThreads) {
-                const int kk = idx / n, i = idx - kk * n;
-                negs[kk * APMS_MAX_WORKERS + i] = __float_as_uint(a.srow[i][c0 + kk]) | 0x80000000u;
+#pragma unroll
+            for (int r = 0; r < kPre; ++r) {
+                const int idx = (int)threadIdx.x + r * kThreads;
+                pre[r] = 0u;
+                if (idx < nchunks * n) {
+                    const int kk = idx / n, i = idx - kk * n;
+                    pre[r] = __float_as_uint(a.srow[i][c0 + kk]) | 0x80000000u;
+                }
             }
-            if (threadIdx.x < nchunks) Sold[threadIdx.x] = a.Sbar[c0 + threadIdx.x];
-            if (consumer_barrier_any(*vfailed != 0)) break;      // -s_i and old scales in place; everybody is done with the previous slab
+            pre_S = ((int)threadIdx.x < nchunks) ? a.Sbar[c0 + threadIdx.x] : 0.0f;
+        };
+        auto store_scales = [&](int buf) {
+#pragma unroll
+            for (int r = 0; r < kPre; ++r) {
+                const int idx = (int)threadIdx.x + r * kThreads;
+                if (idx < kmax * n) {
+                    const int kk = idx / n, i = idx - kk * n;
+                    neg_s[buf][kk * APMS_MAX_WORKERS + i] = pre[r];
+                }
+            }
+            if ((int)threadIdx.x < kmax) S_old_sh[buf][threadIdx.x] = pre_S;
+        };
+        bool leave = false;
+        if (nmine > 0) {
+            fetch_scales(0);
+            store_scales(0);
+        }
+        leave = consumer_barrier_any(*vfailed != 0);                      // the first slab's scales are in place
+        int q = 0;
+        for (int w = 0; w < nmine && !leave; ++w) {
+            const int buf = w & 1;
+            const int64_t base_e = (slab_first + w) * kSlab;
+            const int64_t left = a.t.d - base_e;
+            const int L = (int)(left < kSlab ? left : kSlab);
+            const int64_t c0 = base_e / chunk;
+            const int nchunks = (L + chunk - 1) / chunk;
+            const uint32_t* negs = neg_s[buf];
+            if (w + 1 < nmine) fetch_scales(w + 1);                       // in flight during this slab's arithmetic
             bool ok = true;
             double acc0 = 0.0, acc1 = 0.0;
             {
@@ -581,7 +629,7 @@ k_server_packed(const ServerStagedArgs sa)
                     const int kk0 = k0 < nchunks ? k0 : 0, kk1 = k1 < nchunks ? k1 : 0;
                     signed_scale_sums2<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl,
                                            negs + kk0 * APMS_MAX_WORKERS, negs + kk1 * APMS_MAX_WORKERS, n, sh, s01, s23, t01, t23);
-                    const float So0 = Sold[kk0], So1 = Sold[kk1];
+                    const float So0 = S_old_sh[buf][kk0], So1 = S_old_sh[buf][kk1];
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
 #pragma unroll
@@ -608,32 +656,32 @@ k_server_packed(const ServerStagedArgs sa)
                         if (u) acc1 = acc; else acc0 = acc;
                         st4_checked(a.zbar + base_e, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
                         const uint32_t word = pack_group_words(nibble, lane);
-                        if ((lane & 7) == 0) nb[grp * 4 + wl] = word;        // words past L hold zeros and are never stored
+                        if ((lane & 7) == 0) nb[buf][grp * 4 + wl] = word;    // words past L hold zeros and are never stored
                     }
                 }
                 ++q;
             }
             acc0 = warp_sum(acc0);
             acc1 = warp_sum(acc1);
-            if (lane == 0) { red[g0] = acc0; red[g1] = acc1; }
-            const bool leave = consumer_barrier_any(!ok || *vfailed != 0);   // the groups' sums and the slab's sign words are in shared memory
+            if (lane == 0) { red[buf][g0] = acc0; red[buf][g1] = acc1; }
+            if (w + 1 < nmine) store_scales(buf ^ 1);                     // the next slab's scales, fetched above
+            leave = consumer_barrier_any(!ok || *vfailed != 0);           // the groups' sums and the slab's sign words are in shared memory
             if (leave) break;
+            // The new scale of every chunk of the slab, one chunk per lane (so that a warp runs the binary64
+            // division and square root once), handed to the lanes that need it by shuffles.
+            float S_lane = 0.0f;
+            if (lane < nchunks) {
+                double total = 0.0;
+                for (int r = 0; r < gpc; ++r) total += red[buf][lane * gpc + r];           // group order
+                const int64_t cbeg = (c0 + lane) * (int64_t)chunk;
+                const int64_t Lc = (a.t.d - cbeg < chunk) ? a.t.d - cbeg : chunk;
+                S_lane = (float)sqrt(total / (double)Lc);
+                if (warp == 0) a.Sbar[c0 + lane] = S_lane;
+            }
             // Section 3.3 steps 5-6 for this slab: every group with the new scale of its chunk
             float c_new[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int kk = u ? k1 : k0;
-                float S_new = 0.0f;
-                if (kk < nchunks) {
-                    double total = 0.0;
-                    for (int r = 0; r < gpc; ++r) total += red[kk * gpc + r];          // group order
-                    const int64_t cbeg = (c0 + kk) * (int64_t)chunk;
-                    const int64_t Lc = (a.t.d - cbeg < chunk) ? a.t.d - cbeg : chunk;
-                    S_new = (float)sqrt(total / (double)Lc);
-                    if (lane == 0 && (u ? g1 : g0) == kk * gpc) a.Sbar[c0 + kk] = S_new;     // the warp that holds the chunk's first group
-                }
-                c_new[u] = __fmul_rn(sa.lr, S_new);                  // lr * (+-S) = +-(lr * S)
-            }
+            c_new[0] = __fmul_rn(sa.lr, __shfl_sync(0xffffffffu, S_lane, k0));      // lr * (+-S) = +-(lr * S)
+            c_new[1] = __fmul_rn(sa.lr, __shfl_sync(0xffffffffu, S_lane, k1));
             {
                 const int st = q % kStages;
                 if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
@@ -652,7 +700,7 @@ k_server_packed(const ServerStagedArgs sa)
                     for (int u = 0; u < 2; ++u) {
                         const int grp = u ? g1 : g0;
                         const int k = grp * kGroup + lane * 4;
-                        const uint32_t nib = nb[grp * 4 + wl] >> sh;
+                        const uint32_t nib = nb[buf][grp * 4 + wl] >> sh;
                         xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, c_new[u]);
                         xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new[u]);
                         xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new[u]);
@@ -667,8 +715,8 @@ k_server_packed(const ServerStagedArgs sa)
                 uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
                 const int nwords = (L + 31) / 32;
                 const int w4 = threadIdx.x * 4;
-                if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
-                else for (int r = w4; r < nwords; ++r) ob[r] = nb[r];
+                if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb[buf] + w4));
+                else for (int r = w4; r < nwords; ++r) ob[r] = nb[buf][r];
             }
         }
     }

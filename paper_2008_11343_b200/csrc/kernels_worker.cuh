@@ -139,8 +139,9 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 // Chunks are multiples of 32 elements, so a chunk boundary inside a warp's 512 elements falls
 // between two sign words, i.e. between two 8-lane groups of one 128-element access, and there is at
 // most one of them (chunk >= 512).  With SPLIT (chunks that are not multiples of 512) a warp that
-// sees a boundary reads the scales of both chunks and keeps two sums; every warp then writes two
-// slots: [0] = its elements of the chunk its first element belongs to, [1] = those of the next chunk.
+// sees a boundary reads the scales of both chunks and keeps two sums; a piece then has two slots:
+// [0] = its elements of the chunk its first element belongs to, [1] = those of the next chunk (written
+// and read only where there is one).  A warp without a boundary runs the same code as without SPLIT.
 // Launch order: runs of `run` consecutive tiles of one worker, then the same tiles of the next
 // worker: every stream is read in long sequential pieces (measured: the longer the better for
 // DRAM), while the momentum bits of a run (run * 512 bytes) stay in L2 for the other workers.
@@ -150,6 +151,7 @@ constexpr int kFineU = kFineTile / (kThreads * 4);
 constexpr int kFineSub = kFineTile / kWarps;      // elements per warp = per partial sum
 constexpr int kFineSubWords = kFineSub / 32;
 constexpr int kFineRunDefault = 4096;
+constexpr int64_t kFineLongSlots = 1024;  // chunks with more 512-element pieces than this get a whole CTA in the finalize
 
 struct WorkerFineArgs {
     float* z; int64_t dz;
@@ -162,6 +164,70 @@ struct WorkerFineArgs {
     int i0, ni, run;
     float beta1, omb1;
 };
+
+// One warp's 512 elements (L of them live).  TWO: a chunk boundary lies inside, at sign word `bw`: the lanes whose
+// word lies past it use the next chunk's scales (s_hi, S_hi) and add their squares to acc_hi.
+template <int GT, bool SENDG, bool TWO>
+__device__ __forceinline__ void fine_piece(const WorkerFineArgs& a, const void* __restrict__ g, float* __restrict__ z,
+                                           const uint32_t* __restrict__ mbits, uint32_t* __restrict__ obits, int lane, int L,
+                                           int bw, float s_lo, float S_lo, float s_hi, float S_hi, double& acc, double& acc_hi)
+{
+    if (L == kFineSub) {
+        float4 gv[kFineU], zv[kFineU];
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
+            zv[u] = ld_stream4(z + u * kGroup + lane * 4);
+        }
+        const uint32_t mine = (!SENDG && lane < 4 * kFineU) ? mbits[lane] : 0u;
+        uint32_t outw = 0;
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
+            const bool hi = TWO && (u * 4 + (lane >> 3) >= bw);      // this lane's word lies in the next chunk
+            const float s_old = hi ? s_hi : s_lo, Sbar = hi ? S_hi : S_lo;
+            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+            const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
+            float zn[4];
+            uint32_t nibble = 0;
+            double part = TWO ? 0.0 : acc;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
+                const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
+                zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
+                const double zd = (double)zn[e];
+                part = fma(zd, zd, part);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
+            if (TWO) { acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0; }
+            else acc = part;
+            st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
+            const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
+            if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
+        }
+        if (lane < 4 * kFineU) __stcs(obits + lane, outw);
+    } else {
+        const int ngroups = (L + kGroup - 1) / kGroup;
+        for (int grp = 0; grp < ngroups; ++grp) {
+            const int k = grp * kGroup + lane * 4;
+            const float4 gv = ld_grad4_checked<GT>(g, k, L);
+            const float4 zv = ld4_checked(z, k, L, true);
+            const uint32_t mw = (!SENDG && k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
+            if (TWO) {
+                const bool hi = grp * 4 + (lane >> 3) >= bw;
+                double part = 0.0;
+                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, hi ? s_hi : s_lo, hi ? S_hi : S_lo, gv, zv,
+                                          make_float4(0, 0, 0, 0), mw, part, false, SENDG);
+                acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0;
+            } else {
+                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_lo, S_lo, gv, zv,
+                                          make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
+            }
+        }
+    }
+}
 
 template <int GT, bool SENDG, bool SPLIT>          // SENDG: the gradient-compressing variant (no momentum is read)
 __global__ void __launch_bounds__(kThreads, 4)
@@ -181,7 +247,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + (t * kWarps + warp) * (SPLIT ? 2 : 1);
     const int64_t left = a.d - base;
     if (left <= 0) {                                           // past the end of the vector
-        if (lane == 0) { slot[0] = 0.0; if (SPLIT) slot[1] = 0.0; }
+        if (lane == 0) *slot = 0.0;
         return;
     }
     const int L = (int)(left < kFineSub ? left : kFineSub);
@@ -191,70 +257,20 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
     uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
     const float* __restrict__ srow = a.s + (int64_t)i * a.Cp;
-    // first sign word of this warp's elements that belongs to chunk c + 1 (>= kFineSubWords: none does)
-    const int bw = SPLIT ? (int)(((c + 1) * a.chunk - base) >> 5) : kFineSubWords;
-    const bool two = SPLIT && bw * 32 < L;
     const float s_lo = srow[c], S_lo = a.Sbar[c];
-    const float s_hi = two ? srow[c + 1] : s_lo, S_hi = two ? a.Sbar[c + 1] : S_lo;
     double acc = 0.0, acc_hi = 0.0;
-    if (L == kFineSub) {
-        float4 gv[kFineU], zv[kFineU];
-#pragma unroll
-        for (int u = 0; u < kFineU; ++u) {
-            gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
-            zv[u] = ld_stream4(z + u * kGroup + lane * 4);
-        }
-        const uint32_t mine = (!SENDG && lane < 4 * kFineU) ? mbits[lane] : 0u;
-        uint32_t outw = 0;
-#pragma unroll
-        for (int u = 0; u < kFineU; ++u) {
-            const uint32_t nib = __shfl_sync(0xffffffffu, mine, u * 4 + (lane >> 3)) >> (4 * (lane & 7));
-            const bool hi = SPLIT && (u * 4 + (lane >> 3) >= bw);      // this lane's word lies in chunk c + 1
-            const float s_old = hi ? s_hi : s_lo, Sbar = hi ? S_hi : S_lo;
-            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
-            const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
-            float zn[4];
-            uint32_t nibble = 0;
-            double part = SPLIT ? 0.0 : acc;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float mm = bit_scale((nib >> e) & 1u, Sbar);                    // m = +-Sbar
-                const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));    // local momentum
-                zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old));                   // compensated
-                const double zd = (double)zn[e];
-                part = fma(zd, zd, part);
-                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
-            }
-            if (SPLIT) { acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0; }
-            else acc = part;
-            st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
-            const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
-            const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
-            if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
-        }
-        if (lane < 4 * kFineU) __stcs(obits + lane, outw);
+    // elements of this warp that belong to chunk c + 1 begin at its sign word bw (SPLIT only; rare for long chunks)
+    const int64_t next = (c + 1) * a.chunk - base;
+    if (SPLIT && next < L) {
+        fine_piece<GT, SENDG, true>(a, g, z, mbits, obits, lane, L, (int)(next >> 5), s_lo, S_lo, srow[c + 1], a.Sbar[c + 1], acc, acc_hi);
+        acc = warp_sum(acc);
+        acc_hi = warp_sum(acc_hi);
+        if (lane == 0) { slot[0] = acc; slot[1] = acc_hi; }
     } else {
-        const int ngroups = (L + kGroup - 1) / kGroup;
-        for (int grp = 0; grp < ngroups; ++grp) {
-            const int k = grp * kGroup + lane * 4;
-            const float4 gv = ld_grad4_checked<GT>(g, k, L);
-            const float4 zv = ld4_checked(z, k, L, true);
-            const uint32_t mw = (!SENDG && k < L) ? mbits[grp * 4 + (lane >> 3)] : 0u;
-            const bool hi = SPLIT && (grp * 4 + (lane >> 3) >= bw);
-            if (SPLIT) {
-                double part = 0.0;
-                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, hi ? s_hi : s_lo, hi ? S_hi : S_lo, gv, zv,
-                                          make_float4(0, 0, 0, 0), mw, part, false, SENDG);
-                acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0;
-            } else {
-                worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_lo, S_lo, gv, zv,
-                                          make_float4(0, 0, 0, 0), mw, acc, false, SENDG);
-            }
-        }
+        fine_piece<GT, SENDG, false>(a, g, z, mbits, obits, lane, L, 0, s_lo, S_lo, s_lo, S_lo, acc, acc_hi);
+        acc = warp_sum(acc);
+        if (lane == 0) slot[0] = acc;                          // slot [1] of a piece without a boundary is never read
     }
-    acc = warp_sum(acc);
-    if (SPLIT) acc_hi = warp_sum(acc_hi);
-    if (lane == 0) { slot[0] = acc; if (SPLIT) slot[1] = acc_hi; }
 }
 
 // Scales from the fine form's partial sums (one - or, with chunks that are not multiples of 512, two -
@@ -284,6 +300,27 @@ k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restric
 #pragma unroll
     for (int o = T / 2; o > 0; o >>= 1) total += __shfl_down_sync(0xffffffffu, total, o, T);
     if (live && sub == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+}
+
+// The same for long chunks (thousands of pieces each, few chunks): one CTA per (row, chunk); thread t adds the
+// pieces t, t + 256, ... and the block sum adds the threads in a fixed order.
+__global__ void __launch_bounds__(kThreads)
+k_finalize_fine_cta(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
+                    int rows, int64_t c_first, int64_t C, int64_t d, int64_t chunk, int per)
+{
+    __shared__ double red[kWarps];
+    const int r = (int)(blockIdx.x / C);
+    const int64_t c = c_first + blockIdx.x % C;
+    const int64_t cbeg = c * chunk;
+    const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
+    const int64_t q0 = cbeg / kFineSub, q1 = (cbeg + Lc + kFineSub - 1) / kFineSub;
+    const double* __restrict__ row = partial + (int64_t)r * Pp;
+    double total = 0.0;
+#pragma unroll 4
+    for (int64_t q = q0 + threadIdx.x; q < q1; q += kThreads)
+        total += row[q * per + ((per == 2 && q * kFineSub < cbeg) ? 1 : 0)];
+    total = block_sum(total, red);
+    if (threadIdx.x == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
 }
 
 // Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).

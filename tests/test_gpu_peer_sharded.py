@@ -152,3 +152,30 @@ def test_two_processes_on_one_gpu_exchange_through_mapped_workspaces(tmp_path):
     res = {r: json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)}
     assert res[0][0] and res[1][0], res
     assert max(res[0][1], res[1][1]) < 0.1 * 4 * d * n_local
+
+
+@pytest.mark.parametrize("path,nproc", [("peer", 2), ("sharded", 1), ("peer", 1)])
+def test_bench_runs_the_split_layouts(path, nproc, tmp_path):
+    """bench.py --path peer under a two-process launch with both processes on the one GPU (what a
+    one-process-per-GPU run executes, the peer's memory on the same device), and both split paths with a single
+    process: one JSON line, strong scaling, the workload's workers divided over the processes."""
+    import json
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={nproc}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port),
+           os.path.join(ROOT, "bench.py"), "--gpus", str(nproc), "--path", path, "--config", "1",
+           "--steps", "3", "--warmup", "3", "--no-cpu-baseline"]
+    if nproc > 1:
+        cmd.append("--one-gpu")
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    line = json.loads(lines[0])
+    assert line["scaling"] == "strong" and line["n_gpus"] == nproc and line["value"] > 0
+    assert line["config"]["n_workers"] == 8 and f"{nproc} processes x {8 // nproc} workers" in line["config"]["parallelism"]
+    assert line["gpu_launches"] >= 3 * 3 and "worker" in line["roofline"]["kernel_ms"]

@@ -46,6 +46,9 @@ UNIT = "worker-elements/s"
 # dram__bytes_write.sum per launch) on a smaller case of the same kernel, in bytes per
 # worker-element; scaled by n*d for the benchmarked launch.  Source: profiles/*.md.
 NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT = 11.96    # k_worker_fine, profiles/k_worker_fine_small_case.md
+# The fused server + update kernel, same kind of capture at n = 8 workers (profiles/k_server_staged_small_case.md):
+# 19.49 B per element; each further worker adds its sign words, 1/8 B per element (the traffic grows in proportion).
+NCU_SERVER_FUSED_TRAFFIC_BYTES_PER_ELEMENT_N8 = 19.49
 
 
 def algorithmic_bytes(d: int, n: int, chunk: int, grad_bytes: int = 4) -> dict:
@@ -492,8 +495,13 @@ def main(argv=None) -> int:
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * n_local
                if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32"
                and args.compressor == "onebit" else None)
+    fused = args.compressor == "onebit" and "apply" not in kernel_ms and not split and w.chunk >= 2048
+    traffic_by_kernel = {"worker": traffic,
+                         "server": ((NCU_SERVER_FUSED_TRAFFIC_BYTES_PER_ELEMENT_N8 + (w.n - 8) / 8.0) * w.d
+                                    if fused and args.grad_dtype == "float32" else None)}
     roofline = {"bound": "hbm", "kernel": "k_worker", "achieved": wk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": wk_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": traffic,
+                "traffic_by_kernel": traffic_by_kernel,
                 "algorithmic_bytes_per_launch": ab["worker"],
                 "whole_step": {"algorithmic_bytes": ab["step"], "achieved": step_gbs,
                                "frac": step_gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": step_gbs / 8000.0},

@@ -578,7 +578,7 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
             sa.a = a; sa.status = c->status();
             sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
             sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr; sa.row_align = row_align;
-            const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused);
+            const size_t smem = (size_t)kStages * staged_stage_bytes(a.n, fused) + staged_nb_bytes(c->L.t.tile);
             sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
             const int64_t fill = count / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
             if (sa.span > 1 && fill < sa.span) sa.span = fill < 1 ? 1 : (int)fill;

@@ -232,16 +232,45 @@ __host__ __device__ __forceinline__ size_t staged_stage_bytes(int n, bool fused)
     return (fused && apply > server) ? apply : server;
 }
 
+// Bytes of the buffer of new sign words behind the ring: the words of all slabs of a tile - every consumer warp
+// writes its words of the last slab too, live or not - plus up to three words before the first.
+__host__ __device__ __forceinline__ size_t staged_nb_bytes(int64_t tile_elems)
+{
+    const int64_t nslabs = (tile_elems + kSlab - 1) / kSlab;
+    return (size_t)(nslabs * kSlabWords + 4) * 4;
+}
+
 // Sum over the workers, in worker order, of +-s_i for the lane's 2 x 4 elements of one slab.
 // NT > 0: the number of workers is the compile-time constant NT (fully unrolled).
+// NT >= 8: the running sum starts at zero, so after the first eight workers it is a function of their
+// eight sign bits alone; `prefix8` holds it for all 256 patterns (built once per chunk with the same
+// eight additions in the same order, see build_prefix8).  The lane gathers, per group, its four elements'
+// bits of the eight workers into the four bytes of one word - the nibble times 0x00204081 spreads bits
+// 0..3 to bits 0, 8, 16, 24 (all partial products fall on distinct bits, so nothing carries), shifted
+// left by the worker's index - and looks the four sums up; the other workers are added one by one.
+constexpr int kPrefixWorkers = 8;
+
 template <int NT>
 __device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r0, const uint32_t* __restrict__ r1,
-                                                  const uint32_t* __restrict__ neg_s, int n, int sh,
+                                                  const uint32_t* __restrict__ neg_s, const float* __restrict__ prefix8, int n, int sh,
                                                   float2& s01, float2& s23, float2& t01, float2& t23)
 {
     const int nn = NT > 0 ? NT : n;
+    constexpr int kFirst = NT >= kPrefixWorkers ? kPrefixWorkers : 0;
+    if (NT >= kPrefixWorkers) {
+        uint32_t i0 = 0u, i1 = 0u;
+#pragma unroll
+        for (int i = 0; i < kPrefixWorkers; ++i) {
+            const uint32_t n0 = (r0[i * kRowWords] >> sh) & 0xFu;
+            const uint32_t n1 = (r1[i * kRowWords] >> sh) & 0xFu;
+            i0 |= (n0 * (0x00204081u << i)) & (0x01010101u << i);
+            i1 |= (n1 * (0x00204081u << i)) & (0x01010101u << i);
+        }
+        s01.x = prefix8[i0 & 0xFFu]; s01.y = prefix8[(i0 >> 8) & 0xFFu]; s23.x = prefix8[(i0 >> 16) & 0xFFu]; s23.y = prefix8[i0 >> 24];
+        t01.x = prefix8[i1 & 0xFFu]; t01.y = prefix8[(i1 >> 8) & 0xFFu]; t23.x = prefix8[(i1 >> 16) & 0xFFu]; t23.y = prefix8[i1 >> 24];
+    }
 #pragma unroll(NT > 0 ? NT : 4)
-    for (int i = 0; i < nn; ++i) {
+    for (int i = kFirst; i < nn; ++i) {
         const uint32_t ns = neg_s[i];
         // the lane's four sign bits moved to bits 28..31; a set bit turns -s_i into +s_i
         const uint32_t y0 = r0[i * kRowWords] << (28 - sh);
@@ -258,6 +287,19 @@ __device__ __forceinline__ void signed_scale_sums(const uint32_t* __restrict__ r
     }
 }
 
+// Entry t of the table: 0 + (+-s_0) + (+-s_1) + ... + (+-s_7) in this order, bit i of t set meaning +s_i.
+// `mine` is, in lanes 0..7 of every warp, the bit pattern of -s_lane; one entry per consumer thread.
+__device__ __forceinline__ float prefix8_entry(uint32_t mine, uint32_t t)
+{
+    float acc = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kPrefixWorkers; ++i) {
+        const uint32_t ns = __shfl_sync(0xffffffffu, mine, i);
+        acc = __fadd_rn(acc, __uint_as_float(ns ^ (((t >> i) & 1u) << 31)));
+    }
+    return acc;
+}
+
 // A CTA of the fused form walks `span` consecutive chunks (short chunks are grouped so that a CTA
 // still streams about 32768 elements and the ring never drains between chunks); the unfused form
 // (chunks cut into tiles) handles one tile.  Jobs are numbered across the CTA's whole walk: per
@@ -270,13 +312,15 @@ k_server_staged(const ServerStagedArgs sa)
     const ServerArgs& a = sa.a;
     __shared__ double red[kWarps];
     __shared__ uint64_t full[kStages], empty[kStages];
-    __shared__ uint32_t neg_s[2][APMS_MAX_WORKERS];   // bit patterns of -s_i, double-buffered over the walk
-    __shared__ __align__(16) uint32_t nb[kTileMax / 32 + 4];   // the current tile's new sign words, from the 16-byte boundary below the first
+    __shared__ uint32_t neg_s[APMS_MAX_WORKERS];      // bit patterns of -s_i of the current chunk
+    __shared__ float prefix8[NT >= kPrefixWorkers ? 256 : 1];         // see signed_scale_sums
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n = NT > 0 ? NT : a.n;
     const size_t stage_bytes = staged_stage_bytes(n, FUSED);
+    // behind the ring: the current tile's new sign words, from the 16-byte boundary below the first (staged_nb_bytes)
+    uint32_t* const nb = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes);
     const int span = MULTI ? sa.span : 1;                  // MULTI = false: one item, the walk's loops fold away
     const int64_t item0 = a.item0 + (int64_t)blockIdx.x * span;
     const int nitems = MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1;
@@ -339,14 +383,16 @@ k_server_staged(const ServerStagedArgs sa)
         // all consumers see the same result and leave together, whenever the producer may have set the flag.
         const volatile int* vfailed = &failed;
         int q = 0;
-        // The scales of a chunk are fetched from global memory while the chunk before it is being worked on
-        // (threads 0 .. n-1 one worker's scale each, every thread the server's old scale).
-        static_assert(APMS_MAX_WORKERS <= kThreads, "one scale per thread");
+        // The scales of a chunk are fetched from global memory while the chunk before it is being worked on:
+        // lane i of every warp (and lane i of warps 0, 1 for i + 32 when there are more than 32 workers) holds
+        // -s_i, every thread the server's old scale.
+        static_assert(APMS_MAX_WORKERS <= 64, "two scales per lane of the first two warps at most");
         uint32_t pre_neg = 0u;
         float pre_S = 0.0f;
+        const int my_worker = (warp < 2 && n > 32) ? warp * 32 + lane : lane;     // n <= 32: every warp fetches workers 0..n-1
         {
             const Item it0 = decode_item(a.t, item0);
-            if ((int)threadIdx.x < n) pre_neg = __float_as_uint(a.srow[threadIdx.x][it0.c]) | 0x80000000u;
+            if (my_worker < n) pre_neg = __float_as_uint(a.srow[my_worker][it0.c]) | 0x80000000u;
             pre_S = a.Sbar[it0.c];
         }
         for (int w = 0; w < nitems; ++w) {
@@ -355,12 +401,13 @@ k_server_staged(const ServerStagedArgs sa)
             const int nslabs = (L + kSlab - 1) / kSlab;
             const int64_t wofs = it.base / 32;
             const int off_in = (int)((wofs + sa.row_align) & 3), off_out = (int)(wofs & 3);
-            uint32_t* negs = neg_s[w & 1];
-            if ((int)threadIdx.x < n) negs[threadIdx.x] = pre_neg;
+            const uint32_t* negs = neg_s;
+            if ((warp == 0 || (warp == 1 && n > 32)) && my_worker < n) neg_s[my_worker] = pre_neg;
+            if (NT >= kPrefixWorkers) prefix8[threadIdx.x] = prefix8_entry(pre_neg, threadIdx.x);
             const float S_old = pre_S;
             if (MULTI && w + 1 < nitems) {
                 const Item nx = decode_item(a.t, item0 + w + 1);
-                if ((int)threadIdx.x < n) pre_neg = __float_as_uint(a.srow[threadIdx.x][nx.c]) | 0x80000000u;
+                if (my_worker < n) pre_neg = __float_as_uint(a.srow[my_worker][nx.c]) | 0x80000000u;
                 pre_S = a.Sbar[nx.c];
             }
             if (consumer_barrier_any(*vfailed != 0)) break;      // -s_i in place; everybody is done with the previous chunk
@@ -375,7 +422,7 @@ k_server_staged(const ServerStagedArgs sa)
                 const float4 zo0 = *reinterpret_cast<const float4*>(zs + g0 * kGroup + lane * 4);
                 const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
                 float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
-                signed_scale_sums<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl, negs, n, sh, s01, s23, t01, t23);
+                signed_scale_sums<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl, negs, prefix8, n, sh, s01, s23, t01, t23);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
 #pragma unroll

@@ -63,8 +63,8 @@ typedef enum {
     APMS_ERR_OOM = 4,           /* workspace too small, or allocation failed               */
     APMS_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (reported by the next
                                    synchronising call; the context's state is then undefined) */
-    APMS_ERR_BOUNDS = 6         /* apms_check_guards found guard bytes overwritten: something wrote
-                                   outside an array of the workspace                        */
+    APMS_ERR_BOUNDS = 6         /* apms_check_guards found guard bytes overwritten, or a checked
+                                   accessor of the checked build refused an access          */
 } apms_status;
 
 /* Phases of Algorithm 1. */
@@ -408,6 +408,19 @@ apms_status apms_set_team_mode(apms_ctx* ctx, apms_team_mode mode);
  * contexts created afterwards. */
 apms_status apms_set_guard_bytes(size_t bytes);
 apms_status apms_check_guards(apms_ctx* ctx, int64_t* bad_offset);
+
+/* The checked build of the library (compiled with -DAPMS_BOUNDS_CHECK, `libapms_checked.so`; the debugging aid
+ * that goes with the guard bytes): every global store of the 1-bit step's kernels, of the Adam, update and
+ * finalize kernels, their streaming loads and the sources of their bulk copies are validated on the device
+ * against the live contexts' workspaces and guard regions.  An access that would leave its array is skipped and
+ * recorded; the next synchronising call (and apms_check_guards) returns APMS_ERR_BOUNDS with the offset in
+ * apms_last_error.  Nothing traps or faults.  (Not covered: the top-k kernels and the monitor.)
+ * apms_build_is_checked: 1 in that build, 0 in the ordinary one, where the accessors compile to nothing.
+ * apms_selftest_bounds: checked build with the guard layout only - issues one checked store aimed into the guard
+ * bytes behind x and returns APMS_OK iff it was refused, reported and the guard bytes are untouched; clears the
+ * report.  APMS_ERR_BAD_STATE in the ordinary build. */
+int         apms_build_is_checked(void);
+apms_status apms_selftest_bounds(apms_ctx* ctx);
 
 /* Kernel timing: when enabled, every kernel launch is bracketed by CUDA events on the
  * context's stream.  apms_kernel_time() synchronises the stream, returns the total time

@@ -78,6 +78,8 @@ SIGNATURES = {
     "apms_set_compressor": (C.c_int, [C.c_void_p, C.c_int, C.c_double]),
     "apms_uncompressed_step_typed": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.c_int]),
     "apms_set_team_mode": (C.c_int, [C.c_void_p, C.c_int]),
+    "apms_build_is_checked": (C.c_int, []),
+    "apms_selftest_bounds": (C.c_int, [C.c_void_p]),
     "apms_set_guard_bytes": (C.c_int, [C.c_size_t]),
     "apms_check_guards": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "apms_set_timing": (C.c_int, [C.c_void_p, C.c_int]),
@@ -323,6 +325,14 @@ def apms_set_scale_kind(h, kind: int):
 
 def apms_set_team_mode(h, mode: int):
     _check(h, load().apms_set_team_mode(h, mode))
+
+
+def apms_build_is_checked() -> bool:
+    return bool(load().apms_build_is_checked())
+
+
+def apms_selftest_bounds(h):
+    _check(h, load().apms_selftest_bounds(h))
 
 
 def apms_set_guard_bytes(nbytes: int):

@@ -156,6 +156,8 @@ struct apms_ctx {
     std::vector<EventPair> pool;
     int64_t launches;
     std::vector<GuardRegion> guards;   // empty in the ordinary layout
+    unsigned long long* guard_table;   // checked build: the guard regions as (offset, bytes) pairs on the device
+    bool registered;                   // checked build: this workspace is in the device's table of checked workspaces
     char err[512];
 
     float* x() { return (float*)(ws + L.off_x); }
@@ -214,6 +216,55 @@ apms_status fill_guards(apms_ctx* c)
     return APMS_OK;
 }
 
+#ifdef APMS_BOUNDS_CHECK
+// Checked build: the table of live workspaces the device-side accessors consult (see device_common.cuh).
+std::mutex g_checked_mutex;
+std::vector<CheckedWorkspace> g_checked_host;
+
+apms_status upload_checked_table(apms_ctx* c)
+{
+    const int count = (int)g_checked_host.size();
+    if (count > 0) APMS_CUDA(c, cudaMemcpyToSymbol(g_checked, g_checked_host.data(), sizeof(CheckedWorkspace) * (size_t)count));
+    APMS_CUDA(c, cudaMemcpyToSymbol(g_checked_count, &count, sizeof count));
+    return APMS_OK;
+}
+
+apms_status register_checked(apms_ctx* c)
+{
+    if (c->registered) return APMS_OK;
+    std::lock_guard<std::mutex> lock(g_checked_mutex);
+    if ((int)g_checked_host.size() >= kMaxCheckedWorkspaces) return fail(c, APMS_ERR_OOM, "too many live contexts for the checked build's table");
+    std::vector<unsigned long long> pairs;
+    for (const GuardRegion& g : c->guards) { pairs.push_back(g.off); pairs.push_back(g.bytes); }     // ascending by construction
+    if (!pairs.empty()) {
+        APMS_CUDA(c, cudaMalloc((void**)&c->guard_table, pairs.size() * sizeof(unsigned long long)));
+        APMS_CUDA(c, cudaMemcpy(c->guard_table, pairs.data(), pairs.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    }
+    CheckedWorkspace w;
+    w.lo = (unsigned long long)c->ws; w.hi = w.lo + c->L.total;
+    w.guards = c->guard_table; w.nguards = (int)c->guards.size(); w.status = c->status();
+    APMS_CUDA(c, cudaDeviceSynchronize());
+    g_checked_host.push_back(w);
+    c->registered = true;
+    return upload_checked_table(c);
+}
+
+void unregister_checked(apms_ctx* c)
+{
+    if (!c->registered) return;
+    std::lock_guard<std::mutex> lock(g_checked_mutex);
+    cudaDeviceSynchronize();
+    for (size_t k = 0; k < g_checked_host.size(); ++k)
+        if (g_checked_host[k].lo == (unsigned long long)c->ws) { g_checked_host.erase(g_checked_host.begin() + (long)k); break; }
+    (void)upload_checked_table(c);
+    if (c->guard_table) cudaFree(c->guard_table);
+    c->guard_table = nullptr; c->registered = false;
+}
+#else
+apms_status register_checked(apms_ctx*) { return APMS_OK; }
+void unregister_checked(apms_ctx*) {}
+#endif
+
 // Event bracket around one kernel launch when timing is on.
 struct Timed {
     apms_ctx* c; int k; EventPair ev; bool on;
@@ -271,6 +322,18 @@ apms_status device_status_check(apms_ctx* c)
 {
     int st = 0;
     APMS_CUDA(c, cudaMemcpy(&st, c->status(), sizeof st, cudaMemcpyDeviceToHost));
+    if (st == DEVICE_BOUNDS) {
+        int rec[6] = {0, 0, 0, 0, 0, 0};
+        APMS_CUDA(c, cudaMemcpy(rec, c->status(), sizeof rec, cudaMemcpyDeviceToHost));
+        const unsigned long long addr = ((unsigned long long)(unsigned)rec[3] << 32) | (unsigned)rec[2];
+        const long long off = (long long)(addr - (unsigned long long)c->ws);
+        const char* what = "outside this workspace";
+        for (const GuardRegion& g : c->guards)
+            if (off + rec[4] > (long long)g.off && off < (long long)(g.off + g.bytes)) { what = g.what; break; }
+        snprintf(c->err, sizeof c->err, "a checked accessor refused a %s of %d bytes at workspace offset %lld (guard bytes behind: %s); the access was skipped",
+                 rec[5] ? "store" : "load", rec[4], off, what);
+        return APMS_ERR_BOUNDS;
+    }
     if (st != 0) return fail(c, APMS_ERR_TIMEOUT, "a kernel gave up waiting for its own asynchronous copies; the state of this context is undefined");
     return APMS_OK;
 }
@@ -751,7 +814,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->ws = nullptr; c->ws_bytes = 0; c->owns_ws = false;
     c->stream = nullptr; c->copy_stream = nullptr; c->host_path_ready = false;
     c->device = dev; c->sms = sms; c->timing = false; c->launches = 0; c->err[0] = 0;
-    c->team_mode = APMS_TEAM_AUTO;
+    c->team_mode = APMS_TEAM_AUTO; c->guard_table = nullptr; c->registered = false;
     c->steps = 0; c->has_sched = false; c->substep = 0; c->worker_chunks = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
     c->compressor = APMS_COMPRESSOR_ONEBIT; c->topk_frac = 0.01;
     c->fine_run = kFineRunDefault;
@@ -788,6 +851,8 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.d * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
     st = fill_guards(c);
+    if (st != APMS_OK) return st;
+    st = register_checked(c);
     if (st != APMS_OK) return st;
     if (!src_is_device) APMS_CUDA(c, cudaStreamSynchronize(c->stream));
     c->t = 0; c->steps = 0; c->csteps = 0; c->substep = 0; c->worker_chunks = 0; c->phase = APMS_PHASE_WARMUP; c->m_is_fp32 = true;
@@ -1400,6 +1465,39 @@ apms_status apms_check_guards(apms_ctx* c, int64_t* bad_offset)
     return device_status_check(c);
 }
 
+int apms_build_is_checked(void)
+{
+#ifdef APMS_BOUNDS_CHECK
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+apms_status apms_selftest_bounds(apms_ctx* c)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+#ifdef APMS_BOUNDS_CHECK
+    if (c->guards.empty()) return fail(c, APMS_ERR_BAD_STATE, "the self-test needs the guard layout (apms_set_guard_bytes before apms_create)");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "call apms_set_params first");
+    // a checked 16-byte store to the first whole 16 bytes behind x's d elements: inside the guard bytes that follow x
+    float* target = c->x() + (c->L.d + 3) / 4 * 4;
+    k_selftest_bounds<<<1, 32, 0, c->stream>>>(target);
+    apms_status st = launch_check(c, "k_selftest_bounds");
+    if (st != APMS_OK) return st;
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    st = device_status_check(c);
+    APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
+    if (st != APMS_ERR_BOUNDS) return fail(c, APMS_ERR_BAD_STATE, "the checked accessor did not refuse a store into guard bytes");
+    int64_t bad = -1;
+    st = apms_check_guards(c, &bad);           // the refused store must not have happened
+    if (st != APMS_OK) return st;
+    return APMS_OK;
+#else
+    return fail(c, APMS_ERR_BAD_STATE, "this library was built without checked accessors (-DAPMS_BOUNDS_CHECK)");
+#endif
+}
+
 apms_status apms_set_team_mode(apms_ctx* c, apms_team_mode mode)
 {
     if (!c) return APMS_ERR_INVALID_ARG;
@@ -1441,6 +1539,7 @@ void apms_destroy(apms_ctx* c)
 {
     if (!c) return;
     if (c->stream || c->ws) cudaStreamSynchronize(c->stream);
+    unregister_checked(c);
     for (int k = 0; k < APMS_KERNEL_COUNT; ++k)
         for (EventPair& ev : c->events[k]) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }
     for (EventPair& ev : c->pool) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }

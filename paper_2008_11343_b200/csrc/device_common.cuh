@@ -26,17 +26,86 @@ constexpr int kGroup = 128;              // elements one warp covers per 128-bit
 struct GradPtrs { const void* p[APMS_MAX_WORKERS]; };     // element type given by the kernel's GT template argument
 
 // ------------------------------------------------------------------------------------------
+// Checked build (-DAPMS_BOUNDS_CHECK; stands in for a memory checker): every global store of the step's
+// kernels, their streaming loads and the sources of their bulk copies first look the address up in a table
+// of the live contexts' workspaces and guard regions (the guard layout of apms_set_guard_bytes).  An access
+// that is not wholly inside an array - a store outside every workspace, or any access that touches guard
+// bytes (loads may run up to 16 bytes into them: bulk copies are whole 16-byte pieces) - is NOT performed;
+// the first such access is recorded in the owning context's status words and the next synchronising call
+// returns APMS_ERR_BOUNDS.  Nothing traps.  In the ordinary build the macros below cost nothing.
+
+enum { DEVICE_OK = 0, DEVICE_WAIT_TIMEOUT = 1, DEVICE_BOUNDS = 2 };
+
+#ifdef APMS_BOUNDS_CHECK
+struct CheckedWorkspace {
+    unsigned long long lo, hi;                   // [lo, hi): the workspace
+    const unsigned long long* guards;            // pairs (offset, bytes), ascending by offset
+    int nguards;
+    int* status;                                 // [0] code, [2..3] address, [4] bytes, [5] 1 = store
+};
+constexpr int kMaxCheckedWorkspaces = 64;
+__device__ CheckedWorkspace g_checked[kMaxCheckedWorkspaces];
+__device__ int g_checked_count;
+
+__device__ __noinline__ bool checked_access(const void* p, unsigned bytes, bool store)
+{
+    const unsigned long long a0 = (unsigned long long)p, a1 = a0 + bytes;
+    const int count = g_checked_count;
+    int* report = count > 0 ? g_checked[0].status : nullptr;
+    bool bad = store;                            // a store must land inside some workspace; a load may read the caller's memory
+    for (int w = 0; w < count; ++w) {
+        const CheckedWorkspace& ws = g_checked[w];
+        if (a1 <= ws.lo || a0 >= ws.hi) continue;
+        report = ws.status;
+        bad = a0 < ws.lo || a1 > ws.hi;
+        // the last guard region that begins below the end of the access
+        int lo = 0, hi = ws.nguards;
+        while (lo < hi) {
+            const int mid = (lo + hi) / 2;
+            if (ws.lo + ws.guards[2 * mid] < a1) lo = mid + 1; else hi = mid;
+        }
+        if (lo > 0) {
+            const unsigned long long g0 = ws.lo + ws.guards[2 * (lo - 1)], g1 = g0 + ws.guards[2 * (lo - 1) + 1];
+            const unsigned long long slack = store ? 0ull : 16ull;
+            if (a1 > g0 + slack && a0 < g1) bad = true;
+        }
+        break;
+    }
+    if (bad && report && atomicCAS(report, DEVICE_OK, DEVICE_BOUNDS) == DEVICE_OK) {
+        report[2] = (int)(a0 & 0xffffffffull); report[3] = (int)(a0 >> 32);
+        report[4] = (int)bytes; report[5] = store ? 1 : 0;
+    }
+    return !bad;
+}
+// where a skipped bulk copy reads instead (its byte count is already promised to the mbarrier)
+__device__ __forceinline__ const void* checked_safe_source() { return (const void*)g_checked[0].lo; }
+#define APMS_CAN_LOAD(p, bytes) checked_access((p), (unsigned)(bytes), false)
+#define APMS_CAN_STORE(p, bytes) checked_access((p), (unsigned)(bytes), true)
+#else
+#define APMS_CAN_LOAD(p, bytes) true
+#define APMS_CAN_STORE(p, bytes) true
+#endif
+// a scalar (or vector) store to global memory, skipped when the checked build finds it out of bounds
+#define APMS_STORE(lvalue, value) do { if (APMS_CAN_STORE(&(lvalue), sizeof(lvalue))) (lvalue) = (value); } while (0)
+
+// ------------------------------------------------------------------------------------------
 // small device helpers
 
-__device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ void st_stream4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+__device__ __forceinline__ float4 ld_stream4(const float* p)
+{
+    if (!APMS_CAN_LOAD(p, 16)) return make_float4(0.f, 0.f, 0.f, 0.f);
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream4(float* p, float4 v) { if (APMS_CAN_STORE(p, 16)) __stcs(reinterpret_cast<float4*>(p), v); }
+__device__ __forceinline__ void st_stream_word(uint32_t* p, uint32_t v) { if (APMS_CAN_STORE(p, 4)) __stcs(p, v); }
+__device__ __forceinline__ void st_stream_words4(uint32_t* p, uint4 v) { if (APMS_CAN_STORE(p, 16)) __stcs(reinterpret_cast<uint4*>(p), v); }
 
 // Up to four consecutive floats starting at p[k]; elements at or past `len` read as 0.
 __device__ __forceinline__ float4 ld4_checked(const float* p, int k, int len, bool streaming) {
     float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
     if (k + 3 < len) {
-        r = streaming ? ld_stream4(p + k) : *reinterpret_cast<const float4*>(p + k);
-    } else {
+        r = streaming ? ld_stream4(p + k) : (APMS_CAN_LOAD(p + k, 16) ? *reinterpret_cast<const float4*>(p + k) : r);
+    } else if (k < len && APMS_CAN_LOAD(p + k, 4 * (len - k))) {
         if (k + 0 < len) r.x = p[k + 0];
         if (k + 1 < len) r.y = p[k + 1];
         if (k + 2 < len) r.z = p[k + 2];
@@ -46,7 +115,7 @@ __device__ __forceinline__ float4 ld4_checked(const float* p, int k, int len, bo
 __device__ __forceinline__ void st4_checked(float* p, int k, int len, float4 v) {
     if (k + 3 < len) {
         st_stream4(p + k, v);
-    } else {
+    } else if (k < len && APMS_CAN_STORE(p + k, 4 * (len - k))) {
         if (k + 0 < len) p[k + 0] = v.x;
         if (k + 1 < len) p[k + 1] = v.y;
         if (k + 2 < len) p[k + 2] = v.z;
@@ -65,6 +134,7 @@ template <> struct Grad<APMS_GRAD_BF16> {
     static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const uint16_t*)p + e; }
     static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __uint_as_float((uint32_t)((const uint16_t*)p)[e] << 16); }
     static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        if (!APMS_CAN_LOAD((const uint16_t*)p + k, 8)) return make_float4(0.f, 0.f, 0.f, 0.f);
         const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const uint16_t*)p + k));
         return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
                            __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
@@ -74,6 +144,7 @@ template <> struct Grad<APMS_GRAD_F16> {
     static __device__ __forceinline__ const void* at(const void* p, int64_t e) { return (const __half*)p + e; }
     static __device__ __forceinline__ float ld1(const void* p, int64_t e) { return __half2float(((const __half*)p)[e]); }
     static __device__ __forceinline__ float4 ld4(const void* p, int k) {
+        if (!APMS_CAN_LOAD((const __half*)p + k, 8)) return make_float4(0.f, 0.f, 0.f, 0.f);
         const uint2 r = __ldcs(reinterpret_cast<const uint2*>((const __half*)p + k));
         const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
         const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&r.y));

@@ -53,7 +53,7 @@ k_warmup_adam(const __grid_constant__ GradPtrs G, const AdamArgs a)
             for (int i = 0; i < a.n; ++i) gs = __fadd_rn(gs, Grad<GT>::ld1(G.p[i], e));
             float m = a.m[e], v = a.v[e], x = a.x[e];
             adam_elem(a, gs, m, v, x);
-            a.m[e] = m; a.v[e] = v; a.x[e] = x;
+            APMS_STORE(a.m[e], m); APMS_STORE(a.v[e], v); APMS_STORE(a.x[e], x);
         }
     }
 }

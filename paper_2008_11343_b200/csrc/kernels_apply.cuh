@@ -22,7 +22,7 @@ struct ApplyArgs {
 __global__ void k_make_den(const float* __restrict__ v, float* __restrict__ den, int64_t d, float eps)
 {
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d; j += (int64_t)gridDim.x * blockDim.x)
-        den[j] = __fadd_rn(__fsqrt_rn(v[j]), eps);
+        APMS_STORE(den[j], __fadd_rn(__fsqrt_rn(v[j]), eps));
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -78,7 +78,7 @@ k_apply(const ApplyArgs a)
             st_stream4(x + k, xx);
         } else {
             for (int e = 0; e < 4 && k + e < L; ++e)
-                x[k + e] = apply_stored(x[k + e], v[k + e], (nib >> e) & 1u, cc);
+                APMS_STORE(x[k + e], apply_stored(x[k + e], v[k + e], (nib >> e) & 1u, cc));
         }
     }
 }
@@ -117,8 +117,8 @@ k_apply_gradient(const ApplyGradArgs a)
         } else {
             for (int e = 0; e < 4 && k + e < L; ++e) {
                 const float mn = __fmaf_rn(a.beta1, a.m[j + e], __fmul_rn(a.omb1, bit_scale((nib >> e) & 1u, S)));
-                a.m[j + e] = mn;
-                a.x[j + e] = apply_elem(a.x[j + e], a.v[j + e], mn, a.lr, a.eps);
+                APMS_STORE(a.m[j + e], mn);
+                APMS_STORE(a.x[j + e], apply_elem(a.x[j + e], a.v[j + e], mn, a.lr, a.eps));
             }
         }
     }
@@ -170,7 +170,7 @@ k_uncompressed(const __grid_constant__ GradPtrs G, const UncompressedArgs a)
             for (int i = 0; i < a.n; ++i)
                 acc = __fadd_rn(acc, __fadd_rn(__fmaf_rn(a.beta1, m, __fmul_rn(a.omb1, Grad<GT>::ld1(G.p[i], e))), 0.0f));
             uncompressed_elem(a, acc, m, a.v[e], x);
-            a.m[e] = m; a.x[e] = x;
+            APMS_STORE(a.m[e], m); APMS_STORE(a.x[e], x);
         }
     }
 }

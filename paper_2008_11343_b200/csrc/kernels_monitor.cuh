@@ -50,4 +50,12 @@ __global__ void k_error_norm_rows(const double* __restrict__ partial, int64_t ti
     out[r] = total;
 }
 
+#ifdef APMS_BOUNDS_CHECK
+// Self-test of the checked build: one checked store to an address the host chose inside guard bytes.
+__global__ void k_selftest_bounds(float* target)
+{
+    if (threadIdx.x == 0) st_stream4(target, make_float4(1.f, 2.f, 3.f, 4.f));
+}
+#endif
+
 }  // namespace

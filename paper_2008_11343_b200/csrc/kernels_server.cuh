@@ -79,7 +79,7 @@ __device__ __forceinline__ void server_groups(const ServerArgs& a, const float* 
         if (CHECKED) st4_checked(zb, k, L, out); else st_stream4(zb + k, out);
         const uint32_t word = pack_group_words(nibble, lane);
         const int wk = grp * 4 + wl;
-        if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) ob[wk] = word;
+        if ((lane & 7) == 0 && (!CHECKED || wk * 32 < L)) APMS_STORE(ob[wk], word);
     }
 }
 
@@ -119,8 +119,8 @@ k_server(const ServerArgs a)
         server_groups<1, true>(a, s_sh, wofs, zb, ob, g0, 1, lane, L, S_old, acc);
     const double total = team_sum<WPC>(acc, red);
     if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
-        if (a.t.P == 1) a.Sbar[it.c] = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);
-        else a.partial[it.c * a.t.P + it.p] = total;
+        if (a.t.P == 1) APMS_STORE(a.Sbar[it.c], scale_from_sum(total, (double)it.Lc, a.t.l1 != 0));
+        else APMS_STORE(a.partial[it.c * a.t.P + it.p], total);
     }
 }
 
@@ -148,8 +148,6 @@ constexpr int kStages = 4;
 constexpr int64_t kStagedSpanElems = 32768;   // a CTA of the fused form walks enough chunks to stream about this many elements
 constexpr int kStagedThreads = kThreads + 32;    // eight consumer warps + one producer warp
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about a second of SM clocks
-
-enum { DEVICE_OK = 0, DEVICE_WAIT_TIMEOUT = 1 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -201,6 +199,9 @@ __global__ void k_selftest_wait(int* status, long long limit)
 // Global -> this CTA's shared memory; 16-byte aligned addresses, size a multiple of 16 bytes.
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
 {
+#ifdef APMS_BOUNDS_CHECK
+    if (!APMS_CAN_LOAD(gmem_src, bytes)) gmem_src = checked_safe_source();     // reported; the bytes are owed to the barrier
+#endif
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
@@ -459,7 +460,7 @@ k_server_staged(const ServerStagedArgs sa)
             if (FUSED) {
                 // Section 3.3 steps 5-6 for this chunk: m <- +-Sbar, x <- x - lr m / (sqrt(v) + eps)
                 const float S_new = (float)sqrt(total / (double)it.Lc);
-                if (ok && threadIdx.x == 0) a.Sbar[it.c] = S_new;
+                if (ok && threadIdx.x == 0) APMS_STORE(a.Sbar[it.c], S_new);
                 const float c_new = __fmul_rn(sa.lr, S_new);        // lr * (+-S) = +-(lr * S)
                 for (int j = 0; ok && j < nslabs; ++j, ++q) {
                     const int st = q % kStages;
@@ -487,16 +488,16 @@ k_server_staged(const ServerStagedArgs sa)
                     }
                 }
             } else if (ok && threadIdx.x == 0) {
-                if (a.t.P == 1) a.Sbar[it.c] = (float)sqrt(total / (double)it.Lc);
-                else a.partial[it.c * a.t.P + it.p] = total;
+                if (a.t.P == 1) APMS_STORE(a.Sbar[it.c], (float)sqrt(total / (double)it.Lc));
+                else APMS_STORE(a.partial[it.c * a.t.P + it.p], total);
             }
             // the tile's sign words leave in whole 16-byte pieces (full lines for full tiles)
             if (ok) {
                 uint32_t* __restrict__ ob = a.Bbar + (wofs - off_out);          // 16-byte aligned; the tile's words are [off_out, wend)
                 const int wend = off_out + (L + 31) / 32;
                 for (int w4 = threadIdx.x * 4; w4 < wend; w4 += kThreads * 4) {
-                    if (w4 >= off_out && w4 + 3 < wend) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb + w4));
-                    else for (int r = (w4 < off_out ? off_out : w4); r < w4 + 4 && r < wend; ++r) ob[r] = nb[r];
+                    if (w4 >= off_out && w4 + 3 < wend) st_stream_words4(ob + w4, *reinterpret_cast<const uint4*>(nb + w4));
+                    else for (int r = (w4 < off_out ? off_out : w4); r < w4 + 4 && r < wend; ++r) APMS_STORE(ob[r], nb[r]);
                 }
             }
         }
@@ -723,7 +724,7 @@ k_server_packed(const ServerStagedArgs sa)
                 const int64_t cbeg = (c0 + lane) * (int64_t)chunk;
                 const int64_t Lc = (a.t.d - cbeg < chunk) ? a.t.d - cbeg : chunk;
                 S_lane = (float)sqrt(total / (double)Lc);
-                if (warp == 0) a.Sbar[c0 + lane] = S_lane;
+                if (warp == 0) APMS_STORE(a.Sbar[c0 + lane], S_lane);
             }
             // Section 3.3 steps 5-6 for this slab: every group with the new scale of its chunk
             float c_new[2];
@@ -762,8 +763,8 @@ k_server_packed(const ServerStagedArgs sa)
                 uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
                 const int nwords = (L + 31) / 32;
                 const int w4 = threadIdx.x * 4;
-                if (w4 + 3 < nwords) __stcs(reinterpret_cast<uint4*>(ob + w4), *reinterpret_cast<const uint4*>(nb[buf] + w4));
-                else for (int r = w4; r < nwords; ++r) ob[r] = nb[buf][r];
+                if (w4 + 3 < nwords) st_stream_words4(ob + w4, *reinterpret_cast<const uint4*>(nb[buf] + w4));
+                else for (int r = w4; r < nwords; ++r) APMS_STORE(ob[r], nb[buf][r]);
             }
         }
     }

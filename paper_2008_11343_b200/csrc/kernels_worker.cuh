@@ -61,7 +61,7 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
     const uint32_t word = pack_group_words(nibble, lane);
     if ((lane & 7) == 0) {
         const int wk = grp * 4 + (lane >> 3);
-        if (!CHECKED || wk * 32 < L) __stcs(obits + wk, word);     // streaming: a plain store here costs ~4 % of the kernel
+        if (!CHECKED || wk * 32 < L) st_stream_word(obits + wk, word);     // streaming: a plain store here costs ~4 % of the kernel
     }
 }
 
@@ -123,8 +123,8 @@ k_worker(const __grid_constant__ GradPtrs G, const WorkerArgs a)
 
     const double total = team_sum<WPC>(acc, red);
     if ((WPC == 1) ? (lane == 0) : (threadIdx.x == 0)) {
-        if (a.t.P == 1) *sptr = scale_from_sum(total, (double)it.Lc, a.t.l1 != 0);    // ||z||_2 / sqrt(L)
-        else a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p] = total;
+        if (a.t.P == 1) APMS_STORE(*sptr, scale_from_sum(total, (double)it.Lc, a.t.l1 != 0));    // ||z||_2 / sqrt(L)
+        else APMS_STORE(a.partial[(int64_t)i * a.t.Pp + it.c * a.t.P + it.p], total);
     }
 }
 
@@ -207,7 +207,7 @@ __device__ __forceinline__ void fine_piece(const WorkerFineArgs& a, const void* 
             const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
             if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
         }
-        if (lane < 4 * kFineU) __stcs(obits + lane, outw);
+        if (lane < 4 * kFineU) st_stream_word(obits + lane, outw);
     } else {
         const int ngroups = (L + kGroup - 1) / kGroup;
         for (int grp = 0; grp < ngroups; ++grp) {
@@ -247,7 +247,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + (t * kWarps + warp) * (SPLIT ? 2 : 1);
     const int64_t left = a.d - base;
     if (left <= 0) {                                           // past the end of the vector
-        if (lane == 0) *slot = 0.0;
+        if (lane == 0) APMS_STORE(*slot, 0.0);
         return;
     }
     const int L = (int)(left < kFineSub ? left : kFineSub);
@@ -265,11 +265,11 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
         fine_piece<GT, SENDG, true>(a, g, z, mbits, obits, lane, L, (int)(next >> 5), s_lo, S_lo, srow[c + 1], a.Sbar[c + 1], acc, acc_hi);
         acc = warp_sum(acc);
         acc_hi = warp_sum(acc_hi);
-        if (lane == 0) { slot[0] = acc; slot[1] = acc_hi; }
+        if (lane == 0) { APMS_STORE(slot[0], acc); APMS_STORE(slot[1], acc_hi); }
     } else {
         fine_piece<GT, SENDG, false>(a, g, z, mbits, obits, lane, L, 0, s_lo, S_lo, s_lo, S_lo, acc, acc_hi);
         acc = warp_sum(acc);
-        if (lane == 0) slot[0] = acc;                          // slot [1] of a piece without a boundary is never read
+        if (lane == 0) APMS_STORE(slot[0], acc);                          // slot [1] of a piece without a boundary is never read
     }
 }
 
@@ -299,7 +299,7 @@ k_finalize_fine(const double* __restrict__ partial, int64_t Pp, float* __restric
         total += partial[(int64_t)r * Pp + q * per + ((per == 2 && q * kFineSub < cbeg) ? 1 : 0)];
 #pragma unroll
     for (int o = T / 2; o > 0; o >>= 1) total += __shfl_down_sync(0xffffffffu, total, o, T);
-    if (live && sub == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+    if (live && sub == 0) APMS_STORE(scales[(int64_t)r * Cp + c], (float)sqrt(total / (double)Lc));
 }
 
 // The same for long chunks (thousands of pieces each, few chunks): one CTA per (row, chunk); thread t adds the
@@ -320,7 +320,7 @@ k_finalize_fine_cta(const double* __restrict__ partial, int64_t Pp, float* __res
     for (int64_t q = q0 + threadIdx.x; q < q1; q += kThreads)
         total += row[q * per + ((per == 2 && q * kFineSub < cbeg) ? 1 : 0)];
     total = block_sum(total, red);
-    if (threadIdx.x == 0) scales[(int64_t)r * Cp + c] = (float)sqrt(total / (double)Lc);
+    if (threadIdx.x == 0) APMS_STORE(scales[(int64_t)r * Cp + c], (float)sqrt(total / (double)Lc));
 }
 
 // Scales of split chunks: partial sums added in tile order, then sqrt(sum / L).
@@ -335,7 +335,7 @@ __global__ void k_finalize_scales(const double* __restrict__ partial, float* __r
     const int64_t Lc = (t.d - cbeg < t.chunk) ? t.d - cbeg : t.chunk;
     double total = 0.0;
     for (int p = 0; p < t.P; ++p) total += partial[(int64_t)r * t.Pp + c * t.P + p];
-    scales[(int64_t)r * Cp + c] = scale_from_sum(total, (double)Lc, t.l1 != 0);
+    APMS_STORE(scales[(int64_t)r * Cp + c], scale_from_sum(total, (double)Lc, t.l1 != 0));
 }
 
 }  // namespace

@@ -120,3 +120,28 @@ def test_a_changed_guard_byte_is_found_and_named():
     assert e.value.status == B.ERR_BAD_STATE
     with pytest.raises(B.ApmsError):
         B.apms_set_guard_bytes(100)
+
+
+def test_checked_accessors_refuse_a_store_into_guard_bytes():
+    """Only in the checked build of the library (the same tests are run against it by test_gpu_checked_build.py):
+    a checked store aimed at the guard bytes behind x is skipped and reported, the guard bytes stay untouched,
+    and the context goes on working."""
+    if not B.apms_build_is_checked():
+        w = tiny(100, 2, 32, cfg_id=193)
+        ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        ctx.set_params(wl.initial_params(w))
+        with pytest.raises(B.ApmsError) as e:
+            B.apms_selftest_bounds(ctx._h)                       # the ordinary build has no checked accessors
+        assert e.value.status == B.ERR_BAD_STATE
+        return
+    w = tiny(3 * 1024 + 5, 2, 1024, cfg_id=193)
+    ctx, orc = H.make_pair(w)
+    B.apms_selftest_bounds(ctx._h)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    for step in range(1, 4):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+    H.compare_state(ctx, orc, w, exact=True)
+    ctx.check_guards()

@@ -395,11 +395,13 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     a.tile0 = a.e0 / kFineTile; a.tiles = (a.e1 + kFineTile - 1) / kFineTile - a.tile0;
     a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1;
+    a.inv_chunk = (c->L.C < ((int64_t)1 << 20) && c->L.d < ((int64_t)1 << 40)) ? 1.0f / (float)c->L.chunk : 0.0f;
     a.run = c->fine_run;
     if ((int64_t)a.run > a.tiles) a.run = a.tiles < 1 ? 1 : (int)a.tiles;
     const int64_t stretches = (a.tiles + a.run - 1) / a.run;
     const int64_t blocks = stretches * a.run * ni;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (tile, worker) items for one launch");
+    a.inv_run = 1.0f / (float)a.run; a.inv_per_stretch = 1.0f / ((float)a.run * (float)ni);
     {
         Timed t(c, APMS_KERNEL_WORKER);
         const bool sendg = c->variant == APMS_VARIANT_GRADIENT;
@@ -687,6 +689,7 @@ apms_status launch_apply(apms_ctx* c)
     ApplyArgs a;
     a.Bbar = c->Bbar(); a.Sbar = c->Sbar(); a.den = c->den(); a.x = c->x();
     a.d = c->L.d; a.chunk = c->L.chunk; a.lr = c->lr;
+    a.inv_chunk = (c->L.C < ((int64_t)1 << 20) && c->L.d < ((int64_t)1 << 40)) ? 1.0f / (float)c->L.chunk : 0.0f;
     Timed t(c, APMS_KERNEL_APPLY);
     k_apply<<<(unsigned)((c->L.d + kApplyTile - 1) / kApplyTile), kThreads, 0, c->stream>>>(a);
     return launch_check(c, "k_apply");

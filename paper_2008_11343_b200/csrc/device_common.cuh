@@ -163,6 +163,28 @@ __device__ __forceinline__ float4 ld_grad4_checked(const void* p, int k, int len
     return r;
 }
 
+// floor(a / b) for 0 <= a < 2^40, 0 < b, quotient below 2^21 (checked by the host, which passes 1 / b rounded to
+// binary32): the product of the two binary32 values is within one of the quotient, two multiplications settle it.
+// A general 64-bit division is a subroutine of about seventy instructions - per warp and 512 elements that is a
+// sizeable share of the worker kernel's instructions.
+__device__ __forceinline__ int64_t div_small_quotient(int64_t a, int64_t b, float inv_b)
+{
+    int64_t q = (int64_t)(__ll2float_rz(a) * inv_b);
+    while (q * b > a) --q;                       // at most once for quotients below 2^21
+    while ((q + 1) * b <= a) ++q;
+    return q;
+}
+
+// floor(x / d) for 32-bit operands from an estimate (x times 1 / d in binary32) and exact corrections: the loops
+// run zero times or once for the quotients that occur (block index over tiles per run and the like).
+__device__ __forceinline__ uint32_t div_u32(uint32_t x, uint32_t d, float inv_d)
+{
+    uint32_t q = (uint32_t)(__uint2float_rz(x) * inv_d);
+    while ((uint64_t)q * d > x) --q;
+    while ((uint64_t)(q + 1) * d <= x) ++q;
+    return q;
+}
+
 // +-s with the sign of the compressor: z >= 0 gives +s (so do +0 and -0), NaN gives -s.
 __device__ __forceinline__ float signed_scale(float z, float s) { return (z >= 0.0f) ? s : -s; }
 __device__ __forceinline__ float bit_scale(uint32_t bit, float s) { return bit ? s : -s; }

@@ -16,6 +16,7 @@ constexpr int kApplyU = kApplyTile / (kThreads * 4);
 struct ApplyArgs {
     const uint32_t* Bbar; const float* Sbar; const float* den; float* x;     // den = sqrt(v) + eps, see k_make_den
     int64_t d; int64_t chunk; float lr;
+    float inv_chunk;      // 1 / chunk in binary32 when there are fewer than 2^20 chunks (see div_small_quotient), else 0
 };
 
 // den = sqrt(v) + eps, the denominator of the model update while v is frozen.
@@ -31,9 +32,10 @@ k_apply(const ApplyArgs a)
     const int64_t base = (int64_t)blockIdx.x * kApplyTile;
     const int64_t left = a.d - base;
     const int L = (int)(left < kApplyTile ? left : kApplyTile);
-    const int64_t c0 = base / a.chunk;
+    const int64_t c0 = a.inv_chunk != 0.0f ? div_small_quotient(base, a.chunk, a.inv_chunk) : base / a.chunk;
     const uint32_t off0 = (uint32_t)(base - c0 * a.chunk);
     const uint32_t chunk32 = (uint32_t)a.chunk;
+    const bool long_chunk = a.chunk >= kApplyTile;          // then a tile holds at most one chunk boundary: no division per access
     const uint32_t* __restrict__ bits = a.Bbar + base / 32;
     const float* __restrict__ v = a.den + base;
     float* __restrict__ x = a.x + base;
@@ -49,7 +51,7 @@ k_apply(const ApplyArgs a)
             xx[u] = ld_stream4(x + k);
             nib[u] = bits[k >> 5] >> (k & 31);
             const uint32_t rel = off0 + (uint32_t)k;
-            S[u] = Sb[rel < chunk32 ? 0u : rel / chunk32];
+            S[u] = Sb[long_chunk ? (rel >= chunk32 ? 1u : 0u) : rel / chunk32];
         }
 #pragma unroll
         for (int u = 0; u < kApplyU; ++u) {
@@ -65,7 +67,7 @@ k_apply(const ApplyArgs a)
     }
     for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
         const uint32_t rel = off0 + (uint32_t)k;
-        const float S = Sb[rel < chunk32 ? 0u : rel / chunk32];
+        const float S = Sb[long_chunk ? (rel >= chunk32 ? 1u : 0u) : rel / chunk32];
         const uint32_t nib = bits[k >> 5] >> (k & 31);
         const float cc = __fmul_rn(a.lr, S);
         if (k + 3 < L) {

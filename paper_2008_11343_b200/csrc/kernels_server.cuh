@@ -205,7 +205,9 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
-// Barrier among the 256 consumer threads only (the producer warp never joins it) that also ORs a flag
+// Barrier among the 256 consumer threads only (the producer warp never joins it).
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// The same barrier that also ORs a flag
 // over them: every consumer gets the same answer, so a decision to leave taken on it is uniform even
 // when the flag it is fed from changes while the threads arrive.
 __device__ __forceinline__ bool consumer_barrier_any(bool flag)
@@ -547,20 +549,25 @@ k_server_packed(const ServerStagedArgs sa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const ServerArgs& a = sa.a;
-    // Everything the consumers hand to each other is double-buffered over the walk, so that one barrier per
-    // slab suffices: what slab w+1 writes, slab w-1 was the last to read, and two barriers lie in between.
+    // The model update of a slab lags one slab behind its server step: jobs run in the order
+    //   S(0), S(1), U(0), S(2), U(1), ..., U(last)          (S = steps 4, U = steps 5-6 of Section 3.3)
+    // with ONE barrier per slab, after S(w).  One warp (they take turns) then forms the slab's new scales -
+    // the binary64 division and square root - while the others already update slab w-1, whose scales were
+    // formed a slab earlier: no warp waits for that arithmetic.  Everything the consumers hand to each other is
+    // double-buffered over the walk: what slab w+2 writes, slab w was the last to read, and barrier w+1 lies in between.
     __shared__ double red[2][kPackedMaxChunks];                          // one sum of squares per group of the slab
     __shared__ uint64_t full[kStages], empty[kStages];
     __shared__ uint32_t neg_s[2][kPackedMaxChunks * APMS_MAX_WORKERS];   // -s_i per chunk of the slab
-    __shared__ float S_old_sh[2][kPackedMaxChunks];
-    __shared__ __align__(16) uint32_t nb[2][kSlabWords];                 // the slab's new sign words
+    __shared__ float S_old_sh[2][kPackedMaxChunks], S_new_sh[2][kPackedMaxChunks];
     __shared__ int failed;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n = NT > 0 ? NT : a.n;
     const size_t stage_bytes = staged_stage_bytes(n, true);
-    const int chunk = (int)a.t.chunk;                                  // 128 .. 1024, divides kSlab
-    const int gpc = chunk / kGroup;                                    // groups per chunk
+    const int chunk = (int)a.t.chunk;                                  // 128, 256, 512 or 1024: a power of two that divides kSlab
+    const int cshift = 31 - __clz(chunk);                              // divisions by the chunk length are shifts
+    const int gpc = chunk >> 7;                                        // groups per chunk (kGroup = 128)
+    const int gshift = cshift - 7;
     const int64_t slab_first = a.item0 + (int64_t)blockIdx.x * sa.span;       // items are slabs here
     const int nmine = (int)(a.items - slab_first < sa.span ? a.items - slab_first : sa.span);
 
@@ -575,17 +582,20 @@ k_server_packed(const ServerStagedArgs sa)
         if (lane == 0) {
             int q = 0;
             bool stop = false;
-            for (int w = 0; w < nmine && !stop; ++w) {
-                const int64_t base_e = (slab_first + w) * kSlab;
-                const int64_t left = a.t.d - base_e;
-                const int live = (int)(left < kSlab ? left : kSlab);
-                const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
-                const int64_t wofs = base_e / 32;
-                for (int r = 0; r < 2; ++r, ++q) {
+            // step t issues S(t) (t < nmine) and then U(t-1) (t >= 1): the order the consumers take them in
+            for (int t = 0; t <= nmine && !stop; ++t) {
+                for (int r = 0; r < 2 && !stop; ++r) {
+                    const int w = r == 0 ? t : t - 1;
+                    if (r == 0 ? t >= nmine : t < 1) continue;
+                    const int64_t base_e = (slab_first + w) * kSlab;
+                    const int64_t left = a.t.d - base_e;
+                    const int live = (int)(left < kSlab ? left : kSlab);
+                    const uint32_t zbytes = (uint32_t)((live + 3) / 4) * 16u;
                     const int st = q % kStages;
                     if (q >= kStages && !mbar_wait(&empty[st], (uint32_t)(q / kStages - 1) & 1u)) { failed = 1; stop = true; break; }
                     unsigned char* base = smem + (size_t)st * stage_bytes;
                     if (r == 0) {
+                        const int64_t wofs = base_e / 32;
                         const int off_in = sa.row_align;                 // slabs start at multiples of 64 words
                         const uint32_t wbytes = (uint32_t)((off_in + (live + 31) / 32 + 3) / 4) * 16u;
                         mbar_arrive_expect_tx(&full[st], zbytes + (uint32_t)n * wbytes);
@@ -598,6 +608,7 @@ k_server_packed(const ServerStagedArgs sa)
                         bulk_load(base, sa.den + base_e, zbytes, &full[st]);
                         bulk_load(base + (size_t)kSlab * 4, sa.x + base_e, zbytes, &full[st]);
                     }
+                    ++q;
                 }
             }
             if (failed) {
@@ -609,8 +620,8 @@ k_server_packed(const ServerStagedArgs sa)
         const int sh = 4 * (lane & 7);
         const int wl = lane >> 3;
         const int g0 = warp, g1 = warp + kWarps;
-        const int k0 = g0 / gpc, k1 = g1 / gpc;                          // the chunks (within the slab) of this warp's two groups
-        const int kmax = kSlab / chunk;                                  // chunks per whole slab
+        const int k0 = g0 >> gshift, k1 = g1 >> gshift;                          // the chunks (within the slab) of this warp's two groups
+        const int kmax = kSlab >> cshift;                                  // chunks per whole slab
         const volatile int* vfailed = &failed;
         const int off_in = sa.row_align;
         // this thread's share of a slab's scales: entry idx = kk * n + i for idx = threadIdx.x + 256 r
@@ -621,13 +632,13 @@ k_server_packed(const ServerStagedArgs sa)
             const int64_t base_e = (slab_first + w) * kSlab;
             const int64_t left = a.t.d - base_e;
             const int L = (int)(left < kSlab ? left : kSlab);
-            const int64_t c0 = base_e / chunk;
-            const int nchunks = (L + chunk - 1) / chunk;
+            const int64_t c0 = base_e >> cshift;
+            const int nchunks = (L + chunk - 1) >> cshift;
 #pragma unroll
             for (int r = 0; r < kPre; ++r) {
                 const int idx = (int)threadIdx.x + r * kThreads;
                 pre[r] = 0u;
-                if (idx < nchunks * n) {
+                if (warp * 32 + r * kThreads < nchunks * n && idx < nchunks * n) {      // first test: warp-uniform, skips whole warps
                     const int kk = idx / n, i = idx - kk * n;
                     pre[r] = __float_as_uint(a.srow[i][c0 + kk]) | 0x80000000u;
                 }
@@ -638,31 +649,68 @@ k_server_packed(const ServerStagedArgs sa)
 #pragma unroll
             for (int r = 0; r < kPre; ++r) {
                 const int idx = (int)threadIdx.x + r * kThreads;
-                if (idx < kmax * n) {
+                if (warp * 32 + r * kThreads < kmax * n && idx < kmax * n) {
                     const int kk = idx / n, i = idx - kk * n;
                     neg_s[buf][kk * APMS_MAX_WORKERS + i] = pre[r];
                 }
             }
             if ((int)threadIdx.x < kmax) S_old_sh[buf][threadIdx.x] = pre_S;
         };
-        bool leave = false;
+        int q = 0;
+        bool ok = true;
+        // Steps 5-6 for slab w from its job in the ring, the scales in S_new_sh[w & 1] and this lane's own sign bits.
+        auto update_slab = [&](int w, uint32_t bits0, uint32_t bits1) {
+            const int64_t base_e = (slab_first + w) * kSlab;
+            const int64_t left = a.t.d - base_e;
+            const int L = (int)(left < kSlab ? left : kSlab);
+            const int nchunks = (L + chunk - 1) >> cshift;
+            const float c0n = __fmul_rn(sa.lr, k0 < nchunks ? S_new_sh[w & 1][k0] : 0.0f);      // lr * (+-S) = +-(lr * S)
+            const float c1n = __fmul_rn(sa.lr, k1 < nchunks ? S_new_sh[w & 1][k1] : 0.0f);
+            const int st = q % kStages;
+            if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
+            if (ok) {
+                const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
+                const float* xs = vs + kSlab;
+                float4 vv[2], xx[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
+                    xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[st]);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int k = (u ? g1 : g0) * kGroup + lane * 4;
+                    const uint32_t nib = u ? bits1 : bits0;
+                    const float cn = u ? c1n : c0n;
+                    xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, cn);
+                    xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, cn);
+                    xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, cn);
+                    xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, cn);
+                    st4_checked(sa.x + base_e, k, L, xx[u]);
+                }
+            }
+            ++q;
+        };
         if (nmine > 0) {
             fetch_scales(0);
             store_scales(0);
         }
-        leave = consumer_barrier_any(*vfailed != 0);                      // the first slab's scales are in place
-        int q = 0;
-        for (int w = 0; w < nmine && !leave; ++w) {
+        bool leave = consumer_barrier_any(*vfailed != 0);                 // the first slab's scales are in place
+        uint32_t prev0 = 0u, prev1 = 0u;                                  // this lane's sign bits of the slab before
+        int w = 0;
+        for (; w < nmine && !leave; ++w) {
             const int buf = w & 1;
             const int64_t base_e = (slab_first + w) * kSlab;
             const int64_t left = a.t.d - base_e;
             const int L = (int)(left < kSlab ? left : kSlab);
-            const int64_t c0 = base_e / chunk;
-            const int nchunks = (L + chunk - 1) / chunk;
+            const int64_t c0 = base_e >> cshift;
+            const int nchunks = (L + chunk - 1) >> cshift;
             const uint32_t* negs = neg_s[buf];
             if (w + 1 < nmine) fetch_scales(w + 1);                       // in flight during this slab's arithmetic
-            bool ok = true;
             double acc0 = 0.0, acc1 = 0.0;
+            uint32_t mine0 = 0u, mine1 = 0u;
             {
                 const int st = q % kStages;
                 if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
@@ -680,6 +728,7 @@ k_server_packed(const ServerStagedArgs sa)
                     const float So0 = S_old_sh[buf][kk0], So1 = S_old_sh[buf][kk1];
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
+                    uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const int grp = u ? g1 : g0;
@@ -701,10 +750,12 @@ k_server_packed(const ServerStagedArgs sa)
                                 nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
                             }
                         }
-                        if (u) acc1 = acc; else acc0 = acc;
+                        if (u) { acc1 = acc; mine1 = nibble; } else { acc0 = acc; mine0 = nibble; }
                         st4_checked(a.zbar + base_e, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                        // the group's four new sign words: lanes 0, 8, 16, 24 hold one each - one 16-byte piece per group
                         const uint32_t word = pack_group_words(nibble, lane);
-                        if ((lane & 7) == 0) nb[buf][grp * 4 + wl] = word;    // words past L hold zeros and are never stored
+                        const int wk = grp * 4 + wl;
+                        if ((lane & 7) == 0 && wk * 32 < L) st_stream_word(ob + wk, word);
                     }
                 }
                 ++q;
@@ -713,59 +764,24 @@ k_server_packed(const ServerStagedArgs sa)
             acc1 = warp_sum(acc1);
             if (lane == 0) { red[buf][g0] = acc0; red[buf][g1] = acc1; }
             if (w + 1 < nmine) store_scales(buf ^ 1);                     // the next slab's scales, fetched above
-            leave = consumer_barrier_any(!ok || *vfailed != 0);           // the groups' sums and the slab's sign words are in shared memory
+            leave = consumer_barrier_any(!ok || *vfailed != 0);           // the groups' sums of this slab are in shared memory
             if (leave) break;
-            // The new scale of every chunk of the slab, one chunk per lane (so that a warp runs the binary64
-            // division and square root once), handed to the lanes that need it by shuffles.
-            float S_lane = 0.0f;
-            if (lane < nchunks) {
+            // The new scale of every chunk of the slab, one chunk per lane of one warp (the warps take turns).
+            if (warp == (w & (kWarps - 1)) && lane < nchunks) {
                 double total = 0.0;
                 for (int r = 0; r < gpc; ++r) total += red[buf][lane * gpc + r];           // group order
                 const int64_t cbeg = (c0 + lane) * (int64_t)chunk;
                 const int64_t Lc = (a.t.d - cbeg < chunk) ? a.t.d - cbeg : chunk;
-                S_lane = (float)sqrt(total / (double)Lc);
-                if (warp == 0) APMS_STORE(a.Sbar[c0 + lane], S_lane);
+                const float S_lane = (float)sqrt(total / (double)Lc);
+                S_new_sh[buf][lane] = S_lane;
+                APMS_STORE(a.Sbar[c0 + lane], S_lane);
             }
-            // Section 3.3 steps 5-6 for this slab: every group with the new scale of its chunk
-            float c_new[2];
-            c_new[0] = __fmul_rn(sa.lr, __shfl_sync(0xffffffffu, S_lane, k0));      // lr * (+-S) = +-(lr * S)
-            c_new[1] = __fmul_rn(sa.lr, __shfl_sync(0xffffffffu, S_lane, k1));
-            {
-                const int st = q % kStages;
-                if (!mbar_wait(&full[st], (uint32_t)(q / kStages) & 1u)) { failed = 1; ok = false; }
-                if (ok) {
-                    const float* vs = reinterpret_cast<const float*>(smem + (size_t)st * stage_bytes);
-                    const float* xs = vs + kSlab;
-                    float4 vv[2], xx[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
-                        xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[st]);
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int grp = u ? g1 : g0;
-                        const int k = grp * kGroup + lane * 4;
-                        const uint32_t nib = nb[buf][grp * 4 + wl] >> sh;
-                        xx[u].x = apply_stored(xx[u].x, vv[u].x, nib & 1u, c_new[u]);
-                        xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new[u]);
-                        xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new[u]);
-                        xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, c_new[u]);
-                        st4_checked(sa.x + base_e, k, L, xx[u]);
-                    }
-                }
-                ++q;
-            }
-            // the slab's sign words leave in whole 16-byte pieces
-            if (ok) {
-                uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
-                const int nwords = (L + 31) / 32;
-                const int w4 = threadIdx.x * 4;
-                if (w4 + 3 < nwords) st_stream_words4(ob + w4, *reinterpret_cast<const uint4*>(nb[buf] + w4));
-                else for (int r = w4; r < nwords; ++r) APMS_STORE(ob[r], nb[buf][r]);
-            }
+            if (w >= 1) update_slab(w - 1, prev0, prev1);                 // its scales were formed a slab ago, before this slab's barrier
+            prev0 = mine0; prev1 = mine1;
+        }
+        if (!leave && nmine > 0) {
+            leave = consumer_barrier_any(!ok || *vfailed != 0);           // the last slab's scales are in shared memory
+            if (!leave) update_slab(nmine - 1, prev0, prev1);
         }
     }
     __syncthreads();                                   // every warp has left its loops; shared memory may go

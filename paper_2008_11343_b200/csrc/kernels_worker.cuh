@@ -163,6 +163,8 @@ struct WorkerFineArgs {
     int64_t tile0, e0, e1;            // a launch may cover the elements [e0, e1) of whole chunks only (multiples of 512 without SPLIT)
     int i0, ni, run;
     float beta1, omb1;
+    float inv_chunk;                  // 1 / chunk in binary32 when there are fewer than 2^20 chunks (see div_small_quotient), else 0
+    float inv_run, inv_per_stretch;   // 1 / run and 1 / (ni * run) in binary32 (see div_u32)
 };
 
 // One warp's 512 elements (L of them live).  TWO: a chunk boundary lies inside, at sign word `bw`: the lanes whose
@@ -234,11 +236,11 @@ __global__ void __launch_bounds__(kThreads, 4)
 k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t per_stretch = (int64_t)a.ni * a.run;
-    const int64_t stretch = (int64_t)blockIdx.x / per_stretch;
-    const int rem = (int)((int64_t)blockIdx.x - stretch * per_stretch);
-    const int ii = rem / a.run;
-    const int64_t tl = stretch * a.run + (rem - ii * a.run);
+    const uint32_t per_stretch = (uint32_t)a.ni * (uint32_t)a.run;        // the grid has fewer than 2^31 blocks
+    const uint32_t stretch = div_u32(blockIdx.x, per_stretch, a.inv_per_stretch);
+    const uint32_t rem = blockIdx.x - stretch * per_stretch;
+    const int ii = (int)div_u32(rem, (uint32_t)a.run, a.inv_run);
+    const int64_t tl = (int64_t)stretch * a.run + (rem - (uint32_t)ii * (uint32_t)a.run);
     if (tl >= a.tiles) return;                                 // whole CTA: the last stretch may be short
     const int64_t t = a.tile0 + tl;
     const int i = a.i0 + ii;
@@ -251,7 +253,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
         return;
     }
     const int L = (int)(left < kFineSub ? left : kFineSub);
-    const int64_t c = base / a.chunk;
+    const int64_t c = a.inv_chunk != 0.0f ? div_small_quotient(base, a.chunk, a.inv_chunk) : base / a.chunk;
     const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
     float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
     const uint32_t* __restrict__ mbits = a.Bbar + base / 32;

@@ -81,8 +81,6 @@ class ShardedStep:
         dev = like_bits.device
         mk = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
         self._buffers = {
-            "send_bits": [mk((n, self.row_words[k]), like_bits.dtype) for k in range(self.world)],
-            "send_scales": [mk((n, self.row_scales[k]), like_scales.dtype) for k in range(self.world)],
             "recv_bits": mk((self.world * n, self.row_words[me]), like_bits.dtype),
             "recv_scales": mk((self.world * n, self.row_scales[me]), like_scales.dtype),
             "gather_bits": mk((self.world, max(self.row_words)), like_bits.dtype),
@@ -100,11 +98,15 @@ class ShardedStep:
 
         The worker phase runs range by range, in the order of the serving processes (the same order on every
         process, so that the grouped transfers of a range pair up like one gather and cannot deadlock): as soon
-        as the kernels of range k are enqueued, this process's rows of that range are packed and handed to the
-        transfer to process k, which runs while the later ranges are still being compressed.  Transfers are
+        as the kernels of range k are enqueued, this process's rows of that range are handed - straight from
+        the message buffers, no packing - to the transfer to process k, which runs while the later ranges are
+        still being compressed.  Transfers are
         stream-ordered after the kernels (NCCL) - nothing waits on the host until the server phase needs the
         received rows."""
         b, dist, n, me = self.b, self.dist, self.b.n, self.rank
+        for req in self._sends:                                                 # the previous step's transfers have read the messages
+            req.wait()
+        self._sends = []
         ranged = hasattr(b, "worker_phase_range")
         if not ranged:
             b.worker_phase(grads)                                               # steps 1-2, whole vector
@@ -112,33 +114,30 @@ class ShardedStep:
         if self._buffers is None:
             self._make_buffers(msgs[0][0], msgs[0][1])
         buf = self._buffers
-        for req in self._sends:                                                 # the previous step's send buffers are free again
-            req.wait()
-        self._sends = []
         recvs = []
         for k in range(self.world):
             (w0, w1), (cb, ce) = self.words[k], self.ranges[k]
             if ranged:
                 b.worker_phase_range(grads, cb, ce)                             # steps 1-2 for the chunks process k serves
-            # step 3 (exchange 1): the part of every local message that process k serves goes to process k
-            for i, (bits, scales) in enumerate(msgs):
-                buf["send_bits"][k][i, :w1 - w0].copy_(bits[w0:w1])
-                buf["send_scales"][k][i].copy_(scales[cb:ce])
+            # step 3 (exchange 1): the part of every local message that process k serves goes to process k,
+            # straight from the message buffers (a contiguous piece of each) into the receiver's rows
             ops = []
             if k == me:
                 for q in range(self.world):
-                    rows = slice(q * n, (q + 1) * n)
-                    if q == me:
-                        buf["recv_bits"][rows].copy_(buf["send_bits"][k])
-                        buf["recv_scales"][rows].copy_(buf["send_scales"][k])
-                        continue
-                    peer = self.global_rank(q)
-                    ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][rows], peer, self.group))
-                    ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][rows], peer, self.group))
+                    for i in range(n):
+                        row = q * n + i
+                        if q == me:
+                            buf["recv_bits"][row, :w1 - w0].copy_(msgs[i][0][w0:w1])
+                            buf["recv_scales"][row, :ce - cb].copy_(msgs[i][1][cb:ce])
+                            continue
+                        peer = self.global_rank(q)
+                        ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][row, :w1 - w0], peer, self.group))
+                        ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][row, :ce - cb], peer, self.group))
             else:
                 peer = self.global_rank(k)
-                ops.append(dist.P2POp(dist.isend, buf["send_bits"][k], peer, self.group))
-                ops.append(dist.P2POp(dist.isend, buf["send_scales"][k], peer, self.group))
+                for bits, scales in msgs:
+                    ops.append(dist.P2POp(dist.isend, bits[w0:w1], peer, self.group))
+                    ops.append(dist.P2POp(dist.isend, scales[cb:ce], peer, self.group))
             if ops:
                 (recvs if k == me else self._sends).extend(dist.batch_isend_irecv(ops))
         for req in recvs:
@@ -168,7 +167,7 @@ class ShardedStep:
     def wire_bytes_per_step(self) -> int:
         """Bytes this process sends per step (both exchanges), for comparison with 4 d per worker."""
         n, me = self.b.n, self.rank
-        ex1 = sum(4 * n * (self.row_words[k] + self.row_scales[k]) for k in range(self.world) if k != me)
+        ex1 = sum(4 * n * ((self.words[k][1] - self.words[k][0]) + self.row_scales[k]) for k in range(self.world) if k != me)
         ex2 = (self.world - 1) * 4 * (self.row_words[me] + self.row_scales[me])
         return ex1 + ex2
 

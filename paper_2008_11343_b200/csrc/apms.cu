@@ -373,11 +373,10 @@ apms_status launch_finalize(apms_ctx* c, int first_row, int rows, int64_t cb, in
     return launch_check(c, "k_finalize_scales");
 }
 
-bool use_fine_worker(const apms_ctx* c, bool whole_vector)
+bool use_fine_worker(const apms_ctx* c)
 {
     if (c->team_mode == APMS_TEAM_CTA || c->team_mode == APMS_TEAM_WARP) return false;
     if (c->L.t.l1) return false;             // see use_staged_server
-    if (!whole_vector && c->L.fine_split) return false;      // a range of chunks must end between two warps' pieces
     return (!c->m_is_fp32 || c->variant == APMS_VARIANT_GRADIENT) && c->L.fine_tiles > 0;
 }
 
@@ -463,10 +462,9 @@ apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0
 // Section 3.3 steps 1-2 for workers i0 .. i0+ni-1 on chunks [cb, ce).
 apms_status launch_worker(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni, int64_t cb, int64_t ce)
 {
-    const bool whole = cb == 0 && ce == c->L.C;
     if (c->compressor == APMS_COMPRESSOR_TOPK) return launch_worker_topk(c, G, gtype, i0, ni);      // whole vector only (checked by the callers)
     if (ce <= cb) return APMS_OK;
-    if (use_fine_worker(c, whole)) return launch_worker_fine(c, G, gtype, i0, ni, cb, ce);
+    if (use_fine_worker(c)) return launch_worker_fine(c, G, gtype, i0, ni, cb, ce);
     WorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz;
     a.B = c->B(0); a.Wp = c->L.Wp;

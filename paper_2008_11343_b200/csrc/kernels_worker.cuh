@@ -29,7 +29,7 @@ template <bool M32, bool CHECKED>
 __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __restrict__ z, uint32_t* __restrict__ obits,
                                              int grp, int lane, int L, float s_old, float Sbar,
                                              float4 gv, float4 zv, float4 mv, uint32_t mw, double& acc, bool l1,
-                                             bool send_gradient = false)
+                                             bool send_gradient = false, bool keep = true)      // keep = false: this lane's elements are not this launch's
 {
     const int k = grp * kGroup + lane * 4;
     float mm[4];
@@ -57,9 +57,9 @@ __device__ __forceinline__ void worker_group(float beta1, float omb1, float* __r
         }
     }
     const float4 out = make_float4(zn[0], zn[1], zn[2], zn[3]);
-    if (CHECKED) st4_checked(z, k, L, out); else st_stream4(z + k, out);
+    if (keep) { if (CHECKED) st4_checked(z, k, L, out); else st_stream4(z + k, out); }
     const uint32_t word = pack_group_words(nibble, lane);
-    if ((lane & 7) == 0) {
+    if ((lane & 7) == 0 && keep) {
         const int wk = grp * 4 + (lane >> 3);
         if (!CHECKED || wk * 32 < L) st_stream_word(obits + wk, word);     // streaming: a plain store here costs ~4 % of the kernel
     }
@@ -168,11 +168,14 @@ struct WorkerFineArgs {
 };
 
 // One warp's 512 elements (L of them live).  TWO: a chunk boundary lies inside, at sign word `bw`: the lanes whose
-// word lies past it use the next chunk's scales (s_hi, S_hi) and add their squares to acc_hi.
+// word lies past it use the next chunk's scales (s_hi, S_hi) and add their squares to acc_hi.  `keep`: bit 0 - the
+// elements before the boundary belong to this launch, bit 1 - those past it do (a launch over a range of chunks
+// ends at a chunk boundary, which may be this one; what does not belong is neither stored nor summed).
 template <int GT, bool SENDG, bool TWO>
 __device__ __forceinline__ void fine_piece(const WorkerFineArgs& a, const void* __restrict__ g, float* __restrict__ z,
                                            const uint32_t* __restrict__ mbits, uint32_t* __restrict__ obits, int lane, int L,
-                                           int bw, float s_lo, float S_lo, float s_hi, float S_hi, double& acc, double& acc_hi)
+                                           int bw, float s_lo, float S_lo, float s_hi, float S_hi, double& acc, double& acc_hi,
+                                           int keep = 3)
 {
     if (L == kFineSub) {
         float4 gv[kFineU], zv[kFineU];
@@ -204,12 +207,12 @@ __device__ __forceinline__ void fine_piece(const WorkerFineArgs& a, const void* 
             }
             if (TWO) { acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0; }
             else acc = part;
-            st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            if (!TWO || (keep & (hi ? 2 : 1))) st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
             const uint32_t word = pack_group_words(nibble, lane);       // valid in lanes 0, 8, 16, 24
             const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
             if ((lane >> 2) == u) outw = got;                               // lane 4u + j keeps word j of group u
         }
-        if (lane < 4 * kFineU) st_stream_word(obits + lane, outw);
+        if (lane < 4 * kFineU && (!TWO || (keep & (lane >= bw ? 2 : 1)))) st_stream_word(obits + lane, outw);
     } else {
         const int ngroups = (L + kGroup - 1) / kGroup;
         for (int grp = 0; grp < ngroups; ++grp) {
@@ -221,7 +224,7 @@ __device__ __forceinline__ void fine_piece(const WorkerFineArgs& a, const void* 
                 const bool hi = grp * 4 + (lane >> 3) >= bw;
                 double part = 0.0;
                 worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, hi ? s_hi : s_lo, hi ? S_hi : S_lo, gv, zv,
-                                          make_float4(0, 0, 0, 0), mw, part, false, SENDG);
+                                          make_float4(0, 0, 0, 0), mw, part, false, SENDG, (keep & (hi ? 2 : 1)) != 0);
                 acc += hi ? 0.0 : part; acc_hi += hi ? part : 0.0;
             } else {
                 worker_group<false, true>(a.beta1, a.omb1, z, obits, grp, lane, L, s_lo, S_lo, gv, zv,
@@ -245,7 +248,7 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     const int64_t t = a.tile0 + tl;
     const int i = a.i0 + ii;
     const int64_t base = t * kFineTile + (int64_t)warp * kFineSub;     // this warp's 512 elements
-    if (base < a.e0 || base >= a.e1) return;                   // a launch over a range of chunks: the tiles at its ends are shared
+    if (base + kFineSub <= a.e0 || base >= a.e1) return;       // a launch over a range of chunks: the tiles at its ends are shared
     double* __restrict__ slot = a.partial + (int64_t)ii * a.Pp + (t * kWarps + warp) * (SPLIT ? 2 : 1);
     const int64_t left = a.d - base;
     if (left <= 0) {                                           // past the end of the vector
@@ -264,11 +267,14 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     // elements of this warp that belong to chunk c + 1 begin at its sign word bw (SPLIT only; rare for long chunks)
     const int64_t next = (c + 1) * a.chunk - base;
     if (SPLIT && next < L) {
-        fine_piece<GT, SENDG, true>(a, g, z, mbits, obits, lane, L, (int)(next >> 5), s_lo, S_lo, srow[c + 1], a.Sbar[c + 1], acc, acc_hi);
+        // the boundary may be the start or the end of the launch's range: then only one side is this launch's
+        const int keep = (base + next <= a.e0) ? 2 : ((base + next >= a.e1) ? 1 : 3);
+        fine_piece<GT, SENDG, true>(a, g, z, mbits, obits, lane, L, (int)(next >> 5), s_lo, S_lo, srow[c + 1], a.Sbar[c + 1], acc, acc_hi, keep);
         acc = warp_sum(acc);
         acc_hi = warp_sum(acc_hi);
-        if (lane == 0) { APMS_STORE(slot[0], acc); APMS_STORE(slot[1], acc_hi); }
+        if (lane == 0) { if (keep & 1) APMS_STORE(slot[0], acc); if (keep & 2) APMS_STORE(slot[1], acc_hi); }
     } else {
+        if (base < a.e0) return;                               // (only with SPLIT: a piece before the range that holds no boundary)
         fine_piece<GT, SENDG, false>(a, g, z, mbits, obits, lane, L, 0, s_lo, S_lo, s_lo, S_lo, acc, acc_hi);
         acc = warp_sum(acc);
         if (lane == 0) APMS_STORE(slot[0], acc);                          // slot [1] of a piece without a boundary is never read

@@ -397,7 +397,8 @@ def test_error_norms_match_the_oracle_state():
 @pytest.mark.parametrize("d,n,chunk,cuts", [(9 * 2048 + 300, 4, 2048, (0, 3, 10)), (5 * 4096 + 1, 3, 4096, (0, 1, 5, 6)),
                                             (7 * 96 + 5, 5, 96, (0, 4, 8)), (3 * 70016, 2, 70016, (0, 2, 3)),
                                             (6 * 32768, 16, 32768, (0, 6)), (9 * 4096 + 100, 4, 4096, (0, 2, 3, 7, 10)),
-                                            (5 * 2080 + 100, 3, 2080, (0, 2, 6)), (23 * 512 + 9, 2, 512, (0, 5, 6, 24))])
+                                            (5 * 2080 + 100, 3, 2080, (0, 2, 6)), (23 * 512 + 9, 2, 512, (0, 5, 6, 24)),
+                                            (9 * 1056 + 700, 4, 1056, (0, 1, 2, 5, 9, 10)), (4 * 70016 + 33, 2, 70016, (0, 1, 3, 5))])
 def test_phase_wise_step_equals_the_whole_step(d, n, chunk, cuts):
     """worker phase, the server phase range by range from COPIES of the messages laid out as a receiver would
     hold them (rows = senders, word 0 = first word of the range), apply phase: bit-identical to apms_compressed_step."""

@@ -303,6 +303,32 @@ __device__ __forceinline__ float prefix8_entry(uint32_t mine, uint32_t t)
     return acc;
 }
 
+// One lane's four elements of a group after the sums over the workers: average, plus the implied old error,
+// stored as the new compensated values; returns the four sign bits and adds the squares to acc.
+// CHECKED = false: the whole slab lies inside the tile (no element needs a bounds test).
+template <bool CHECKED>
+__device__ __forceinline__ uint32_t server_finish_group(float4 zo4, float sum0, float sum1, float sum2, float sum3, float S_old,
+                                                        float inv_n, float nf, float* __restrict__ zdst, int k, int L, double& acc)
+{
+    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
+    const float sum[4] = {sum0, sum1, sum2, sum3};
+    float zn[4];
+    uint32_t nibble = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float avg = (inv_n != 0.0f) ? __fmul_rn(sum[e], inv_n) : __fdiv_rn(sum[e], nf);
+        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
+        if (!CHECKED || k + e < L) {
+            const double zd = (double)zn[e];
+            acc = fma(zd, zd, acc);
+            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+        }
+    }
+    if (CHECKED) st4_checked(zdst, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+    else st_stream4(zdst + k, make_float4(zn[0], zn[1], zn[2], zn[3]));
+    return nibble;
+}
+
 // A CTA of the fused form walks `span` consecutive chunks (short chunks are grouped so that a CTA
 // still streams about 32768 elements and the ring never drains between chunks); the unfused form
 // (chunks cut into tiles) handles one tile.  Jobs are numbered across the CTA's whole walk: per
@@ -428,26 +454,16 @@ k_server_staged(const ServerStagedArgs sa)
                 signed_scale_sums<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl, negs, prefix8, n, sh, s01, s23, t01, t23);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
+                const bool whole = (j + 1) * kSlab <= L;                 // no element of this slab needs a bounds test (warp-uniform)
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int grp = j * kSlabGroups + (u ? g1 : g0);
                     const int k = grp * kGroup + lane * 4;
                     const float4 zo4 = u ? zo1 : zo0;
-                    const float zo[4] = {zo4.x, zo4.y, zo4.z, zo4.w};
-                    const float sum[4] = {u ? t01.x : s01.x, u ? t01.y : s01.y, u ? t23.x : s23.x, u ? t23.y : s23.y};
-                    float zn[4];
-                    uint32_t nibble = 0;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float avg = (sa.inv_n != 0.0f) ? __fmul_rn(sum[e], sa.inv_n) : __fdiv_rn(sum[e], a.nf);
-                        zn[e] = __fadd_rn(avg, implied_error(zo[e], S_old));
-                        if (k + e < L) {
-                            const double zd = (double)zn[e];
-                            acc = fma(zd, zd, acc);
-                            nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
-                        }
-                    }
-                    st4_checked(a.zbar + it.base, k, L, make_float4(zn[0], zn[1], zn[2], zn[3]));
+                    const float2 lo = u ? t01 : s01, hi = u ? t23 : s23;
+                    const uint32_t nibble = whole
+                        ? server_finish_group<false>(zo4, lo.x, lo.y, hi.x, hi.y, S_old, sa.inv_n, a.nf, a.zbar + it.base, k, L, acc)
+                        : server_finish_group<true>(zo4, lo.x, lo.y, hi.x, hi.y, S_old, sa.inv_n, a.nf, a.zbar + it.base, k, L, acc);
                     const uint32_t word = pack_group_words(nibble, lane);
                     if ((lane & 7) == 0) nb[off_out + grp * 4 + wl] = word;   // words past L hold zeros and are never stored
                 }
@@ -486,7 +502,8 @@ k_server_staged(const ServerStagedArgs sa)
                         xx[u].y = apply_stored(xx[u].y, vv[u].y, nib & 2u, c_new);
                         xx[u].z = apply_stored(xx[u].z, vv[u].z, nib & 4u, c_new);
                         xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, c_new);
-                        st4_checked(sa.x + it.base, k, L, xx[u]);
+                        if ((j + 1) * kSlab <= L) st_stream4(sa.x + it.base + k, xx[u]);
+                        else st4_checked(sa.x + it.base, k, L, xx[u]);
                     }
                 }
             } else if (ok && threadIdx.x == 0) {

@@ -128,7 +128,7 @@ typedef enum {
  * that the server does not keep is left untouched by the model update when that is exact (lr >= +0,
  * eps > 0, no negative or NaN entry in v); otherwise every element is updated.  Chosen with
  * apms_set_compressor until the first compression-phase step has run; TOPK works with the momentum
- * variant, the l2 scale setting and the whole-step functions. */
+ * variant and the l2 scale setting, through the whole-step functions and the apms_topk_* phase-wise calls. */
 typedef enum {
     APMS_COMPRESSOR_ONEBIT = 0,
     APMS_COMPRESSOR_TOPK = 1
@@ -264,6 +264,42 @@ apms_status apms_server_phase(apms_ctx* ctx, const uint32_t* bits_rows_dev, int6
                               const float* scale_rows_dev, int64_t row_scales, int rows,
                               int64_t chunk_begin, int64_t chunk_end);
 apms_status apms_apply_phase(apms_ctx* ctx);
+
+/* The phase-wise step with the top-k compressor (Section 5.1, second item; the compressor the paper runs on 8 GPUs
+ * for ResNet-18).  On the wire a top-k message is a selection mask (one bit per element, the layout of the sign
+ * words) plus the kept values in index order: K = ceil(fraction * L) values per chunk of L elements, stored
+ * apms_topk_values_per_chunk() = ceil(fraction * chunk) apart (the last, shorter chunk fills fewer).  Inside a
+ * context the values stay where they are (the compensated vectors); these calls pack and unpack them:
+ *
+ *   apms_worker_phase       (whole vector) steps 1-2; worker i's mask is its message's sign-word buffer
+ *                           (apms_get_message);
+ *   apms_topk_pack_values   writes the kept values of worker `worker` (-1: of the server's message, after the
+ *                           server phase) for chunks [chunk_begin, chunk_end) to vals_dev (device,
+ *                           (chunk_end - chunk_begin) * values_per_chunk floats);
+ *   [exchange 1: masks and packed values of the chunks a peer serves go to that peer]
+ *   apms_topk_server_phase  step 4 and, for the kept elements of these chunks, steps 5-6: `rows` received messages
+ *                           (row j: row_words mask words from mask_rows_dev + j * row_words, word 0 = first word of
+ *                           chunk chunk_begin; row_vals packed values from val_rows_dev + j * row_vals), summed in
+ *                           row order.  scratch_dev: caller-owned device memory of
+ *                           apms_topk_server_scratch_bytes(ctx, rows, chunk_begin, chunk_end) bytes, 16-byte aligned
+ *                           (the rows are spread out there); may be reused by the next call;
+ *   [exchange 2: every process's range of the server's message - mask words (apms_get_message(ctx, -1)) and packed
+ *    values (apms_topk_pack_values(ctx, -1, ...)) - goes to all peers]
+ *   apms_topk_put_server_range  takes over a range computed elsewhere: mask words (word 0 = first word of chunk
+ *                           chunk_begin), the kept values to their places, steps 5-6 for them;
+ *   apms_apply_phase        ends the step.
+ *
+ * The phase-wise top-k step needs the conditions under which an element that is not kept does not move (lr >= +0,
+ * eps > 0, no negative or NaN entry in v; APMS_ERR_BAD_STATE otherwise).  With rows in global worker order and the
+ * ranges covering every chunk once the result equals apms_compressed_step of one context holding all workers. */
+int64_t     apms_topk_values_per_chunk(const apms_ctx* ctx);
+apms_status apms_topk_pack_values(apms_ctx* ctx, int worker, int64_t chunk_begin, int64_t chunk_end, float* vals_dev);
+size_t      apms_topk_server_scratch_bytes(const apms_ctx* ctx, int rows, int64_t chunk_begin, int64_t chunk_end);
+apms_status apms_topk_server_phase(apms_ctx* ctx, const uint32_t* mask_rows_dev, int64_t row_words,
+                                   const float* val_rows_dev, int64_t row_vals, int rows,
+                                   int64_t chunk_begin, int64_t chunk_end, void* scratch_dev, size_t scratch_bytes);
+apms_status apms_topk_put_server_range(apms_ctx* ctx, const uint32_t* mask_words_dev, const float* vals_dev,
+                                       int64_t chunk_begin, int64_t chunk_end);
 
 /* The same step with the exchanges done by the GPUs themselves, for processes on one node whose
  * GPUs reach each other's memory (NVLink / NVSwitch peers): every process maps its peers' workspaces

@@ -54,6 +54,12 @@ SIGNATURES = {
     "apms_get_message": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
     "apms_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64]),
     "apms_apply_phase": (C.c_int, [C.c_void_p]),
+    "apms_topk_values_per_chunk": (C.c_int64, [C.c_void_p]),
+    "apms_topk_pack_values": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
+    "apms_topk_server_scratch_bytes": (C.c_size_t, [C.c_void_p, C.c_int, C.c_int64, C.c_int64]),
+    "apms_topk_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64,
+                                         C.c_void_p, C.c_size_t]),
+    "apms_topk_put_server_range": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64]),
     "apms_server_phase_rows": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64]),
     "apms_put_server_range": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64]),
     "apms_message_offsets": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
@@ -184,6 +190,28 @@ def apms_worker_phase(h, grad_ptrs: Sequence[int], grad_type: int):
 
 def apms_worker_phase_range(h, grad_ptrs: Sequence[int], grad_type: int, chunk_begin: int, chunk_end: int):
     _check(h, load().apms_worker_phase_range(h, _ptr_array(grad_ptrs), grad_type, chunk_begin, chunk_end))
+
+
+def apms_topk_values_per_chunk(h) -> int:
+    return int(load().apms_topk_values_per_chunk(h))
+
+
+def apms_topk_pack_values(h, worker: int, chunk_begin: int, chunk_end: int, vals_ptr: int):
+    _check(h, load().apms_topk_pack_values(h, worker, chunk_begin, chunk_end, vals_ptr))
+
+
+def apms_topk_server_scratch_bytes(h, rows: int, chunk_begin: int, chunk_end: int) -> int:
+    return int(load().apms_topk_server_scratch_bytes(h, rows, chunk_begin, chunk_end))
+
+
+def apms_topk_server_phase(h, mask_rows_ptr: int, row_words: int, val_rows_ptr: int, row_vals: int, rows: int,
+                           chunk_begin: int, chunk_end: int, scratch_ptr: int, scratch_bytes: int):
+    _check(h, load().apms_topk_server_phase(h, mask_rows_ptr, row_words, val_rows_ptr, row_vals, rows, chunk_begin, chunk_end,
+                                            scratch_ptr, scratch_bytes))
+
+
+def apms_topk_put_server_range(h, mask_words_ptr: int, vals_ptr: int, chunk_begin: int, chunk_end: int):
+    _check(h, load().apms_topk_put_server_range(h, mask_words_ptr, vals_ptr, chunk_begin, chunk_end))
 
 
 def apms_get_message(h, worker: int):
@@ -408,6 +436,7 @@ class Context:
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self._h = apms_create(d, n, beta1, beta2, eps, lr, chunk)
+        self.topk = False
         nbytes = apms_workspace_bytes(d, n, chunk)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         if library_workspace:
@@ -601,6 +630,31 @@ class Context:
 
     def set_compressor(self, kind: int, topk_fraction: float = 0.01):
         apms_set_compressor(self._h, kind, topk_fraction)
+        self.topk = kind == COMPRESSOR_TOPK
+
+    # phase-wise step with the top-k compressor: masks travel as the sign words do, the kept values packed
+    def topk_values_per_chunk(self) -> int:
+        return apms_topk_values_per_chunk(self._h)
+
+    def topk_pack_values(self, worker: int, chunk_begin: int, chunk_end: int, out):
+        """out: float32 CUDA tensor of (chunk_end - chunk_begin) * topk_values_per_chunk() elements."""
+        assert out.is_cuda and out.is_contiguous() and out.numel() >= (chunk_end - chunk_begin) * self.topk_values_per_chunk()
+        apms_topk_pack_values(self._h, worker, chunk_begin, chunk_end, out.data_ptr())
+
+    def topk_server_phase(self, mask_rows, val_rows, chunk_begin: int, chunk_end: int):
+        """mask_rows: int32 CUDA tensor [rows, row_words]; val_rows: float32 CUDA tensor [rows, row_vals]."""
+        import torch
+
+        assert mask_rows.is_contiguous() and val_rows.is_contiguous() and mask_rows.shape[0] == val_rows.shape[0]
+        need = apms_topk_server_scratch_bytes(self._h, mask_rows.shape[0], chunk_begin, chunk_end)
+        if getattr(self, "_topk_scratch", None) is None or self._topk_scratch.numel() < need:
+            self._topk_scratch = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device)
+        apms_topk_server_phase(self._h, mask_rows.data_ptr(), mask_rows.shape[1], val_rows.data_ptr(), val_rows.shape[1],
+                               mask_rows.shape[0], chunk_begin, chunk_end, self._topk_scratch.data_ptr(), self._topk_scratch.numel())
+
+    def topk_put_server_range(self, mask_words, vals, chunk_begin: int, chunk_end: int):
+        assert mask_words.is_cuda and vals.is_cuda and mask_words.is_contiguous() and vals.is_contiguous()
+        apms_topk_put_server_range(self._h, mask_words.data_ptr(), vals.data_ptr(), chunk_begin, chunk_end)
 
     def set_variant(self, variant: int):
         apms_set_variant(self._h, variant)

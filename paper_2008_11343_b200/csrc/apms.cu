@@ -738,7 +738,7 @@ apms_status launch_server_and_apply(apms_ctx* c)
         a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp;
         a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n; a.lr = c->lr; a.eps = c->eps;
-        a.frac = c->topk_frac;
+        a.frac = c->topk_frac; a.c0 = 0;
         if (c->L.C > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");
         Timed t(c, APMS_KERNEL_SERVER);
         k_topk_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
@@ -941,8 +941,15 @@ apms_status apms_worker_phase_range(apms_ctx* c, const void* const* grads_dev, a
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_worker_phase needs the COMPRESSED phase (call apms_freeze_v first)");
     if (c->substep > 1 || (c->substep == 1 && c->worker_chunks >= c->L.C))
         return fail(c, APMS_ERR_BAD_STATE, "the worker phase of this step is complete (continue with the server and apply phases)");
-    if (c->compressor != APMS_COMPRESSOR_ONEBIT) return fail(c, APMS_ERR_BAD_STATE, "the phase-wise step exists for the 1-bit compressor only");
     if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (c->compressor == APMS_COMPRESSOR_TOPK) {
+        if (chunk_begin != 0 || chunk_end != c->L.C) return fail(c, APMS_ERR_INVALID_ARG, "with the top-k compressor the worker phase covers the whole vector in one call");
+        if (c->variant != APMS_VARIANT_MOMENTUM) return fail(c, APMS_ERR_BAD_STATE, "top-k runs with the momentum variant");
+        bool sparse = false;
+        apms_status sst = topk_sparse_update_allowed(c, &sparse);
+        if (sst != APMS_OK) return sst;
+        if (!sparse) return fail(c, APMS_ERR_BAD_STATE, "the phase-wise top-k step needs lr >= +0, eps > 0 and a variance without negative or NaN entries");
+    }
     if (c->worker_chunks + (chunk_end - chunk_begin) > c->L.C) return fail(c, APMS_ERR_INVALID_ARG, "the ranges of one step's worker phase cover more chunks than there are");
     GradPtrs G;
     apms_status st = check_grads(c, grads_dev, (int)type, &G, c->L.n);
@@ -971,6 +978,7 @@ apms_status apms_server_phase(apms_ctx* c, const uint32_t* bits_rows_dev, int64_
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase needs the COMPRESSED phase");
     if (c->substep < 1 || c->worker_chunks < c->L.C) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase follows a complete worker phase (every chunk once)");
+    if (c->compressor != APMS_COMPRESSOR_ONEBIT) return fail(c, APMS_ERR_BAD_STATE, "top-k messages go through apms_topk_server_phase");
     if (!bits_rows_dev || !scale_rows_dev) return fail(c, APMS_ERR_INVALID_ARG, "a message pointer is NULL");
     if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
     if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
@@ -995,6 +1003,7 @@ apms_status apms_server_phase_rows(apms_ctx* c, const uint32_t* const* bits_rows
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows needs the COMPRESSED phase");
     if (c->substep < 1 || c->worker_chunks < c->L.C) return fail(c, APMS_ERR_BAD_STATE, "apms_server_phase_rows follows a complete worker phase (every chunk once)");
+    if (c->compressor != APMS_COMPRESSOR_ONEBIT) return fail(c, APMS_ERR_BAD_STATE, "top-k messages go through apms_topk_server_phase");
     if (!bits_rows || !scale_rows) return fail(c, APMS_ERR_INVALID_ARG, "a pointer array is NULL");
     if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
     if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
@@ -1040,6 +1049,116 @@ apms_status apms_message_offsets(apms_ctx* c, int worker, size_t* bits_offset, s
     if (bits_offset) *bits_offset = (size_t)((char*)(worker < 0 ? c->Bbar() : c->B(worker)) - c->ws);
     if (scales_offset) *scales_offset = (size_t)((char*)(worker < 0 ? c->Sbar() : c->s(worker)) - c->ws);
     return APMS_OK;
+}
+
+int64_t apms_topk_values_per_chunk(const apms_ctx* c)
+{
+    if (!c || c->compressor != APMS_COMPRESSOR_TOPK) return 0;
+    long long K = (long long)ceil(c->topk_frac * (double)c->L.chunk);
+    if (K < 1) K = 1;
+    if (K > c->L.chunk) K = c->L.chunk;
+    return (int64_t)K;
+}
+
+apms_status apms_topk_pack_values(apms_ctx* c, int worker, int64_t chunk_begin, int64_t chunk_end, float* vals_dev)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->compressor != APMS_COMPRESSOR_TOPK) return fail(c, APMS_ERR_BAD_STATE, "the context does not run the top-k compressor");
+    if (c->phase != APMS_PHASE_COMPRESSED || c->substep < 1) return fail(c, APMS_ERR_BAD_STATE, "apms_topk_pack_values belongs to a phase-wise step (after apms_worker_phase)");
+    if (worker < -1 || worker >= c->L.n) return fail(c, APMS_ERR_INVALID_ARG, "worker index out of range (-1 = the server's message)");
+    if (worker < 0 && c->substep < 2) return fail(c, APMS_ERR_BAD_STATE, "the server's message exists after apms_topk_server_phase");
+    if (!vals_dev) return fail(c, APMS_ERR_INVALID_ARG, "vals_dev is NULL");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (chunk_begin == chunk_end) return APMS_OK;
+    TopkPackArgs a;
+    a.z = worker < 0 ? c->zbar() : c->z(worker); a.dz = c->L.dz;
+    a.mask = worker < 0 ? c->Bbar() : c->B(worker); a.Wp = c->L.Wp;
+    a.vals = vals_dev; a.vstride = 0;
+    a.d = c->L.d; a.chunk = c->L.chunk; a.c0 = chunk_begin; a.nchunks = chunk_end - chunk_begin;
+    a.kmax = (int)apms_topk_values_per_chunk(c);
+    if (a.nchunks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");
+    k_topk_pack<<<(unsigned)a.nchunks, kThreads, 0, c->stream>>>(a);
+    return launch_check(c, "k_topk_pack");
+}
+
+size_t apms_topk_server_scratch_bytes(const apms_ctx* c, int rows, int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c || rows < 1 || chunk_begin < 0 || chunk_end > c->L.C || chunk_begin >= chunk_end) return 0;
+    const int64_t elems = (chunk_end - chunk_begin) * c->L.chunk;
+    return (size_t)rows * round_up((size_t)elems, 64) * 4;
+}
+
+apms_status apms_topk_server_phase(apms_ctx* c, const uint32_t* mask_rows_dev, int64_t row_words, const float* val_rows_dev,
+                                   int64_t row_vals, int rows, int64_t chunk_begin, int64_t chunk_end, void* scratch_dev, size_t scratch_bytes)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->compressor != APMS_COMPRESSOR_TOPK) return fail(c, APMS_ERR_BAD_STATE, "the context does not run the top-k compressor");
+    if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_topk_server_phase needs the COMPRESSED phase");
+    if (c->substep < 1 || c->worker_chunks < c->L.C) return fail(c, APMS_ERR_BAD_STATE, "apms_topk_server_phase follows apms_worker_phase");
+    if (!mask_rows_dev || !val_rows_dev || !scratch_dev) return fail(c, APMS_ERR_INVALID_ARG, "a buffer pointer is NULL");
+    if (rows < 1 || rows > APMS_MAX_WORKERS) return fail(c, APMS_ERR_INVALID_ARG, "rows must be between 1 and APMS_MAX_WORKERS");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (chunk_begin == chunk_end) { c->substep = 2; return APMS_OK; }
+    const int64_t nchunks = chunk_end - chunk_begin;
+    const int kmax = (int)apms_topk_values_per_chunk(c);
+    const int64_t first_elem = chunk_begin * c->L.chunk;
+    const int64_t last_elem = chunk_end * c->L.chunk < c->L.d ? chunk_end * c->L.chunk : c->L.d;
+    const int64_t need_words = (last_elem - first_elem + 31) / 32;
+    if (row_words < need_words || row_vals < nchunks * kmax)
+        return fail(c, APMS_ERR_INVALID_ARG, "rows too short: row_words must cover the range's mask words, row_vals its chunks times apms_topk_values_per_chunk");
+    if (scratch_bytes < apms_topk_server_scratch_bytes(c, rows, chunk_begin, chunk_end) || ((uintptr_t)scratch_dev & 15u))
+        return fail(c, APMS_ERR_INVALID_ARG, "scratch too small (apms_topk_server_scratch_bytes) or not 16-byte aligned");
+    if (nchunks * rows > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (row, chunk) pairs for one launch");
+    bool sparse = false;
+    apms_status st = topk_sparse_update_allowed(c, &sparse);
+    if (st != APMS_OK) return st;
+    if (!sparse) return fail(c, APMS_ERR_BAD_STATE, "the phase-wise top-k step needs lr >= +0, eps > 0 and a variance without negative or NaN entries");
+    const int64_t dstride = (int64_t)round_up((size_t)(nchunks * c->L.chunk), 64);
+    TopkUnpackArgs u;
+    u.mask = mask_rows_dev; u.row_words = row_words; u.vals = val_rows_dev; u.row_vals = row_vals;
+    u.dense = (float*)scratch_dev; u.dstride = dstride;
+    u.d = c->L.d; u.chunk = c->L.chunk; u.c0 = chunk_begin; u.nchunks = nchunks; u.kmax = kmax;
+    {
+        Timed t(c, APMS_KERNEL_SERVER);
+        k_topk_unpack<<<(unsigned)(nchunks * rows), kThreads, 0, c->stream>>>(u);
+        st = launch_check(c, "k_topk_unpack");
+        if (st != APMS_OK) return st;
+        // the server kernel addresses rows by absolute element / word: shift the received rows back to where index 0 would be
+        TopkServerArgs a;
+        a.sparse = 1;
+        a.z = (const float*)scratch_dev - first_elem; a.dz = dstride;
+        a.B = mask_rows_dev - first_elem / 32; a.Wp = row_words;
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
+        a.d = c->L.d; a.chunk = c->L.chunk; a.n = rows; a.nf = (float)rows; a.lr = c->lr; a.eps = c->eps;
+        a.frac = c->topk_frac; a.c0 = chunk_begin;
+        k_topk_server<<<(unsigned)nchunks, kThreads, 0, c->stream>>>(a);
+        st = launch_check(c, "k_topk_server");
+        if (st != APMS_OK) return st;
+    }
+    c->substep = 2;
+    return APMS_OK;
+}
+
+apms_status apms_topk_put_server_range(apms_ctx* c, const uint32_t* mask_words_dev, const float* vals_dev, int64_t chunk_begin, int64_t chunk_end)
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (c->compressor != APMS_COMPRESSOR_TOPK) return fail(c, APMS_ERR_BAD_STATE, "the context does not run the top-k compressor");
+    if (c->phase != APMS_PHASE_COMPRESSED || c->substep < 1 || c->worker_chunks < c->L.C)
+        return fail(c, APMS_ERR_BAD_STATE, "apms_topk_put_server_range belongs to a phase-wise step (after apms_worker_phase)");
+    if (!mask_words_dev || !vals_dev) return fail(c, APMS_ERR_INVALID_ARG, "a buffer pointer is NULL");
+    if (chunk_begin < 0 || chunk_end > c->L.C || chunk_begin > chunk_end) return fail(c, APMS_ERR_INVALID_ARG, "chunk range out of bounds");
+    if (chunk_begin == chunk_end) { c->substep = 2; return APMS_OK; }
+    if (chunk_end - chunk_begin > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");
+    TopkPutArgs a;
+    a.mask = mask_words_dev; a.vals = vals_dev;
+    a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.v = c->v(); a.x = c->x();
+    a.d = c->L.d; a.chunk = c->L.chunk; a.c0 = chunk_begin;
+    a.kmax = (int)apms_topk_values_per_chunk(c); a.lr = c->lr; a.eps = c->eps;
+    Timed t(c, APMS_KERNEL_APPLY);
+    k_topk_put<<<(unsigned)(chunk_end - chunk_begin), kThreads, 0, c->stream>>>(a);
+    apms_status st = launch_check(c, "k_topk_put");
+    if (st == APMS_OK) c->substep = 2;
+    return st;
 }
 
 apms_status apms_ipc_export(apms_ctx* c, void* handle_out)
@@ -1089,6 +1208,14 @@ apms_status apms_apply_phase(apms_ctx* c)
     if (!c) return APMS_ERR_INVALID_ARG;
     if (c->phase != APMS_PHASE_COMPRESSED) return fail(c, APMS_ERR_BAD_STATE, "apms_apply_phase needs the COMPRESSED phase");
     if (c->substep != 2) return fail(c, APMS_ERR_BAD_STATE, "apms_apply_phase follows apms_server_phase");
+    if (c->compressor == APMS_COMPRESSOR_TOPK) {
+        // the kept elements were updated where their server range was computed (apms_topk_server_phase) or taken
+        // over (apms_topk_put_server_range); the momentum stays implicit in (zbar, mask)
+        c->m_is_fp32 = false;
+        c->csteps += 1;
+        c->substep = 0; c->worker_chunks = 0;
+        return APMS_OK;
+    }
     apms_status st = launch_apply(c);
     if (st != APMS_OK) return st;
     c->m_is_fp32 = c->variant == APMS_VARIANT_GRADIENT;

@@ -430,6 +430,7 @@ struct TopkServerArgs {
     int64_t d, chunk;
     int n; float nf, lr, eps;
     double frac;
+    int64_t c0;                       // first chunk of this launch (a launch may serve a range of chunks from received rows)
     // An element that is not kept has m = +0, and x - (lr * 0) / (sqrt(v) + eps) is x itself whenever
     // lr >= +0, eps > 0 and v is neither negative nor NaN (the host checks all three).  Then only the
     // kept elements are touched (sparse != 0): the momentum stays implicit in (zbar, mask), v and x are read
@@ -446,7 +447,7 @@ k_topk_server(const TopkServerArgs a)
     __shared__ uint32_t sh[2];
     __shared__ uint32_t warp_ties[kWarps];
     __shared__ TopkList list;
-    const int64_t c = blockIdx.x;
+    const int64_t c = a.c0 + blockIdx.x;
     const int64_t base = c * a.chunk;
     const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
     const int nwords = (L + 31) / 32;
@@ -632,6 +633,120 @@ k_topk_server(const TopkServerArgs a)
             for (int e = 0; e < 4 && k + e < L; ++e) { acc[k + e] = mm[e]; x[k + e] = xx[e]; }
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// The top-k message on the wire (phase-wise step, one process per GPU): a selection mask plus the kept values in
+// index order, K per chunk.  The kernels below turn the library's in-place form (mask + the compensated vector)
+// into that message and back.  One CTA per (row, chunk); thread t owns a contiguous run of the chunk's mask words,
+// a block-wide exclusive scan of the runs' popcounts gives every kept element its position in the message.
+
+// Calls fn(j, rank) for every set bit j (element index in the chunk, ascending per thread) of words[0..nwords).
+template <typename F>
+__device__ __forceinline__ void topk_for_each_kept(const uint32_t* __restrict__ words, int nwords, uint32_t* scan /* kThreads + 1 words of shared memory */, F fn)
+{
+    const int per = (nwords + kThreads - 1) / kThreads;
+    const int w0 = threadIdx.x * per, w1 = (w0 + per < nwords) ? w0 + per : nwords;
+    uint32_t mine = 0;
+    for (int w = w0; w < w1; ++w) mine += __popc(words[w]);
+    scan[threadIdx.x + 1] = mine;
+    if (threadIdx.x == 0) scan[0] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) for (int t = 1; t <= kThreads; ++t) scan[t] += scan[t - 1];      // 256 additions: not worth a tree
+    __syncthreads();
+    uint32_t rank = scan[threadIdx.x];
+    for (int w = w0; w < w1; ++w) {
+        uint32_t word = words[w];
+        while (word) {
+            const int j = w * 32 + (__ffs(word) - 1);
+            word &= word - 1;
+            fn(j, rank);
+            ++rank;
+        }
+    }
+}
+
+struct TopkPackArgs {
+    const float* z; int64_t dz;            // rows of compensated vectors (row stride dz)
+    const uint32_t* mask; int64_t Wp;      // rows of selection masks
+    float* vals; int64_t vstride;          // out: rows of packed values, (chunk - c0) * kmax + rank within a row
+    int64_t d, chunk, c0, nchunks;
+    int kmax;
+};
+
+// grid: rows * nchunks.  vals[row][(c - c0) * kmax + rank] = z[row][element of that rank in chunk c].
+__global__ void __launch_bounds__(kThreads)
+k_topk_pack(const TopkPackArgs a)
+{
+    __shared__ uint32_t scan[kThreads + 1];
+    const int row = (int)(blockIdx.x / a.nchunks);
+    const int64_t c = a.c0 + blockIdx.x % a.nchunks;
+    const int64_t base = c * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const float* __restrict__ z = a.z + (int64_t)row * a.dz + base;
+    float* __restrict__ out = a.vals + (int64_t)row * a.vstride + (c - a.c0) * a.kmax;
+    const int kmax = a.kmax;
+    topk_for_each_kept(a.mask + (int64_t)row * a.Wp + base / 32, (L + 31) / 32, scan,
+                       [&](int j, uint32_t rank) { if (j < L && rank < (uint32_t)kmax) out[rank] = z[j]; });
+}
+
+struct TopkUnpackArgs {
+    const uint32_t* mask; int64_t row_words;     // received rows: word 0 = first word of chunk c0
+    const float* vals; int64_t row_vals;         // received rows of packed values
+    float* dense; int64_t dstride;               // out: rows of compensated values, element 0 = first element of chunk c0
+    int64_t d, chunk, c0, nchunks;
+    int kmax;
+};
+
+// grid: rows * nchunks.  The kept values of every received row go back to their positions in a dense row.
+__global__ void __launch_bounds__(kThreads)
+k_topk_unpack(const TopkUnpackArgs a)
+{
+    __shared__ uint32_t scan[kThreads + 1];
+    const int row = (int)(blockIdx.x / a.nchunks);
+    const int64_t cr = blockIdx.x % a.nchunks;                  // chunk within the range
+    const int64_t base = (a.c0 + cr) * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const float* __restrict__ in = a.vals + (int64_t)row * a.row_vals + cr * a.kmax;
+    float* __restrict__ out = a.dense + (int64_t)row * a.dstride + cr * a.chunk;
+    const int kmax = a.kmax;
+    topk_for_each_kept(a.mask + (int64_t)row * a.row_words + cr * (a.chunk / 32), (L + 31) / 32, scan,
+                       [&](int j, uint32_t rank) { if (j < L && rank < (uint32_t)kmax) out[j] = in[rank]; });
+}
+
+struct TopkPutArgs {
+    const uint32_t* mask;                        // the range's server mask words, word 0 = first word of chunk c0
+    const float* vals;                           // its kept values, cr * kmax + rank
+    float* zbar; uint32_t* Bbar; const float* v; float* x;
+    int64_t d, chunk, c0;
+    int kmax; float lr, eps;
+};
+
+// grid: chunks of the range.  A server range computed elsewhere becomes this context's: mask words, the kept
+// values at their places in zbar (where the workers read the momentum C[zbar] under the mask), and Section 3.3
+// step 6 for the kept elements (the others have momentum +0 and do not move: see TopkServerArgs::sparse).
+__global__ void __launch_bounds__(kThreads)
+k_topk_put(const TopkPutArgs a)
+{
+    __shared__ uint32_t scan[kThreads + 1];
+    const int64_t cr = blockIdx.x;
+    const int64_t base = (a.c0 + cr) * a.chunk;
+    const int L = (int)((a.d - base < a.chunk) ? a.d - base : a.chunk);
+    const int nwords = (L + 31) / 32;
+    const uint32_t* __restrict__ words = a.mask + cr * (a.chunk / 32);
+    const float* __restrict__ in = a.vals + cr * a.kmax;
+    float* __restrict__ zb = a.zbar + base;
+    const float* __restrict__ v = a.v + base;
+    float* __restrict__ x = a.x + base;
+    const int kmax = a.kmax;
+    topk_for_each_kept(words, nwords, scan, [&](int j, uint32_t rank) {
+        if (j < L && rank < (uint32_t)kmax) {
+            const float m = in[rank];
+            zb[j] = m;
+            x[j] = apply_elem(x[j], v[j], m, a.lr, a.eps);
+        }
+    });
+    for (int w = threadIdx.x; w < nwords; w += kThreads) a.Bbar[base / 32 + w] = words[w];
 }
 
 // Sets *flag if any v[j] is negative or NaN (v >= 0 fails); -0 and +inf pass.

@@ -69,9 +69,14 @@ class ShardedStep:
         self.ranges = chunk_ranges(backend.C, self.world)
         self.words = [word_range(cb, ce, backend.chunk, backend.d) for cb, ce in self.ranges]
         self.row_words = [_round4(w1 - w0) for w0, w1 in self.words]
-        self.row_scales = [ce - cb for cb, ce in self.ranges]
+        # what accompanies the sign words: one scale per chunk - or, with the top-k compressor, where the words are
+        # a selection mask, the chunk's kept values (`per` = ceil(fraction * chunk) floats per chunk)
+        self.topk = bool(getattr(backend, "topk", False))
+        self.per = backend.topk_values_per_chunk() if self.topk else 1
+        self.row_scales = [(ce - cb) * self.per for cb, ce in self.ranges]
         self._buffers = None
         self._sends = []
+        self._packed = None
 
     # ------------------------------------------------------------------ buffers (made once)
     def _make_buffers(self, like_bits, like_scales):
@@ -107,13 +112,22 @@ class ShardedStep:
         for req in self._sends:                                                 # the previous step's transfers have read the messages
             req.wait()
         self._sends = []
-        ranged = hasattr(b, "worker_phase_range")
+        ranged = hasattr(b, "worker_phase_range") and not self.topk
         if not ranged:
             b.worker_phase(grads)                                               # steps 1-2, whole vector
         msgs = [b.message(i) for i in range(n)]
+        if self.topk:                                                           # the kept values, packed chunk by chunk
+            import torch
+
+            if self._packed is None:
+                self._packed = [torch.zeros(b.C * self.per, dtype=torch.float32, device=msgs[0][0].device) for _ in range(n + 1)]
+            for i in range(n):
+                b.topk_pack_values(i, 0, b.C, self._packed[i])
+            msgs = [(msgs[i][0], self._packed[i]) for i in range(n)]
         if self._buffers is None:
             self._make_buffers(msgs[0][0], msgs[0][1])
         buf = self._buffers
+        per = self.per
         recvs = []
         for k in range(self.world):
             (w0, w1), (cb, ce) = self.words[k], self.ranges[k]
@@ -128,16 +142,16 @@ class ShardedStep:
                         row = q * n + i
                         if q == me:
                             buf["recv_bits"][row, :w1 - w0].copy_(msgs[i][0][w0:w1])
-                            buf["recv_scales"][row, :ce - cb].copy_(msgs[i][1][cb:ce])
+                            buf["recv_scales"][row, :(ce - cb) * per].copy_(msgs[i][1][cb * per:ce * per])
                             continue
                         peer = self.global_rank(q)
                         ops.append(dist.P2POp(dist.irecv, buf["recv_bits"][row, :w1 - w0], peer, self.group))
-                        ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][row, :ce - cb], peer, self.group))
+                        ops.append(dist.P2POp(dist.irecv, buf["recv_scales"][row, :(ce - cb) * per], peer, self.group))
             else:
                 peer = self.global_rank(k)
                 for bits, scales in msgs:
                     ops.append(dist.P2POp(dist.isend, bits[w0:w1], peer, self.group))
-                    ops.append(dist.P2POp(dist.isend, scales[cb:ce], peer, self.group))
+                    ops.append(dist.P2POp(dist.isend, scales[cb * per:ce * per], peer, self.group))
             if ops:
                 (recvs if k == me else self._sends).extend(dist.batch_isend_irecv(ops))
         for req in recvs:
@@ -145,13 +159,20 @@ class ShardedStep:
 
         # step 4: average and recompress the chunks this process serves
         cb, ce = self.ranges[me]
-        b.server_phase(buf["recv_bits"], buf["recv_scales"], cb, ce)
+        if self.topk:
+            b.topk_server_phase(buf["recv_bits"], buf["recv_scales"], cb, ce)   # and steps 5-6 for the elements it keeps
+        else:
+            b.server_phase(buf["recv_bits"], buf["recv_scales"], cb, ce)
 
         # step 5 (exchange 2): every process's range of the server message goes to everybody
         sbits, sscales = b.message(-1)
         w0, w1 = self.words[me]
         buf["mine_bits"][:w1 - w0].copy_(sbits[w0:w1])
-        buf["mine_scales"][:ce - cb].copy_(sscales[cb:ce])
+        if self.topk:
+            b.topk_pack_values(-1, cb, ce, self._packed[n])
+            buf["mine_scales"][:(ce - cb) * per].copy_(self._packed[n][:(ce - cb) * per])
+        else:
+            buf["mine_scales"][:ce - cb].copy_(sscales[cb:ce])
         if self.world > 1:
             dist.all_gather_into_tensor(buf["gather_bits"].view(-1), buf["mine_bits"], group=self.group)
             dist.all_gather_into_tensor(buf["gather_scales"].view(-1), buf["mine_scales"], group=self.group)
@@ -159,8 +180,11 @@ class ShardedStep:
                 if k == me:
                     continue
                 (v0, v1), (kb, ke) = self.words[k], self.ranges[k]
-                sbits[v0:v1].copy_(buf["gather_bits"][k, :v1 - v0])
-                sscales[kb:ke].copy_(buf["gather_scales"][k, :ke - kb])
+                if self.topk:                                                   # mask, kept values to their places, steps 5-6 for them
+                    b.topk_put_server_range(buf["gather_bits"][k], buf["gather_scales"][k], kb, ke)
+                else:
+                    sbits[v0:v1].copy_(buf["gather_bits"][k, :v1 - v0])
+                    sscales[kb:ke].copy_(buf["gather_scales"][k, :ke - kb])
 
         b.apply_phase()                                                         # steps 5-6
 

@@ -66,6 +66,18 @@ def test_topk_steps_leave_the_guard_bytes_alone(d, n, chunk, frac):
     assert np.array_equal(ctx.get_state(B.STATE_X).view(np.uint32), orc.x.view(np.uint32))
     ctx.error_norms()
     ctx.check_guards()
+    # one more step through the phase-wise calls: messages packed, unpacked, served in two ranges
+    from test_gpu_parity import _topk_rows
+
+    gs = wl.host_gradients(w, 6)
+    ctx.worker_phase(H.upload(gs)); orc.compressed_step(gs)
+    mid = ctx.C // 2
+    for cb, ce in ((0, mid), (mid, ctx.C)):
+        masks, vals = _topk_rows([ctx], cb, ce)
+        ctx.topk_server_phase(masks, vals, cb, ce)
+    ctx.apply_phase()
+    assert np.array_equal(ctx.get_state(B.STATE_X).view(np.uint32), orc.x.view(np.uint32))
+    ctx.check_guards()
 
 
 @pytest.mark.parametrize("d,n,chunk,cuts", [(9 * 2048 + 300, 4, 2048, (0, 3, 10)), (7 * 96 + 5, 5, 96, (0, 4, 8)), (3 * 70016, 2, 70016, (0, 2, 3)),

@@ -269,9 +269,6 @@ def test_topk_compressor_bit_identical(d, n, chunk, frac):
     with pytest.raises(B.ApmsError) as e:
         ctx.set_compressor(B.COMPRESSOR_ONEBIT)               # fixed once a compression-phase step has run
     assert e.value.status == B.ERR_BAD_STATE
-    with pytest.raises(B.ApmsError) as e:
-        ctx.worker_phase(H.upload(wl.host_gradients(w, 9)))
-    assert e.value.status == B.ERR_BAD_STATE
 
 
 def test_topk_ties_and_teacher_forced_errors():
@@ -345,6 +342,162 @@ def test_topk_long_free_run(frac):
         ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
         if step % 10 == 0:
             _topk_compare(ctx, orc, w, step)
+
+
+def _topk_rows(ctxs, cb, ce):
+    """The messages of all workers of `ctxs` for chunks [cb, ce) as a receiver holds them: mask rows (word 0 = first
+    word of chunk cb) and rows of packed values, in worker order."""
+    import torch
+
+    c0 = ctxs[0]
+    per = c0.topk_values_per_chunk()
+    w0, w1 = cb * c0.chunk // 32, (min(c0.d, ce * c0.chunk) + 31) // 32
+    masks, vals = [], []
+    for ctx in ctxs:
+        for i in range(ctx.n):
+            masks.append(ctx.message(i)[0][w0:w1].clone())
+            v = torch.full(((ce - cb) * per,), float("nan"), dtype=torch.float32, device="cuda")
+            ctx.topk_pack_values(i, cb, ce, v)
+            vals.append(v)
+    return torch.stack(masks).contiguous(), torch.stack(vals).contiguous()
+
+
+@pytest.mark.parametrize("d,n,chunk,frac,cuts", [(5 * 4096 + 1234, 3, 4096, 0.01, (0, 2, 6)), (7 * 96 + 5, 4, 96, 0.1, (0, 1, 5, 8)),
+                                                 (2 * 32768 + 23552, 4, 32768, 0.05, (0, 1, 3)), (131072 + 5000, 2, 131072, 0.01, (0, 1, 2)),
+                                                 (9 * 512 + 3, 2, 512, 0.5, (0, 4, 10)), (3 * 2080 + 64, 2, 2080, 1.0, (0, 3, 4))])
+def test_topk_phase_wise_step_equals_the_whole_step(d, n, chunk, frac, cuts):
+    """Top-k through the phase-wise calls: worker phase, the server phase range by range from packed messages
+    (masks + the kept values, as they would arrive from other processes), apply phase - bit-identical to
+    apms_compressed_step and to the oracle, over steps that take the kernels' different routes."""
+    w = tiny(d, n, chunk, cfg_id=185)
+    a, orc = H.make_pair(w)
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b.set_params(wl.initial_params(w))
+    for c in (a, b):
+        c.set_compressor(B.COMPRESSOR_TOPK, frac)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+    gs = wl.host_gradients(w, 0)
+    for c in (a, b):
+        c.warmup_step(H.upload(gs))
+        c.freeze_v()
+    orc.warmup_step(gs); orc.freeze_v()
+    assert cuts[-1] == a.C
+    for step in range(1, 6):
+        host = wl.host_gradients(w, step)
+        gs = H.upload(host)
+        a.compressed_step(gs)
+        orc.compressed_step(host)
+        b.worker_phase(gs)
+        with pytest.raises(B.ApmsError) as e:
+            b.server_phase_rows([b.message_ptrs(i)[0] for i in range(n)], [b.message_ptrs(i)[1] for i in range(n)], 0, b.C)
+        assert e.value.status == B.ERR_BAD_STATE                    # top-k messages have their own server call
+        for cb, ce in zip(cuts, cuts[1:]):
+            masks, vals = _topk_rows([b], cb, ce)
+            b.topk_server_phase(masks, vals, cb, ce)
+        b.apply_phase()
+        _topk_compare(a, orc, w, step)
+        for k in (B.STATE_X, B.STATE_M, B.STATE_SERVER_ERR, B.STATE_SERVER_BITS):
+            assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32)), (step, k)
+        for i in range(n):
+            for k in (B.STATE_WORKER_ERR, B.STATE_WORKER_BITS):
+                assert np.array_equal(a.get_state(k, i).view(np.uint32), b.get_state(k, i).view(np.uint32)), (step, k, i)
+    with pytest.raises(B.ApmsError) as e:
+        b.worker_phase_range(H.upload(wl.host_gradients(w, 9)), 0, 1)       # top-k compresses the whole vector at once
+    assert e.value.status in (B.ERR_INVALID_ARG, B.ERR_BAD_STATE)
+
+
+@pytest.mark.parametrize("d,chunk,frac", [(11 * 2048 + 77, 2048, 0.02), (3 * 32768 + 23552, 32768, 0.01), (9 * 96 + 5, 96, 0.25)])
+def test_topk_two_emulated_ranks_equal_one_four_worker_run(d, chunk, frac):
+    """Two contexts of two workers each stand for two processes: each serves half of the chunks from all four workers'
+    packed messages and hands its range of the server's message (mask + kept values) to the other, which takes it over.
+    Equal, bit for bit, to one context with all four workers and to the oracle."""
+    import torch
+
+    w = tiny(d, 4, chunk, cfg_id=186)
+    whole, orc = H.make_pair(w)
+    ranks = [B.Context(w.d, 2, w.beta1, w.beta2, w.eps, w.lr, w.chunk) for _ in range(2)]
+    for c in [whole] + ranks:
+        c.set_compressor(B.COMPRESSOR_TOPK, frac)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+    x0 = wl.initial_params(w)
+    for c in ranks:
+        c.set_params(x0)
+    host = wl.host_gradients(w, 0)
+    gs = H.upload(host)
+    whole.warmup_step(gs); orc.warmup_step(host)
+    for r in range(2):                                   # the warmup phase averages all four workers' gradients everywhere
+        ranks[r].restore(0, B.PHASE_WARMUP)
+    whole.freeze_v(); orc.freeze_v()
+    for r in range(2):
+        for k in (B.STATE_X, B.STATE_V, B.STATE_M):
+            ranks[r].set_state(k, whole.get_state(k))
+        ranks[r].restore(1, B.PHASE_COMPRESSED)
+    from paper_2008_11343_b200 import sharded
+    ranges = sharded.chunk_ranges(whole.C, 2)
+    per = whole.topk_values_per_chunk()
+    for step in range(1, 5):
+        host = wl.host_gradients(w, step)
+        gs = H.upload(host)
+        whole.compressed_step(gs)
+        orc.compressed_step(host)
+        for r in range(2):
+            ranks[r].worker_phase(gs[2 * r:2 * r + 2])
+        for r in range(2):
+            cb, ce = ranges[r]
+            masks, vals = _topk_rows(ranks, cb, ce)
+            ranks[r].topk_server_phase(masks, vals, cb, ce)
+        for r in range(2):                               # exchange 2: my range of the server's message to the other rank
+            cb, ce = ranges[r]
+            w0, w1 = cb * chunk // 32, (min(d, ce * chunk) + 31) // 32
+            mask = ranks[r].message(-1)[0][w0:w1].clone()
+            vals = torch.zeros((ce - cb) * per, dtype=torch.float32, device="cuda")
+            ranks[r].topk_pack_values(-1, cb, ce, vals)
+            ranks[1 - r].topk_put_server_range(mask, vals, cb, ce)
+        for r in range(2):
+            ranks[r].apply_phase()
+        _topk_compare(whole, orc, w, step)
+        for r in range(2):
+            for which in (B.STATE_X, B.STATE_M, B.STATE_SERVER_BITS):
+                assert np.array_equal(ranks[r].get_state(which).view(np.uint32), whole.get_state(which).view(np.uint32)), (step, r, which)
+            lo, hi = ranges[r][0] * chunk, min(d, ranges[r][1] * chunk)
+            assert np.array_equal(ranks[r].get_state(B.STATE_SERVER_ERR)[lo:hi].view(np.uint32),
+                                  whole.get_state(B.STATE_SERVER_ERR)[lo:hi].view(np.uint32))
+            for i in range(2):
+                assert np.array_equal(ranks[r].get_state(B.STATE_WORKER_ERR, i).view(np.uint32),
+                                      whole.get_state(B.STATE_WORKER_ERR, 2 * r + i).view(np.uint32))
+
+
+def test_sharded_step_with_the_topk_compressor_equals_the_whole_step():
+    import socket
+
+    import torch.distributed as dist
+
+    from paper_2008_11343_b200 import sharded
+
+    w = tiny(11 * 2048 + 77, 4, 2048, cfg_id=187)
+    a = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    b = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+    for c in (a, b):
+        c.set_compressor(B.COMPRESSOR_TOPK, 0.03)
+        c.set_params(wl.initial_params(w))
+        c.warmup_step(H.upload(wl.host_gradients(w, 0)))
+        c.freeze_v()
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    try:
+        step = sharded.ShardedStep(b)
+        for k in range(1, 5):
+            gs = H.upload(wl.host_gradients(w, k))
+            a.compressed_step(gs)
+            step.step(gs)
+        for k in (B.STATE_X, B.STATE_M, B.STATE_SERVER_ERR, B.STATE_SERVER_BITS):
+            assert np.array_equal(a.get_state(k).view(np.uint32), b.get_state(k).view(np.uint32))
+        for i in range(w.n):
+            assert np.array_equal(a.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), b.get_state(B.STATE_WORKER_ERR, i).view(np.uint32))
+    finally:
+        dist.destroy_process_group()
 
 
 # ------------------------------------------------------------------ phase driver and error monitor

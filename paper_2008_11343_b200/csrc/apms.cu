@@ -59,7 +59,7 @@ struct GuardRegion { size_t off, bytes; const char* what; };
 struct Layout {
     int64_t d, chunk, C, W, dz, Wp, Cp;
     int64_t fine_tiles, fine_Pp;   // 4096-element tiles of the fine worker form (0 when the chunk length does not allow it)
-    int fine_split;
+    int fine_split, fine_words;
     int n;
     Tiling t;
     size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
@@ -109,9 +109,10 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L, size_t guard = 0, s
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64) + (int64_t)(guard / 8);
     L->off_part = take("partial sums of split chunks", L->t.P > 1 ? un + 1 : 0, L->t.Pp, (size_t)(L->C * L->t.P), 8);   // n worker rows + 1 server row
-    L->fine_tiles = (chunk >= kFineSub) ? (d + kFineTile - 1) / kFineTile : 0;
+    L->fine_tiles = (d + kFineTile - 1) / kFineTile;
     L->fine_split = (chunk % kFineSub != 0) ? 1 : 0;     // a warp's 512 elements may lie in two chunks: two partial sums each
-    const size_t fine_used = (size_t)L->fine_tiles * kWarps * (size_t)(L->fine_split ? 2 : 1);
+    L->fine_words = chunk < kFineSub ? 1 : 0;            // ... or in several: one partial sum per sign word
+    const size_t fine_used = L->fine_words ? (size_t)L->W : (size_t)L->fine_tiles * kWarps * (size_t)(L->fine_split ? 2 : 1);
     L->fine_Pp = (int64_t)round_up(fine_used, 64) + (int64_t)(guard / 8);
     L->off_fine = take("partial sums of the fine worker form", un, L->fine_Pp, fine_used, 8);
     L->off_stage = take("staging buffers", 2, L->dz, ud, 4);
@@ -404,6 +405,16 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     {
         Timed t(c, APMS_KERNEL_WORKER);
         const bool sendg = c->variant == APMS_VARIANT_GRADIENT;
+        if (c->L.fine_words) {                     // chunks below 512 elements: per-word scales and sums
+            if (sendg) APMS_DISPATCH_GRAD(gtype, k_worker_fine_words<GT, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+            else       APMS_DISPATCH_GRAD(gtype, k_worker_fine_words<GT, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+            apms_status st = launch_check(c, "k_worker_fine_words");
+            if (st != APMS_OK) return st;
+            const int64_t total = (int64_t)ni * (ce - cb);
+            k_finalize_words<<<(unsigned)((total + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->fine_partial(i0), c->L.fine_Pp, c->s(i0), c->L.Cp,
+                                                                                                    ni, cb, ce - cb, c->L.d, c->L.chunk);
+            return launch_check(c, "k_finalize_words");
+        }
         if (c->L.fine_split) {
             if (sendg) APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, true, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
             else       APMS_DISPATCH_GRAD(gtype, k_worker_fine<GT, false, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));

@@ -281,6 +281,125 @@ k_worker_fine(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
     }
 }
 
+// The same tiling for chunks below 512 elements: a warp's 512 elements then hold several chunks, but a sign word
+// (32 elements = the 8 lanes of one access) still lies in one chunk.  Every lane looks up the scales of its word's
+// chunk, the squares are summed per word (three shuffle steps inside the 8 lanes) into one slot per word, and
+// k_finalize_words adds a chunk's words in order.  A launch over a range of chunks skips the words outside it.
+template <int GT, bool SENDG>
+__global__ void __launch_bounds__(kThreads, 4)
+k_worker_fine_words(const __grid_constant__ GradPtrs G, const WorkerFineArgs a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t per_stretch = (uint32_t)a.ni * (uint32_t)a.run;
+    const uint32_t stretch = div_u32(blockIdx.x, per_stretch, a.inv_per_stretch);
+    const uint32_t rem = blockIdx.x - stretch * per_stretch;
+    const int ii = (int)div_u32(rem, (uint32_t)a.run, a.inv_run);
+    const int64_t tl = (int64_t)stretch * a.run + (rem - (uint32_t)ii * (uint32_t)a.run);
+    if (tl >= a.tiles) return;
+    const int64_t t = a.tile0 + tl;
+    const int i = a.i0 + ii;
+    const int64_t base = t * kFineTile + (int64_t)warp * kFineSub;
+    if (base + kFineSub <= a.e0 || base >= a.e1 || base >= a.d) return;
+    const int64_t left = a.d - base;
+    const int L = (int)(left < kFineSub ? left : kFineSub);
+    const void* __restrict__ g = Grad<GT>::at(G.p[ii], base);
+    float* __restrict__ z = a.z + (int64_t)i * a.dz + base;
+    const uint32_t* __restrict__ mbits = a.Bbar + base / 32;
+    uint32_t* __restrict__ obits = a.B + (int64_t)i * a.Wp + base / 32;
+    const float* __restrict__ srow = a.s + (int64_t)i * a.Cp;
+    double* __restrict__ slots = a.partial + (int64_t)ii * a.Pp + base / 32;      // one slot per sign word
+    // the chunk of this lane's word in each of the four accesses: first chunk of the piece plus a small quotient
+    const int64_t c_first = base / a.chunk;
+    const uint32_t rel0 = (uint32_t)(base - c_first * a.chunk), chunk32 = (uint32_t)a.chunk;
+    const float inv_c = 1.0f / (float)chunk32;
+    const int wl = lane >> 3;
+    float s_old[kFineU], Sb[kFineU];
+    bool mine[kFineU];                                          // the word exists and belongs to this launch's range
+#pragma unroll
+    for (int u = 0; u < kFineU; ++u) {
+        const int wi = u * 4 + wl;
+        const int64_t e = base + 32 * wi;
+        mine[u] = 32 * wi < L && e >= a.e0 && e < a.e1;
+        const int64_t cw = c_first + div_u32(rel0 + 32u * (uint32_t)wi, chunk32, inv_c);
+        s_old[u] = 32 * wi < L ? srow[cw] : 0.0f;
+        Sb[u] = 32 * wi < L ? a.Sbar[cw] : 0.0f;
+    }
+    if (L == kFineSub) {
+        float4 gv[kFineU], zv[kFineU];
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            gv[u] = Grad<GT>::ld4(g, u * kGroup + lane * 4);
+            zv[u] = ld_stream4(z + u * kGroup + lane * 4);
+        }
+        const uint32_t mw = (!SENDG && lane < 4 * kFineU) ? mbits[lane] : 0u;
+        uint32_t outw = 0;
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            const uint32_t nib = __shfl_sync(0xffffffffu, mw, u * 4 + wl) >> (4 * (lane & 7));
+            const float gg[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+            const float zo[4] = {zv[u].x, zv[u].y, zv[u].z, zv[u].w};
+            float zn[4];
+            uint32_t nibble = 0;
+            double part = 0.0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float mm = bit_scale((nib >> e) & 1u, Sb[u]);
+                const float mi = SENDG ? gg[e] : __fmaf_rn(a.beta1, mm, __fmul_rn(a.omb1, gg[e]));
+                zn[e] = __fadd_rn(mi, implied_error(zo[e], s_old[u]));
+                const double zd = (double)zn[e];
+                part = fma(zd, zd, part);
+                nibble |= (zn[e] >= 0.0f ? 1u : 0u) << e;
+            }
+            if (mine[u]) st_stream4(z + u * kGroup + lane * 4, make_float4(zn[0], zn[1], zn[2], zn[3]));
+            part += __shfl_xor_sync(0xffffffffu, part, 1);      // the word's 32 squares: lanes 8k .. 8k+7
+            part += __shfl_xor_sync(0xffffffffu, part, 2);
+            part += __shfl_xor_sync(0xffffffffu, part, 4);
+            if ((lane & 7) == 0 && mine[u]) APMS_STORE(slots[u * 4 + wl], part);
+            const uint32_t word = pack_group_words(nibble, lane);
+            const uint32_t got = __shfl_sync(0xffffffffu, word, (lane & 3) * 8);
+            if ((lane >> 2) == u) outw = got;
+        }
+        if (lane < 4 * kFineU) {                                // lane j keeps word j: stored if it belongs to the range
+            const int64_t e = base + 32 * lane;
+            if (e >= a.e0 && e < a.e1) st_stream_word(obits + lane, outw);
+        }
+    } else {
+        const int ngroups = (L + kGroup - 1) / kGroup;
+#pragma unroll
+        for (int u = 0; u < kFineU; ++u) {
+            if (u >= ngroups) break;
+            const int k = u * kGroup + lane * 4;
+            const float4 gv = ld_grad4_checked<GT>(g, k, L);
+            const float4 zv = ld4_checked(z, k, L, true);
+            const uint32_t mw = (!SENDG && k < L) ? mbits[u * 4 + wl] : 0u;
+            double part = 0.0;
+            worker_group<false, true>(a.beta1, a.omb1, z, obits, u, lane, L, s_old[u], Sb[u], gv, zv,
+                                      make_float4(0, 0, 0, 0), mw, part, false, SENDG, mine[u]);
+            part += __shfl_xor_sync(0xffffffffu, part, 1);
+            part += __shfl_xor_sync(0xffffffffu, part, 2);
+            part += __shfl_xor_sync(0xffffffffu, part, 4);
+            if ((lane & 7) == 0 && mine[u]) APMS_STORE(slots[u * 4 + wl], part);
+        }
+    }
+}
+
+// Scales from one sum of squares per sign word: a thread per (row, chunk) adds the chunk's words in order.
+__global__ void __launch_bounds__(kThreads)
+k_finalize_words(const double* __restrict__ partial, int64_t Pp, float* __restrict__ scales, int64_t Cp,
+                 int rows, int64_t c_first, int64_t C, int64_t d, int64_t chunk)
+{
+    const int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (idx >= (int64_t)rows * C) return;
+    const int r = (int)(idx / C);
+    const int64_t c = c_first + idx % C;
+    const int64_t cbeg = c * chunk;
+    const int64_t Lc = (d - cbeg < chunk) ? d - cbeg : chunk;
+    const double* __restrict__ p = partial + (int64_t)r * Pp + cbeg / 32;
+    double total = 0.0;
+    for (int w = 0; w < (int)((Lc + 31) / 32); ++w) total += p[w];
+    APMS_STORE(scales[(int64_t)r * Cp + c], (float)sqrt(total / (double)Lc));
+}
+
 // Scales from the fine form's partial sums (one - or, with chunks that are not multiples of 512, two -
 // per 512 elements): a team of T lanes per (row, chunk) adds the chunk's slots in a fixed order (lane l
 // of the team takes the 512-element pieces l, l + T, ..., then the shuffle tree) and takes sqrt(sum / L).

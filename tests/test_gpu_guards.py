@@ -73,6 +73,8 @@ def test_topk_steps_leave_the_guard_bytes_alone(d, n, chunk, frac):
     ctx.worker_phase(H.upload(gs)); orc.compressed_step(gs)
     mid = ctx.C // 2
     for cb, ce in ((0, mid), (mid, ctx.C)):
+        if cb == ce:
+            continue
         masks, vals = _topk_rows([ctx], cb, ce)
         ctx.topk_server_phase(masks, vals, cb, ce)
     ctx.apply_phase()

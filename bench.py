@@ -291,6 +291,8 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
     ctx.set_timing(True)
     for kid in range(len(B.KERNEL_NAMES)):
         ctx.kernel_time(kid)
+    if args.compressor == "topk":
+        ctx.topk_route_counts()                        # reset: the counts below are those of the timed steps
     launches0 = ctx.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
@@ -317,10 +319,16 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
         if cnt:
             kernel_ms[name] = ms / cnt
     ctx.set_timing(False)
+    routes = None
+    if args.compressor == "topk":                     # how the chunks' selections were settled (exact on every route)
+        names = ("predicted_list", "two_passes", "general", "missed_above", "missed_below", "missed_overflow")
+        wr, sr = ctx.topk_route_counts()
+        routes = {"worker": dict(zip(names, wr)), "server": dict(zip(names, sr))}
     work = n_total if split else world * w.n          # worker vectors the whole job compresses per step
     out = {"ms_per_step": seconds * 1e3 / args.steps, "value": work * w.d * args.steps / seconds,
            "ms_per_step_min": per_step_ms[0], "ms_per_step_median": per_step_ms[len(per_step_ms) // 2],
-           "kernel_ms": kernel_ms, "launches": launches, "clocks": clocks.summary(), "adam": adam, "e2e": None}
+           "kernel_ms": kernel_ms, "launches": launches, "clocks": clocks.summary(), "adam": adam, "e2e": None,
+           "topk_routes": routes}
 
     # end to end through the host-gradient entry point: H2D of the n gradients and D2H of x
     # inside the timed region, every step
@@ -523,6 +531,8 @@ def main(argv=None) -> int:
                 "ms_per_step_min": m["ms_per_step_min"], "ms_per_step_median": m["ms_per_step_median"]}
         if m["adam"]:
             line["warmup_adam"] = m["adam"]
+        if m.get("topk_routes"):
+            line["topk_routes"] = m["topk_routes"]
         if "wire_bytes_per_step" in m:
             line["wire_bytes_per_step_per_process"] = m["wire_bytes_per_step"]
         print(json.dumps(line))

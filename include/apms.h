@@ -293,6 +293,13 @@ apms_status apms_apply_phase(apms_ctx* ctx);
  * eps > 0, no negative or NaN entry in v; APMS_ERR_BAD_STATE otherwise).  With rows in global worker order and the
  * ranges covering every chunk once the result equals apms_compressed_step of one context holding all workers. */
 int64_t     apms_topk_values_per_chunk(const apms_ctx* ctx);
+/* Diagnostics of the top-k kernels (no counterpart in the paper; the selection is exact on every route): how many
+ * (worker, chunk) and server chunk selections, since the last call, were settled [0] by the list of keys around the
+ * threshold predicted from the earlier steps (the chunk is read once), [1] by two passes over the chunk, [2] by the
+ * general radix select; and how many predictions missed (those chunks then took route 1 or 2) because the K-th key
+ * lay [3] above or [4] below the listed keys or [5] the list overflowed.  Synchronises the stream and resets the
+ * counters. */
+apms_status apms_topk_route_counts(apms_ctx* ctx, int64_t worker_routes[6], int64_t server_routes[6]);
 apms_status apms_topk_pack_values(apms_ctx* ctx, int worker, int64_t chunk_begin, int64_t chunk_end, float* vals_dev);
 size_t      apms_topk_server_scratch_bytes(const apms_ctx* ctx, int rows, int64_t chunk_begin, int64_t chunk_end);
 apms_status apms_topk_server_phase(apms_ctx* ctx, const uint32_t* mask_rows_dev, int64_t row_words,

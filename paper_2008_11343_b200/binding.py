@@ -55,6 +55,7 @@ SIGNATURES = {
     "apms_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64]),
     "apms_apply_phase": (C.c_int, [C.c_void_p]),
     "apms_topk_values_per_chunk": (C.c_int64, [C.c_void_p]),
+    "apms_topk_route_counts": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "apms_topk_pack_values": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p]),
     "apms_topk_server_scratch_bytes": (C.c_size_t, [C.c_void_p, C.c_int, C.c_int64, C.c_int64]),
     "apms_topk_server_phase": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int64,
@@ -194,6 +195,13 @@ def apms_worker_phase_range(h, grad_ptrs: Sequence[int], grad_type: int, chunk_b
 
 def apms_topk_values_per_chunk(h) -> int:
     return int(load().apms_topk_values_per_chunk(h))
+
+
+def apms_topk_route_counts(h):
+    """(worker routes, server routes): 6 counters each, reset by the call."""
+    wr, sr = (C.c_int64 * 6)(), (C.c_int64 * 6)()
+    _check(h, load().apms_topk_route_counts(h, wr, sr))
+    return list(wr), list(sr)
 
 
 def apms_topk_pack_values(h, worker: int, chunk_begin: int, chunk_end: int, vals_ptr: int):
@@ -635,6 +643,9 @@ class Context:
     # phase-wise step with the top-k compressor: masks travel as the sign words do, the kept values packed
     def topk_values_per_chunk(self) -> int:
         return apms_topk_values_per_chunk(self._h)
+
+    def topk_route_counts(self):
+        return apms_topk_route_counts(self._h)
 
     def topk_pack_values(self, worker: int, chunk_begin: int, chunk_end: int, out):
         """out: float32 CUDA tensor of (chunk_end - chunk_begin) * topk_values_per_chunk() elements."""

@@ -62,7 +62,7 @@ struct Layout {
     int fine_split, fine_words;
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_hint, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
     size_t guard;                  // guard bytes behind every row of every array (0 = the ordinary layout)
 };
 
@@ -104,6 +104,8 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L, size_t guard = 0, s
     L->off_Bbar = take("Bbar", 1, L->Wp, L->W, 4);
     L->off_s = take("s_i", un, L->Cp, L->C, 4);
     L->off_Sbar = take("Sbar", 1, L->Cp, L->C, 4);
+    // top-k: the thresholds of the step before last (n worker rows + 1 server row), then as many rows of learned bands
+    L->off_hint = take("threshold hints", 2 * (un + 1), L->Cp, L->C, 4);
     L->t.d = d; L->t.chunk = chunk;
     if (chunk <= kTileMax) { L->t.tile = chunk; L->t.P = 1; }
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
@@ -170,6 +172,8 @@ struct apms_ctx {
     uint32_t* Bbar() { return (uint32_t*)(ws + L.off_Bbar); }
     float* s(int i) { return (float*)(ws + L.off_s) + (int64_t)i * L.Cp; }
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
+    float* hint(int i) { return (float*)(ws + L.off_hint) + (int64_t)i * L.Cp; }   // i = n: the server's
+    float* learned(int i) { return hint(L.n + 1 + i); }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
     int* status() { return (int*)(ws + L.off_status); }
     float* den() { return (float*)(ws + L.off_den); }
@@ -454,19 +458,28 @@ apms_status launch_worker_fine(apms_ctx* c, const GradPtrs& G, int gtype, int i0
     return APMS_OK;
 }
 
+// Where the top-k kernels count the routes their chunks took (ints of the status block).
+constexpr int kRouteWorker = 16, kRouteServer = 24, kRoutes = 6;
+
 apms_status launch_worker_topk(apms_ctx* c, const GradPtrs& G, int gtype, int i0, int ni)
 {
     TopkWorkerArgs a;
     a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp; a.m32 = c->m();
     a.zbar = c->zbar(); a.Bbar = c->Bbar();
-    a.thr = c->s(0); a.Cp = c->L.Cp;
+    a.thr = c->s(0); a.hint = c->hint(0); a.learned = c->learned(0); a.route = c->status() + kRouteWorker; a.Cp = c->L.Cp;
     a.d = c->L.d; a.chunk = c->L.chunk; a.C = c->L.C; a.i0 = i0; a.ni = ni;
     a.beta1 = c->beta1; a.omb1 = 1.0f - c->beta1; a.frac = c->topk_frac;
     const int64_t blocks = c->L.C * ni;
     if (blocks > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many (chunk, worker) items for one launch");
+    const bool band = 6 * apms_topk_values_per_chunk(c) > kTopkList;       // too many for the one-sided window
     Timed t(c, APMS_KERNEL_WORKER);
-    if (c->m_is_fp32) APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, true><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
-    else              APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, false><<<(unsigned)blocks, kThreads, 0, c->stream>>>(G, a));
+    if (c->m_is_fp32) {
+        if (band) APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, true, true><<<(unsigned)blocks, kTopkThreads, 0, c->stream>>>(G, a));
+        else      APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, true, false><<<(unsigned)blocks, kTopkThreads, 0, c->stream>>>(G, a));
+    } else {
+        if (band) APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, false, true><<<(unsigned)blocks, kTopkThreads, 0, c->stream>>>(G, a));
+        else      APMS_DISPATCH_GRAD(gtype, k_topk_worker<GT, false, false><<<(unsigned)blocks, kTopkThreads, 0, c->stream>>>(G, a));
+    }
     return launch_check(c, "k_topk_worker");
 }
 
@@ -747,12 +760,12 @@ apms_status launch_server_and_apply(apms_ctx* c)
         TopkServerArgs a;
         a.sparse = sparse ? 1 : 0;
         a.z = c->z(0); a.dz = c->L.dz; a.B = c->B(0); a.Wp = c->L.Wp;
-        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.hint = c->hint(c->L.n); a.learned = c->learned(c->L.n); a.route = c->status() + kRouteServer; a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.n = c->L.n; a.nf = (float)c->L.n; a.lr = c->lr; a.eps = c->eps;
         a.frac = c->topk_frac; a.c0 = 0;
         if (c->L.C > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunks for one launch");
         Timed t(c, APMS_KERNEL_SERVER);
-        k_topk_server<<<(unsigned)c->L.C, kThreads, 0, c->stream>>>(a);
+        k_topk_server<<<(unsigned)c->L.C, kTopkThreads, 0, c->stream>>>(a);
         apms_status st = launch_check(c, "k_topk_server");
         if (st != APMS_OK) return st;
         c->m_is_fp32 = !sparse;    // sparse update: the momentum stays implicit in (zbar, Bbar)
@@ -1062,6 +1075,20 @@ apms_status apms_message_offsets(apms_ctx* c, int worker, size_t* bits_offset, s
     return APMS_OK;
 }
 
+apms_status apms_topk_route_counts(apms_ctx* c, int64_t worker_routes[6], int64_t server_routes[6])
+{
+    if (!c) return APMS_ERR_INVALID_ARG;
+    if (!worker_routes || !server_routes) return fail(c, APMS_ERR_INVALID_ARG, "an output array is NULL");
+    if (c->phase == APMS_PHASE_CREATED) return fail(c, APMS_ERR_BAD_STATE, "no workspace yet");
+    int counts[16];
+    static_assert(kRouteServer - kRouteWorker + kRoutes <= 16 && kRouteServer + kRoutes <= 64, "the counters lie inside the status block");
+    APMS_CUDA(c, cudaMemcpyAsync(counts, c->status() + kRouteWorker, sizeof counts, cudaMemcpyDeviceToHost, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->status() + kRouteWorker, 0, sizeof counts, c->stream));
+    APMS_CUDA(c, cudaStreamSynchronize(c->stream));
+    for (int r = 0; r < kRoutes; ++r) { worker_routes[r] = counts[r]; server_routes[r] = counts[kRouteServer - kRouteWorker + r]; }
+    return APMS_OK;
+}
+
 int64_t apms_topk_values_per_chunk(const apms_ctx* c)
 {
     if (!c || c->compressor != APMS_COMPRESSOR_TOPK) return 0;
@@ -1139,10 +1166,10 @@ apms_status apms_topk_server_phase(apms_ctx* c, const uint32_t* mask_rows_dev, i
         a.sparse = 1;
         a.z = (const float*)scratch_dev - first_elem; a.dz = dstride;
         a.B = mask_rows_dev - first_elem / 32; a.Wp = row_words;
-        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.v = c->v(); a.x = c->x();
+        a.zbar = c->zbar(); a.Bbar = c->Bbar(); a.m32 = c->m(); a.thr = c->Sbar(); a.hint = c->hint(c->L.n); a.learned = c->learned(c->L.n); a.route = c->status() + kRouteServer; a.v = c->v(); a.x = c->x();
         a.d = c->L.d; a.chunk = c->L.chunk; a.n = rows; a.nf = (float)rows; a.lr = c->lr; a.eps = c->eps;
         a.frac = c->topk_frac; a.c0 = chunk_begin;
-        k_topk_server<<<(unsigned)nchunks, kThreads, 0, c->stream>>>(a);
+        k_topk_server<<<(unsigned)nchunks, kTopkThreads, 0, c->stream>>>(a);
         st = launch_check(c, "k_topk_server");
         if (st != APMS_OK) return st;
     }

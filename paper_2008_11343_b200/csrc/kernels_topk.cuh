@@ -24,6 +24,16 @@ namespace {
 
 constexpr int kTopkBins = 2048;
 
+// CTA shape of the top-k kernels.  Their passes are latency-bound, so resident threads matter more than registers:
+// 1536 threads per SM at 40 registers measured fastest (at 2048 threads and 32 registers the spills cost more than
+// the extra warps give).  As 3 CTAs of 512 threads rather than 6 of 256: a chunk is then finished in half the
+// time, half as many chunks are in flight (444 x 128 KB of compensated values), and the later passes over a chunk
+// find it in L2 - with 888 chunks in flight they came from DRAM again (ncu, two-pass route, 8 workers x 116 M
+// elements: 11.5 GB read against 8.1 GB).
+constexpr int kTopkResident = 3;
+constexpr int kTopkThreads = 512, kTopkWarps = kTopkThreads / 32;
+
+
 __device__ __forceinline__ uint32_t mag_key(float z) { return __float_as_uint(z) & 0x7fffffffu; }
 
 // C[z] and the error it leaves, from a stored compensated value and its selection bit (the subtraction is
@@ -65,11 +75,11 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
                                                uint32_t& tau, uint32_t& ties)
 {
     const uint32_t b0 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    for (int b = threadIdx.x; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
     // the lower levels spread over many bins: plain atomics (combining equal bins costs more than it saves there)
 #pragma unroll 4
-    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+    for (int k = threadIdx.x * 4; k < L; k += kTopkThreads * 4) {
         const float4 zv = ld4_checked(zc, k, L, false);
         const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
 #pragma unroll
@@ -77,11 +87,11 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
             if (k + e < L && (key[e] >> 20) == b0) atomicAdd(&hist[(key[e] >> 9) & 0x7ffu], 1u);
     }
     const uint32_t b1 = (uint32_t)topk_find_bin(hist, kTopkBins, K, sh);
-    for (int b = threadIdx.x; b < 512; b += kThreads) hist[b] = 0;
+    for (int b = threadIdx.x; b < 512; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
     const uint32_t top = (b0 << 11) | b1;
 #pragma unroll 4
-    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+    for (int k = threadIdx.x * 4; k < L; k += kTopkThreads * 4) {
         const float4 zv = ld4_checked(zc, k, L, false);
         const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
 #pragma unroll
@@ -94,22 +104,93 @@ __device__ __forceinline__ void topk_threshold(const float* zc, int L, uint32_t 
 }
 
 // Last step's threshold of the same (worker, chunk) predicts this step's: only the keys at or above a
-// floor a little below it (key lowered by 2^20, an eighth of an exponent step: 0.92 of the threshold) are
+// floor a little below it (key lowered by up to 2^20, an eighth of an exponent step: 0.92 of the threshold) are
 // looked at for the selection, which is exact either way - a chunk whose window turns out to hold fewer
-// than K keys, or more than the list below can take, goes the general route (histograms over the whole
-// chunk, re-read from L2).  Error feedback piles the unsent elements up just under the threshold, and while
+// than K keys, or more than the list below can take, is counted in a further pass and goes the two-pass
+// route.  Error feedback piles the unsent elements up just under the threshold, and while
 // the errors still build up the threshold rises by 5 to 10 % a step, so the window holds several times K
-// keys (about 4 K on the benchmark's gradients at k = 1 %).  Hence a window only for K <= kTopkList / 6;
-// for larger K the first pass builds the top-level histogram of all keys itself.  A stored threshold of 0
+// keys (about 4 K on the benchmark's gradients at k = 1 %).  Hence a window only for K <= kTopkList / 6
+// (larger K: the two-sided band below), and every (worker, chunk) adapts how far below the threshold its window
+// reaches to how many keys it listed last step (topk_window_learn).  A stored threshold of 0
 // (first step) also means no window.  The list is kept small on purpose: shared memory comes out of the L1
 // cache, which the first pass, the general route and the server's sparse sum live on (a list of 4096 entries
 // made the worker 45 % and the server 30 % slower).
 constexpr int kTopkList = 2048;
-constexpr uint32_t kTopkFloorDrop = 1u << 20;
-__device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K)
+constexpr uint32_t kTopkFloorDrop = 1u << 20, kTopkFloorDropMin = 1u << 16;
+__device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K, uint32_t drop)
 {
     const uint32_t key = mag_key(last_threshold);
-    return (6 * K <= (uint32_t)kTopkList && key > kTopkFloorDrop) ? key - kTopkFloorDrop : 0u;
+    return (6 * K <= (uint32_t)kTopkList && key > drop) ? key - drop : 0u;
+}
+__device__ __forceinline__ uint32_t topk_window_drop(float learned)
+{
+    const uint32_t drop = __float_as_uint(learned);
+    return (drop >= kTopkFloorDropMin && drop <= kTopkFloorDrop) ? drop : kTopkFloorDrop;
+}
+__device__ __forceinline__ uint32_t topk_window_learn(uint32_t drop, uint32_t listed, uint32_t K)
+{
+    if (listed > 3u * kTopkList / 4) return drop / 2 >= kTopkFloorDropMin ? drop / 2 : kTopkFloorDropMin;
+    if (listed < K || listed < (uint32_t)kTopkList / 4) return drop * 2 <= kTopkFloorDrop ? drop * 2 : kTopkFloorDrop;
+    return drop;
+}
+
+// Larger K: the window would hold more keys than the list takes, so the prediction has to be two-sided: keys at
+// or above a band around the predicted threshold are kept at once, keys inside the band go to the list, which
+// settles them, and the chunk is read once.  How wide the band may be depends on how densely the keys lie around
+// the threshold, and error feedback piles them up there as the steps go on (measured on the benchmark's
+// gradients: from 330 to more than 700 keys per 4 % of the value, of a chunk of 32768 at k = 10 %), so every
+// (worker, chunk) learns its own band from its last step (topk_learn): the half-width that would have listed
+// about kTopkBandTarget keys, and which of three simple predictions (topk_predict) came closest (keys are close
+// to a logarithmic scale: a linear step in the key is a ratio in the value).  The
+// band is only used if that prediction would have hit a band 0.7 times as wide last step; otherwise, and when
+// the band misses after all (the K-th key outside it, or more keys inside than the list takes: the chunk is then
+// counted in a further pass), the two-pass route runs and learns again.  Exact on every route.
+constexpr uint32_t kTopkBandTarget = 1000;
+constexpr uint32_t kTopkBandMaxHalf = 3u << 18;      // one and a half bins of a sixteenth of an exponent step: -6 % .. +7 %
+constexpr uint32_t kTopkBandMinHalf = 1u << 12;
+constexpr int64_t kTopkBandMaxStep = 4 << 19;
+__device__ __forceinline__ int64_t topk_trend(uint32_t last_key, uint32_t prev_key)
+{
+    if (prev_key == 0) return 0;
+    const int64_t step = (int64_t)last_key - (int64_t)prev_key;
+    return step > kTopkBandMaxStep ? kTopkBandMaxStep : (step < -kTopkBandMaxStep ? -kTopkBandMaxStep : step);
+}
+// The candidates for this step's threshold key: 0 the last step's, 1 its extrapolation by the step before, 2 the
+// key of the step before (a threshold that alternates, as it does when the same few batches come round).
+__device__ __forceinline__ int64_t topk_predict(int which, uint32_t last_key, uint32_t prev_key)
+{
+    if (which == 1) return (int64_t)last_key + topk_trend(last_key, prev_key);
+    if (which == 2 && prev_key != 0) return (int64_t)prev_key;
+    return (int64_t)last_key;
+}
+// learned: the half-width (a multiple of 4) + the candidate to use; 0 = no band.
+__device__ __forceinline__ void topk_band(uint32_t last_key, uint32_t prev_key, uint32_t learned, uint32_t& lo, uint32_t& hi)
+{
+    lo = hi = 0;
+    const uint32_t half = learned & ~3u;
+    if (half == 0 || last_key == 0) return;
+    const int64_t pred = topk_predict((int)(learned & 3u), last_key, prev_key);
+    if (pred <= (int64_t)(1u << 23) || pred >= (int64_t)0x7f000000) return;
+    lo = (uint32_t)pred - half;
+    hi = (uint32_t)pred + half;
+}
+// After a step: `count` keys were seen in `width` key units around the new threshold tau (the band's list, or the
+// K-th key's bin of the two-pass route; width 0: nothing learned).  Returns what topk_band takes next step.
+__device__ __forceinline__ uint32_t topk_learn(uint32_t tau, uint32_t last_key, uint32_t prev_key, uint32_t count, uint32_t width)
+{
+    if (width == 0 || last_key == 0) return 0;
+    uint64_t half = count ? (uint64_t)width * (kTopkBandTarget / 2) / count : kTopkBandMaxHalf;
+    if (half > kTopkBandMaxHalf) half = kTopkBandMaxHalf;
+    if (half < kTopkBandMinHalf) return 0;
+    int best = 0;
+    int64_t err = llabs((int64_t)tau - topk_predict(0, last_key, prev_key));
+#pragma unroll
+    for (int which = 1; which < 3; ++which) {
+        const int64_t e = llabs((int64_t)tau - topk_predict(which, last_key, prev_key));
+        if (e < err) { err = e; best = which; }
+    }
+    if (err * 10 > (int64_t)half * 7) return 0;
+    return ((uint32_t)half & ~3u) | (uint32_t)best;
 }
 
 // The keys inside the window are appended, with their positions in the chunk (16 bits: the list is used
@@ -119,11 +200,6 @@ __device__ __forceinline__ uint32_t topk_floor(float last_threshold, uint32_t K)
 // on 16 workers, 335 M elements, the scattered form takes 2.7 / 3.7 / 5.9 / 12.4 ms at k = 0.1 / 1 / 3 / 10 %,
 // the register form 3.8 / 4.6 / 5.2 / 5.9 ms.
 constexpr double kTopkDenseSum = 0.02;
-// Resident CTAs per SM the top-k kernels are compiled for.  Their passes are latency-bound, so residency
-// matters more than registers, but at eight (32 registers) the spills cost more than the two CTAs give:
-// six measured fastest (worker 16.5 ms against 23.2 at eight and 17.9 at four, 16 workers, 335 M elements).
-constexpr int kTopkResident = 6;
-
 struct TopkList { uint32_t key[kTopkList]; uint16_t idx[kTopkList]; uint32_t count; };
 
 __device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_t idx)
@@ -138,30 +214,30 @@ __device__ __forceinline__ void topk_list_add(TopkList& l, uint32_t key, uint32_
 // to scan.  Returns false, with nothing decided, when the K-th key lies in the clipped bin (it is then
 // more than four times the floor).  Also returns how many keys equal tau in all (ties_total); ties <=
 // ties_total of them are to be kept.
-static_assert(kThreads == 256, "one histogram bin per thread");
+static_assert(kTopkThreads >= 256, "one histogram bin per thread");
 __device__ __forceinline__ bool topk_threshold_list(const TopkList& l, int n, uint32_t floor_key, uint32_t K,
                                                     uint32_t* hist /* 256 bins */, uint32_t* sh,
                                                     uint32_t& tau, uint32_t& ties, uint32_t& ties_total)
 {
-    hist[threadIdx.x] = 0;
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
     __syncthreads();
-    for (int p = threadIdx.x; p < n; p += kThreads) {
+    for (int p = threadIdx.x; p < n; p += kTopkThreads) {
         const uint32_t rel = l.key[p] - floor_key;
         atomicAdd(&hist[rel >> 16 < 255u ? rel >> 16 : 255u], 1u);
     }
     const uint32_t b0 = (uint32_t)topk_find_bin(hist, 256, K, sh);
     if (b0 == 255u) return false;                      // the same value in every thread
-    hist[threadIdx.x] = 0;
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
     __syncthreads();
-    for (int p = threadIdx.x; p < n; p += kThreads) {
+    for (int p = threadIdx.x; p < n; p += kTopkThreads) {
         const uint32_t rel = l.key[p] - floor_key;
         if (rel >> 16 == b0) atomicAdd(&hist[(rel >> 8) & 0xffu], 1u);
     }
     const uint32_t b1 = (uint32_t)topk_find_bin(hist, 256, K, sh);
-    hist[threadIdx.x] = 0;
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
     __syncthreads();
     const uint32_t top = (b0 << 8) | b1;
-    for (int p = threadIdx.x; p < n; p += kThreads) {
+    for (int p = threadIdx.x; p < n; p += kTopkThreads) {
         const uint32_t rel = l.key[p] - floor_key;
         if (rel >> 8 == top) atomicAdd(&hist[rel & 0xffu], 1u);
     }
@@ -208,9 +284,9 @@ __device__ __forceinline__ int topk_bin(uint32_t key, int shift, int base)
 // Top-level histogram over the whole chunk (general route).
 __device__ __forceinline__ void topk_full_hist(const float* zc, int L, uint32_t* hist)
 {
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    for (int b = threadIdx.x; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
-    for (int j = threadIdx.x; j < L; j += kThreads) atomicAdd(&hist[mag_key(zc[j]) >> 20], 1u);
+    for (int j = threadIdx.x; j < L; j += kTopkThreads) atomicAdd(&hist[mag_key(zc[j]) >> 20], 1u);
 }
 
 // One wave (1024 elements) of the ordered pass: the thread holds the keys of 4 consecutive elements
@@ -233,7 +309,7 @@ __device__ __forceinline__ uint32_t topk_select_wave(const uint32_t key[4], uint
     __syncthreads();
     uint32_t before = seen, total = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) { const uint32_t c = warp_ties[w]; if (w < warp) before += c; total += c; }
+    for (int w = 0; w < kTopkWarps; ++w) { const uint32_t c = warp_ties[w]; if (w < warp) before += c; total += c; }
     before += incl - cnt;
     seen += total;
     __syncthreads();                                   // warp_ties may be rewritten by the next wave
@@ -255,6 +331,9 @@ struct TopkWorkerArgs {
     const float* m32;                 // the momentum in binary32 (M32 form of the kernel) ...
     const float* zbar; const uint32_t* Bbar;   // ... or as the server left it: m = C[zbar] = mask ? zbar : 0
     float* thr; int64_t Cp;           // per (worker, chunk): the magnitude of the K-th element of the last step
+    float* hint; float* learned;      // ... of the step before, and what topk_learn made of it (same stride): only ever prediction aids
+    int* route;                       // 6 counters: chunks settled by the predicted list / by two passes / by the general route;
+                                      // predictions missed because the K-th key lay above / below the listed keys / the list overflowed
     int64_t d, chunk, C;
     int i0, ni;
     float beta1, omb1;
@@ -272,14 +351,17 @@ __device__ __forceinline__ uint32_t topk_count(double frac, int L)
 // M32: the momentum is read from the binary32 buffer (first step of the phase, after a state upload, or
 // when the server applies densely); otherwise it is taken from the server's compensated vector where the
 // server's mask has a bit, so that the server need not write a momentum vector at all.
-template <int GT, bool M32>
-__global__ void __launch_bounds__(kThreads, kTopkResident)
+// BAND: K is too large for the one-sided window (chosen by the host from the full chunk's K); the first pass
+// then uses the two-sided band where both earlier thresholds are known.
+template <int GT, bool M32, bool BAND>
+__global__ void __launch_bounds__(kTopkThreads, kTopkResident)
 k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
     __shared__ uint32_t bins8[256];
     __shared__ uint32_t sh[2];
-    __shared__ uint32_t warp_ties[kWarps];
+    __shared__ uint32_t above_total;
+    __shared__ uint32_t warp_ties[kTopkWarps];
     __shared__ TopkList list;
     const int ii = (int)(blockIdx.x % a.ni);
     const int64_t c = blockIdx.x / a.ni;
@@ -292,30 +374,50 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     const float* __restrict__ m = (M32 ? a.m32 : a.zbar) + base;
     const uint32_t* __restrict__ mbar = a.Bbar + base / 32;
     float* thr = a.thr + (int64_t)i * a.Cp + c;
+    float* hint = a.hint + (int64_t)i * a.Cp + c;
+    const float last_thr = *thr;
     const uint32_t K = topk_count(a.frac, L);
     const int nwords = (L + 31) / 32;
     const bool small = nwords <= kTopkBins;            // the mask fits the shared-memory words: list routes possible
-    const uint32_t floor_key = small ? topk_floor(*thr, K) : 0u;
-    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(*thr) : 0;
+    float* learned = a.learned + (int64_t)i * a.Cp + c;
+    const uint32_t drop = topk_window_drop(*learned);
+    const uint32_t floor_key = (small && !BAND) ? topk_floor(last_thr, K, drop) : 0u;
+    const uint32_t last_key = mag_key(last_thr), prev_key = mag_key(*hint);
+    uint32_t band_lo = 0, band_hi = 0;
+    if (BAND && small) topk_band(last_key, prev_key, __float_as_uint(*learned), band_lo, band_hi);
+    const bool band = BAND && band_lo != 0;
+    uint32_t learn_count = 0, learn_width = 0;
+    const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(last_thr) : 0;
+    const int lane = threadIdx.x & 31;
+    uint32_t above = 0;                                // band: this thread's keys at or above it
 
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
-    if (threadIdx.x == 0) list.count = 0;
+    for (int b = threadIdx.x; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
+    if (threadIdx.x == 0) { list.count = 0; above_total = 0; }
     __syncthreads();
     // pass A: z = (b1 m + (1-b1) g) + delta_old, with delta_old from the stored z and last step's mask;
     // whole 1024-element sweeps without bounds checks, two sweeps' loads in flight, then the ragged rest
-    const int Lfull = L & ~(kThreads * 4 - 1);
+    const int Lfull = L & ~(kTopkThreads * 4 - 1);
     auto sweep = [&](int k, float4 gv, float4 zv, float4 mv, uint32_t nib, bool checked) {
         const float gg[4] = {gv.x, gv.y, gv.z, gv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w}, mm[4] = {mv.x, mv.y, mv.z, mv.w};
         float zn[4];
+        uint32_t kept = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float mi = __fmaf_rn(a.beta1, mm[e], __fmul_rn(a.omb1, gg[e]));
             zn[e] = __fadd_rn(mi, topk_error(zo[e], (nib >> e) & 1u));
             if (!checked || k + e < L) {
                 const uint32_t key = mag_key(zn[e]);
-                if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);     // no window: every key counts
+                if (BAND && band) {
+                    if (key >= band_hi) kept |= 1u << e;
+                    else if (key >= band_lo) topk_list_add(list, key, (uint32_t)(k + e));
+                } else if (floor_key == 0) atomicAdd(&hist[topk_bin(key, shift, bin0)], 1u);     // no prediction: every key counts
                 else if (key >= floor_key) topk_list_add(list, key, (uint32_t)(k + e));
             }
+        }
+        if (BAND && band) {                            // every sweep is taken by whole warps
+            above += __popc(kept);
+            const uint32_t word = pack_group_words(kept, lane);     // valid in lanes 0, 8, 16, 24
+            if ((lane & 7) == 0 && (!checked || k < L)) hist[k >> 5] = word;
         }
         if (!checked || k + 3 < L) *reinterpret_cast<float4*>(zc + k) = make_float4(zn[0], zn[1], zn[2], zn[3]);
         else for (int e = 0; e < 4 && k + e < L; ++e) zc[k + e] = zn[e];
@@ -323,14 +425,14 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
     // the momentum of elements k..k+3
     auto momentum = [&](int k, bool checked) -> float4 {
         if (M32) return checked ? ld4_checked(m, k, L, false) : *reinterpret_cast<const float4*>(m + k);
-        const uint32_t nb = (mbar[k >> 5] >> (k & 31)) & 0xfu;
+        const uint32_t nb = (!checked || k < L) ? (mbar[k >> 5] >> (k & 31)) & 0xfu : 0u;
         // loaded whether or not a bit is set: a load that waits for the mask word costs more than it saves
         const float4 zb = checked ? ld4_checked(m, k, L, false) : *reinterpret_cast<const float4*>(m + k);
         return make_float4((nb & 1u) ? zb.x : 0.0f, (nb & 2u) ? zb.y : 0.0f, (nb & 4u) ? zb.z : 0.0f, (nb & 8u) ? zb.w : 0.0f);
     };
     int k = threadIdx.x * 4;
-    for (; k + kThreads * 4 < Lfull; k += 2 * kThreads * 4) {
-        const int k2 = k + kThreads * 4;
+    for (; k + kTopkThreads * 4 < Lfull; k += 2 * kTopkThreads * 4) {
+        const int k2 = k + kTopkThreads * 4;
         const float4 g0 = Grad<GT>::ld4(g, k), g1 = Grad<GT>::ld4(g, k2);
         const float4 z0 = *reinterpret_cast<const float4*>(zc + k), z1 = *reinterpret_cast<const float4*>(zc + k2);
         const float4 m0 = momentum(k, false), m1 = momentum(k2, false);
@@ -338,25 +440,67 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
         sweep(k, g0, z0, m0, n0, false);
         sweep(k2, g1, z1, m1, n1, false);
     }
-    for (; k < Lfull; k += kThreads * 4)
+    for (; k < Lfull; k += kTopkThreads * 4)
         sweep(k, Grad<GT>::ld4(g, k), *reinterpret_cast<const float4*>(zc + k), momentum(k, false),
               maskw[k >> 5] >> (k & 31), false);
-    for (; k < L; k += kThreads * 4)
+    for (int w0 = k - threadIdx.x * 4; w0 < L; w0 += kTopkThreads * 4) {          // the ragged rest, by whole warps
+        k = w0 + threadIdx.x * 4;
         sweep(k, ld_grad4_checked<GT>(g, k, L), ld4_checked(zc, k, L, false), momentum(k, true),
-              maskw[k >> 5] >> (k & 31), true);
-    __syncthreads();                                   // z stores, histogram and list are complete
-    const int lane = threadIdx.x & 31;
+              k < L ? maskw[k >> 5] >> (k & 31) : 0u, true);
+    }
+    if (BAND && band) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
+        if (lane == 0) atomicAdd(&above_total, above);
+    }
+    __syncthreads();                                   // z stores, histogram (or mask so far) and list are complete
     int n_list = 0;                                    // > 0: the list decides, hist[0..nwords) holds the mask so far
     uint32_t K_list = K, floor_list = floor_key;
-    if (floor_key != 0) {                              // window route: the mask words are still all zero
+    bool counted = !band && floor_key == 0;            // hist holds the fine counts of all keys
+    bool two_pass = false, missed = false;
+    uint32_t learned_next = BAND ? 0u : drop;
+    if (BAND && band) {
+        const uint32_t listed = list.count, over = above_total;
+        if (over < K && K <= over + listed && listed <= (uint32_t)kTopkList) {
+            n_list = (int)listed; K_list = K - over; floor_list = band_lo;
+            learn_count = listed; learn_width = band_hi - band_lo;
+        } else {
+            missed = true;
+            if (threadIdx.x == 0) atomicAdd(a.route + (listed > (uint32_t)kTopkList ? 5 : (over >= K ? 3 : 4)), 1);
+        }
+    } else if (floor_key != 0) {                       // window route: the mask words are still all zero
         const uint32_t listed = list.count;
+        learned_next = topk_window_learn(drop, listed, K);
         if (listed >= K && listed <= (uint32_t)kTopkList) n_list = (int)listed;
-    } else if (small) {                                // two-pass route
+        else {
+            missed = true;
+            if (threadIdx.x == 0) atomicAdd(a.route + (listed < K ? 4 : 5), 1);
+        }
+    }
+    if (missed) {                                      // the prediction missed: count every key after all
+        __syncthreads();
+        for (int b = threadIdx.x; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
+        if (threadIdx.x == 0) list.count = 0;
+        __syncthreads();
+        for (int kk = threadIdx.x * 4; kk < L; kk += kTopkThreads * 4) {
+            const float4 zv = ld4_checked(zc, kk, L, false);
+            const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (kk + e < L) atomicAdd(&hist[topk_bin(key[e], shift, bin0)], 1u);
+        }
+        counted = true;
+    }
+    if (n_list > 0) {
+        // settled by the list below
+    } else if (small && counted) {                     // two-pass route
         uint32_t Kb = K;
         const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
         const uint32_t inbin = hist[b0];
         __syncthreads();                               // everybody has read the histogram: its words become the mask
         if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            two_pass = true;
+            learn_count = inbin; learn_width = 1u << 19;
             auto settle = [&](int k, float4 zv, bool checked) {
                 const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
                 uint32_t nibble = 0;
@@ -372,15 +516,15 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
                 if ((lane & 7) == 0 && (!checked || k < L)) hist[k >> 5] = word;
             };
             int w0 = 0;
-            for (; w0 + 4 * kThreads * 4 <= L; w0 += 4 * kThreads * 4) {      // four sweeps' loads in flight
+            for (; w0 + 4 * kTopkThreads * 4 <= L; w0 += 4 * kTopkThreads * 4) {      // four sweeps' loads in flight
                 const int k = w0 + threadIdx.x * 4;
                 float4 zv[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zc + k + u * kThreads * 4);
+                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zc + k + u * kTopkThreads * 4);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) settle(k + u * kThreads * 4, zv[u], false);
+                for (int u = 0; u < 4; ++u) settle(k + u * kTopkThreads * 4, zv[u], false);
             }
-            for (; w0 < L; w0 += kThreads * 4) {
+            for (; w0 < L; w0 += kTopkThreads * 4) {
                 const int k = w0 + threadIdx.x * 4;
                 settle(k, ld4_checked(zc, k, L, false), true);
             }
@@ -394,22 +538,26 @@ k_topk_worker(const __grid_constant__ GradPtrs G, const TopkWorkerArgs a)
         uint32_t ties_total;
         have_tau = topk_threshold_list(list, n_list, floor_list, K_list, bins8, sh, tau, ties, ties_total);
         if (have_tau) {
-            for (int p = threadIdx.x; p < n_list; p += kThreads)
+            for (int p = threadIdx.x; p < n_list; p += kTopkThreads)
                 if (topk_list_selected(list, n_list, p, tau, ties, ties_total))
                     atomicOr(&hist[list.idx[p] >> 5], 1u << (list.idx[p] & 31u));
             __syncthreads();
-            for (int w = threadIdx.x; w < nwords; w += kThreads) maskw[w] = hist[w];
-            if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+            for (int w = threadIdx.x; w < nwords; w += kTopkThreads) maskw[w] = hist[w];
+            if (threadIdx.x == 0) {
+                *thr = __uint_as_float(tau); *hint = last_thr;
+                *learned = __uint_as_float(BAND ? topk_learn(tau, last_key, prev_key, learn_count, learn_width) : learned_next);
+                atomicAdd(a.route + (two_pass ? 1 : 0), 1);
+            }
             return;
         }
     }
     // general route: histograms over the whole chunk
     if (small) topk_full_hist(zc, L, hist);
     topk_threshold(zc, L, K, hist, sh, tau, ties);
-    if (threadIdx.x == 0) *thr = __uint_as_float(tau);
+    if (threadIdx.x == 0) { *thr = __uint_as_float(tau); *hint = last_thr; *learned = __uint_as_float(learned_next); atomicAdd(a.route + 2, 1); }
     // ordered pass over the chunk: the selection mask with the tie rule
     uint32_t seen = 0;
-    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+    for (int w0 = 0; w0 < L; w0 += kTopkThreads * 4) {
         const int k = w0 + threadIdx.x * 4;
         const float4 zv = ld4_checked(zc, k, L, false);
         const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
@@ -426,6 +574,8 @@ struct TopkServerArgs {
     float* zbar; uint32_t* Bbar;      // the server's compensated vector and mask
     float* m32;                       // accumulator during the step; the new momentum after it where the chunk was applied densely
     float* thr;                       // per chunk: the magnitude of the K-th element of the last step
+    float* hint; float* learned;      // ... of the step before, and what topk_learn made of it
+    int* route;                       // as in TopkWorkerArgs
     const float* v; float* x;
     int64_t d, chunk;
     int n; float nf, lr, eps;
@@ -439,13 +589,13 @@ struct TopkServerArgs {
     int sparse;
 };
 
-__global__ void __launch_bounds__(kThreads, kTopkResident)
+__global__ void __launch_bounds__(kTopkThreads, kTopkResident)
 k_topk_server(const TopkServerArgs a)
 {
     __shared__ uint32_t hist[kTopkBins];
     __shared__ uint32_t bins8[256];
     __shared__ uint32_t sh[2];
-    __shared__ uint32_t warp_ties[kWarps];
+    __shared__ uint32_t warp_ties[kTopkWarps];
     __shared__ TopkList list;
     const int64_t c = a.c0 + blockIdx.x;
     const int64_t base = c * a.chunk;
@@ -455,7 +605,7 @@ k_topk_server(const TopkServerArgs a)
     float* zb = a.zbar + base;
     uint32_t* maskbar = a.Bbar + base / 32;
 
-    for (int b = threadIdx.x; b < kTopkBins; b += kThreads) hist[b] = 0;
+    for (int b = threadIdx.x; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
     if (threadIdx.x == 0) list.count = 0;
     // The sum of the n sparse messages, in worker order, has two forms.  Few kept elements (k below
     // kTopkDenseSum): scattered, through the momentum buffer - a thread owns the same mask words for every
@@ -463,12 +613,12 @@ k_topk_server(const TopkServerArgs a)
     // the mask words of eight workers are fetched together.  Many: in registers inside pass A (below).
     const bool dense = a.frac >= kTopkDenseSum;
     if (!dense) {
-        for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+        for (int k = threadIdx.x * 4; k < L; k += kTopkThreads * 4) {
             if (k + 3 < L) *reinterpret_cast<float4*>(acc + k) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             else for (int e = 0; k + e < L; ++e) acc[k + e] = 0.0f;
         }
         __syncthreads();
-        for (int w = threadIdx.x; w < nwords; w += kThreads) {
+        for (int w = threadIdx.x; w < nwords; w += kTopkThreads) {
             for (int i0 = 0; i0 < a.n; i0 += 8) {
                 uint32_t mw[8];
 #pragma unroll
@@ -492,12 +642,23 @@ k_topk_server(const TopkServerArgs a)
     // of them is set.
     const uint32_t K = topk_count(a.frac, L);
     const bool small = nwords <= kTopkBins && a.sparse != 0;      // list routes: the mask fits the shared-memory words, sparse update allowed
-    const uint32_t floor_key = small ? topk_floor(a.thr[c], K) : 0u;
+    const uint32_t drop = topk_window_drop(a.learned[c]);
+    const uint32_t floor_key = small ? topk_floor(a.thr[c], K, drop) : 0u;
     const int shift = small ? 19 : 20, bin0 = small ? topk_fine_base(a.thr[c]) : 0;
-    for (int k = threadIdx.x * 4; k < L; k += kThreads * 4) {
+    // The dense form waits on memory twice per four workers (mask words, then the values under them), so it asks
+    // for the mask lines of the sweep after next ahead of time.
+    auto ask_masks = [&](int k0) {                     // k0: first element of a sweep (64 mask words a worker: two lines, three when not aligned)
+        if (dense && (int)threadIdx.x < 4 * a.n && (threadIdx.x & 3) != 3 && k0 < L) {
+            const int w = (k0 >> 5) + ((threadIdx.x & 3) == 2 ? 63 : 32 * (int)(threadIdx.x & 3));
+            if (w < nwords) prefetch_l1(a.B + (int64_t)(threadIdx.x >> 2) * a.Wp + base / 32 + w);
+        }
+    };
+    ask_masks(0); ask_masks(kTopkThreads * 4);
+    for (int k = threadIdx.x * 4; k < L; k += kTopkThreads * 4) {
         float aa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         const uint32_t* mrow = a.B + base / 32 + (k >> 5);
         const float* zrow = a.z + base;
+        ask_masks(k - (int)threadIdx.x * 4 + 2 * kTopkThreads * 4);
         if (!dense) {
             const float4 av = ld4_checked(acc, k, L, false);
             aa[0] = av.x; aa[1] = av.y; aa[2] = av.z; aa[3] = av.w;
@@ -541,15 +702,35 @@ k_topk_server(const TopkServerArgs a)
     uint32_t tau, ties;
     int n_list = 0;                                    // > 0: the list decides, hist[0..nwords) holds the mask so far
     uint32_t K_list = K, floor_list = floor_key;
+    bool two_pass = false, counted = small && floor_key == 0;
+    uint32_t learned_next = drop;
     if (floor_key != 0) {                              // window route: the mask words are still all zero
         const uint32_t listed = list.count;
+        learned_next = topk_window_learn(drop, listed, K);
         if (listed >= K && listed <= (uint32_t)kTopkList) n_list = (int)listed;
-    } else if (small) {                                // two-pass route
+        else {                                         // the window missed: count every key after all
+            if (threadIdx.x == 0) atomicAdd(a.route + (listed < K ? 4 : 5), 1);
+            __syncthreads();
+            if (threadIdx.x == 0) list.count = 0;
+            for (int kk = threadIdx.x * 4; kk < L; kk += kTopkThreads * 4) {       // (the bins are still all zero)
+                const float4 zv = ld4_checked(zb, kk, L, false);
+                const uint32_t key[4] = {mag_key(zv.x), mag_key(zv.y), mag_key(zv.z), mag_key(zv.w)};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (kk + e < L) atomicAdd(&hist[topk_bin(key[e], shift, bin0)], 1u);
+            }
+            counted = true;
+        }
+    }
+    if (n_list > 0) {
+        // settled by the list below
+    } else if (counted) {                              // two-pass route
         uint32_t Kb = K;
         const int b0 = topk_find_bin(hist, kTopkBins, Kb, sh);
         const uint32_t inbin = hist[b0];
         __syncthreads();                               // everybody has read the histogram: its words become the mask
         if (b0 > 0 && b0 < kTopkBins - 1 && inbin <= (uint32_t)kTopkList) {
+            two_pass = true;
             // second pass: the elements above the bin of the K-th key are kept - mask bit, model update
             // (Section 3.3 steps 5-6) - and those of that bin go to the list
             auto settle = [&](int k, float4 zv, bool checked) {
@@ -572,15 +753,15 @@ k_topk_server(const TopkServerArgs a)
                 if ((lane & 7) == 0 && (!checked || k < L)) hist[k >> 5] = word;
             };
             int w0 = 0;
-            for (; w0 + 4 * kThreads * 4 <= L; w0 += 4 * kThreads * 4) {      // four sweeps' loads in flight
+            for (; w0 + 4 * kTopkThreads * 4 <= L; w0 += 4 * kTopkThreads * 4) {      // four sweeps' loads in flight
                 const int k = w0 + threadIdx.x * 4;
                 float4 zv[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zb + k + u * kThreads * 4);
+                for (int u = 0; u < 4; ++u) zv[u] = *reinterpret_cast<const float4*>(zb + k + u * kTopkThreads * 4);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) settle(k + u * kThreads * 4, zv[u], false);
+                for (int u = 0; u < 4; ++u) settle(k + u * kTopkThreads * 4, zv[u], false);
             }
-            for (; w0 < L; w0 += kThreads * 4) {
+            for (; w0 < L; w0 += kTopkThreads * 4) {
                 const int k = w0 + threadIdx.x * 4;
                 settle(k, ld4_checked(zb, k, L, false), true);
             }
@@ -593,25 +774,28 @@ k_topk_server(const TopkServerArgs a)
         uint32_t ties_total;
         have_tau = topk_threshold_list(list, n_list, floor_list, K_list, bins8, sh, tau, ties, ties_total);
         if (have_tau) {
-            for (int p = threadIdx.x; p < n_list; p += kThreads) {              // the listed elements, one by one
+            for (int p = threadIdx.x; p < n_list; p += kTopkThreads) {              // the listed elements, one by one
                 if (!topk_list_selected(list, n_list, p, tau, ties, ties_total)) continue;
                 const int j = (int)list.idx[p];
                 x[j] = apply_elem(x[j], v[j], zb[j], a.lr, a.eps);
                 atomicOr(&hist[j >> 5], 1u << (j & 31));
             }
             __syncthreads();
-            for (int w = threadIdx.x; w < nwords; w += kThreads) maskbar[w] = hist[w];
-            if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
+            for (int w = threadIdx.x; w < nwords; w += kTopkThreads) maskbar[w] = hist[w];
+            if (threadIdx.x == 0) {
+                a.thr[c] = __uint_as_float(tau); a.learned[c] = __uint_as_float(learned_next);
+                atomicAdd(a.route + (two_pass ? 1 : 0), 1);
+            }
             return;
         }
     }
     // general route: histograms over the whole chunk
     if (small) topk_full_hist(zb, L, hist);
     topk_threshold(zb, L, K, hist, sh, tau, ties);
-    if (threadIdx.x == 0) a.thr[c] = __uint_as_float(tau);
+    if (threadIdx.x == 0) { a.thr[c] = __uint_as_float(tau); a.learned[c] = __uint_as_float(learned_next); atomicAdd(a.route + 2, 1); }
     // ordered pass: mask, momentum m = C[zbar] written out, model update (Section 3.3 steps 5-6) of every element
     uint32_t seen = 0;
-    for (int w0 = 0; w0 < L; w0 += kThreads * 4) {
+    for (int w0 = 0; w0 < L; w0 += kTopkThreads * 4) {
         const int k = w0 + threadIdx.x * 4;
         const float4 zv = ld4_checked(zb, k, L, false);
         const float4 vv = ld4_checked(v, k, L, true);

@@ -15,7 +15,7 @@ import json
 import sys
 
 
-def _setup(d, n, chunk, compressor=None, variant=None, team=None, first_step=False, grad_dtype="float32"):
+def _setup(d, n, chunk, compressor=None, variant=None, team=None, first_step=False, grad_dtype="float32", steps=1):
     import torch
 
     from . import binding as B
@@ -41,7 +41,8 @@ def _setup(d, n, chunk, compressor=None, variant=None, team=None, first_step=Fal
     ctx.warmup_step(grads)
     ctx.freeze_v()
     if not first_step:
-        ctx.compressed_step(grads)          # the first step of the phase reads the binary32 momentum: not the steady state
+        for _ in range(steps):              # the first step of the phase reads the binary32 momentum: not the steady state
+            ctx.compressed_step(grads)      # (top-k: the predicted-threshold routes need a few steps of history)
     torch.cuda.synchronize()
     return ctx, w, grads
 
@@ -60,7 +61,11 @@ def _cases(args):
                                     bytes=lambda w: w.n * (12 * w.d + w.d // 8) + w.d // 8),
         "k_worker_fine_bf16": dict(setup=dict(chunk=32768, grad_dtype="bfloat16"), call="worker_phase", timer=B.KERNEL_WORKER,
                                    bytes=lambda w: w.n * (10 * w.d + w.d // 8) + w.d // 8),
-        "k_worker": dict(setup=dict(chunk=160), call="worker_phase", timer=B.KERNEL_WORKER,
+        "k_worker_fine_words": dict(setup=dict(chunk=128), call="worker_phase", timer=B.KERNEL_WORKER,
+                                    bytes=lambda w: w.n * (12 * w.d + w.d // 8) + w.d // 8),
+        "k_finalize_words": dict(setup=dict(chunk=128), call="worker_phase", timer=B.KERNEL_WORKER,
+                                 bytes=lambda w: w.n * (8 * (w.d // 32) + 4 * w.n_chunks)),
+        "k_worker": dict(setup=dict(chunk=160, team=B.TEAM_WARP), call="worker_phase", timer=B.KERNEL_WORKER,
                          bytes=lambda w: w.n * (12 * w.d + w.d // 8) + w.d // 8),
         "k_worker_m32": dict(setup=dict(chunk=32768, first_step=True), call="first_worker_phase", timer=B.KERNEL_WORKER,
                              bytes=lambda w: w.n * (12 * w.d + w.d // 8) + 4 * w.d),
@@ -87,6 +92,12 @@ def _cases(args):
                               bytes=lambda w: w.n * (12 * w.d + w.d // 4) + 4 * w.d),
         "k_topk_server": dict(setup=dict(chunk=32768, compressor=0.01), call="step", timer=B.KERNEL_SERVER,
                               bytes=lambda w: w.n * (w.d // 8 + int(0.04 * w.d)) + 24 * w.d + w.d // 8),
+        "k_topk_worker_band": dict(setup=dict(chunk=32768, compressor=0.03, steps=8), call="step", timer=B.KERNEL_WORKER,
+                                   bytes=lambda w: w.n * (12 * w.d + w.d // 4) + 4 * w.d),
+        "k_topk_worker_two_pass": dict(setup=dict(chunk=32768, compressor=0.1, steps=1), call="step", timer=B.KERNEL_WORKER,
+                                       bytes=lambda w: w.n * (12 * w.d + w.d // 4) + 4 * w.d),
+        "k_topk_server_dense": dict(setup=dict(chunk=32768, compressor=0.03, steps=8), call="step", timer=B.KERNEL_SERVER,
+                                    bytes=lambda w: w.n * (w.d // 8 + int(0.12 * w.d)) + 24 * w.d + w.d // 8),
         "k_error_norm_tiles": dict(setup=dict(chunk=32768), call="error_norms", timer=None,
                                    bytes=lambda w: 4 * (w.n + 1) * w.d),
     }

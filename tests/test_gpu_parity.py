@@ -326,11 +326,11 @@ def test_topk_updates_every_element_when_skipping_is_not_exact(lr, eps):
         _topk_compare(ctx, orc, w, step)
 
 
-@pytest.mark.parametrize("frac", [0.01, 0.1])
-def test_topk_long_free_run(frac):
-    """60 free-running top-k steps: the predicted-threshold routes run on thresholds that drift as the errors
-    build up; masks, errors, momentum and model stay bit-identical."""
-    w = tiny(6 * 8192 + 500, 3, 8192, cfg_id=183)
+@pytest.mark.parametrize("frac,chunk", [(0.01, 8192), (0.1, 8192), (0.03, 32768), (0.1, 32768), (0.25, 4096)])
+def test_topk_long_free_run(frac, chunk):
+    """60 free-running top-k steps: the predicted-threshold routes (one-sided window, two-sided band) run on
+    thresholds that drift as the errors build up; masks, errors, momentum and model stay bit-identical."""
+    w = tiny((6 if chunk < 32768 else 2) * chunk + 500, 3, chunk, cfg_id=183)
     ctx, orc = H.make_pair(w)
     ctx.set_compressor(B.COMPRESSOR_TOPK, frac)
     orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
@@ -342,6 +342,30 @@ def test_topk_long_free_run(frac):
         ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
         if step % 10 == 0:
             _topk_compare(ctx, orc, w, step)
+
+
+def test_topk_route_counts_add_up():
+    """Every (worker, chunk) and every server chunk is settled on exactly one of the three routes each step, and
+    with enough history the predicted list settles some of them (K = 984 of 32768: the two-sided band)."""
+    w = tiny(4 * 32768 + 999, 3, 32768, cfg_id=189)
+    ctx, orc = H.make_pair(w)
+    ctx.set_compressor(B.COMPRESSOR_TOPK, 0.03)
+    orc.set_compressor(ao.TOPK); orc.set_topk_fraction(0.03)
+    gs = wl.host_gradients(w, 0)
+    ctx.warmup_step(H.upload(gs)); orc.warmup_step(gs)
+    ctx.freeze_v(); orc.freeze_v()
+    ctx.topk_route_counts()
+    predicted = 0
+    for step in range(1, 25):
+        gs = wl.host_gradients(w, step)
+        ctx.compressed_step(H.upload(gs)); orc.compressed_step(gs)
+        wr, sr = ctx.topk_route_counts()
+        assert sum(wr[:3]) == w.n * w.n_chunks and sum(sr[:3]) == w.n_chunks, (step, wr, sr)
+        assert sum(wr[3:]) <= w.n * w.n_chunks and min(wr) >= 0 and min(sr) >= 0
+        predicted += wr[0]
+    assert ctx.topk_route_counts() == ([0] * 6, [0] * 6)            # reset by the call
+    assert predicted > 0
+    _topk_compare(ctx, orc, w, 24)
 
 
 def _topk_rows(ctxs, cb, ce):

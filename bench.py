@@ -228,7 +228,7 @@ def measure(w, args, rank, world, local_rank, dist, want_adam=False, want_e2e=Tr
         assert n_total % world == 0, "the worker count must be a multiple of the number of processes"
         w = w.with_(n=n_total // world)
     ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk, device=f"cuda:{local_rank}",
-                    library_workspace=(args.path == "peer"))
+                    library_workspace=(args.path == "peer" and args.compressor == "onebit"))   # top-k: the peers share receive rows, not workspaces
     if args.compressor == "topk":
         ctx.set_compressor(B.COMPRESSOR_TOPK, args.topk_fraction)
     x0 = torch.empty(w.d, dtype=torch.float32, device=dev).normal_(0.0, w.x0_std)

@@ -251,9 +251,12 @@ class PeerShardedStep:
     their messages is complete.  The worker phase runs range by range, every process starting with the range
     after its own, so the range a process serves is finished everywhere one range before the end of the
     worker phase: its server phase does not wait for the slowest process's last kernel.
+
+    With the top-k compressor (a backend with a torch workspace and set_compressor(TOPK) done) the messages are
+    stored, not loaded: see _init_topk.
     """
 
-    def __init__(self, backend, group=None, peers=None, timeout_s: float = 120.0):
+    def __init__(self, backend, group=None, peers=None, timeout_s: float = 120.0, share=None):
         import torch.distributed as dist
 
         self.b, self.dist, self.group = backend, dist, group
@@ -264,6 +267,12 @@ class PeerShardedStep:
             from . import binding as peers
         self._peers = peers
         self.ranges = chunk_ranges(backend.C, self.world)
+        self.steps = 0
+        self.base = []
+        self.topk = bool(getattr(backend, "topk", False))
+        if self.topk:
+            self._init_topk(share, timeout_s)
+            return
         n = backend.n
         self.off = {i: backend.message_offsets(i) for i in range(-1, n)}
         mine = (backend.ipc_export(), (backend.d, n, backend.chunk), tuple(sorted(self.off.items())))
@@ -276,9 +285,77 @@ class PeerShardedStep:
         self.base = [own_base if r == self.rank else peers.apms_ipc_open(h) for r, (h, _, _) in enumerate(everyone)]
         # stages 0 .. world-1: "my workers' messages for range k are complete"; stage world: "my server range is stored everywhere"
         self.flags = HostFlags(dist, group, self.world, self.world + 1, timeout_s)
-        self.steps = 0
         self.order = [(self.rank + 1 + j) % self.world for j in range(self.world)]      # own range last
         dist.barrier(group=group)
+
+    # ------------------------------------------------------------------ the top-k compressor
+    def _init_topk(self, share, timeout_s):
+        """With the top-k compressor a message is a selection mask plus the kept values, packed (Section 5.1);
+        packing is a kernel of its own, so it writes straight into the serving process's receive rows: device
+        buffers that every process makes for its own range and shares with its peers (`share`: a pair of
+        functions (export(tensor) -> picklable, open(picklable) -> tensor); by default torch's CUDA IPC
+        reductions).  The backend needs a torch workspace here (the masks are read through its message views)."""
+        import torch
+
+        b, dist, n, me = self.b, self.dist, self.b.n, self.rank
+        if share is None:
+            from torch.multiprocessing.reductions import reduce_tensor
+
+            share = (reduce_tensor, lambda handle: handle[0](*handle[1]))
+        export, open_ = share
+        self.per = b.topk_values_per_chunk()
+        self.words = [word_range(cb, ce, b.chunk, b.d) for cb, ce in self.ranges]
+        self.row_words = [_round4(w1 - w0) for w0, w1 in self.words]
+        self.row_vals = [(ce - cb) * self.per for cb, ce in self.ranges]
+        bits0 = b.message(0)[0]
+        mk = lambda shape, dt: torch.zeros(shape, dtype=dt, device=bits0.device)
+        self.own = {"recv_bits": mk((self.world * n, self.row_words[me]), bits0.dtype),
+                    "recv_vals": mk((self.world * n, self.row_vals[me]), torch.float32),
+                    "gather_bits": mk((self.world, max(self.row_words)), bits0.dtype),
+                    "gather_vals": mk((self.world, max(self.row_vals)), torch.float32)}
+        mine = ({k: export(t) for k, t in self.own.items()}, (b.d, n, b.chunk, self.per))
+        everyone = [None] * self.world
+        dist.all_gather_object(everyone, mine, group=self.group)
+        for r, (_, shape) in enumerate(everyone):
+            if shape != mine[1]:
+                raise ValueError(f"process {r} holds a context of another shape: {shape} against {mine[1]}")
+        self.bufs = [self.own if r == me else {k: open_(h) for k, h in handles.items()} for r, (handles, _) in enumerate(everyone)]
+        # stage 0: "my workers' rows are stored in every serving process"; stage 1: "my server range is stored everywhere"
+        self.flags = HostFlags(dist, self.group, self.world, 2, timeout_s)
+        dist.barrier(group=self.group)
+
+    def _step_topk(self, grads: Sequence) -> None:
+        b, n, me, flags, per = self.b, self.b.n, self.rank, self.flags, self.per
+        self.steps += 1
+        b.worker_phase(grads)                                                   # steps 1-2 (top-k: the whole vector)
+        for k in range(self.world):                                             # step 3: masks and packed values into process k's rows
+            (w0, w1), (cb, ce) = self.words[k], self.ranges[k]
+            dst = self.bufs[k]
+            for i in range(n):
+                row = me * n + i
+                dst["recv_bits"][row, :w1 - w0].copy_(b.message(i)[0][w0:w1])
+                b.topk_pack_values(i, cb, ce, dst["recv_vals"][row, :(ce - cb) * per])
+        b.synchronize()
+        flags.post(0, self.steps)
+        flags.wait_all(0, self.steps)                                           # every process's rows of my range have arrived
+        cb, ce = self.ranges[me]
+        w0, w1 = self.words[me]
+        b.topk_server_phase(self.own["recv_bits"], self.own["recv_vals"], cb, ce)   # step 4, and steps 5-6 for the elements it keeps
+        mine_vals = self.own["gather_vals"][me, :(ce - cb) * per]
+        b.topk_pack_values(-1, cb, ce, mine_vals)
+        sbits = b.message(-1)[0]
+        for r in range(self.world):                                             # step 5: my range of the server's message to every peer
+            if r != me:
+                self.bufs[r]["gather_bits"][me, :w1 - w0].copy_(sbits[w0:w1])
+                self.bufs[r]["gather_vals"][me, :(ce - cb) * per].copy_(mine_vals)
+        b.synchronize()
+        flags.post(1, self.steps)
+        flags.wait_all(1, self.steps)                                           # every range is stored everywhere
+        for k in range(self.world):
+            if k != me:
+                kb, ke = self.ranges[k]
+                b.topk_put_server_range(self.own["gather_bits"][k], self.own["gather_vals"][k], kb, ke)
+        b.apply_phase()
 
     def row_pointers(self):
         """(sign-word addresses, scale addresses) of all world * n senders' rows for this process's chunk range,
@@ -290,6 +367,8 @@ class PeerShardedStep:
         return bits, scales
 
     def step(self, grads: Sequence) -> None:
+        if self.topk:
+            return self._step_topk(grads)
         b, me, flags = self.b, self.rank, self.flags
         self.steps += 1
         events = []
@@ -315,6 +394,9 @@ class PeerShardedStep:
         """Unmaps the peers' workspaces.  Collective: returns when every process has unmapped, so that each may
         then free its own workspace."""
         self.dist.barrier(group=self.group)                                     # nobody reads a mapping that goes away
+        if self.topk:
+            self.b.synchronize()
+            self.bufs = []                                                      # the peers' buffers are unmapped with their last reference
         for r, base in enumerate(self.base):
             if r != self.rank and base is not None:
                 self._peers.apms_ipc_close(base)
@@ -327,5 +409,8 @@ class PeerShardedStep:
         range it stores to them."""
         cb, ce = self.ranges[self.rank]
         w0, w1 = word_range(cb, ce, self.b.chunk, self.b.d)
+        if self.topk:                                                           # what it stores into peers: its workers' rows, its server range
+            ex1 = sum(4 * self.b.n * ((self.words[k][1] - self.words[k][0]) + self.row_vals[k]) for k in range(self.world) if k != self.rank)
+            return ex1 + (self.world - 1) * 4 * ((w1 - w0) + self.row_vals[self.rank])
         per_row = 4 * (w1 - w0) + 4 * (ce - cb)
         return (self.world - 1) * self.b.n * per_row + (self.world - 1) * per_row

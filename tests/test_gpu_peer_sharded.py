@@ -154,8 +154,75 @@ def test_two_processes_on_one_gpu_exchange_through_mapped_workspaces(tmp_path):
     assert max(res[0][1], res[1][1]) < 0.1 * 4 * d * n_local
 
 
-@pytest.mark.parametrize("path,nproc", [("peer", 2), ("sharded", 1), ("peer", 1)])
-def test_bench_runs_the_split_layouts(path, nproc, tmp_path):
+def _rank_main_topk(rank, world, port, d, chunk, n_local, steps, frac, outdir):
+    import torch
+    import torch.distributed as dist
+
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    try:
+        torch.cuda.set_device(0)
+        dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+        w = tiny(d, world * n_local, chunk, cfg_id=145)
+        ctx = B.Context(w.d, n_local, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        ctx.set_compressor(B.COMPRESSOR_TOPK, frac)
+        orc = ao.Oracle(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        orc.set_compressor(ao.TOPK); orc.set_topk_fraction(frac)
+        x0 = wl.initial_params(w)
+        ctx.set_params(x0); orc.set_params(x0)
+        ctx.freeze_v(); orc.freeze_v()
+        step = sharded.PeerShardedStep(ctx)
+        for k in range(1, steps + 1):
+            host = wl.host_gradients(w, k)
+            step.step(H.upload(host[rank * n_local:(rank + 1) * n_local]))
+            orc.compressed_step(host)
+        idx = np.arange(w.d)
+        mask = (ctx.get_state(B.STATE_SERVER_BITS)[idx // 32] >> (idx % 32).astype(np.uint32)) & 1
+        bad = []
+        if not np.array_equal(mask.astype(np.uint8), orc.server_selected):
+            bad.append("server mask")
+        for name, which, ref in (("x", B.STATE_X, orc.x), ("m", B.STATE_M, orc.m)):
+            if not np.array_equal(ctx.get_state(which).view(np.uint32), ref.view(np.uint32)):
+                bad.append(name)
+        cb, ce = step.ranges[rank]                                  # a range's server error lives where the range is served
+        e0, e1 = cb * w.chunk, min(ce * w.chunk, w.d)
+        if not np.array_equal(ctx.get_state(B.STATE_SERVER_ERR)[e0:e1].view(np.uint32), orc.server_err[e0:e1].view(np.uint32)):
+            bad.append("server error")
+        for i in range(n_local):
+            if not np.array_equal(ctx.get_state(B.STATE_WORKER_ERR, i).view(np.uint32), orc.worker_err(rank * n_local + i).view(np.uint32)):
+                bad.append(f"error of worker {rank * n_local + i}")
+        wire = step.wire_bytes_per_step()
+        step.close()
+        ctx.close()
+        _report(outdir, rank, [not bad, wire, ", ".join(bad)])
+        dist.destroy_process_group()
+    except Exception as exc:                                        # reported to the parent, which fails the test
+        _report(outdir, rank, [False, 0, repr(exc)])
+        raise
+
+
+@pytest.mark.parametrize("d,chunk,frac", [(9 * 2048 + 300, 2048, 0.03), (5 * 4096 + 77, 4096, 0.25)])
+def test_two_processes_on_one_gpu_carry_the_topk_compressor(d, chunk, frac, tmp_path):
+    """The peer form with the top-k compressor: every process packs its workers' kept values straight into the
+    serving process's receive rows (device buffers shared through CUDA IPC), the server ranges go back the same
+    way; state equal, bit for bit, to the oracle holding all workers."""
+    import json
+
+    import torch.multiprocessing as mp
+
+    n_local, world = 2, 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    mp.spawn(_rank_main_topk, args=(world, port, d, chunk, n_local, 4, frac, str(tmp_path)), nprocs=world, join=True)
+    res = {r: json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)}
+    assert res[0][0] and res[1][0], res
+    assert max(res[0][1], res[1][1]) < (0.1 + 2 * frac) * 4 * d * n_local
+
+
+@pytest.mark.parametrize("path,nproc,extra", [("peer", 2, ()), ("sharded", 1, ()), ("peer", 1, ()),
+                                              ("peer", 2, ("--compressor", "topk", "--topk-fraction", "0.01"))])
+def test_bench_runs_the_split_layouts(path, nproc, extra, tmp_path):
     """bench.py --path peer under a two-process launch with both processes on the one GPU (what a
     one-process-per-GPU run executes, the peer's memory on the same device), and both split paths with a single
     process: one JSON line, strong scaling, the workload's workers divided over the processes."""
@@ -168,7 +235,7 @@ def test_bench_runs_the_split_layouts(path, nproc, tmp_path):
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={nproc}",
            "--master-addr", "127.0.0.1", "--master-port", str(port),
            os.path.join(ROOT, "bench.py"), "--gpus", str(nproc), "--path", path, "--config", "1",
-           "--steps", "3", "--warmup", "3", "--no-cpu-baseline"]
+           "--steps", "3", "--warmup", "3", "--no-cpu-baseline", *extra]
     if nproc > 1:
         cmd.append("--one-gpu")
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=900, cwd=ROOT)

@@ -500,10 +500,11 @@ def main(argv=None) -> int:
         ab["step"] = ab["worker"] + ab["server"]
     wk_gbs = ab["worker"] / (kernel_ms["worker"] * 1e-3) / 1e9
     step_gbs = ab["step"] / (ms_per_step * 1e-3) / 1e9
+    # the ncu figures are those of k_worker_fine (chunks of 512 elements and more) and of the per-chunk fused server kernel
     traffic = (NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT * w.d * n_local
                if NCU_WORKER_TRAFFIC_BYTES_PER_WORKER_ELEMENT and args.grad_dtype == "float32"
-               and args.compressor == "onebit" else None)
-    fused = args.compressor == "onebit" and "apply" not in kernel_ms and not split and w.chunk >= 2048
+               and args.compressor == "onebit" and w.chunk >= 512 else None)
+    fused = args.compressor == "onebit" and "apply" not in kernel_ms and not split and 2048 <= w.chunk <= 65536
     traffic_by_kernel = {"worker": traffic,
                          "server": ((NCU_SERVER_FUSED_TRAFFIC_BYTES_PER_ELEMENT_N8 + (w.n - 8) / 8.0) * w.d
                                     if fused and args.grad_dtype == "float32" else None)}

@@ -191,3 +191,46 @@ def test_topk_sampled_chunks_at_full_size(frac):
             words = _gather_words(ctx, B.STATE_WORKER_BITS, sl, worker=i)
             assert np.array_equal(((words[idx // 32] >> (idx % 32).astype(np.uint32)) & 1).astype(np.uint8),
                                   orc.worker_selected(i)), (step, i, "mask")
+
+
+@pytest.mark.parametrize("chunk", [None, "d/16", 1024], ids=["chunk-32768", "one-chunk-per-server", "chunk-1024"])
+def test_two_runs_at_full_size_leave_the_same_state(chunk):
+    """Thousands of CTAs of the step's kernels overlap in time at full size and in changing order; the state they
+    leave must not depend on it: two runs from the same inputs, the whole server message and the whole model
+    compared bit for bit after every compressed step (checksums on the host)."""
+    import zlib
+
+    import torch
+
+    w = wl.config(3)
+    if chunk is not None:
+        w = w.with_(chunk=w.d // 16 if chunk == "d/16" else chunk)
+    gc.collect(); torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < B.apms_workspace_bytes(w.d, w.n, w.chunk) + (w.n + 2) * 4 * w.d + (4 << 30):
+        pytest.skip("not enough device memory for the full-size workload")
+    grads = [torch.empty(w.d, dtype=torch.float32, device="cuda") for _ in range(w.n)]
+    x0 = torch.from_numpy(wl.initial_params(w)).cuda()
+    crc = lambda a: zlib.crc32(np.ascontiguousarray(a).tobytes())
+    runs = []
+    for rep in range(2):
+        ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        ctx.set_params(x0)
+        rec = []
+        for step in range(5):
+            for i in range(w.n):
+                wl.device_gradient(w, step, i, grads[i])
+            if step < 2:
+                ctx.warmup_step(grads)
+                if step == 1:
+                    ctx.freeze_v()
+                continue
+            ctx.compressed_step(grads)
+            rec.append((crc(ctx.get_state(B.STATE_SERVER_SCALES)), crc(ctx.get_state(B.STATE_SERVER_BITS)),
+                        crc(ctx.get_state(B.STATE_SERVER_ERR)), crc(ctx.get_state(B.STATE_X)),
+                        crc(ctx.get_state(B.STATE_WORKER_SCALES, w.n - 1)), crc(ctx.get_state(B.STATE_WORKER_BITS, w.n - 1))))
+        runs.append(rec)
+        ctx.close()
+        del ctx
+        gc.collect(); torch.cuda.empty_cache()
+    assert runs[0] == runs[1]

@@ -62,7 +62,7 @@ struct Layout {
     int fine_split, fine_words;
     int n;
     Tiling t;
-    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_hint, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
+    size_t off_x, off_v, off_m, off_zbar, off_z, off_B, off_Bbar, off_s, off_Sbar, off_hint, off_tiles, off_part, off_fine, off_stage, off_mon, off_den, off_status, total;
     size_t guard;                  // guard bytes behind every row of every array (0 = the ordinary layout)
 };
 
@@ -109,6 +109,8 @@ bool make_layout(int64_t d, int n, int64_t chunk, Layout* L, size_t guard = 0, s
     L->t.d = d; L->t.chunk = chunk;
     if (chunk <= kTileMax) { L->t.tile = chunk; L->t.P = 1; }
     else { L->t.tile = kTileSplit; L->t.P = (int)((chunk + kTileSplit - 1) / kTileSplit); }
+    // counters of the lagged server form (chunks cut into tiles): 64 words for the ticket, then per chunk the tiles done and the ready flag
+    L->off_tiles = take("server tile counters", 1, 64 + 2 * (size_t)L->Cp, L->t.P > 1 ? 64 + 2 * (size_t)L->Cp - guard / 4 : 0, 4);
     L->t.Pp = (int64_t)round_up((size_t)(L->C * L->t.P), 64) + (int64_t)(guard / 8);
     L->off_part = take("partial sums of split chunks", L->t.P > 1 ? un + 1 : 0, L->t.Pp, (size_t)(L->C * L->t.P), 8);   // n worker rows + 1 server row
     L->fine_tiles = (d + kFineTile - 1) / kFineTile;
@@ -155,6 +157,7 @@ struct apms_ctx {
     bool timing;
     apms_team_mode team_mode;
     int fine_run;            // tiles of one worker launched back to back in the fine worker form
+    unsigned int tile_epoch; // launches of the lagged server form so far (never 0 in a launch)
     std::vector<EventPair> events[APMS_KERNEL_COUNT];
     std::vector<EventPair> pool;
     int64_t launches;
@@ -174,6 +177,9 @@ struct apms_ctx {
     float* Sbar() { return (float*)(ws + L.off_Sbar); }
     float* hint(int i) { return (float*)(ws + L.off_hint) + (int64_t)i * L.Cp; }   // i = n: the server's
     float* learned(int i) { return hint(L.n + 1 + i); }
+    unsigned int* tile_ticket() { return (unsigned int*)(ws + L.off_tiles); }
+    unsigned int* tiles_done() { return tile_ticket() + 64; }
+    unsigned int* tiles_ready() { return tiles_done() + L.Cp; }
     float* stage(int b) { return (float*)(ws + L.off_stage) + (int64_t)b * L.dz; }
     int* status() { return (int*)(ws + L.off_status); }
     float* den() { return (float*)(ws + L.off_den); }
@@ -657,11 +663,21 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
         Timed t(c, APMS_KERNEL_SERVER);
         if (staged) {
             const bool fused = may_fuse && c->L.t.P == 1;   // the CTA sees the whole chunk, so it knows the new scale
-            if (fused) {
+            // chunks cut into tiles, whole vector: steps 5-6 follow `lag` tiles behind in the same kernel
+            const bool lagged = may_fuse && c->L.t.P > 1 && cb == 0 && ce == c->L.C && c->team_mode == APMS_TEAM_AUTO;
+            if (fused || lagged) {
                 apms_status dst = ensure_den(c);
                 if (dst != APMS_OK) return dst;
             }
             ServerStagedArgs sa;
+            sa.lag = 0; sa.ticket = sa.done = sa.ready = nullptr; sa.epoch = 0;
+            if (lagged) {
+                // at least the tiles of a chunk (no deadlock, see the kernel); about the resident CTAs more, so that the wait is rare
+                sa.lag = (int64_t)c->L.t.P + 3 * (int64_t)c->sms;
+                sa.ticket = c->tile_ticket(); sa.done = c->tiles_done(); sa.ready = c->tiles_ready();
+                if (++c->tile_epoch == 0) c->tile_epoch = 1;
+                sa.epoch = c->tile_epoch;
+            }
             sa.a = a; sa.status = c->status();
             sa.inv_n = ((a.n & (a.n - 1)) == 0) ? 1.0f / (float)a.n : 0.0f;
             sa.den = c->den(); sa.x = c->x(); sa.lr = c->lr; sa.row_align = row_align;
@@ -669,14 +685,16 @@ apms_status launch_server(apms_ctx* c, const ServerSource& src, int64_t cb, int6
             sa.span = fused ? (int)((kStagedSpanElems + c->L.chunk - 1) / c->L.chunk) : 1;
             const int64_t fill = count / (2 * (int64_t)c->sms);       // small problems: keep at least two CTAs per SM
             if (sa.span > 1 && fill < sa.span) sa.span = fill < 1 ? 1 : (int)fill;
-            const int64_t ctas = (count + sa.span - 1) / sa.span;
+            const int64_t ctas = (count + sa.span - 1) / sa.span + sa.lag;
+            if (ctas > 0x7fffffff) return fail(c, APMS_ERR_INVALID_ARG, "too many chunk tiles for one launch");
             cudaError_t e = fused ? launch_staged_n<true>(sa, (unsigned)ctas, smem, c->stream)
                                   : launch_staged_n<false>(sa, (unsigned)ctas, smem, c->stream);
             if (e != cudaSuccess) {
                 snprintf(c->err, sizeof c->err, "setting up k_server_staged failed: %s", cudaGetErrorString(e));
                 return APMS_ERR_CUDA;
             }
-            *applied = fused;
+            *applied = fused || lagged;
+            if (lagged) return launch_check(c, "k_server_staged");      // the chunks' scales are stored by their last tiles
         }
         else if (warp_teams) k_server<APMS_SERVER_U, 1><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
         else            k_server<APMS_SERVER_U, kWarps><<<(unsigned)blocks, kThreads, 0, c->stream>>>(a);
@@ -843,6 +861,7 @@ apms_status apms_create(apms_ctx** out, int64_t d, int n, float beta1, float bet
     c->steps = 0; c->has_sched = false; c->substep = 0; c->worker_chunks = 0; c->variant = APMS_VARIANT_MOMENTUM; c->csteps = 0;
     c->compressor = APMS_COMPRESSOR_ONEBIT; c->topk_frac = 0.01;
     c->fine_run = kFineRunDefault;
+    c->tile_epoch = 0;
     if ((int64_t)c->fine_run > L.fine_tiles && L.fine_tiles > 0) c->fine_run = (int)L.fine_tiles;
     *out = c;
     return APMS_OK;
@@ -875,6 +894,7 @@ apms_status apms_set_params(apms_ctx* c, const float* x0, int src_is_device)
     APMS_CUDA(c, cudaMemsetAsync(c->m(), 0, (size_t)c->L.d * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->v(), 0, (size_t)c->L.d * 4, c->stream));
     APMS_CUDA(c, cudaMemsetAsync(c->status(), 0, 256, c->stream));
+    APMS_CUDA(c, cudaMemsetAsync(c->tile_ticket(), 0, (64 + 2 * (size_t)c->L.Cp) * 4, c->stream));
     st = fill_guards(c);
     if (st != APMS_OK) return st;
     st = register_checked(c);

@@ -225,6 +225,12 @@ struct ServerStagedArgs {
     const float* den; float* x; float lr;        // steps 5-6 (fused form only): den = sqrt(v) + eps, see k_make_den
     int span;             // chunks per CTA of the fused form
     int row_align;        // (address of every row's word 0 / 4) mod 4: the rows' common distance from a 16-byte boundary, in words
+    // Lagged form (chunks cut into several tiles, whole step): see k_server_staged.  lag = 0: off.
+    int64_t lag;          // a CTA applies the model update of the tile `lag` tickets before its own
+    unsigned int* ticket; // the next tile to hand out
+    unsigned int* done;   // per chunk: tiles finished so far in this launch
+    unsigned int* ready;  // per chunk: `epoch` once the chunk's new scale is stored
+    unsigned int epoch;   // differs from launch to launch, never 0
 };
 
 // Bytes of one ring stage: a slab of zbar plus n rows of sign words, or (fused form) a slab of v and of x.
@@ -345,21 +351,34 @@ k_server_staged(const ServerStagedArgs sa)
     __shared__ float prefix8[NT >= kPrefixWorkers ? 256 : 1];         // see signed_scale_sums
     __shared__ int failed;
 
+    __shared__ unsigned int my_ticket;
+
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n = NT > 0 ? NT : a.n;
     const size_t stage_bytes = staged_stage_bytes(n, FUSED);
     // behind the ring: the current tile's new sign words, from the 16-byte boundary below the first (staged_nb_bytes)
     uint32_t* const nb = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes);
     const int span = MULTI ? sa.span : 1;                  // MULTI = false: one item, the walk's loops fold away
-    const int64_t item0 = a.item0 + (int64_t)blockIdx.x * span;
-    const int nitems = MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1;
+    // Lagged form.  A chunk cut into P tiles knows its new scale only when its last tile is done, so steps 5-6
+    // cannot follow step 4 inside the tile's CTA; run as a kernel of their own they cost the step 3 % (the
+    // server part is bound by instruction issue, the update by memory: one after the other neither unit is busy).
+    // Here the CTAs take their tiles from a ticket counter, in order; a CTA does step 4 for tile t, counts it in
+    // (the chunk's last tile adds the P partial sums in tile order, stores the scale and raises the chunk's flag),
+    // and then does steps 5-6 for tile t - lag, whose chunk is complete or about to be: with lag >= P all of its
+    // tiles hold lower tickets, so they belong to CTAs that are already running and that wait for nobody
+    // before they have counted their tile in - the wait (bounded like every other) cannot deadlock.  `lag` more
+    // CTAs than tiles do the last updates.
+    const bool lagged = !FUSED && !MULTI && sa.lag > 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
         failed = 0;
+        if (lagged) my_ticket = atomicAdd(sa.ticket, 1u);
         mbar_fence_init();
     }
     __syncthreads();
+    const int64_t item0 = lagged ? a.item0 + (int64_t)my_ticket : a.item0 + (int64_t)blockIdx.x * span;
+    const int nitems = lagged ? (item0 < a.items ? 1 : 0) : (MULTI ? (int)(a.items - item0 < span ? a.items - item0 : span) : 1);
 
     if (warp == kWarps) {
         // ---- producer warp: one lane feeds the ring (only whole 16-byte pieces that hold live elements)
@@ -419,11 +438,12 @@ k_server_staged(const ServerStagedArgs sa)
         uint32_t pre_neg = 0u;
         float pre_S = 0.0f;
         const int my_worker = (warp < 2 && n > 32) ? warp * 32 + lane : lane;     // n <= 32: every warp fetches workers 0..n-1
-        {
+        if (nitems > 0) {
             const Item it0 = decode_item(a.t, item0);
             if (my_worker < n) pre_neg = __float_as_uint(a.srow[my_worker][it0.c]) | 0x80000000u;
             pre_S = a.Sbar[it0.c];
         }
+        bool tile_done = false;
         for (int w = 0; w < nitems; ++w) {
             const Item it = decode_item(a.t, item0 + w);
             const int L = it.L;
@@ -452,8 +472,6 @@ k_server_staged(const ServerStagedArgs sa)
                 const float4 zo1 = *reinterpret_cast<const float4*>(zs + g1 * kGroup + lane * 4);
                 float2 s01 = make_float2(0.f, 0.f), s23 = s01, t01 = s01, t23 = s01;   // running sums, worker order
                 signed_scale_sums<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl, negs, prefix8, n, sh, s01, s23, t01, t23);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
                 const bool whole = (j + 1) * kSlab <= L;                 // no element of this slab needs a bounds test (warp-uniform)
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
@@ -467,6 +485,11 @@ k_server_staged(const ServerStagedArgs sa)
                     const uint32_t word = pack_group_words(nibble, lane);
                     if ((lane & 7) == 0) nb[off_out + grp * 4 + wl] = word;   // words past L hold zeros and are never stored
                 }
+                // The stage is handed back only now: the stores above needed every value this warp loaded from it, so
+                // the loads have returned.  (Handed back right after the loads were issued, the stage was now and then
+                // refilled before a load had read it, when the SM's load/store path was backed up.)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[st]);
             }
             acc = warp_sum(acc);
             if (lane == 0) red[warp] = acc;
@@ -491,8 +514,6 @@ k_server_staged(const ServerStagedArgs sa)
                         vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
                         xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[st]);
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const int grp = j * kSlabGroups + (u ? g1 : g0);
@@ -505,6 +526,8 @@ k_server_staged(const ServerStagedArgs sa)
                         if ((j + 1) * kSlab <= L) st_stream4(sa.x + it.base + k, xx[u]);
                         else st4_checked(sa.x + it.base, k, L, xx[u]);
                     }
+                    __syncwarp();                                        // after the stores: see above
+                    if (lane == 0) mbar_arrive(&empty[st]);
                 }
             } else if (ok && threadIdx.x == 0) {
                 if (a.t.P == 1) APMS_STORE(a.Sbar[it.c], (float)sqrt(total / (double)it.Lc));
@@ -519,6 +542,76 @@ k_server_staged(const ServerStagedArgs sa)
                     else for (int r = (w4 < off_out ? off_out : w4); r < w4 + 4 && r < wend; ++r) APMS_STORE(ob[r], nb[r]);
                 }
             }
+            tile_done = ok;
+        }
+        if (lagged) {
+            if (nitems > 0 && tile_done) {
+                __threadfence();                       // this thread's sign words, thread 0's partial sum: visible before the count
+                consumer_barrier();
+                if (threadIdx.x == 0) {
+                    const Item it = decode_item(a.t, item0);
+                    if (atomicAdd(sa.done + it.c, 1u) + 1u == (unsigned int)a.t.P) {
+                        __threadfence();
+                        double total = 0.0;            // as k_finalize_scales: the tiles' sums in tile order
+                        for (int p = 0; p < a.t.P; ++p) total += __ldcg(a.partial + it.c * a.t.P + p);
+                        APMS_STORE(a.Sbar[it.c], scale_from_sum(total, (double)it.Lc, a.t.l1 != 0));
+                        sa.done[it.c] = 0u;            // for the next launch
+                        __threadfence();
+                        atomicExch(sa.ready + it.c, sa.epoch);
+                    }
+                }
+            }
+            const int64_t u = item0 - sa.lag;
+            if (u >= a.item0 && u < a.items) {
+                const Item iu = decode_item(a.t, u);
+                if (threadIdx.x == 0 && *vfailed == 0) {
+                    const volatile unsigned int* flag = sa.ready + iu.c;
+                    const volatile int* status = sa.status;
+                    const long long t0 = clock64();
+                    while (*flag != sa.epoch) {
+                        if (*status != DEVICE_OK || clock64() - t0 > kWaitCycles) { failed = 1; break; }
+                        __nanosleep(200);
+                    }
+                    __threadfence();
+                }
+                if (!consumer_barrier_any(*vfailed != 0)) {
+                    const float c_new = __fmul_rn(sa.lr, __ldcg(a.Sbar + iu.c));
+                    const uint32_t* __restrict__ bw = a.Bbar + iu.base / 32;
+                    const float* __restrict__ dn = sa.den + iu.base;
+                    float* __restrict__ xo = sa.x + iu.base;
+                    constexpr int kAhead = 4;                                 // sweeps whose loads are in flight together
+                    const int Lfull = iu.L - iu.L % (kAhead * kThreads * 4);
+                    int k = threadIdx.x * 4;
+                    for (; k < Lfull; k += kAhead * kThreads * 4) {
+                        float4 dd[kAhead], xx[kAhead];
+                        uint32_t nn[kAhead];
+#pragma unroll
+                        for (int u2 = 0; u2 < kAhead; ++u2) {
+                            const int kk = k + u2 * kThreads * 4;
+                            dd[u2] = ld_stream4(dn + kk);
+                            xx[u2] = ld_stream4(xo + kk);
+                            nn[u2] = __ldcg(bw + (kk >> 5)) >> (kk & 31);
+                        }
+#pragma unroll
+                        for (int u2 = 0; u2 < kAhead; ++u2) {
+                            xx[u2].x = apply_stored(xx[u2].x, dd[u2].x, nn[u2] & 1u, c_new);
+                            xx[u2].y = apply_stored(xx[u2].y, dd[u2].y, nn[u2] & 2u, c_new);
+                            xx[u2].z = apply_stored(xx[u2].z, dd[u2].z, nn[u2] & 4u, c_new);
+                            xx[u2].w = apply_stored(xx[u2].w, dd[u2].w, nn[u2] & 8u, c_new);
+                            st_stream4(xo + k + u2 * kThreads * 4, xx[u2]);
+                        }
+                    }
+                    for (; k < iu.L; k += kThreads * 4) {
+                        const float4 d0 = ld4_checked(dn, k, iu.L, true);
+                        float4 x0 = ld4_checked(xo, k, iu.L, true);
+                        const uint32_t n0 = __ldcg(bw + (k >> 5)) >> (k & 31);
+                        x0.x = apply_stored(x0.x, d0.x, n0 & 1u, c_new); x0.y = apply_stored(x0.y, d0.y, n0 & 2u, c_new);
+                        x0.z = apply_stored(x0.z, d0.z, n0 & 4u, c_new); x0.w = apply_stored(x0.w, d0.w, n0 & 8u, c_new);
+                        st4_checked(xo, k, iu.L, x0);
+                    }
+                }
+            }
+            if (threadIdx.x == 0 && my_ticket + 1u == gridDim.x) *sa.ticket = 0u;    // every ticket has been handed out
         }
     }
     __syncthreads();                                   // every warp has left its loops; shared memory may go
@@ -694,8 +787,6 @@ k_server_packed(const ServerStagedArgs sa)
                     vv[u] = *reinterpret_cast<const float4*>(vs + (u ? g1 : g0) * kGroup + lane * 4);
                     xx[u] = *reinterpret_cast<const float4*>(xs + (u ? g1 : g0) * kGroup + lane * 4);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int k = (u ? g1 : g0) * kGroup + lane * 4;
@@ -707,6 +798,8 @@ k_server_packed(const ServerStagedArgs sa)
                     xx[u].w = apply_stored(xx[u].w, vv[u].w, nib & 8u, cn);
                     st4_checked(sa.x + base_e, k, L, xx[u]);
                 }
+                __syncwarp();                                            // the stage goes back after the stores that needed its values
+                if (lane == 0) mbar_arrive(&empty[st]);
             }
             ++q;
         };
@@ -743,8 +836,6 @@ k_server_packed(const ServerStagedArgs sa)
                     signed_scale_sums2<NT>(rows + off_in + g0 * 4 + wl, rows + off_in + g1 * 4 + wl,
                                            negs + kk0 * APMS_MAX_WORKERS, negs + kk1 * APMS_MAX_WORKERS, n, sh, s01, s23, t01, t23);
                     const float So0 = S_old_sh[buf][kk0], So1 = S_old_sh[buf][kk1];
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[st]);                  // this warp is done with the stage
                     uint32_t* __restrict__ ob = a.Bbar + base_e / 32;
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
@@ -774,6 +865,8 @@ k_server_packed(const ServerStagedArgs sa)
                         const int wk = grp * 4 + wl;
                         if ((lane & 7) == 0 && wk * 32 < L) st_stream_word(ob + wk, word);
                     }
+                    __syncwarp();                                            // the stage goes back after the stores that needed its values
+                    if (lane == 0) mbar_arrive(&empty[st]);
                 }
                 ++q;
             }

@@ -73,8 +73,10 @@ def _cases(args):
                                 bytes=lambda w: w.n * (8 * (w.d // 512) + 4 * w.n_chunks)),
         "k_server_staged": dict(setup=dict(chunk=32768), call="step", timer=B.KERNEL_SERVER,
                                 bytes=lambda w: w.n * w.d // 8 + 8 * w.d + w.d // 8 + 12 * w.d),
-        "k_server_staged_unfused": dict(setup=dict(chunk=4 * 65536), call="step", timer=B.KERNEL_SERVER,
+        "k_server_staged_unfused": dict(setup=dict(chunk=4 * 65536), call="worker_phase", timer=B.KERNEL_SERVER,
                                         bytes=lambda w: w.n * w.d // 8 + 8 * w.d + w.d // 8),
+        "k_server_staged_lagged": dict(setup=dict(chunk=4 * 65536), call="step", timer=B.KERNEL_SERVER,
+                                       bytes=lambda w: w.n * w.d // 8 + 8 * w.d + w.d // 4 + 12 * w.d),
         "k_server_packed": dict(setup=dict(chunk=1024), call="step", timer=B.KERNEL_SERVER,
                                 bytes=lambda w: w.n * w.d // 8 + 8 * w.d + w.d // 8 + 12 * w.d),
         "k_server": dict(setup=dict(chunk=160), call="step", timer=B.KERNEL_SERVER,

@@ -193,8 +193,9 @@ def test_topk_sampled_chunks_at_full_size(frac):
                                   orc.worker_selected(i)), (step, i, "mask")
 
 
-@pytest.mark.parametrize("chunk", [None, "d/16", 1024], ids=["chunk-32768", "one-chunk-per-server", "chunk-1024"])
-def test_two_runs_at_full_size_leave_the_same_state(chunk):
+@pytest.mark.parametrize("chunk,topk", [(None, None), ("d/16", None), (1024, None), (128, None), (None, 0.01), (None, 0.03)],
+                         ids=["chunk-32768", "one-chunk-per-server", "chunk-1024", "chunk-128", "topk-1%", "topk-3%"])
+def test_two_runs_at_full_size_leave_the_same_state(chunk, topk):
     """Thousands of CTAs of the step's kernels overlap in time at full size and in changing order; the state they
     leave must not depend on it: two runs from the same inputs, the whole server message and the whole model
     compared bit for bit after every compressed step (checksums on the host)."""
@@ -215,9 +216,11 @@ def test_two_runs_at_full_size_leave_the_same_state(chunk):
     runs = []
     for rep in range(2):
         ctx = B.Context(w.d, w.n, w.beta1, w.beta2, w.eps, w.lr, w.chunk)
+        if topk is not None:
+            ctx.set_compressor(B.COMPRESSOR_TOPK, topk)
         ctx.set_params(x0)
         rec = []
-        for step in range(5):
+        for step in range(5 if topk is None else 8):       # top-k: the predicted-threshold routes need a few steps of history
             for i in range(w.n):
                 wl.device_gradient(w, step, i, grads[i])
             if step < 2:

@@ -97,6 +97,83 @@ class OracleBackend:
             self.x[lo:hi] = self.x[lo:hi] - (np.float32(LR) * q) / (np.sqrt(self.v[lo:hi]) + np.float32(EPS))
 
 
+FRAC = 0.05
+
+
+def _pack_mask(sel):
+    pad = (-sel.size) % 32
+    return np.packbits(np.concatenate([sel, np.zeros(pad, np.uint8)]), bitorder="little").view(np.uint32)
+
+
+def _unpack_mask(words, length):
+    return np.unpackbits(np.ascontiguousarray(words).view(np.uint8), bitorder="little")[:length].astype(bool)
+
+
+class TopkOracleBackend(OracleBackend):
+    """The same stand-in with the top-k compressor (Section 5.1): a message is the selection mask plus the kept
+    values in index order, `per` slots per chunk."""
+
+    topk = True
+
+    def __init__(self, *args):
+        super().__init__(*args)
+        self.q = [np.zeros(self.d, np.float32) for _ in range(self.n + 1)]      # C[z] of every worker, last = server
+
+    def topk_values_per_chunk(self):
+        return self.ao.topk_count(FRAC, self.chunk)
+
+    def worker_phase(self, grads):
+        omb1 = np.float32(1.0) - np.float32(BETA1)
+        for i, g in enumerate(grads):
+            g = g.numpy()
+            for c, lo, hi in self._chunks(0, self.C):
+                z = _fma32(np.float32(BETA1), self.m[lo:hi], omb1 * g[lo:hi]) + self.err[i][lo:hi]
+                q, sel = self.ao.compress_topk(z, self.ao.topk_count(FRAC, hi - lo))
+                self.err[i][lo:hi] = z - q
+                self.q[i][lo:hi] = q
+                words = _pack_mask(sel)
+                self.bits[i].numpy().view(np.uint32)[lo // 32:lo // 32 + words.size] = words
+
+    def topk_pack_values(self, worker, cb, ce, out):
+        per = self.topk_values_per_chunk()
+        for c, lo, hi in self._chunks(cb, ce):
+            sel = _unpack_mask(self.bits[worker].numpy().view(np.uint32)[lo // 32:(hi + 31) // 32], hi - lo)
+            vals = self.q[worker][lo:hi][sel]
+            out[(c - cb) * per:(c - cb) * per + vals.size] = torch.from_numpy(vals)
+
+    def _take_over(self, c, lo, hi, q, sel):
+        self.q[-1][lo:hi] = q
+        words = _pack_mask(sel.astype(np.uint8))
+        self.bits[-1].numpy().view(np.uint32)[lo // 32:lo // 32 + words.size] = words
+        self.m[lo:hi] = q
+        self.x[lo:hi] = self.x[lo:hi] - (np.float32(LR) * q) / (np.sqrt(self.v[lo:hi]) + np.float32(EPS))
+
+    def topk_server_phase(self, mask_rows, val_rows, cb, ce):
+        per, rows, w_first = self.topk_values_per_chunk(), mask_rows.shape[0], cb * self.chunk // 32
+        for c, lo, hi in self._chunks(cb, ce):
+            acc = np.zeros(hi - lo, np.float32)
+            for j in range(rows):                                   # row order = global worker order
+                sel = _unpack_mask(mask_rows[j].numpy().view(np.uint32)[lo // 32 - w_first:(hi + 31) // 32 - w_first], hi - lo)
+                qj = np.zeros(hi - lo, np.float32)
+                qj[sel] = val_rows[j, (c - cb) * per:(c - cb) * per + int(sel.sum())].numpy()
+                acc = acc + qj
+            z = acc / np.float32(rows) + self.server_err[lo:hi]
+            q, sel = self.ao.compress_topk(z, self.ao.topk_count(FRAC, hi - lo))
+            self.server_err[lo:hi] = z - q
+            self._take_over(c, lo, hi, q, sel)
+
+    def topk_put_server_range(self, mask_words, vals, kb, ke):
+        per, w_first = self.topk_values_per_chunk(), kb * self.chunk // 32
+        for c, lo, hi in self._chunks(kb, ke):
+            sel = _unpack_mask(mask_words.numpy().view(np.uint32)[lo // 32 - w_first:(hi + 31) // 32 - w_first], hi - lo)
+            q = np.zeros(hi - lo, np.float32)
+            q[sel] = vals[(c - kb) * per:(c - kb) * per + int(sel.sum())].numpy()
+            self._take_over(c, lo, hi, q, sel)
+
+    def apply_phase(self):                                          # the kept elements were updated where their range was served or taken over
+        pass
+
+
 def _inputs():
     rng = np.random.default_rng(77)
     x0 = (rng.standard_normal(D) * 0.02).astype(np.float32)
@@ -155,6 +232,49 @@ def test_two_ranks_two_workers_each_equal_one_four_worker_run():
     assert res[0][0] and res[1][0]
     # the wire carries packed sign words and scales only: far below 4 d bytes per worker
     assert max(res[0][1], res[1][1]) < 0.1 * 4 * D * (N_TOTAL // world)
+
+
+def _rank_main_topk(rank, world, port, out):
+    from oracle import apms_oracle as ao
+    from paper_2008_11343_b200 import sharded
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    x0, v, m, grads = _inputs()
+    n_local = N_TOTAL // world
+    backend = TopkOracleBackend(D, n_local, CHUNK, x0, v, m)
+    step = sharded.ShardedStep(backend)
+    for gs in grads:
+        step.step([torch.from_numpy(g) for g in gs[rank * n_local:(rank + 1) * n_local]])
+    ref = ao.Oracle(D, N_TOTAL, BETA1, 0.999, EPS, LR, CHUNK)
+    ref.set_compressor(ao.TOPK); ref.set_topk_fraction(FRAC)
+    ref.set_params(x0)
+    ref.freeze_v()
+    ref.v[:], ref.m[:] = v, m
+    for gs in grads:
+        ref.compressed_step(gs)
+    ok = bool(np.array_equal(backend.x, ref.x) and np.array_equal(backend.m, ref.m)
+              and np.array_equal(_unpack_mask(backend.bits[-1].numpy().view(np.uint32), D), ref.server_selected.astype(bool)))
+    for i in range(n_local):
+        ok = ok and bool(np.array_equal(backend.err[i], ref.worker_err(rank * n_local + i)))
+    cb, ce = step.ranges[rank]
+    lo, hi = cb * CHUNK, min(D, ce * CHUNK)
+    ok = ok and bool(np.array_equal(backend.server_err[lo:hi], ref.server_err[lo:hi]))
+    out[rank] = (ok, step.wire_bytes_per_step())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_carry_the_topk_compressor():
+    """ShardedStep with the top-k compressor over two gloo ranks: masks and packed kept values cross the wire, the
+    result equals one four-worker run of the C oracle with the same compressor."""
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_rank_main_topk, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0][0] and res[1][0]
+    assert max(res[0][1], res[1][1]) < (0.1 + 2 * FRAC) * 4 * D * (N_TOTAL // world)
 
 
 def test_chunk_and_word_ranges_tile_the_vector():
